@@ -1,0 +1,607 @@
+/*
+ * CPU oracle for StreamingTOM's Online Quantized Memory (OQM).
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is a plain, slow restatement of the
+ * method, step by step, in the paper's order and notation.  It shares no
+ * code, header, table or helper with the CUDA library, and the CUDA library
+ * never calls it.  Only the test-suite, the smoke check and the benchmark's
+ * CPU-baseline leg load it.
+ *
+ * Every pointer is a HOST pointer.  Floating point that decides an integer
+ * (the 4-bit codes) is done in IEEE binary32 exactly as written here; all
+ * other reductions (means, norms, dot products, softmax) are done in
+ * binary64.  Build with  gcc -O2 -ffp-contract=off -fno-fast-math  so the
+ * compiler neither fuses nor reorders the binary32 operations.
+ *
+ * Passages followed (paper section / equation):
+ *   - group quantizer, scale and offset ........ Sec. 3.4 "Online Quantized
+ *     Memory", the Q_4 equation and the (s_t, m_t) equation
+ *   - representative key ...................... Sec. 3.4 (mean of the keys
+ *     before quantization); appendix "Layer-wise vision memory"
+ *   - dequantization .......................... Sec. 3.4, the Q_4^{-1} equation
+ *   - question embedding, cosine top-K ........ appendix "Question-guided
+ *     single-pass retrieval" (the q^(l) equation and the K = min(..) equation)
+ *   - active cache ............................ Sec. 3.4, the KV_active
+ *     equation; appendix "Cache reconstruction for decoding"
+ *   - storage accounting ...................... Sec. 3.1 memory-growth
+ *     equation and its footnote; Sec. 3.2 ratio 4N/G; ablation table "Ratio"
+ *
+ * Readings taken where the paper is silent (kept in one place so they can be
+ * checked by eye):
+ *   - forward map: code = clamp(rne((x - m) / s), 0, 15), true division,
+ *     round-half-to-even; if s == 0 the channel is constant (or its range
+ *     underflows) and every code is 0;
+ *   - packing: along the channel axis, even channel in the low nibble;
+ *   - inverse map: fmaf(code, s, m), then one rounding to the output type;
+ *   - GQA: query head h_q belongs to kv head h_q / (H_q / H_k);
+ *   - zero norms: each norm is clamped below by 1e-12 (score becomes 0);
+ *   - ties in top-K: the lower group index wins.
+ *
+ * Pin status: every exported function is pinned by tests that do not call it
+ * to produce their own expectation (closed forms, invariants, brute force,
+ * library routines, values printed in the paper), except the byte layout of
+ * the packed codes (nibble order), which the paper does not fix:
+ * "parity unpinned" for the nibble order only.
+ */
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define ORC_OK 0
+#define ORC_ERR_ARG (-1)
+
+enum { ORC_BF16 = 0, ORC_FP16 = 1, ORC_FP32 = 2 };
+enum { ORC_PER_LAYER = 0, ORC_PER_HEAD = 1 };
+
+/* Same field order as the CUDA library's config so one Python-side recipe
+ * can fill either; declared here independently on purpose. */
+typedef struct {
+    int32_t n_layers;        /* L   */
+    int32_t n_q_heads;       /* H_q */
+    int32_t n_kv_heads;      /* H_k */
+    int32_t head_dim;        /* d   */
+    int32_t group_tokens;    /* G   */
+    int32_t capacity_groups; /* groups the store can hold per layer */
+    int32_t bits;            /* 4 or 2 */
+    int32_t kv_dtype;        /* ORC_BF16 | ORC_FP16 | ORC_FP32 */
+    int32_t score_mode;      /* ORC_PER_LAYER | ORC_PER_HEAD */
+} orc_config;
+
+/* Arrays of the memory bank, all indexed [layer][group][kv head]... */
+typedef struct {
+    uint8_t *codes_k;  /* [L][cap][H_k][G][d*bits/8] */
+    uint8_t *codes_v;  /* same                         */
+    float *scale_k;    /* [L][cap][H_k][d]             */
+    float *zero_k;     /* [L][cap][H_k][d]             */
+    float *scale_v;    /* [L][cap][H_k][d]             */
+    float *zero_v;     /* [L][cap][H_k][d]             */
+    float *rep_key;    /* [L][cap][H_k][d]  k-bar      */
+    float *rep_norm2;  /* [L][cap][H_k]     |k-bar_h|^2 */
+} orc_store;
+
+/* ------------------------------------------------------------------ */
+/* number formats                                                      */
+/* ------------------------------------------------------------------ */
+
+static float bits_to_f32(uint32_t u) { float f; memcpy(&f, &u, 4); return f; }
+static uint32_t f32_to_bits(float f) { uint32_t u; memcpy(&u, &f, 4); return u; }
+
+/* bfloat16 is the upper half of a binary32 */
+float orc_bf16_to_f32(uint16_t h) { return bits_to_f32((uint32_t)h << 16); }
+
+/* binary32 -> bfloat16, round to nearest, ties to even */
+uint16_t orc_f32_to_bf16(float f) {
+    uint32_t u = f32_to_bits(f);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x0040u); /* NaN */
+    uint32_t lower = u & 0xffffu;
+    uint32_t upper = u >> 16;
+    if (lower > 0x8000u || (lower == 0x8000u && (upper & 1u))) upper += 1u;
+    return (uint16_t)upper;
+}
+
+/* IEEE binary16 -> binary32 (exact) */
+float orc_f16_to_f32(uint16_t h) {
+    uint32_t sign = (uint32_t)(h >> 15) << 31;
+    int32_t e = (h >> 10) & 0x1f;
+    uint32_t frac = h & 0x3ffu;
+    if (e == 0x1f) return bits_to_f32(sign | 0x7f800000u | (frac << 13));
+    if (e == 0) {
+        /* subnormal: frac * 2^-24 */
+        float v = (float)frac * 5.9604644775390625e-08f;
+        return sign ? -v : v;
+    }
+    return bits_to_f32(sign | ((uint32_t)(e - 15 + 127) << 23) | (frac << 13));
+}
+
+/* binary32 -> IEEE binary16, round to nearest, ties to even */
+uint16_t orc_f32_to_f16(float f) {
+    uint32_t u = f32_to_bits(f);
+    uint16_t sign = (uint16_t)((u >> 16) & 0x8000u);
+    uint32_t a = u & 0x7fffffffu;
+    if (a > 0x7f800000u) return (uint16_t)(sign | 0x7e00u);  /* NaN */
+    if (a >= 0x477ff000u) return (uint16_t)(sign | 0x7c00u); /* >= 65520 rounds to inf */
+    double mag = fabs((double)f);
+    if (mag < 6.103515625e-05) {
+        /* subnormal target: multiples of 2^-24 */
+        double q = mag * 16777216.0;
+        double r = nearbyint(q); /* ties to even in the default mode */
+        return (uint16_t)(sign | (uint16_t)r); /* r == 1024 gives the smallest normal */
+    }
+    int e;
+    double fr = frexp(mag, &e); /* mag = fr * 2^e, fr in [0.5,1) */
+    double sig = fr * 2048.0;   /* in [1024, 2048) */
+    double r = nearbyint(sig);
+    int ee = e - 1;             /* unbiased exponent of the leading bit */
+    if (r == 2048.0) { r = 1024.0; ee += 1; }
+    return (uint16_t)(sign | (uint16_t)((ee + 15) << 10) | ((uint16_t)r - 1024u));
+}
+
+static float load_elem(const void *p, int64_t i, int dtype) {
+    switch (dtype) {
+    case ORC_BF16: return orc_bf16_to_f32(((const uint16_t *)p)[i]);
+    case ORC_FP16: return orc_f16_to_f32(((const uint16_t *)p)[i]);
+    default: return ((const float *)p)[i];
+    }
+}
+
+void orc_convert_to_f32(const void *src, int dtype, int64_t n, float *dst) {
+    for (int64_t i = 0; i < n; ++i) dst[i] = load_elem(src, i, dtype);
+}
+
+void orc_convert_from_f32(const float *src, int dtype, int64_t n, void *dst) {
+    for (int64_t i = 0; i < n; ++i) {
+        if (dtype == ORC_BF16) ((uint16_t *)dst)[i] = orc_f32_to_bf16(src[i]);
+        else if (dtype == ORC_FP16) ((uint16_t *)dst)[i] = orc_f32_to_f16(src[i]);
+        else ((float *)dst)[i] = src[i];
+    }
+}
+
+/* ------------------------------------------------------------------ */
+/* O1  group quantizer (Sec. 3.4, Q_4 and the (s_t, m_t) equation)     */
+/* ------------------------------------------------------------------ */
+
+static int levels_of(int bits) { return (1 << bits) - 1; } /* 15 for 4-bit, 3 for 2-bit */
+
+/*
+ * X is one group tensor [H][G][d] in binary32.  Statistics are taken per
+ * head and per channel across the G tokens.  codes is [H][G][d] with one
+ * code per byte (not yet packed); s and m are [H][d].
+ */
+void orc_quantize_group(const float *X, int H, int G, int d, int bits,
+                        uint8_t *codes, float *s, float *m) {
+    const float nlev = (float)levels_of(bits);
+    for (int h = 0; h < H; ++h) {
+        for (int c = 0; c < d; ++c) {
+            float mn = X[((int64_t)h * G + 0) * d + c];
+            float mx = mn;
+            for (int g = 1; g < G; ++g) {
+                float x = X[((int64_t)h * G + g) * d + c];
+                if (x < mn) mn = x;
+                if (x > mx) mx = x;
+            }
+            float range = mx - mn;
+            float sc = range / nlev;
+            s[h * d + c] = sc;
+            m[h * d + c] = mn;
+            for (int g = 0; g < G; ++g) {
+                float x = X[((int64_t)h * G + g) * d + c];
+                int code = 0;
+                if (sc != 0.0f) {
+                    float diff = x - mn;
+                    float t = diff / sc;
+                    float r = nearbyintf(t); /* default mode: ties to even */
+                    if (r < 0.0f) r = 0.0f;
+                    if (r > nlev) r = nlev;
+                    code = (int)r;
+                }
+                codes[((int64_t)h * G + g) * d + c] = (uint8_t)code;
+            }
+        }
+    }
+}
+
+/* Pack one row of d codes: bits=4 -> 2 per byte, bits=2 -> 4 per byte; the
+ * lowest channel sits in the lowest bits. */
+void orc_pack_row(const uint8_t *codes, int d, int bits, uint8_t *out) {
+    int per = 8 / bits;
+    for (int j = 0; j < d / per; ++j) {
+        unsigned b = 0;
+        for (int i = 0; i < per; ++i) b |= (unsigned)codes[j * per + i] << (bits * i);
+        out[j] = (uint8_t)b;
+    }
+}
+
+void orc_unpack_row(const uint8_t *packed, int d, int bits, uint8_t *codes) {
+    int per = 8 / bits;
+    unsigned mask = (1u << bits) - 1u;
+    for (int j = 0; j < d / per; ++j)
+        for (int i = 0; i < per; ++i) codes[j * per + i] = (uint8_t)((packed[j] >> (bits * i)) & mask);
+}
+
+/* Sec. 3.4, Q_4^{-1}: depack(X) * s + m, evaluated as one fused multiply-add */
+float orc_dequant_value(int code, float s, float m) { return fmaf((float)code, s, m); }
+
+/* ------------------------------------------------------------------ */
+/* O2  representative key (Sec. 3.4; appendix "Layer-wise vision        */
+/*     memory": k_t = (1/G) sum_{i in G_t} K_i)                         */
+/* ------------------------------------------------------------------ */
+
+void orc_rep_key(const float *K, int H, int G, int d, float *rep, float *norm2) {
+    for (int h = 0; h < H; ++h) {
+        double n2 = 0.0;
+        for (int c = 0; c < d; ++c) {
+            double acc = 0.0;
+            for (int g = 0; g < G; ++g) acc += (double)K[((int64_t)h * G + g) * d + c];
+            float kb = (float)(acc / (double)G);
+            rep[h * d + c] = kb;
+            n2 += (double)kb * (double)kb;
+        }
+        norm2[h] = (float)n2;
+    }
+}
+
+/* ------------------------------------------------------------------ */
+/* store addressing                                                     */
+/* ------------------------------------------------------------------ */
+
+static int64_t code_row_bytes(const orc_config *c) { return (int64_t)c->head_dim * c->bits / 8; }
+static int64_t codes_off(const orc_config *c, int l, int t, int h) {
+    return ((((int64_t)l * c->capacity_groups + t) * c->n_kv_heads + h) * c->group_tokens) * code_row_bytes(c);
+}
+static int64_t meta_off(const orc_config *c, int l, int t, int h) {
+    return (((int64_t)l * c->capacity_groups + t) * c->n_kv_heads + h) * c->head_dim;
+}
+static int64_t norm_off(const orc_config *c, int l, int t, int h) {
+    return ((int64_t)l * c->capacity_groups + t) * c->n_kv_heads + h;
+}
+
+static int check_cfg(const orc_config *c) {
+    if (!c) return 0;
+    if (c->n_layers < 1 || c->n_kv_heads < 1 || c->n_q_heads < 1) return 0;
+    if (c->n_q_heads % c->n_kv_heads) return 0;
+    if (c->head_dim < 1 || c->group_tokens < 1 || c->capacity_groups < 1) return 0;
+    if (c->bits != 4 && c->bits != 2) return 0;
+    if ((c->head_dim * c->bits) % 8) return 0;
+    if (c->kv_dtype < 0 || c->kv_dtype > 2) return 0;
+    if (c->score_mode < 0 || c->score_mode > 1) return 0;
+    return 1;
+}
+
+/* ------------------------------------------------------------------ */
+/* A1  quantize the groups of newly arrived frames and append them      */
+/* ------------------------------------------------------------------ */
+
+/*
+ * K, V: element (l, f, h, tok, c) lives at
+ *   (l - layer_begin)*stride_layer + f*stride_group + h*stride_head
+ *   + tok*stride_token + c            (strides in elements)
+ * with tok = token_idx ? token_idx[f*G + g] : g  for g in [0, G).
+ * K_summary (nullable) has the same addressing and supplies the keys the
+ * representative key is averaged from (keys before rotary embedding).
+ * Writes store slots [group_begin, group_begin + group_count) of layers
+ * [layer_begin, layer_begin + layer_count); never reads older groups.
+ */
+int32_t orc_quantize_frame(const orc_config *cfg, const orc_store *st,
+                           int32_t layer_begin, int32_t layer_count,
+                           int32_t group_begin, int32_t group_count,
+                           const void *K, const void *V,
+                           int64_t stride_layer, int64_t stride_group,
+                           int64_t stride_head, int64_t stride_token,
+                           const void *K_summary, const int32_t *token_idx,
+                           int32_t tokens_per_frame_in, int32_t n_threads) {
+    if (!check_cfg(cfg) || !st || !K || !V) return ORC_ERR_ARG;
+    if (layer_begin < 0 || layer_count < 0 || layer_begin + layer_count > cfg->n_layers) return ORC_ERR_ARG;
+    if (group_begin < 0 || group_count < 0 || group_begin + group_count > cfg->capacity_groups) return ORC_ERR_ARG;
+    const int H = cfg->n_kv_heads, G = cfg->group_tokens, d = cfg->head_dim;
+    if (token_idx) { /* tokens_per_frame_in only bounds token_idx */
+        for (int64_t i = 0; i < (int64_t)group_count * G; ++i)
+            if (token_idx[i] < 0 || token_idx[i] >= tokens_per_frame_in) return ORC_ERR_ARG;
+    }
+    const int64_t units = (int64_t)layer_count * group_count;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#endif
+    int failed = 0;
+#pragma omp parallel for schedule(static)
+    for (int64_t u = 0; u < units; ++u) {
+        const int li = (int)(u / group_count), f = (int)(u % group_count);
+        const int l = layer_begin + li, t = group_begin + f;
+        float *X = (float *)malloc(sizeof(float) * (size_t)H * G * d);
+        float *Ks = (float *)malloc(sizeof(float) * (size_t)H * G * d);
+        uint8_t *codes = (uint8_t *)malloc((size_t)H * G * d);
+        if (!X || !Ks || !codes) { failed = 1; free(X); free(Ks); free(codes); continue; }
+        for (int which = 0; which < 2; ++which) { /* 0: keys, 1: values */
+            const void *src = which ? V : K;
+            for (int h = 0; h < H; ++h)
+                for (int g = 0; g < G; ++g) {
+                    int tok = token_idx ? token_idx[(int64_t)f * G + g] : g;
+                    int64_t base = (int64_t)li * stride_layer + (int64_t)f * stride_group +
+                                   (int64_t)h * stride_head + (int64_t)tok * stride_token;
+                    for (int c = 0; c < d; ++c) {
+                        X[((int64_t)h * G + g) * d + c] = load_elem(src, base + c, cfg->kv_dtype);
+                        if (!which)
+                            Ks[((int64_t)h * G + g) * d + c] =
+                                load_elem(K_summary ? K_summary : K, base + c, cfg->kv_dtype);
+                    }
+                }
+            float *s = (which ? st->scale_v : st->scale_k) + meta_off(cfg, l, t, 0);
+            float *m = (which ? st->zero_v : st->zero_k) + meta_off(cfg, l, t, 0);
+            orc_quantize_group(X, H, G, d, cfg->bits, codes, s, m);
+            uint8_t *dst = (which ? st->codes_v : st->codes_k) + codes_off(cfg, l, t, 0);
+            for (int64_t r = 0; r < (int64_t)H * G; ++r)
+                orc_pack_row(codes + r * d, d, cfg->bits, dst + r * code_row_bytes(cfg));
+            if (!which)
+                orc_rep_key(Ks, H, G, d, st->rep_key + meta_off(cfg, l, t, 0),
+                            st->rep_norm2 + norm_off(cfg, l, t, 0));
+        }
+        free(X); free(Ks); free(codes);
+    }
+    return failed ? ORC_ERR_ARG : ORC_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* A2  question embedding and cosine scores (appendix "Question-guided  */
+/*     single-pass retrieval")                                          */
+/* ------------------------------------------------------------------ */
+
+/*
+ * Q element (l, h_q, j, c) at (l-layer_begin)*q_stride_layer + h_q*q_stride_head
+ * + j*q_stride_token + c.  qemb is [H_k][d] binary64: the mean over the query
+ * heads of each GQA block and over the T_q tokens.
+ */
+void orc_query_embedding(const orc_config *cfg, const void *Q, int q_dtype, int64_t layer_off,
+                         int32_t T_q, int64_t q_stride_head, int64_t q_stride_token, double *qemb) {
+    const int H = cfg->n_kv_heads, d = cfg->head_dim, rep = cfg->n_q_heads / cfg->n_kv_heads;
+    for (int h = 0; h < H; ++h)
+        for (int c = 0; c < d; ++c) {
+            double head_acc = 0.0;
+            for (int r = 0; r < rep; ++r) {
+                int hq = h * rep + r;
+                double tok_acc = 0.0;
+                for (int j = 0; j < T_q; ++j)
+                    tok_acc += (double)load_elem(Q, layer_off + hq * q_stride_head + j * q_stride_token + c, q_dtype);
+                head_acc += tok_acc / (double)T_q;
+            }
+            qemb[h * d + c] = head_acc / (double)rep;
+        }
+}
+
+/*
+ * scores: PER_LAYER -> [layer_count][n_groups]; PER_HEAD -> [layer_count][H_k][n_groups].
+ * score = <q, k-bar_t> / (max(|q|, eps) * max(|k-bar_t|, eps)), eps = 1e-12.
+ */
+int32_t orc_score_groups(const orc_config *cfg, const orc_store *st,
+                         int32_t layer_begin, int32_t layer_count, int32_t n_groups,
+                         const void *Q, int32_t T_q, int64_t q_stride_layer,
+                         int64_t q_stride_head, int64_t q_stride_token,
+                         float *scores, int32_t n_threads) {
+    if (!check_cfg(cfg) || !st || !Q || !scores || T_q < 1) return ORC_ERR_ARG;
+    if (layer_begin < 0 || layer_count < 0 || layer_begin + layer_count > cfg->n_layers) return ORC_ERR_ARG;
+    if (n_groups < 0 || n_groups > cfg->capacity_groups) return ORC_ERR_ARG;
+    const int H = cfg->n_kv_heads, d = cfg->head_dim;
+    const double eps = 1e-12;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#endif
+    for (int li = 0; li < layer_count; ++li) {
+        const int l = layer_begin + li;
+        double *q = (double *)malloc(sizeof(double) * (size_t)H * d);
+        if (!q) return ORC_ERR_ARG;
+        orc_query_embedding(cfg, Q, cfg->kv_dtype, (int64_t)li * q_stride_layer, T_q, q_stride_head, q_stride_token, q);
+#pragma omp parallel for schedule(static)
+        for (int t = 0; t < n_groups; ++t) {
+            const float *kb = st->rep_key + meta_off(cfg, l, t, 0);
+            if (cfg->score_mode == ORC_PER_LAYER) {
+                double dot = 0.0, qn = 0.0, kn = 0.0;
+                for (int i = 0; i < H * d; ++i) {
+                    dot += q[i] * (double)kb[i];
+                    qn += q[i] * q[i];
+                    kn += (double)kb[i] * (double)kb[i];
+                }
+                double den = fmax(sqrt(qn), eps) * fmax(sqrt(kn), eps);
+                scores[(int64_t)li * n_groups + t] = (float)(dot / den);
+            } else {
+                for (int h = 0; h < H; ++h) {
+                    double dot = 0.0, qn = 0.0, kn = 0.0;
+                    for (int c = 0; c < d; ++c) {
+                        double qv = q[h * d + c], kv = (double)kb[h * d + c];
+                        dot += qv * kv; qn += qv * qv; kn += kv * kv;
+                    }
+                    double den = fmax(sqrt(qn), eps) * fmax(sqrt(kn), eps);
+                    scores[((int64_t)li * H + h) * n_groups + t] = (float)(dot / den);
+                }
+            }
+        }
+        free(q);
+    }
+    return ORC_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* A3  top-K (appendix: K = min(ceil(B/G), T/G); indices kept sorted)   */
+/* ------------------------------------------------------------------ */
+
+int32_t orc_budget_to_k(int64_t budget_tokens, int32_t G, int32_t stored_groups) {
+    int64_t k = (budget_tokens + G - 1) / G;
+    return (int32_t)(k < stored_groups ? k : stored_groups);
+}
+
+typedef struct { float score; int32_t idx; } orc_pair;
+
+static int cmp_score_desc_idx_asc(const void *a, const void *b) {
+    const orc_pair *x = (const orc_pair *)a, *y = (const orc_pair *)b;
+    if (x->score > y->score) return -1;
+    if (x->score < y->score) return 1;
+    return (x->idx > y->idx) - (x->idx < y->idx);
+}
+static int cmp_idx_asc(const void *a, const void *b) {
+    const orc_pair *x = (const orc_pair *)a, *y = (const orc_pair *)b;
+    return (x->idx > y->idx) - (x->idx < y->idx);
+}
+
+/*
+ * For each row: the min(k, n) largest scores (ties: lower index first), then
+ * those indices in ascending order.  Unused slots of idx_out are -1 (their
+ * score_out is 0).  n_sel_out[row] = min(k, n).
+ */
+int32_t orc_topk(const float *scores, int32_t rows, int32_t n, int64_t row_stride, int32_t k,
+                 int32_t *idx_out, float *score_out, int32_t *n_sel_out) {
+    if (!scores || !idx_out || rows < 0 || n < 0 || k < 1) return ORC_ERR_ARG;
+    const int ksel = k < n ? k : n;
+    for (int r = 0; r < rows; ++r) {
+        orc_pair *p = (orc_pair *)malloc(sizeof(orc_pair) * (size_t)(n > 0 ? n : 1));
+        if (!p) return ORC_ERR_ARG;
+        for (int i = 0; i < n; ++i) { p[i].score = scores[(int64_t)r * row_stride + i]; p[i].idx = i; }
+        qsort(p, (size_t)n, sizeof(orc_pair), cmp_score_desc_idx_asc);
+        qsort(p, (size_t)ksel, sizeof(orc_pair), cmp_idx_asc);
+        for (int j = 0; j < k; ++j) {
+            idx_out[(int64_t)r * k + j] = j < ksel ? p[j].idx : -1;
+            if (score_out) score_out[(int64_t)r * k + j] = j < ksel ? p[j].score : 0.0f;
+        }
+        if (n_sel_out) n_sel_out[r] = ksel;
+        free(p);
+    }
+    return ORC_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* A4  dequantize the selected groups into the active cache             */
+/*     (Sec. 3.4 KV_active; appendix "Cache reconstruction")            */
+/* ------------------------------------------------------------------ */
+
+static void store_out(void *p, int64_t i, int dtype, float v) {
+    if (dtype == ORC_BF16) ((uint16_t *)p)[i] = orc_f32_to_bf16(v);
+    else if (dtype == ORC_FP16) ((uint16_t *)p)[i] = orc_f32_to_f16(v);
+    else ((float *)p)[i] = v;
+}
+
+/*
+ * idx: PER_LAYER -> [layer_count][k]; PER_HEAD -> [layer_count][H_k][k].
+ * Slot j of a row lands at tokens token_offset + j*G .. + G-1 of the active
+ * cache; element (l, h, tok, c) of k_active / v_active is at
+ * (l-layer_begin)*stride_layer + h*stride_head + tok*stride_token + c.
+ * Entries equal to -1 are skipped (their slot is left untouched).
+ */
+int32_t orc_dequant_gather(const orc_config *cfg, const orc_store *st,
+                           int32_t layer_begin, int32_t layer_count,
+                           const int32_t *idx, int32_t k, int32_t n_groups,
+                           void *k_active, void *v_active, int32_t out_dtype,
+                           int64_t stride_layer, int64_t stride_head, int64_t stride_token,
+                           int32_t token_offset, int32_t n_threads) {
+    if (!check_cfg(cfg) || !st || !idx || !k_active || !v_active || k < 1) return ORC_ERR_ARG;
+    if (layer_begin < 0 || layer_count < 0 || layer_begin + layer_count > cfg->n_layers) return ORC_ERR_ARG;
+    const int H = cfg->n_kv_heads, G = cfg->group_tokens, d = cfg->head_dim;
+    const int per_head = cfg->score_mode == ORC_PER_HEAD;
+    const int64_t nidx = (int64_t)layer_count * (per_head ? H : 1) * k;
+    for (int64_t i = 0; i < nidx; ++i)
+        if (idx[i] < -1 || idx[i] >= n_groups) return ORC_ERR_ARG;
+#ifdef _OPENMP
+    if (n_threads > 0) omp_set_num_threads(n_threads);
+#endif
+    const int64_t units = (int64_t)layer_count * k;
+#pragma omp parallel for schedule(static)
+    for (int64_t u = 0; u < units; ++u) {
+        const int li = (int)(u / k), j = (int)(u % k), l = layer_begin + li;
+        uint8_t *row = (uint8_t *)malloc((size_t)d);
+        for (int h = 0; h < H; ++h) {
+            const int t = per_head ? idx[((int64_t)li * H + h) * k + j] : idx[(int64_t)li * k + j];
+            if (t < 0) continue;
+            for (int which = 0; which < 2; ++which) {
+                const uint8_t *codes = (which ? st->codes_v : st->codes_k) + codes_off(cfg, l, t, h);
+                const float *s = (which ? st->scale_v : st->scale_k) + meta_off(cfg, l, t, h);
+                const float *m = (which ? st->zero_v : st->zero_k) + meta_off(cfg, l, t, h);
+                void *out = which ? v_active : k_active;
+                for (int g = 0; g < G; ++g) {
+                    orc_unpack_row(codes + (int64_t)g * code_row_bytes(cfg), d, cfg->bits, row);
+                    int64_t base = (int64_t)li * stride_layer + (int64_t)h * stride_head +
+                                   ((int64_t)token_offset + (int64_t)j * G + g) * stride_token;
+                    for (int c = 0; c < d; ++c)
+                        store_out(out, base + c, out_dtype, orc_dequant_value(row[c], s[c], m[c]));
+                }
+            }
+        }
+        free(row);
+    }
+    return ORC_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* A5  decode attention over [system tokens || selected groups]         */
+/*     (Sec. 3.4: decoding attends to the bounded active kv)            */
+/* ------------------------------------------------------------------ */
+
+/*
+ * One layer.  q_dec [H_q][d] (dtype q_dtype).  Keys/values are the active
+ * cache as orc_dequant_gather leaves it: element (h, tok, c) at
+ * h*stride_head + tok*stride_token + c, n_tokens tokens, dtype kv_dtype
+ * (values already rounded to that type, as the materialised cache holds
+ * them).  out [H_q][d] rounded to out_dtype.  Plain softmax(q k^T * scale) v
+ * in binary64.
+ */
+int32_t orc_attend(int32_t H_q, int32_t H_k, int32_t d, const void *q_dec, int32_t q_dtype,
+                   const void *k_cache, const void *v_cache, int32_t kv_dtype,
+                   int64_t stride_head, int64_t stride_token, int32_t n_tokens,
+                   double softmax_scale, void *out, int32_t out_dtype) {
+    if (H_q < 1 || H_k < 1 || H_q % H_k || d < 1 || n_tokens < 1) return ORC_ERR_ARG;
+    const int rep = H_q / H_k;
+    double *p = (double *)malloc(sizeof(double) * (size_t)n_tokens);
+    double *acc = (double *)malloc(sizeof(double) * (size_t)d);
+    if (!p || !acc) { free(p); free(acc); return ORC_ERR_ARG; }
+    for (int hq = 0; hq < H_q; ++hq) {
+        const int h = hq / rep;
+        double mx = -INFINITY;
+        for (int t = 0; t < n_tokens; ++t) {
+            double dot = 0.0;
+            for (int c = 0; c < d; ++c)
+                dot += (double)load_elem(q_dec, (int64_t)hq * d + c, q_dtype) *
+                       (double)load_elem(k_cache, h * stride_head + t * stride_token + c, kv_dtype);
+            p[t] = dot * softmax_scale;
+            if (p[t] > mx) mx = p[t];
+        }
+        double den = 0.0;
+        for (int t = 0; t < n_tokens; ++t) { p[t] = exp(p[t] - mx); den += p[t]; }
+        for (int c = 0; c < d; ++c) acc[c] = 0.0;
+        for (int t = 0; t < n_tokens; ++t)
+            for (int c = 0; c < d; ++c)
+                acc[c] += p[t] * (double)load_elem(v_cache, h * stride_head + t * stride_token + c, kv_dtype);
+        for (int c = 0; c < d; ++c) store_out(out, (int64_t)hq * d + c, out_dtype, (float)(acc[c] / den));
+    }
+    free(p); free(acc);
+    return ORC_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* O8  storage accounting                                               */
+/* ------------------------------------------------------------------ */
+
+/* Sec. 3.2 / Sec. 3.4: (N*d*16 bits) / (G*d*bits) = 16N / (bits*G); 4N/G at 4 bits */
+double orc_paper_ratio(int32_t N, int32_t G, int32_t bits) { return (16.0 * N) / ((double)bits * G); }
+
+/* ablation table "Ratio (%)": stored bits relative to N tokens at 16 bit */
+double orc_ratio_percent(int32_t N, int32_t G, int32_t bits) { return 100.0 * ((double)G * bits) / (16.0 * N); }
+
+/* Sec. 3.1 growth equation integrated: 2 (K and V) * L * frames * N * H_kv * d_h * sizeof */
+double orc_fp16_kv_bytes(int32_t L, int64_t frames, int32_t N, int32_t H_kv, int32_t d_h, int32_t elem_bytes) {
+    return 2.0 * L * (double)frames * N * H_kv * d_h * elem_bytes;
+}
+
+/* bytes this store really holds for `groups` groups per layer, metadata included */
+double orc_store_bytes(const orc_config *c, int64_t groups, int32_t with_metadata) {
+    double per_head_codes = 2.0 * c->group_tokens * (double)code_row_bytes(c); /* K and V */
+    double per_head_meta = 4.0 * c->head_dim * 4.0 /* sK mK sV mV */ + c->head_dim * 4.0 /* k-bar */ + 4.0;
+    double per = per_head_codes + (with_metadata ? per_head_meta : 0.0);
+    return per * c->n_kv_heads * (double)groups * c->n_layers;
+}
+
+int32_t orc_max_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
