@@ -1,0 +1,135 @@
+// Internal helpers shared by the translation units of libstom_oqm.so.
+// Host side: argument validation, bank addressing, CUDA error bookkeeping.
+// Device side: vector loads and number-format helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "stom_oqm.h"
+
+namespace stom {
+
+// ---------------------------------------------------------------- host
+
+void set_last_cuda_error(cudaError_t e);
+
+// Validates the geometry; returns STOM_OK or an error code.
+int32_t check_config(const stom_oqm_config *cfg);
+int32_t check_store(const stom_oqm_store *st);
+int32_t check_layers(const stom_oqm_config *cfg, int32_t layer_begin, int32_t layer_count);
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+inline int elem_bytes(int dtype) { return dtype == STOM_FP32 ? 4 : 2; }
+inline bool stride_ok(int64_t stride_elems, int dtype) { return (stride_elems * elem_bytes(dtype)) % 16 == 0; }
+
+inline int32_t finish_launch() {
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) {
+        set_last_cuda_error(e);
+        return STOM_ERR_CUDA;
+    }
+    return STOM_OK;
+}
+
+// Bank geometry passed by value to kernels.
+struct BankGeom {
+    int32_t H;        // kv heads
+    int32_t G;        // tokens per group
+    int32_t d;        // head dim
+    int32_t cap;      // groups per layer
+    int32_t row_bytes;  // packed bytes per token row = d/2
+};
+
+inline BankGeom bank_geom(const stom_oqm_config *c) {
+    return BankGeom{c->n_kv_heads, c->group_tokens, c->head_dim, c->capacity_groups, c->head_dim * c->bits / 8};
+}
+
+// ---------------------------------------------------------------- device
+
+#ifdef __CUDACC__
+
+// Index of (layer, group, head) in the [L][cap][H] lattice every bank array shares.
+__device__ __forceinline__ int64_t bank_slot(const BankGeom &g, int l, int t, int h) {
+    return ((int64_t)l * g.cap + t) * g.H + h;
+}
+
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// Two packed 16-bit elements -> two floats (exact).
+template <typename T>
+__device__ __forceinline__ void unpack2(uint32_t w, float &a, float &b);
+template <>
+__device__ __forceinline__ void unpack2<__nv_bfloat16>(uint32_t w, float &a, float &b) {
+    a = bf16lo(w);
+    b = bf16hi(w);
+}
+template <>
+__device__ __forceinline__ void unpack2<__half>(uint32_t w, float &a, float &b) {
+    __half2 h = *reinterpret_cast<__half2 *>(&w);
+    float2 f = __half22float2(h);
+    a = f.x;
+    b = f.y;
+}
+
+// Two floats -> two packed 16-bit elements, round to nearest even.
+template <typename T>
+__device__ __forceinline__ uint32_t pack2(float a, float b);
+template <>
+__device__ __forceinline__ uint32_t pack2<__nv_bfloat16>(float a, float b) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+template <>
+__device__ __forceinline__ uint32_t pack2<__half>(float a, float b) {
+    __half2 v = __floats2half2_rn(a, b);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// W consecutive 32-bit words from global memory through the read-only path.
+template <int W>
+struct Words {
+    uint32_t w[W];
+};
+
+template <int W>
+__device__ __forceinline__ Words<W> load_words(const void *p) {
+    Words<W> r;
+    if constexpr (W == 1) {
+        r.w[0] = __ldg(reinterpret_cast<const uint32_t *>(p));
+    } else if constexpr (W == 2) {
+        uint2 v = __ldg(reinterpret_cast<const uint2 *>(p));
+        r.w[0] = v.x;
+        r.w[1] = v.y;
+    } else {
+        static_assert(W % 4 == 0, "word count");
+#pragma unroll
+        for (int i = 0; i < W / 4; ++i) {
+            uint4 v = __ldg(reinterpret_cast<const uint4 *>(p) + i);
+            r.w[4 * i + 0] = v.x;
+            r.w[4 * i + 1] = v.y;
+            r.w[4 * i + 2] = v.z;
+            r.w[4 * i + 3] = v.w;
+        }
+    }
+    return r;
+}
+
+// Element j of a register-resident row fragment as float.
+template <typename T, int W>
+__device__ __forceinline__ float elem_of(const Words<W> &r, int j) {
+    if constexpr (sizeof(T) == 4) {
+        return __uint_as_float(r.w[j]);
+    } else {
+        float a, b;
+        unpack2<T>(r.w[j >> 1], a, b);
+        return (j & 1) ? b : a;
+    }
+}
+
+#endif  // __CUDACC__
+
+}  // namespace stom

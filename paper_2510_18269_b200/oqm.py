@@ -1,0 +1,199 @@
+"""Thin Python binding of libstom_oqm.so (argument marshalling only).
+
+Every step of the path runs in the library's CUDA kernels; PyTorch is used for
+device memory and streams.  There is no CPU fallback: if the library is not
+built, importing `lib()` raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+from pathlib import Path
+
+import torch
+
+_PKG = Path(__file__).resolve().parent
+LIB_PATH = _PKG / "libstom_oqm.so"
+
+BF16, FP16, FP32 = 0, 1, 2
+PER_LAYER, PER_HEAD = 0, 1
+FLAG_BAD_INDEX = 1
+
+_TORCH_DTYPE = {BF16: torch.bfloat16, FP16: torch.float16, FP32: torch.float32}
+_DTYPE_CODE = {v: k for k, v in _TORCH_DTYPE.items()}
+
+EXPORTS = (
+    "stom_oqm_store_layout", "stom_oqm_store_bind", "stom_oqm_budget_to_k", "stom_oqm_score_workspace_bytes",
+    "stom_status_string", "stom_last_cuda_error", "stom_oqm_quantize_frame", "stom_oqm_score_groups",
+    "stom_oqm_topk", "stom_oqm_dequant_gather", "stom_oqm_retrieve",
+)
+
+
+class Config(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in (
+        "n_layers", "n_q_heads", "n_kv_heads", "head_dim", "group_tokens",
+        "capacity_groups", "bits", "kv_dtype", "score_mode")]
+
+
+class StoreDesc(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in (
+        "codes_k", "codes_v", "scale_k", "zero_k", "scale_v", "zero_v", "rep_key", "rep_norm2")]
+
+
+class Layout(C.Structure):
+    _fields_ = [(n, C.c_int64) for n in (
+        "bytes_total", "off_codes_k", "off_codes_v", "off_scale_k", "off_zero_k", "off_scale_v", "off_zero_v",
+        "off_rep_key", "off_rep_norm2", "bytes_codes", "bytes_meta", "bytes_norm2")]
+
+
+class StomError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().stom_status_string(code).decode()
+        super().__init__(f"{where}: {msg} (status {code}, cuda error {lib().stom_last_cuda_error()})")
+
+
+_lib = None
+
+
+def lib():
+    """The loaded C-ABI library.  Fails loudly when it has not been built."""
+    global _lib
+    if _lib is None:
+        if not LIB_PATH.exists():
+            raise ImportError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2510_18269_b200.build` "
+                "(there is no fallback path)")
+        L = C.CDLL(str(LIB_PATH))
+        L.stom_status_string.restype = C.c_char_p
+        L.stom_status_string.argtypes = [C.c_int32]
+        L.stom_oqm_score_workspace_bytes.restype = C.c_int64
+        L.stom_oqm_score_workspace_bytes.argtypes = [C.POINTER(Config), C.c_int32]
+        L.stom_oqm_budget_to_k.argtypes = [C.c_int64, C.c_int32, C.c_int32]
+        for name in EXPORTS:
+            fn = getattr(L, name)
+            if fn.restype is C.c_int:
+                fn.restype = C.c_int32
+        _lib = L
+    return _lib
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _check(rc: int, where: str):
+    if rc != 0:
+        raise StomError(rc, where)
+
+
+def make_config(n_layers, n_q_heads, n_kv_heads, head_dim, group_tokens, capacity_groups,
+                bits=4, kv_dtype=BF16, score_mode=PER_LAYER) -> Config:
+    return Config(n_layers, n_q_heads, n_kv_heads, head_dim, group_tokens, capacity_groups,
+                  bits, kv_dtype, score_mode)
+
+
+def dtype_code(t: torch.dtype) -> int:
+    return _DTYPE_CODE[t]
+
+
+def stom_oqm_store_layout(cfg: Config) -> Layout:
+    lay = Layout()
+    _check(lib().stom_oqm_store_layout(C.byref(cfg), C.byref(lay)), "stom_oqm_store_layout")
+    return lay
+
+
+def stom_oqm_budget_to_k(budget_tokens: int, group_tokens: int, stored_groups: int) -> int:
+    return int(lib().stom_oqm_budget_to_k(budget_tokens, group_tokens, stored_groups))
+
+
+def stom_oqm_score_workspace_bytes(cfg: Config, layer_count: int) -> int:
+    return int(lib().stom_oqm_score_workspace_bytes(C.byref(cfg), layer_count))
+
+
+class Store:
+    """One device arena holding the memory bank, plus typed tensor views of its arrays."""
+
+    def __init__(self, cfg: Config, device="cuda", zero: bool = True):
+        self.cfg = cfg
+        self.layout = stom_oqm_store_layout(cfg)
+        alloc = torch.zeros if zero else torch.empty
+        self.arena = alloc(self.layout.bytes_total + 256, dtype=torch.uint8, device=device)
+        shift = (-self.arena.data_ptr()) % 256
+        self.base = self.arena[shift:shift + self.layout.bytes_total]
+        self.desc = StoreDesc()
+        _check(lib().stom_oqm_store_bind(C.byref(cfg), C.c_void_p(self.base.data_ptr()), C.byref(self.desc)),
+               "stom_oqm_store_bind")
+        L, T, H, G, d = cfg.n_layers, cfg.capacity_groups, cfg.n_kv_heads, cfg.group_tokens, cfg.head_dim
+        lay = self.layout
+
+        def view(off, nbytes, dtype, shape):
+            return self.base[off:off + nbytes].view(dtype).view(*shape)
+
+        self.codes_k = view(lay.off_codes_k, lay.bytes_codes, torch.uint8, (L, T, H, G, d * cfg.bits // 8))
+        self.codes_v = view(lay.off_codes_v, lay.bytes_codes, torch.uint8, (L, T, H, G, d * cfg.bits // 8))
+        self.scale_k = view(lay.off_scale_k, lay.bytes_meta, torch.float32, (L, T, H, d))
+        self.zero_k = view(lay.off_zero_k, lay.bytes_meta, torch.float32, (L, T, H, d))
+        self.scale_v = view(lay.off_scale_v, lay.bytes_meta, torch.float32, (L, T, H, d))
+        self.zero_v = view(lay.off_zero_v, lay.bytes_meta, torch.float32, (L, T, H, d))
+        self.rep_key = view(lay.off_rep_key, lay.bytes_meta, torch.float32, (L, T, H, d))
+        self.rep_norm2 = view(lay.off_rep_norm2, lay.bytes_norm2, torch.float32, (L, T, H))
+
+
+def stom_oqm_quantize_frame(cfg: Config, store: Store, layer_begin, layer_count, group_begin, group_count,
+                            K, V, strides, K_summary=None, token_idx=None, tokens_per_frame_in=0,
+                            dev_flags=None, stream=None):
+    """strides = (layer, group, head, token) in elements of K / V."""
+    sl, sg, sh, st = strides
+    rc = lib().stom_oqm_quantize_frame(
+        C.byref(cfg), C.byref(store.desc), C.c_int32(layer_begin), C.c_int32(layer_count),
+        C.c_int32(group_begin), C.c_int32(group_count), _ptr(K), _ptr(V),
+        C.c_int64(sl), C.c_int64(sg), C.c_int64(sh), C.c_int64(st), _ptr(K_summary), _ptr(token_idx),
+        C.c_int32(tokens_per_frame_in), _ptr(dev_flags), _stream(stream))
+    _check(rc, "stom_oqm_quantize_frame")
+
+
+def stom_oqm_score_groups(cfg: Config, store: Store, layer_begin, layer_count, n_groups, Q, T_q, q_strides,
+                          scores, workspace, stream=None):
+    ql, qh, qt = q_strides
+    rc = lib().stom_oqm_score_groups(
+        C.byref(cfg), C.byref(store.desc), C.c_int32(layer_begin), C.c_int32(layer_count), C.c_int32(n_groups),
+        _ptr(Q), C.c_int32(T_q), C.c_int64(ql), C.c_int64(qh), C.c_int64(qt), _ptr(scores), _ptr(workspace),
+        C.c_int64(0 if workspace is None else workspace.numel() * workspace.element_size()), _stream(stream))
+    _check(rc, "stom_oqm_score_groups")
+
+
+def stom_oqm_topk(scores, rows, n, row_stride, k, idx_out, score_out=None, n_sel_out=None, stream=None):
+    rc = lib().stom_oqm_topk(_ptr(scores), C.c_int32(rows), C.c_int32(n), C.c_int64(row_stride), C.c_int32(k),
+                             _ptr(idx_out), _ptr(score_out), _ptr(n_sel_out), _stream(stream))
+    _check(rc, "stom_oqm_topk")
+
+
+def stom_oqm_dequant_gather(cfg: Config, store: Store, layer_begin, layer_count, idx, k, n_groups,
+                            k_active, v_active, out_dtype, strides, token_offset, dev_flags=None, stream=None):
+    """strides = (layer, head, token) in elements of the active cache."""
+    sl, sh, st = strides
+    rc = lib().stom_oqm_dequant_gather(
+        C.byref(cfg), C.byref(store.desc), C.c_int32(layer_begin), C.c_int32(layer_count), _ptr(idx),
+        C.c_int32(k), C.c_int32(n_groups), _ptr(k_active), _ptr(v_active), C.c_int32(out_dtype),
+        C.c_int64(sl), C.c_int64(sh), C.c_int64(st), C.c_int32(token_offset), _ptr(dev_flags), _stream(stream))
+    _check(rc, "stom_oqm_dequant_gather")
+
+
+def stom_oqm_retrieve(cfg: Config, store: Store, layer_begin, layer_count, n_groups, Q, T_q, q_strides, k,
+                      scores, idx, k_active, v_active, out_dtype, strides, token_offset, workspace,
+                      dev_flags=None, stream=None):
+    ql, qh, qt = q_strides
+    sl, sh, st = strides
+    rc = lib().stom_oqm_retrieve(
+        C.byref(cfg), C.byref(store.desc), C.c_int32(layer_begin), C.c_int32(layer_count), C.c_int32(n_groups),
+        _ptr(Q), C.c_int32(T_q), C.c_int64(ql), C.c_int64(qh), C.c_int64(qt), C.c_int32(k), _ptr(scores),
+        _ptr(idx), _ptr(k_active), _ptr(v_active), C.c_int32(out_dtype), C.c_int64(sl), C.c_int64(sh),
+        C.c_int64(st), C.c_int32(token_offset), _ptr(workspace),
+        C.c_int64(0 if workspace is None else workspace.numel() * workspace.element_size()), _ptr(dev_flags),
+        _stream(stream))
+    _check(rc, "stom_oqm_retrieve")

@@ -1,0 +1,121 @@
+"""Shared helpers of the GPU parity tests: run the same seeded inputs through the
+CPU oracle and through the C-ABI CUDA library, and compare element by element.
+
+Tolerances (stated here, used by every parity test):
+  * packed 4-bit codes ........ bit-exact
+  * scale s ................... bit-exact (two binary32 operations on both sides)
+  * offset m .................. equal as numbers (+0 and -0 compare equal)
+  * representative key ........ |d| <= 2^-24 * sum_g|x_g| + 2^-23 * |k-bar|   (binary32 summation of G terms
+                                against the oracle's binary64 mean), norms to 1e-5 relative
+  * scores .................... |d| <= 1e-5 absolute (scores lie in [-1, 1])
+  * selected indices .......... identical, except members whose oracle score is within 1e-5 relative of the
+                                oracle's K-th score (ties)
+  * dequantized values ........ |a - b| <= 1e-3 * max(|b|, s); in fact expected bit-identical (same fmaf, same
+                                rounding), and the mismatch count is asserted to be 0
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from paper_2510_18269_b200 import synth
+
+GUARD = 64  # sentinel elements kept after every output buffer
+
+
+def dt_code(dtype: str) -> int:
+    return {"bf16": 0, "fp16": 1, "fp32": 2}[dtype]
+
+
+def contiguous_strides(sh, tokens):
+    """Element strides (layer, group, head, token) of a [L][T][H_k][tokens][d] tensor."""
+    return (sh.T * sh.H_k * tokens * sh.d, sh.H_k * tokens * sh.d, tokens * sh.d, sh.d)
+
+
+def q_strides(sh):
+    return (sh.H_q * sh.T_q * sh.d, sh.T_q * sh.d, sh.d)
+
+
+def oracle_cfg(orc, sh, mode=0, cap=None):
+    return orc.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, cap or sh.T, 4, dt_code(sh.dtype), mode)
+
+
+def gpu_cfg(oqm, sh, mode=0, cap=None):
+    return oqm.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, cap or sh.T, 4, dt_code(sh.dtype), mode)
+
+
+def compare_store(gst, ost, K_f32, groups=None, layers=None):
+    """gst: oqm.Store (device); ost: oracle Store (host); K_f32: float32 numpy [L][T][H][G][d] of the keys the
+    representative key was averaged from (for its error bound)."""
+    L = gst.cfg.n_layers
+    layers = range(L) if layers is None else layers
+    gsel = slice(None) if groups is None else groups
+    for l in layers:
+        for name in ("codes_k", "codes_v"):
+            g = getattr(gst, name)[l, gsel].cpu().numpy()
+            o = getattr(ost, name)[l, gsel]
+            bad = int((g != o).sum())
+            assert bad == 0, f"{name} layer {l}: {bad} packed bytes differ"
+        for name in ("scale_k", "scale_v"):
+            g = getattr(gst, name)[l, gsel].cpu().numpy()
+            o = getattr(ost, name)[l, gsel]
+            assert np.array_equal(g.view(np.uint32), o.view(np.uint32)), f"{name} layer {l} not bit-exact"
+        for name in ("zero_k", "zero_v"):
+            g = getattr(gst, name)[l, gsel].cpu().numpy()
+            o = getattr(ost, name)[l, gsel]
+            assert np.array_equal(g, o), f"{name} layer {l} differs"
+        g = gst.rep_key[l, gsel].cpu().numpy().astype(np.float64)
+        o = ost.rep_key[l, gsel].astype(np.float64)
+        absum = np.abs(K_f32[l, gsel]).astype(np.float64).sum(axis=-2)         # [T][H][d]
+        tol = 2.0 ** -24 * absum + 2.0 ** -23 * np.abs(o) + 1e-30
+        assert np.all(np.abs(g - o) <= tol), f"rep_key layer {l}: max excess {(np.abs(g - o) - tol).max()}"
+        gn = gst.rep_norm2[l, gsel].cpu().numpy().astype(np.float64)
+        on = ost.rep_norm2[l, gsel].astype(np.float64)
+        assert np.all(np.abs(gn - on) <= 1e-5 * np.abs(on) + 1e-30), f"rep_norm2 layer {l}"
+
+
+def compare_scores(g_scores: torch.Tensor, o_scores: np.ndarray):
+    g = g_scores.cpu().numpy().reshape(o_scores.shape)
+    err = np.abs(g.astype(np.float64) - o_scores.astype(np.float64))
+    assert err.max() <= 1e-5, f"scores differ by {err.max()}"
+
+
+def compare_topk(g_idx: torch.Tensor, o_idx: np.ndarray, o_scores_rows: np.ndarray, k: int):
+    """g_idx, o_idx: [rows][k]; o_scores_rows: [rows][n] oracle scores."""
+    g = g_idx.cpu().numpy().reshape(o_idx.shape)
+    n = o_scores_rows.shape[1]
+    ksel = min(k, n)
+    exact_rows = 0
+    for r in range(o_idx.shape[0]):
+        gr, orr = g[r], o_idx[r]
+        assert np.all(gr[ksel:] == -1), "unused slots must be -1"
+        sel = gr[:ksel]
+        assert np.all((sel >= 0) & (sel < n)) and np.all(np.diff(sel) > 0), "selection must be ascending and in range"
+        if np.array_equal(sel, orr[:ksel]):
+            exact_rows += 1
+            continue
+        kth = o_scores_rows[r, orr[:ksel]].min()
+        diff = np.setxor1d(sel, orr[:ksel])
+        sc = o_scores_rows[r, diff]
+        assert np.all(np.abs(sc - kth) <= 1e-5 * max(abs(kth), 1e-30)), \
+            f"row {r}: selections differ beyond score ties: {diff}, scores {sc}, kth {kth}"
+    return exact_rows
+
+
+def out_buffers(sh, layer_count, S_tokens, torch_dtype, device, sentinel):
+    """Active cache [layer_count][H_k][S_tokens][d] with a guard band after it, filled with a sentinel."""
+    n = layer_count * sh.H_k * S_tokens * sh.d
+    flat = torch.full((n + GUARD,), sentinel, dtype=torch_dtype, device=device)
+    return flat, flat[:n].view(layer_count, sh.H_k, S_tokens, sh.d)
+
+
+def active_strides(sh, S_tokens):
+    return (sh.H_k * S_tokens * sh.d, S_tokens * sh.d, sh.d)
+
+
+def as_np16(t: torch.Tensor) -> np.ndarray:
+    return synth.as_u16(t)
+
+
+def f32_of(orc, arr: np.ndarray, dtype: str) -> np.ndarray:
+    return arr if dtype == "fp32" else orc.to_f32(arr, dt_code(dtype))
