@@ -205,7 +205,8 @@ def test_exact_ties_constant_and_tiny_channels(orc, oqm):
     V[:, 2, :, :, 6] = torch.tensor([0.0, 1e-45] * 15 + [0.0])   # range underflows: s == 0
     V[:, 3, :, :, 7] *= 1e-30                                # scale below the fast-path window
     V[:, 4, :, :, 8] *= 1e30                                 # scale above the fast-path window
-    K[:, 5, :, :, 9] = torch.linspace(-1e38, 1e38, sh.G)     # huge but finite range
+    V[:, 5, :, :, 9] = torch.linspace(-1e38, 1e38, sh.G)     # huge but finite range (values only: the key mean
+                                                             # is accumulated in binary32 and would overflow)
     gst, ost, gcfg, ocfg = _quantize_both(orc, oqm, sh, K, V)
     P.compare_store(gst, ost, K.numpy())
     ties = (K[0, 0, 0, :, 0] % 2 == 1).sum()
