@@ -1,0 +1,429 @@
+#!/usr/bin/env python
+"""Benchmark of the OQM hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--config C3|C2|C5]
+
+One step = one pass of the whole path over one synthetic stream:
+    A1  quantize every frame's kv groups of every layer into the memory bank
+    A2  question embedding + cosine scores over all stored groups
+    A3  top-K groups per layer
+    A4  dequantize-and-gather the selected groups into the active bf16 cache
+Inputs are resident in HBM before the timed region; the input stream (20.6 GB
+at C3) is far larger than L2 and a 512 MB L2 flush separates A1 from A2-A4.
+
+Rank 0 prints ONE JSON line.  `value` is the retrieve+dequant (A2+A3+A4)
+throughput in algorithmic GB/s summed over ranks; the quantize throughput in
+tokens/s and the per-query latency ride along in `submetrics`.  `e2e` measures
+the same thing through the host-buffer C-ABI entry points with the
+host<->device copies inside the timed region.  `--impl reference` times the CPU
+oracle (a deliberately plain program) on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+FALLBACK_HBM_GBS = 6650.0
+
+# dram bytes per unit of work measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum) on a reduced
+# case of the same kernel and scaled by the units one launch processes; see profiles/*.md.  None = not captured.
+NCU_TRAFFIC_PER_UNIT = {
+    "quantize_kernel": None,        # bytes per (layer, frame)
+    "dequant_gather_kernel": None,  # bytes per (layer, selected group)
+    "score_kernel": None,           # bytes per (layer, stored group)
+}
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="C3")
+    ap.add_argument("--frames-per-call", type=int, default=0, help="0: the whole stream in one quantize call")
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--cpu-sample-frames", type=int, default=256)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--layers", type=int, default=0, help="override L (reduced case for profiler captures)")
+    ap.add_argument("--frames", type=int, default=0, help="override T (reduced case for profiler captures)")
+    return ap.parse_args()
+
+
+# ---------------------------------------------------------------- byte accounting (algorithmic bytes)
+
+def bytes_quantize(sh, frames):
+    e = 4 if sh.dtype == "fp32" else 2
+    per = 2 * sh.H_k * sh.G * sh.d * e + 2 * sh.H_k * sh.G * sh.d // 2 + 4 * sh.H_k * sh.d * 4 + sh.H_k * sh.d * 4 + sh.H_k * 4
+    return per * frames * sh.L
+
+
+def bytes_score(sh, groups):
+    return (sh.H_k * sh.d * 4 + sh.H_k * 4 + 4) * groups * sh.L + sh.L * sh.H_q * sh.T_q * sh.d * 2
+
+
+def bytes_topk(sh, groups):
+    return sh.L * (groups * 4 + sh.k * 4)
+
+
+def bytes_gather(sh, k):
+    per = 2 * sh.H_k * sh.G * sh.d // 2 + 4 * sh.H_k * sh.d * 4 + 2 * sh.H_k * sh.G * sh.d * 2
+    return per * k * sh.L
+
+
+def measured_peak():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+# ---------------------------------------------------------------- clocks
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int):
+        super().__init__(daemon=True)
+        self.index, self.samples, self.reasons, self.stop_flag, self.max_mhz = index, [], set(), False, None
+
+    def run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            names = {
+                nv.nvmlClocksThrottleReasonHwSlowdown: "hw_slowdown",
+                nv.nvmlClocksThrottleReasonHwThermalSlowdown: "hw_thermal_slowdown",
+                nv.nvmlClocksThrottleReasonSwThermalSlowdown: "sw_thermal_slowdown",
+                nv.nvmlClocksThrottleReasonSwPowerCap: "sw_power_cap",
+            }
+            while not self.stop_flag:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+                time.sleep(0.05)
+        except Exception as ex:  # pragma: no cover
+            self.reasons.add(f"nvml-unavailable:{type(ex).__name__}")
+
+    def result(self):
+        self.stop_flag = True
+        self.join(timeout=2)
+        med = statistics.median(self.samples) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons)}
+
+
+def nvml_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+# ---------------------------------------------------------------- CPU oracle leg
+
+def oracle_sample(sh, K_cpu, V_cpu, Q_cpu, frames, threads=0):
+    """Times the oracle on `frames` frames of every layer: quantize, score, top-K, gather.  Returns seconds per stage."""
+    from oracle import oqm_oracle as orc
+    from paper_2510_18269_b200 import synth
+    import numpy as np
+    k = min(sh.k, frames)
+    cfg = orc.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, frames, 4, {"bf16": 0, "fp16": 1, "fp32": 2}[sh.dtype])
+    st = orc.Store(cfg)
+    kn, vn, qn = synth.as_u16(K_cpu), synth.as_u16(V_cpu), synth.as_u16(Q_cpu)
+    strides = (frames * sh.H_k * sh.G * sh.d, sh.H_k * sh.G * sh.d, sh.G * sh.d, sh.d)
+    t0 = time.perf_counter()
+    assert orc.quantize_frame(cfg, st, 0, sh.L, 0, frames, kn, vn, strides, n_threads=threads) == 0
+    t1 = time.perf_counter()
+    sc = orc.score_groups(cfg, st, 0, sh.L, frames, qn, sh.T_q, (sh.H_q * sh.T_q * sh.d, sh.T_q * sh.d, sh.d),
+                          n_threads=threads)
+    idx, _, _ = orc.topk(sc, k)
+    S = k * sh.G
+    ka = np.zeros((sh.L, sh.H_k, S, sh.d), np.uint16)
+    va = np.zeros_like(ka)
+    assert orc.dequant_gather(cfg, st, 0, sh.L, idx, k, frames, ka, va, orc.BF16,
+                              (sh.H_k * S * sh.d, S * sh.d, sh.d), 0, n_threads=threads) == 0
+    t2 = time.perf_counter()
+    return {"quantize_s": t1 - t0, "retrieve_s": t2 - t1, "k": k, "threads": orc.max_threads() if threads == 0 else threads,
+            "cores": orc.host_cores()}
+
+
+def cpu_inputs(sh, frames):
+    """The first `frames` frames of every layer, generated on the CPU with the same recipe."""
+    import dataclasses
+    import torch
+    from paper_2510_18269_b200 import synth
+    small = dataclasses.replace(sh, T=frames)
+    planted = synth.planted_groups(small, min(sh.k // 2, frames))
+    K = torch.empty(sh.L, frames, sh.H_k, sh.G, sh.d, dtype=synth.DTYPES[sh.dtype])
+    V = torch.empty_like(K)
+    for l in range(sh.L):
+        K[l], V[l] = synth.kv_chunk(small, l, 0, frames, "cpu", planted)
+    return K, V, synth.queries(small)
+
+
+def run_reference(args, sh):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    frames = args.cpu_sample_frames
+    K, V, Q = cpu_inputs(sh, frames)
+    for _ in range(min(args.warmup, 1)):
+        oracle_sample(sh, K, V, Q, min(frames, 16))
+    rs, qs = [], []
+    info = None
+    for _ in range(args.steps):
+        info = oracle_sample(sh, K, V, Q, frames)
+        rs.append(info["retrieve_s"])
+        qs.append(info["quantize_s"])
+    k = info["k"]
+    rbytes = bytes_score(sh, frames) + bytes_topk(sh, frames) + bytes_gather(sh, k)
+    rt = statistics.mean(rs)
+    value = rbytes / rt / 1e9
+    sample = f"first {frames} frames of all {sh.L} layers (of {sh.T}); top-{k} groups gathered per layer"
+    out = {
+        "impl": "reference", "metric": "OQM retrieve+dequant throughput", "value": value, "unit": "GB/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": min(args.warmup, 1),
+        "ms_per_step": 1e3 * (statistics.mean(qs) + rt), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": sh.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": info["threads"], "kind": "oracle", "sample": sample,
+                         "quantize_tokens_per_s": frames * sh.G / statistics.mean(qs)},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(out))
+
+
+# ---------------------------------------------------------------- CUDA leg
+
+def run_ours(args, sh):
+    import torch
+    import torch.distributed as dist
+    from paper_2510_18269_b200 import oqm, synth, dist as sdist
+
+    rank, world, local = sdist.init_from_env(args.gpus)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    oqm.lib()
+    peak, peak_src = measured_peak()
+
+    # independent streams per rank (weak scaling: every GPU serves its own video stream)
+    import dataclasses
+    sh = dataclasses.replace(sh, seed=sh.seed + 17 * rank)
+    cfg = oqm.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, sh.T, 4, oqm.dtype_code(synth.DTYPES[sh.dtype]))
+    store = oqm.Store(cfg, device=dev, zero=False)
+    K, V = synth.kv_stream(sh, dev)
+    Q = synth.queries(sh, dev)
+    strides = (sh.T * sh.H_k * sh.G * sh.d, sh.H_k * sh.G * sh.d, sh.G * sh.d, sh.d)
+    qs = (sh.H_q * sh.T_q * sh.d, sh.T_q * sh.d, sh.d)
+    sys_len = 0
+    S = sys_len + sh.k * sh.G
+    act = (sh.H_k * S * sh.d, S * sh.d, sh.d)
+    scores = torch.empty(sh.L, sh.T, dtype=torch.float32, device=dev)
+    idx = torch.empty(sh.L, sh.k, dtype=torch.int32, device=dev)
+    ka = torch.empty(sh.L, sh.H_k, S, sh.d, dtype=torch.bfloat16, device=dev)
+    va = torch.empty_like(ka)
+    ws = torch.empty(oqm.stom_oqm_score_workspace_bytes(cfg, sh.L), dtype=torch.uint8, device=dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+    flags = torch.zeros(1, dtype=torch.int32, device=dev)
+    fpc = args.frames_per_call or sh.T
+    n_qcalls = (sh.T + fpc - 1) // fpc
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def step(timers=None):
+        e = [ev() for _ in range(6)] if timers is not None else None
+        if e: e[0].record()
+        for f0 in range(0, sh.T, fpc):
+            n = min(fpc, sh.T - f0)
+            oqm.stom_oqm_quantize_frame(cfg, store, 0, sh.L, f0, n, K.view(-1)[f0 * strides[1]:],
+                                        V.view(-1)[f0 * strides[1]:], strides, dev_flags=flags)
+        if e: e[1].record()
+        flush.fill_(1)                       # evict freshly written codes / keys from L2
+        if e: e[2].record()
+        oqm.stom_oqm_score_groups(cfg, store, 0, sh.L, sh.T, Q, sh.T_q, qs, scores, ws)
+        if e: e[3].record()
+        oqm.stom_oqm_topk(scores, sh.L, sh.T, sh.T, sh.k, idx)
+        if e: e[4].record()
+        oqm.stom_oqm_dequant_gather(cfg, store, 0, sh.L, idx, sh.k, sh.T, ka, va, oqm.BF16, act, sys_len,
+                                    dev_flags=flags)
+        if e: e[5].record()
+        if timers is not None:
+            timers.append(e)
+
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+    sdist.barrier()
+
+    sampler = ClockSampler(nvml_index(local))
+    sampler.start()
+    timers = []
+    t_start, t_end = ev(), ev()
+    torch.cuda.synchronize()
+    t_start.record()
+    for _ in range(args.steps):
+        step(timers)
+    t_end.record()
+    torch.cuda.synchronize()
+    clocks = sampler.result()
+    total_ms = t_start.elapsed_time(t_end)
+    total_ms = sdist.max_over_ranks(total_ms)
+
+    def mean_ms(a, b):
+        return statistics.mean(t[a].elapsed_time(t[b]) for t in timers)
+
+    q_ms, sc_ms, tk_ms, ga_ms = mean_ms(0, 1), mean_ms(2, 3), mean_ms(3, 4), mean_ms(4, 5)
+    r_ms = mean_ms(2, 5)
+    q_ms, sc_ms, tk_ms, ga_ms, r_ms = (sdist.max_over_ranks(x) for x in (q_ms, sc_ms, tk_ms, ga_ms, r_ms))
+    assert int(flags.item()) == 0, "a kernel flagged a bad index"
+
+    rbytes = bytes_score(sh, sh.T) + bytes_topk(sh, sh.T) + bytes_gather(sh, sh.k)
+    value = world * rbytes / (r_ms * 1e-3) / 1e9
+    qbytes = bytes_quantize(sh, sh.T)
+
+    def roof(name, nbytes, ms, launches, unit_count):
+        a = nbytes / launches / (ms / launches * 1e-3) / 1e9
+        tpu = NCU_TRAFFIC_PER_UNIT.get(name)
+        return {"kernel": name, "bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s", "frac": a / peak,
+                "traffic": None if tpu is None else tpu * unit_count / launches, "peak_source": peak_src,
+                "algorithmic_bytes_per_launch": nbytes / launches, "ms_per_launch": ms / launches}
+
+    roofs = [
+        roof("quantize_kernel", qbytes, q_ms, n_qcalls, sh.L * sh.T),
+        roof("dequant_gather_kernel", bytes_gather(sh, sh.k), ga_ms, 1, sh.L * sh.k),
+        roof("score_kernel", bytes_score(sh, sh.T), sc_ms, 1, sh.L * sh.T),
+    ]
+    out = {
+        "metric": "OQM retrieve+dequant throughput", "value": value, "unit": "GB/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": sh.name, "L": sh.L, "H_q": sh.H_q, "H_k": sh.H_k, "d": sh.d, "G": sh.G, "T": sh.T,
+                   "T_q": sh.T_q, "k": sh.k, "kv_dtype": sh.dtype, "frames_per_quantize_call": fpc,
+                   "l2": "inputs 20.6 GB >> L2; 512 MB flush between quantize and retrieve",
+                   "multi_gpu": "independent stream per rank, no collective"},
+        "submetrics": {
+            "retrieve_dequant_GBps": value, "retrieve_dequant_frac_of_measured_hbm": value / world / peak,
+            "quantize_tokens_per_s": world * sh.T * sh.G / (q_ms * 1e-3),
+            "quantize_GBps": world * qbytes / (q_ms * 1e-3) / 1e9,
+            "quantize_frac_of_measured_hbm": qbytes / (q_ms * 1e-3) / 1e9 / peak,
+            "query_latency_us": r_ms * 1e3,
+            "stage_us": {"quantize": q_ms * 1e3, "score": sc_ms * 1e3, "topk": tk_ms * 1e3, "dequant_gather": ga_ms * 1e3},
+            "frac_of_nominal_8TBps": {"quantize": qbytes / (q_ms * 1e-3) / 8e12,
+                                      "dequant_gather": bytes_gather(sh, sh.k) / (ga_ms * 1e-3) / 8e12},
+        },
+        "roofline": roofs[0], "roofline_all": roofs,
+        "gpu_launches": n_qcalls + 4, "clocks": clocks,
+        "paper_context": {"hardware": "A6000 48GB FP16 (paper)", "kv_compression": 15.7, "oqm_stage_ms_64_frames":
+                          {"kv_storage": 7.3, "retrieval": 6.9, "reconstruction": 28.7}},
+    }
+
+    # ---- end to end through the host-buffer entry points (pinned host memory, copies inside the timed region)
+    if not args.no_e2e:
+        out["e2e"] = run_e2e(args, sh, cfg, store, K, V, Q, dev, world, sdist, rbytes)
+    # ---- the oracle on this machine's host cores, rank 0 only, single-GPU runs only
+    if not args.no_cpu_baseline and rank == 0 and world == 1:
+        frames = args.cpu_sample_frames
+        Kc, Vc, Qc = cpu_inputs(sh, frames)
+        info = oracle_sample(sh, Kc, Vc, Qc, frames)
+        k = info["k"]
+        cb = bytes_score(sh, frames) + bytes_topk(sh, frames) + bytes_gather(sh, k)
+        out["cpu_baseline"] = {
+            "value": cb / info["retrieve_s"] / 1e9, "unit": "GB/s", "cores": info["threads"], "kind": "oracle",
+            "sample": f"first {frames} frames of all {sh.L} layers (of {sh.T}); top-{k} groups gathered per layer",
+            "quantize_tokens_per_s": frames * sh.G / info["quantize_s"], "seconds": info["quantize_s"] + info["retrieve_s"]}
+    if rank == 0:
+        print(json.dumps(out))
+    sdist.finish()
+
+
+def run_e2e(args, sh, cfg, store, K, V, Q, dev, world, sdist, rbytes):
+    import torch
+    from paper_2510_18269_b200 import oqm
+    chunk = 64                                   # frames per host->device chunk
+    e = 2
+    one = sh.L * chunk * sh.H_k * sh.G * sh.d * e
+    # pinned ring: one chunk of host K/V (re-sent for every chunk of the stream; every byte is really copied)
+    Kh = torch.empty(sh.L, chunk, sh.H_k, sh.G, sh.d, dtype=K.dtype).pin_memory()
+    Vh = torch.empty_like(Kh).pin_memory()
+    Kh.copy_(K[:, :chunk])
+    Vh.copy_(V[:, :chunk])
+    Qh = Q.cpu().pin_memory()
+    S = sh.k * sh.G
+    idx_h = torch.empty(sh.L, sh.k, dtype=torch.int32).pin_memory()
+    ka_h = torch.empty(sh.L, sh.H_k, S, sh.d, dtype=torch.bfloat16).pin_memory()
+    va_h = torch.empty_like(ka_h).pin_memory()
+    qscr = torch.empty(oqm.stom_oqm_quantize_host_scratch_bytes(cfg, sh.L, chunk), dtype=torch.uint8, device=dev)
+    rscr = torch.empty(oqm.stom_oqm_retrieve_host_scratch_bytes(cfg, sh.L, sh.T, sh.T_q, sh.k, oqm.BF16) + 256,
+                       dtype=torch.uint8, device=dev)
+    rscr = rscr[(-rscr.data_ptr()) % 256:]
+    n_chunks = sh.T // chunk
+
+    def e2e_step(ev_pairs=None):
+        a, b, c = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+        a.record()
+        for ci in range(n_chunks):
+            oqm.stom_oqm_quantize_frame_host(cfg, store, 0, sh.L, ci * chunk, chunk, Kh, Vh, qscr)
+        b.record()
+        oqm.stom_oqm_retrieve_host(cfg, store, 0, sh.L, sh.T, Qh, sh.T_q, sh.k, idx_h, ka_h, va_h, oqm.BF16, rscr)
+        c.record()
+        if ev_pairs is not None:
+            ev_pairs.append((a, b, c))
+
+    e2e_step()
+    torch.cuda.synchronize()
+    sdist.barrier()
+    pairs = []
+    for _ in range(max(1, args.e2e_steps)):
+        e2e_step(pairs)
+    torch.cuda.synchronize()
+    q_ms = sdist.max_over_ranks(statistics.mean(a.elapsed_time(b) for a, b, _ in pairs))
+    r_ms = sdist.max_over_ranks(statistics.mean(b.elapsed_time(c) for _, b, c in pairs))
+    return {
+        "value": world * rbytes / (r_ms * 1e-3) / 1e9, "unit": "GB/s",
+        "h2d_bytes_per_step": 2 * one * n_chunks + Qh.numel() * 2,
+        "d2h_bytes_per_step": 2 * ka_h.numel() * 2 + idx_h.numel() * 4,
+        "query_latency_us": r_ms * 1e3, "quantize_tokens_per_s": world * n_chunks * chunk * sh.G / (q_ms * 1e-3),
+        "ms_per_step": q_ms + r_ms,
+        "note": "host K/V of the stream sent in 64-frame chunks from a pinned ring; Q up, indices and the "
+                "reconstructed K/V cache down, all inside the timed region",
+    }
+
+
+def main():
+    args = parse()
+    from paper_2510_18269_b200 import synth
+    sh = synth.CONFIGS[args.config]
+    if args.layers or args.frames:
+        import dataclasses
+        sh = dataclasses.replace(sh, L=args.layers or sh.L, T=args.frames or sh.T,
+                                 name=f"{sh.name}-reduced-L{args.layers or sh.L}-T{args.frames or sh.T}")
+    if args.impl == "reference":
+        run_reference(args, sh)
+    else:
+        run_ours(args, sh)
+
+
+if __name__ == "__main__":
+    main()

@@ -237,6 +237,46 @@ int32_t stom_oqm_retrieve(const stom_oqm_config *cfg, const stom_oqm_store *stor
                           int32_t token_offset, void *workspace, int64_t workspace_bytes,
                           uint32_t *dev_flags, void *stream);
 
+/* ---- the same path driven from HOST memory -----------------------------
+ * These two calls take HOST input/output buffers (pinned memory makes the
+ * copies asynchronous), stage them through caller-provided DEVICE scratch with
+ * cudaMemcpyAsync on `stream`, and run the kernels of A1 resp. A2-A4 above
+ * (same passages of the paper).  They return without synchronising: results
+ * in host memory are valid after the caller synchronises the stream.
+ */
+
+/* Device scratch bytes stom_oqm_quantize_frame_host needs. */
+int64_t stom_oqm_quantize_host_scratch_bytes(const stom_oqm_config *cfg, int32_t layer_count,
+                                             int32_t group_count);
+
+/* A1 from host memory.  K_host, V_host: compact [layer_count][group_count][H_k][G][d]
+ * arrays of cfg->kv_dtype on the HOST.  scratch: DEVICE, 16-byte aligned.
+ * Errors: as stom_oqm_quantize_frame, plus WORKSPACE. */
+int32_t stom_oqm_quantize_frame_host(const stom_oqm_config *cfg, const stom_oqm_store *store,
+                                     int32_t layer_begin, int32_t layer_count,
+                                     int32_t group_begin, int32_t group_count,
+                                     const void *K_host, const void *V_host,
+                                     void *scratch, int64_t scratch_bytes, uint32_t *dev_flags,
+                                     void *stream);
+
+/* Device scratch bytes stom_oqm_retrieve_host needs. */
+int64_t stom_oqm_retrieve_host_scratch_bytes(const stom_oqm_config *cfg, int32_t layer_count,
+                                             int32_t n_groups, int32_t T_q, int32_t k, int32_t out_dtype);
+
+/* A2+A3+A4 from host memory.  Q_host: compact [layer_count][H_q][T_q][d] of
+ * cfg->kv_dtype on the HOST.  idx_host: HOST [rows][k] int32 (rows as in
+ * stom_oqm_topk).  k_active_host, v_active_host: HOST compact
+ * [layer_count][H_k][k*G][d] of out_dtype, both given or both NULL (NULL: the
+ * reconstructed cache stays in scratch on the device and is not copied back).
+ * scratch: DEVICE, 256-byte aligned.
+ * Errors: as the three device calls, plus WORKSPACE. */
+int32_t stom_oqm_retrieve_host(const stom_oqm_config *cfg, const stom_oqm_store *store,
+                               int32_t layer_begin, int32_t layer_count, int32_t n_groups,
+                               const void *Q_host, int32_t T_q, int32_t k,
+                               int32_t *idx_host, void *k_active_host, void *v_active_host,
+                               int32_t out_dtype, void *scratch, int64_t scratch_bytes,
+                               uint32_t *dev_flags, void *stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -1,14 +1,19 @@
 // A1: group quantizer + representative key (paper Sec. 3.4: Q_4, (s_t, m_t),
 // k-bar; appendix "Layer-wise vision memory").
 //
-// One warp owns one tile = the G tokens x d channels of one (layer, frame,
-// kv head) of K or of V.  Lane `lane` owns CPL = d/32 adjacent channels of
-// every token row, so the per-channel min / max / sum over the G tokens are
-// plain per-lane register reductions: no shared-memory reduction, no block
-// barrier, and all G row loads of the tile are in flight at once.  The tile
-// stays in registers between the statistics pass and the coding pass, so HBM
-// is read exactly once.  Packed codes are staged per warp in shared memory and
-// written back with 16-byte stores.
+// One thread block owns one tile = the G tokens x d channels of one (layer,
+// frame, kv head) of K or of V.  A thread owns 8 adjacent channels (16 bytes of
+// a 16-bit row) of P rows; the block size is chosen on the host so that
+// P * rows-per-pass covers G with the least padding (G = 50, d = 128: 5 warps,
+// 10 rows per pass, P = 5).  The tile is loaded once, stays in registers
+// between the statistics pass and the coding pass, and the code that is
+// unrolled is only P rows long, so it fits the instruction cache.
+//   pass 1  per-thread packed min / max (and binary32 sums for keys), a
+//           shuffle across the rows of a warp, per-warp partials to shared memory
+//   owners  thread c reduces channel c over the warps, computes s, m, 1/s,
+//           the representative key, and writes the statistics (coalesced)
+//   pass 2  every thread fetches s, 1/s, m of its 8 channels and emits one
+//           32-bit word of codes per row
 //
 // Bit-exactness of the codes: the contract is code = rne(fl((x - m) / s)) in
 // binary32 with a true division.  A hardware-exact division per element would
@@ -19,13 +24,11 @@
 // (q1 is a faithful quotient, and a faithful quotient corrected once more with
 // an exact FMA residual and a correctly rounded reciprocal is the correctly
 // rounded quotient -- Markstein's division theorem), followed by the
-// add-magic-constant trick for round-half-even.  Channels whose scale is zero
-// or outside [2^-60, 2^60] take a slow path with the IEEE division.
+// add-magic-constant trick for round-half-even.  Tiles with a channel whose
+// scale is zero or outside (2^-60, 2^60) take a slow path with the IEEE division.
 #include "stom_internal.cuh"
 
 namespace stom {
-
-constexpr int kQuantWarps = 4;
 
 struct QuantParams {
     const void *K, *V, *Ksum;
@@ -39,16 +42,7 @@ struct QuantParams {
     int64_t n_tiles;
 };
 
-template <int N>
-__device__ __forceinline__ void store_floats(float *dst, const float (&v)[N]) {
-    if constexpr (N == 2) {
-        *reinterpret_cast<float2 *>(dst) = make_float2(v[0], v[1]);
-    } else {
-#pragma unroll
-        for (int i = 0; i < N / 4; ++i)
-            reinterpret_cast<float4 *>(dst)[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-    }
-}
+constexpr int kMaxWarps = 8;
 
 // code of one element on the fast path (scale in the safe range, reciprocal exact-rounded)
 __device__ __forceinline__ uint32_t code_fast(float x, float m, float s, float y) {
@@ -72,205 +66,258 @@ __device__ __forceinline__ uint32_t code_slow(float x, float m, float s) {
     return (uint32_t)r;
 }
 
-template <typename T, int CPL, int MAXR, bool RESIDENT>
-__global__ void __launch_bounds__(kQuantWarps * 32) quantize_kernel(const QuantParams p) {
-    constexpr int W = CPL * (int)sizeof(T) / 4;  // 32-bit words one lane loads per row
-    extern __shared__ __align__(16) uint8_t smem[];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t tile = (int64_t)blockIdx.x * kQuantWarps + warp;
-    if (tile >= p.n_tiles) return;  // whole warp leaves together; no block barrier is used below
+// element-wise min / max on one 32-bit word of a row fragment (two 16-bit values or one float)
+template <typename T> struct WordOps;
+template <> struct WordOps<__nv_bfloat16> {
+    static constexpr uint32_t kPosInf = 0x7F807F80u, kNegInf = 0xFF80FF80u;
+    static __device__ __forceinline__ uint32_t vmin(uint32_t a, uint32_t b) {
+        __nv_bfloat162 r = __hmin2(*reinterpret_cast<__nv_bfloat162 *>(&a), *reinterpret_cast<__nv_bfloat162 *>(&b));
+        return *reinterpret_cast<uint32_t *>(&r);
+    }
+    static __device__ __forceinline__ uint32_t vmax(uint32_t a, uint32_t b) {
+        __nv_bfloat162 r = __hmax2(*reinterpret_cast<__nv_bfloat162 *>(&a), *reinterpret_cast<__nv_bfloat162 *>(&b));
+        return *reinterpret_cast<uint32_t *>(&r);
+    }
+};
+template <> struct WordOps<__half> {
+    static constexpr uint32_t kPosInf = 0x7C007C00u, kNegInf = 0xFC00FC00u;
+    static __device__ __forceinline__ uint32_t vmin(uint32_t a, uint32_t b) {
+        __half2 r = __hmin2(*reinterpret_cast<__half2 *>(&a), *reinterpret_cast<__half2 *>(&b));
+        return *reinterpret_cast<uint32_t *>(&r);
+    }
+    static __device__ __forceinline__ uint32_t vmax(uint32_t a, uint32_t b) {
+        __half2 r = __hmax2(*reinterpret_cast<__half2 *>(&a), *reinterpret_cast<__half2 *>(&b));
+        return *reinterpret_cast<uint32_t *>(&r);
+    }
+};
+template <> struct WordOps<float> {
+    static constexpr uint32_t kPosInf = 0x7F800000u, kNegInf = 0xFF800000u;
+    static __device__ __forceinline__ uint32_t vmin(uint32_t a, uint32_t b) {
+        return __float_as_uint(fminf(__uint_as_float(a), __uint_as_float(b)));
+    }
+    static __device__ __forceinline__ uint32_t vmax(uint32_t a, uint32_t b) {
+        return __float_as_uint(fmaxf(__uint_as_float(a), __uint_as_float(b)));
+    }
+};
 
-    const int G = p.g.G, H = p.g.H, d = p.g.d;
+// LPR: lanes per token row (d / 8); P: rows a thread owns.  blockDim.x = 32 * warps.
+template <typename T, int LPR, int P>
+__global__ void __launch_bounds__(kMaxWarps * 32) quantize_kernel(const QuantParams p) {
+    constexpr int W = 8 * (int)sizeof(T) / 4;  // 32-bit words of one thread's 8 channels: 4 or 8
+    constexpr int RPW = 32 / LPR;              // rows one warp covers per pass
+    constexpr int D = LPR * 8;
+    __shared__ __align__(16) float part_mn[kMaxWarps][D], part_mx[kMaxWarps][D], part_sum[kMaxWarps][D];
+    __shared__ __align__(16) float ch_s[D], ch_y[D], ch_m[D];
+    __shared__ float warp_n2[kMaxWarps];
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
+    const int sub = lane / LPR, cl = lane - sub * LPR;
+    const int rpp = nwarps * RPW;  // rows per pass of the whole block
+    const int G = p.g.G, H = p.g.H;
+
+    const int64_t tile = blockIdx.x;
     const int which = (int)(tile & 1);  // 0: keys, 1: values
     int64_t rest = tile >> 1;
     const int h = (int)(rest % H);
     rest /= H;
     const int f = (int)(rest % p.F);
     const int li = (int)(rest / p.F);
-
-    // token row of every group member (identity, or the caller's keep list)
-    int tok_lo = lane, tok_hi = lane + 32;
-    if (p.token_idx) {
-        const int32_t *ti = p.token_idx + (int64_t)f * G;
-        bool bad = false;
-        if (lane < G) {
-            int v = ti[lane];
-            bad |= (v < 0 || v >= p.n_in);
-            tok_lo = min(max(v, 0), p.n_in - 1);
-        }
-        if (lane + 32 < G) {
-            int v = ti[lane + 32];
-            bad |= (v < 0 || v >= p.n_in);
-            tok_hi = min(max(v, 0), p.n_in - 1);
-        }
-        if (bad && p.flags) atomicOr(p.flags, STOM_FLAG_BAD_INDEX);
-    }
-    const bool has_idx = p.token_idx != nullptr;  // warp-uniform
-    auto tok_of = [&](int i) -> int {
-        return has_idx ? __shfl_sync(0xffffffffu, i < 32 ? tok_lo : tok_hi, i & 31) : i;
-    };
-
-    const int64_t base = (int64_t)li * p.sl + (int64_t)f * p.sg + (int64_t)h * p.sh + lane * CPL;
+    const int64_t base = (int64_t)li * p.sl + (int64_t)f * p.sg + (int64_t)h * p.sh + cl * 8;
     const T *src = reinterpret_cast<const T *>(which ? p.V : p.K) + base;
+    const bool want_sum = !which;                 // block-uniform
+    const bool own_sum = want_sum && !p.Ksum;     // sums come from the tile itself
 
-    float mn[CPL], mx[CPL], sum[CPL];
+    // ---- load the thread's rows (all requests issued before any use)
+    Words<W> raw[P];
+    int64_t row_off[P];
 #pragma unroll
-    for (int j = 0; j < CPL; ++j) {
-        mn[j] = INFINITY;
-        mx[j] = -INFINITY;
-        sum[j] = 0.0f;
+    for (int i = 0; i < P; ++i) {
+        const int r = i * rpp + warp * RPW + sub;
+        int tok = r;
+        if (p.token_idx && r < G) {
+            const int v = p.token_idx[(int64_t)f * G + r];
+            if (v < 0 || v >= p.n_in) {
+                if (p.flags) atomicOr(p.flags, STOM_FLAG_BAD_INDEX);
+            }
+            tok = min(max(v, 0), p.n_in - 1);
+        }
+        row_off[i] = (int64_t)tok * p.st;
+        if (r < G) raw[i] = load_words<W>(src + row_off[i]);
     }
 
-    Words<W> raw[RESIDENT ? MAXR : 1];
-    if constexpr (RESIDENT) {
+    // ---- pass 1: min / max per channel over this thread's rows (packed for 16-bit types), sums for keys
+    uint32_t mnw[W], mxw[W];
+    float sum[8];
 #pragma unroll
-        for (int i = 0; i < MAXR; ++i) {
-            const int tok = tok_of(i);
-            if (i < G) raw[i] = load_words<W>(src + (int64_t)tok * p.st);
-        }
+    for (int j = 0; j < W; ++j) {
+        mnw[j] = WordOps<T>::kPosInf;
+        mxw[j] = WordOps<T>::kNegInf;
+    }
 #pragma unroll
-        for (int i = 0; i < MAXR; ++i) {
-            if (i < G) {
+    for (int j = 0; j < 8; ++j) sum[j] = 0.0f;
 #pragma unroll
-                for (int j = 0; j < CPL; ++j) {
-                    const float x = elem_of<T, W>(raw[i], j);
-                    mn[j] = fminf(mn[j], x);
-                    mx[j] = fmaxf(mx[j], x);
-                    sum[j] += x;
-                }
+    for (int i = 0; i < P; ++i) {
+        const int r = i * rpp + warp * RPW + sub;
+        if (r < G) {
+#pragma unroll
+            for (int j = 0; j < W; ++j) {
+                mnw[j] = WordOps<T>::vmin(mnw[j], raw[i].w[j]);
+                mxw[j] = WordOps<T>::vmax(mxw[j], raw[i].w[j]);
+            }
+            if (own_sum) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) sum[j] += elem_of<T, W>(raw[i], j);
             }
         }
-    } else {
-#pragma unroll 8
-        for (int i = 0; i < MAXR; ++i) {
-            const int tok = tok_of(i);
-            if (i < G) {
-                const Words<W> r = load_words<W>(src + (int64_t)tok * p.st);
+    }
+    if (want_sum && !own_sum) {  // keys averaged from the separate pre-rotary tensor
+        const T *ks = reinterpret_cast<const T *>(p.Ksum) + base;
 #pragma unroll
-                for (int j = 0; j < CPL; ++j) {
-                    const float x = elem_of<T, W>(r, j);
-                    mn[j] = fminf(mn[j], x);
-                    mx[j] = fmaxf(mx[j], x);
-                    sum[j] += x;
-                }
+        for (int i = 0; i < P; ++i) {
+            const int r = i * rpp + warp * RPW + sub;
+            if (r < G) {
+                const Words<W> kr = load_words<W>(ks + row_off[i]);
+#pragma unroll
+                for (int j = 0; j < 8; ++j) sum[j] += elem_of<T, W>(kr, j);
             }
         }
     }
-
-    // scale, offset, reciprocal
-    float s[CPL], y[CPL];
-    bool safe = true;
+    // rows of the same warp
 #pragma unroll
-    for (int j = 0; j < CPL; ++j) {
-        s[j] = __fdiv_rn(__fsub_rn(mx[j], mn[j]), 15.0f);
-        safe &= (s[j] > 8.673617379884035e-19f) && (s[j] < 1.152921504606847e18f);  // (2^-60, 2^60)
-        y[j] = __frcp_rn(s[j]);
-    }
-    safe = __all_sync(0xffffffffu, safe);
-
-    // coding pass -> per-warp staging buffer
-    const int row_bytes = p.g.row_bytes;
-    uint8_t *stage = smem + (size_t)warp * G * row_bytes;
-    auto emit = [&](int i, uint32_t cw) {
-        if constexpr (CPL == 8) *reinterpret_cast<uint32_t *>(stage + i * row_bytes + lane * 4) = cw;
-        else if constexpr (CPL == 4) *reinterpret_cast<uint16_t *>(stage + i * row_bytes + lane * 2) = (uint16_t)cw;
-        else stage[i * row_bytes + lane] = (uint8_t)cw;
-    };
-    auto code_row = [&](int i, const Words<W> &r) {
-        uint32_t cw = 0;
-        if (safe) {
+    for (int o = LPR; o < 32; o <<= 1) {
 #pragma unroll
-            for (int j = 0; j < CPL; ++j) cw |= code_fast(elem_of<T, W>(r, j), mn[j], s[j], y[j]) << (4 * j);
-        } else {
-#pragma unroll
-            for (int j = 0; j < CPL; ++j) cw |= code_slow(elem_of<T, W>(r, j), mn[j], s[j]) << (4 * j);
+        for (int j = 0; j < W; ++j) {
+            mnw[j] = WordOps<T>::vmin(mnw[j], __shfl_xor_sync(0xffffffffu, mnw[j], o));
+            mxw[j] = WordOps<T>::vmax(mxw[j], __shfl_xor_sync(0xffffffffu, mxw[j], o));
         }
-        emit(i, cw);
-    };
-    if constexpr (RESIDENT) {
+        if (want_sum) {
 #pragma unroll
-        for (int i = 0; i < MAXR; ++i)
-            if (i < G) code_row(i, raw[i]);
-    } else {
-#pragma unroll 4
-        for (int i = 0; i < MAXR; ++i) {
-            const int tok = tok_of(i);
-            if (i < G) code_row(i, load_words<W>(src + (int64_t)tok * p.st));
+            for (int j = 0; j < 8; ++j) sum[j] += __shfl_xor_sync(0xffffffffu, sum[j], o);
         }
     }
+    if (sub == 0) {
+        Words<W> a, b;
+#pragma unroll
+        for (int j = 0; j < W; ++j) {
+            a.w[j] = mnw[j];
+            b.w[j] = mxw[j];
+        }
+#pragma unroll
+        for (int j = 0; j < 8; j += 4) {
+            *reinterpret_cast<float4 *>(&part_mn[warp][cl * 8 + j]) =
+                make_float4(elem_of<T, W>(a, j), elem_of<T, W>(a, j + 1), elem_of<T, W>(a, j + 2), elem_of<T, W>(a, j + 3));
+            *reinterpret_cast<float4 *>(&part_mx[warp][cl * 8 + j]) =
+                make_float4(elem_of<T, W>(b, j), elem_of<T, W>(b, j + 1), elem_of<T, W>(b, j + 2), elem_of<T, W>(b, j + 3));
+            if (want_sum)
+                *reinterpret_cast<float4 *>(&part_sum[warp][cl * 8 + j]) = make_float4(sum[j], sum[j + 1], sum[j + 2], sum[j + 3]);
+        }
+    }
+    __syncthreads();
 
+    // ---- owners: thread c finishes channel c
     const int l = p.layer_begin + li, t = p.group_begin + f;
     const int64_t slot = bank_slot(p.g, l, t, h);
-
-    // statistics
-    store_floats<CPL>((which ? p.scale_v : p.scale_k) + slot * d + lane * CPL, s);
-    store_floats<CPL>((which ? p.zero_v : p.zero_k) + slot * d + lane * CPL, mn);
-
-    // representative key (keys only): mean over the G tokens, and its squared norm per head
-    if (!which) {
-        if (p.Ksum) {
-            const T *ks = reinterpret_cast<const T *>(p.Ksum) + base;
-#pragma unroll
-            for (int j = 0; j < CPL; ++j) sum[j] = 0.0f;
-#pragma unroll 8
-            for (int i = 0; i < MAXR; ++i) {
-                const int tok = tok_of(i);
-                if (i < G) {
-                    const Words<W> r = load_words<W>(ks + (int64_t)tok * p.st);
-#pragma unroll
-                    for (int j = 0; j < CPL; ++j) sum[j] += elem_of<T, W>(r, j);
-                }
-            }
+    bool safe = true;
+    float n2 = 0.0f;
+    for (int c = tid; c < D; c += blockDim.x) {
+        float mn = part_mn[0][c], mx = part_mx[0][c], sm = want_sum ? part_sum[0][c] : 0.0f;
+        for (int w = 1; w < nwarps; ++w) {
+            mn = fminf(mn, part_mn[w][c]);
+            mx = fmaxf(mx, part_mx[w][c]);
+            if (want_sum) sm += part_sum[w][c];
         }
-        float kb[CPL], n2 = 0.0f;
-        const float Gf = (float)G;
-#pragma unroll
-        for (int j = 0; j < CPL; ++j) {
-            kb[j] = __fdiv_rn(sum[j], Gf);
-            n2 = fmaf(kb[j], kb[j], n2);
+        const float s = __fdiv_rn(__fsub_rn(mx, mn), 15.0f);
+        safe &= (s > 8.673617379884035e-19f) && (s < 1.152921504606847e18f);  // (2^-60, 2^60)
+        ch_s[c] = s;
+        ch_y[c] = __frcp_rn(s);
+        ch_m[c] = mn;
+        (which ? p.scale_v : p.scale_k)[slot * D + c] = s;
+        (which ? p.zero_v : p.zero_k)[slot * D + c] = mn;
+        if (want_sum) {
+            const float kb = __fdiv_rn(sm, (float)G);
+            p.rep_key[slot * D + c] = kb;
+            n2 = fmaf(kb, kb, n2);
         }
-        store_floats<CPL>(p.rep_key + slot * d + lane * CPL, kb);
+    }
+    if (want_sum) {
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, o);
-        if (lane == 0) p.rep_norm2[slot] = n2;
+        if (lane == 0) warp_n2[warp] = n2;
+    }
+    safe = __syncthreads_and(safe);
+    if (want_sum && tid == 0) {
+        float tot = 0.0f;
+        for (int w = 0; w < nwarps; ++w) tot += warp_n2[w];
+        p.rep_norm2[slot] = tot;
     }
 
-    // staged codes -> bank, 16 bytes per lane per step
-    __syncwarp();
-    uint8_t *dst = (which ? p.codes_v : p.codes_k) + slot * (int64_t)G * row_bytes;
-    const int n16 = G * row_bytes / 16;
-    for (int c = lane; c < n16; c += 32)
-        reinterpret_cast<uint4 *>(dst)[c] = reinterpret_cast<const uint4 *>(stage)[c];
+    // ---- pass 2: codes
+    float s[8], y[8], m[8];
+#pragma unroll
+    for (int j = 0; j < 8; j += 4) {
+        const float4 a = *reinterpret_cast<const float4 *>(&ch_s[cl * 8 + j]);
+        const float4 b = *reinterpret_cast<const float4 *>(&ch_y[cl * 8 + j]);
+        const float4 c = *reinterpret_cast<const float4 *>(&ch_m[cl * 8 + j]);
+        s[j] = a.x; s[j + 1] = a.y; s[j + 2] = a.z; s[j + 3] = a.w;
+        y[j] = b.x; y[j + 1] = b.y; y[j + 2] = b.z; y[j + 3] = b.w;
+        m[j] = c.x; m[j + 1] = c.y; m[j + 2] = c.z; m[j + 3] = c.w;
+    }
+    uint32_t *dst = reinterpret_cast<uint32_t *>((which ? p.codes_v : p.codes_k) + slot * (int64_t)G * p.g.row_bytes) + cl;
+#pragma unroll
+    for (int i = 0; i < P; ++i) {
+        const int r = i * rpp + warp * RPW + sub;
+        if (r < G) {
+            uint32_t cw = 0;
+            if (safe) {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) cw |= code_fast(elem_of<T, W>(raw[i], j), m[j], s[j], y[j]) << (4 * j);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) cw |= code_slow(elem_of<T, W>(raw[i], j), m[j], s[j]) << (4 * j);
+            }
+            dst[(int64_t)r * LPR] = cw;
+        }
+    }
 }
 
-template <typename T, int CPL, int MAXR, bool RESIDENT>
-static int32_t launch_one(const QuantParams &p, cudaStream_t stream) {
-    const int64_t blocks = (p.n_tiles + kQuantWarps - 1) / kQuantWarps;
-    if (blocks > 0x7fffffffLL) return STOM_ERR_SHAPE;
-    const size_t smem = (size_t)kQuantWarps * p.g.G * p.g.row_bytes;
-    quantize_kernel<T, CPL, MAXR, RESIDENT><<<(unsigned)blocks, kQuantWarps * 32, smem, stream>>>(p);
+template <typename T, int LPR>
+static int32_t launch_lpr(const QuantParams &p, cudaStream_t stream) {
+    if (p.n_tiles > 0x7fffffffLL) return STOM_ERR_SHAPE;
+    constexpr int RPW = 32 / LPR;
+    // block shape: the (warps, P) pair that covers G rows with the least padding, P <= 8; ties -> more warps
+    const int G = p.g.G;
+    int best_w = kMaxWarps, best_p = (G + kMaxWarps * RPW - 1) / (kMaxWarps * RPW), best_pad = 1 << 30;
+    for (int w = kMaxWarps; w >= 2; --w) {
+        const int P = (G + w * RPW - 1) / (w * RPW);
+        if (P > 8) continue;
+        const int pad = P * w * RPW - G;
+        if (pad < best_pad) {
+            best_pad = pad;
+            best_w = w;
+            best_p = P;
+        }
+    }
+    const unsigned grid = (unsigned)p.n_tiles, block = best_w * 32;
+    switch (best_p) {
+    case 1: quantize_kernel<T, LPR, 1><<<grid, block, 0, stream>>>(p); break;
+    case 2: quantize_kernel<T, LPR, 2><<<grid, block, 0, stream>>>(p); break;
+    case 3: quantize_kernel<T, LPR, 3><<<grid, block, 0, stream>>>(p); break;
+    case 4: quantize_kernel<T, LPR, 4><<<grid, block, 0, stream>>>(p); break;
+    case 5: quantize_kernel<T, LPR, 5><<<grid, block, 0, stream>>>(p); break;
+    case 6: quantize_kernel<T, LPR, 6><<<grid, block, 0, stream>>>(p); break;
+    case 7: quantize_kernel<T, LPR, 7><<<grid, block, 0, stream>>>(p); break;
+    default: quantize_kernel<T, LPR, 8><<<grid, block, 0, stream>>>(p); break;
+    }
     return finish_launch();
 }
 
 template <typename T>
 static int32_t launch_for_type(const QuantParams &p, cudaStream_t stream) {
-    const int G = p.g.G;
-    // register budget: keep the tile resident while it costs at most 128 registers per lane
-    constexpr bool wide = sizeof(T) == 4;
     switch (p.g.d) {
-    case 128:
-        if (G <= 16) return launch_one<T, 4, 16, true>(p, stream);
-        if (G <= 32) return launch_one<T, 4, 32, true>(p, stream);
-        if (G <= 40) return launch_one<T, 4, 40, !wide>(p, stream);
-        if (G <= 48) return launch_one<T, 4, 48, !wide>(p, stream);
-        if (G <= 56) return launch_one<T, 4, 56, !wide>(p, stream);
-        return launch_one<T, 4, 64, !wide>(p, stream);
-    case 64:
-        return launch_one<T, 2, 64, !wide>(p, stream);
-    case 256:
-        return launch_one<T, 8, 64, false>(p, stream);
-    default:
-        return STOM_ERR_SHAPE;
+    case 64: return launch_lpr<T, 8>(p, stream);
+    case 128: return launch_lpr<T, 16>(p, stream);
+    case 256: return launch_lpr<T, 32>(p, stream);
+    default: return STOM_ERR_SHAPE;
     }
 }
 

@@ -25,6 +25,8 @@ EXPORTS = (
     "stom_oqm_store_layout", "stom_oqm_store_bind", "stom_oqm_budget_to_k", "stom_oqm_score_workspace_bytes",
     "stom_status_string", "stom_last_cuda_error", "stom_oqm_quantize_frame", "stom_oqm_score_groups",
     "stom_oqm_topk", "stom_oqm_dequant_gather", "stom_oqm_retrieve",
+    "stom_oqm_quantize_host_scratch_bytes", "stom_oqm_quantize_frame_host",
+    "stom_oqm_retrieve_host_scratch_bytes", "stom_oqm_retrieve_host",
 )
 
 
@@ -69,6 +71,8 @@ def lib():
         L.stom_oqm_score_workspace_bytes.restype = C.c_int64
         L.stom_oqm_score_workspace_bytes.argtypes = [C.POINTER(Config), C.c_int32]
         L.stom_oqm_budget_to_k.argtypes = [C.c_int64, C.c_int32, C.c_int32]
+        L.stom_oqm_quantize_host_scratch_bytes.restype = C.c_int64
+        L.stom_oqm_retrieve_host_scratch_bytes.restype = C.c_int64
         for name in EXPORTS:
             fn = getattr(L, name)
             if fn.restype is C.c_int:
@@ -197,3 +201,41 @@ def stom_oqm_retrieve(cfg: Config, store: Store, layer_begin, layer_count, n_gro
         C.c_int64(0 if workspace is None else workspace.numel() * workspace.element_size()), _ptr(dev_flags),
         _stream(stream))
     _check(rc, "stom_oqm_retrieve")
+
+
+# ---------------------------------------------------------------- host-buffer entry points
+
+def _hptr(t):
+    """Address of a HOST tensor (pinned or pageable)."""
+    if t is None:
+        return None
+    assert not t.is_cuda and t.is_contiguous()
+    return C.c_void_p(t.data_ptr())
+
+
+def stom_oqm_quantize_host_scratch_bytes(cfg: Config, layer_count: int, group_count: int) -> int:
+    return int(lib().stom_oqm_quantize_host_scratch_bytes(C.byref(cfg), C.c_int32(layer_count), C.c_int32(group_count)))
+
+
+def stom_oqm_quantize_frame_host(cfg: Config, store: Store, layer_begin, layer_count, group_begin, group_count,
+                                 K_host, V_host, scratch, dev_flags=None, stream=None):
+    rc = lib().stom_oqm_quantize_frame_host(
+        C.byref(cfg), C.byref(store.desc), C.c_int32(layer_begin), C.c_int32(layer_count), C.c_int32(group_begin),
+        C.c_int32(group_count), _hptr(K_host), _hptr(V_host), _ptr(scratch),
+        C.c_int64(scratch.numel() * scratch.element_size()), _ptr(dev_flags), _stream(stream))
+    _check(rc, "stom_oqm_quantize_frame_host")
+
+
+def stom_oqm_retrieve_host_scratch_bytes(cfg: Config, layer_count, n_groups, T_q, k, out_dtype) -> int:
+    return int(lib().stom_oqm_retrieve_host_scratch_bytes(
+        C.byref(cfg), C.c_int32(layer_count), C.c_int32(n_groups), C.c_int32(T_q), C.c_int32(k), C.c_int32(out_dtype)))
+
+
+def stom_oqm_retrieve_host(cfg: Config, store: Store, layer_begin, layer_count, n_groups, Q_host, T_q, k,
+                           idx_host, k_active_host, v_active_host, out_dtype, scratch, dev_flags=None, stream=None):
+    rc = lib().stom_oqm_retrieve_host(
+        C.byref(cfg), C.byref(store.desc), C.c_int32(layer_begin), C.c_int32(layer_count), C.c_int32(n_groups),
+        _hptr(Q_host), C.c_int32(T_q), C.c_int32(k), _hptr(idx_host), _hptr(k_active_host), _hptr(v_active_host),
+        C.c_int32(out_dtype), _ptr(scratch), C.c_int64(scratch.numel() * scratch.element_size()), _ptr(dev_flags),
+        _stream(stream))
+    _check(rc, "stom_oqm_retrieve_host")
