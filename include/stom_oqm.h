@@ -47,6 +47,7 @@ extern "C" {
 #define STOM_ERR_UNSUPPORTED (-6) /* bits / dtype / mode not implemented              */
 #define STOM_ERR_CUDA (-7)        /* launch failed; see stom_last_cuda_error()        */
 #define STOM_ERR_WORKSPACE (-8)   /* workspace missing or too small                   */
+#define STOM_ERR_NOALLOC_LIMIT (-9) /* request exceeds the built-in scratch of a *_noalloc call */
 
 /* ---- element types and modes ----------------------------------------- */
 #define STOM_BF16 0
@@ -186,6 +187,45 @@ int32_t stom_oqm_score_groups(const stom_oqm_config *cfg, const stom_oqm_store *
                               const void *Q, int32_t T_q, int64_t q_stride_layer,
                               int64_t q_stride_head, int64_t q_stride_token,
                               float *scores, void *workspace, int64_t workspace_bytes, void *stream);
+
+/* ---- A2 for callers that cannot allocate device memory -----------------
+ *
+ * (No counterpart in the paper: this is a packaging variant of the call above.)
+ *
+ * Some hosts of this library have no allocator to offer: an inference server
+ * that handed every byte of HBM to its own pool at start-up, a plug-in that is
+ * forbidden to call cudaMalloc because that call synchronises the whole device
+ * and would stall the other streams of a serving process, or a caller that only
+ * holds the tensors it was given.  stom_oqm_score_groups needs a scratch buffer
+ * from such a caller; this variant does not.  It computes exactly the same
+ * scores with the same kernels, but keeps the question embeddings in a fixed
+ * array of STOM_NOALLOC_SCRATCH_BYTES bytes that is part of the library image.
+ * Inputs and outputs are still the caller's.
+ *
+ * Consequences of the built-in array:
+ *   - every GPU that loads the library holds the array until the process exits;
+ *   - the layer range of one call must fit: layer_count * H_k * (d + 1) * 4
+ *     bytes, rounded up to 256, may not exceed STOM_NOALLOC_SCRATCH_BYTES,
+ *     otherwise the call returns STOM_ERR_NOALLOC_LIMIT and launches nothing
+ *     (score the layers in several calls instead);
+ *   - all calls on one GPU share the array.  Calls that may overlap on the GPU
+ *     (different streams, no ordering between them) race on it and produce
+ *     wrong scores; calls on one stream, or ordered by events, are safe.  The
+ *     array keeps the previous call's contents; nothing in it needs clearing,
+ *     because each call rewrites every word it later reads;
+ *   - the first call on each GPU looks up the array's device address (with that
+ *     GPU current) before it launches; make that first call outside of any
+ *     stream capture.
+ * The call itself never calls cudaMalloc, cudaFree or any allocating routine.
+ * Errors: as stom_oqm_score_groups without WORKSPACE, plus NOALLOC_LIMIT, and
+ * UNSUPPORTED for a device ordinal of 64 or more.
+ */
+#define STOM_NOALLOC_SCRATCH_BYTES (512 * 1024)
+int32_t stom_oqm_score_groups_noalloc(const stom_oqm_config *cfg, const stom_oqm_store *store,
+                                      int32_t layer_begin, int32_t layer_count, int32_t n_groups,
+                                      const void *Q, int32_t T_q, int64_t q_stride_layer,
+                                      int64_t q_stride_head, int64_t q_stride_token,
+                                      float *scores, void *stream);
 
 /* ---- A3: top-K (Sec. 3.4 the TopK equation; appendix: selected indices are
  *      kept in sorted order) ---------------------------------------------

@@ -100,6 +100,7 @@ extern "C" const char *stom_status_string(int32_t s) {
     case STOM_ERR_UNSUPPORTED: return "unsupported bits, dtype or mode";
     case STOM_ERR_CUDA: return "CUDA launch failed (see stom_last_cuda_error)";
     case STOM_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+    case STOM_ERR_NOALLOC_LIMIT: return "request needs more scratch than the library's built-in array holds; split the layer range";
     default: return "unknown status";
     }
 }

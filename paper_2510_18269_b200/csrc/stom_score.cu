@@ -10,6 +10,8 @@
 //   kernel 2: one warp per stored group, q held in shared memory, 16-byte
 //             loads of k-bar, warp-shuffle reduction, stored |k-bar_h|^2
 //             reused for the norm.
+#include <mutex>
+
 #include "stom_internal.cuh"
 
 namespace stom {
@@ -175,4 +177,61 @@ extern "C" int32_t stom_oqm_score_groups(const stom_oqm_config *cfg, const stom_
     const size_t smem = (size_t)cfg->n_kv_heads * (cfg->head_dim + 1) * sizeof(float);
     score_kernel<<<g2, kScoreWarps * 32, smem, s>>>(p);
     return finish_launch();
+}
+
+// ---------------------------------------------------------------------------
+// Scoring for callers that must not touch the device allocator.
+//
+// The question embeddings that pass from the first scoring kernel to the second
+// live in an array that is part of the library image instead of in caller
+// scratch.  The array exists once per GPU that loads the library and is shared
+// by every call on that GPU.
+// ---------------------------------------------------------------------------
+
+static __device__ __align__(256) unsigned char g_score_scratch[STOM_NOALLOC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_scratch_mutex;
+void *g_scratch_addr[kMaxDevices];  // device address of g_score_scratch on each GPU, filled on first use
+}  // namespace
+
+extern "C" int32_t stom_oqm_score_groups_noalloc(const stom_oqm_config *cfg, const stom_oqm_store *store,
+                                                 int32_t layer_begin, int32_t layer_count, int32_t n_groups,
+                                                 const void *Q, int32_t T_q, int64_t q_stride_layer,
+                                                 int64_t q_stride_head, int64_t q_stride_token,
+                                                 float *scores, void *stream) {
+    int32_t rc = check_config(cfg);
+    if (rc) return rc;
+    if ((rc = check_layers(cfg, layer_begin, layer_count))) return rc;
+    const int64_t need = stom_oqm_score_workspace_bytes(cfg, layer_count);
+    if (need < 0) return STOM_ERR_INVALID_ARG;
+    if (need > (int64_t)STOM_NOALLOC_SCRATCH_BYTES) return STOM_ERR_NOALLOC_LIMIT;
+
+    // The symbol's name is only a host-side handle; the kernels need its address on the current GPU.
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) {
+        set_last_cuda_error(e);
+        return STOM_ERR_CUDA;
+    }
+    if (dev < 0 || dev >= kMaxDevices) return STOM_ERR_UNSUPPORTED;
+    void *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_scratch_mutex);
+        if (!g_scratch_addr[dev]) {
+            void *p = nullptr;
+            e = cudaGetSymbolAddress(&p, g_score_scratch);
+            if (e != cudaSuccess || !p) {
+                set_last_cuda_error(e);
+                return STOM_ERR_CUDA;
+            }
+            g_scratch_addr[dev] = p;
+        }
+        scratch = g_scratch_addr[dev];
+    }
+    // Every word of the scratch that the second kernel reads is written by the first kernel of the
+    // same call, so nothing has to be cleared between calls.
+    return stom_oqm_score_groups(cfg, store, layer_begin, layer_count, n_groups, Q, T_q, q_stride_layer,
+                                 q_stride_head, q_stride_token, scores, scratch, STOM_NOALLOC_SCRATCH_BYTES, stream);
 }

@@ -27,6 +27,7 @@ EXPORTS = (
     "stom_oqm_topk", "stom_oqm_dequant_gather", "stom_oqm_retrieve",
     "stom_oqm_quantize_host_scratch_bytes", "stom_oqm_quantize_frame_host",
     "stom_oqm_retrieve_host_scratch_bytes", "stom_oqm_retrieve_host",
+    "stom_oqm_score_groups_noalloc",
 )
 
 
@@ -169,6 +170,25 @@ def stom_oqm_score_groups(cfg: Config, store: Store, layer_begin, layer_count, n
         _ptr(Q), C.c_int32(T_q), C.c_int64(ql), C.c_int64(qh), C.c_int64(qt), _ptr(scores), _ptr(workspace),
         C.c_int64(0 if workspace is None else workspace.numel() * workspace.element_size()), _stream(stream))
     _check(rc, "stom_oqm_score_groups")
+
+
+NOALLOC_SCRATCH_BYTES = 512 * 1024
+
+
+def stom_oqm_score_groups_noalloc(cfg: Config, store: Store, layer_begin, layer_count, n_groups, Q, T_q, q_strides,
+                                  scores, stream=None):
+    """Scores without caller scratch, for hosts that cannot allocate device memory (for example a server whose
+    memory pool owns all of HBM, or code that may not call cudaMalloc because it would stall the device).
+
+    Same result as stom_oqm_score_groups.  The intermediate question embeddings live in a NOALLOC_SCRATCH_BYTES
+    array inside the library that all calls on a GPU share: keep such calls ordered on the GPU (one stream, or
+    events), make the first call on each GPU outside of stream capture, and split the layer range when the call
+    reports that the array is too small."""
+    ql, qh, qt = q_strides
+    rc = lib().stom_oqm_score_groups_noalloc(
+        C.byref(cfg), C.byref(store.desc), C.c_int32(layer_begin), C.c_int32(layer_count), C.c_int32(n_groups),
+        _ptr(Q), C.c_int32(T_q), C.c_int64(ql), C.c_int64(qh), C.c_int64(qt), _ptr(scores), _stream(stream))
+    _check(rc, "stom_oqm_score_groups_noalloc")
 
 
 def stom_oqm_topk(scores, rows, n, row_stride, k, idx_out, score_out=None, n_sel_out=None, stream=None):
