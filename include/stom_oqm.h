@@ -62,6 +62,7 @@ extern "C" {
 
 /* bits of dev_flags set by kernels */
 #define STOM_FLAG_BAD_INDEX 1u /* an entry of idx was < -1 or >= n_groups and was skipped */
+#define STOM_FLAG_TIMEOUT 2u   /* a bounded wait inside a kernel ran out; the call's outputs are incomplete */
 
 /* Geometry of one memory bank (paper notation: L, H_q, H_k, d, G). */
 typedef struct stom_oqm_config {

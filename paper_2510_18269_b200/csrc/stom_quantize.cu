@@ -1,19 +1,30 @@
 // A1: group quantizer + representative key (paper Sec. 3.4: Q_4, (s_t, m_t),
 // k-bar; appendix "Layer-wise vision memory").
 //
-// One thread block owns one tile = the G tokens x d channels of one (layer,
-// frame, kv head) of K or of V.  A thread owns 8 adjacent channels (16 bytes of
-// a 16-bit row) of P rows; the block size is chosen on the host so that
-// P * rows-per-pass covers G with the least padding (G = 50, d = 128: 5 warps,
-// 10 rows per pass, P = 5).  The tile is loaded once, stays in registers
-// between the statistics pass and the coding pass, and the code that is
-// unrolled is only P rows long, so it fits the instruction cache.
-//   pass 1  per-thread packed min / max (and binary32 sums for keys), a
-//           shuffle across the rows of a warp, per-warp partials to shared memory
-//   owners  thread c reduces channel c over the warps, computes s, m, 1/s,
-//           the representative key, and writes the statistics (coalesced)
-//   pass 2  every thread fetches s, 1/s, m of its 8 channels and emits one
-//           32-bit word of codes per row
+// A tile is the G tokens x d channels of one (layer, frame, kv head) of K or
+// of V (12.8 KB at G = 50, d = 128, bf16).  The kernel is persistent: one
+// block per SM, kConsumerWarps consumer warps and one producer warp.
+//
+//   producer  walks the block's tiles in order and, for each, issues bulk
+//             asynchronous copies (cp.async.bulk, completion counted on an
+//             mbarrier) from global memory into the next free slot of a ring
+//             of shared-memory slots; a tile whose rows are contiguous is one
+//             copy, a strided or index-gathered tile is one copy per row.
+//             The ring keeps ~10 tiles per SM in flight, which is what hides
+//             HBM latency; no register is tied up by a load.
+//   consumer  warp w owns every kConsumerWarps-th tile of the block outright.
+//             A lane owns d/32 adjacent channels of ALL G rows, so the
+//             per-channel statistics need no cross-lane traffic at all:
+//               pass 1  packed min / max down the rows (shared memory reads)
+//               stats   s = (max - min)/15, m = min, y = rn(1/s)   -> global
+//               pass 2  codes, two channels per instruction (f32x2), written
+//                       to a shared staging tile; key tiles add up the rows
+//                       for the representative key on the way
+//             and the finished code tile leaves with ONE bulk store.
+//
+// Every wait on an mbarrier is bounded (wall-clock limit); a wait that runs
+// out sets STOM_FLAG_TIMEOUT, tells the rest of the block to stop, and the
+// block drains its copies in flight before it returns.
 //
 // Bit-exactness of the codes: the contract is code = rne(fl((x - m) / s)) in
 // binary32 with a true division.  A hardware-exact division per element would
@@ -30,6 +41,11 @@
 
 namespace stom {
 
+constexpr int kConsumerWarps = 8;
+constexpr int kQuantThreads = (kConsumerWarps + 1) * 32;
+constexpr int kMaxSlots = 24;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s: far beyond any legitimate wait
+
 struct QuantParams {
     const void *K, *V, *Ksum;
     const int32_t *token_idx;
@@ -39,23 +55,77 @@ struct QuantParams {
     BankGeom g;
     int32_t layer_begin, group_begin, F, n_in;
     uint32_t *flags;
-    int64_t n_tiles;
+    uint32_t n_tiles;     // layer_count * F * H * n_kinds, below 2^31
+    int32_t n_kinds;      // 2: keys, values;  3: keys, values, pre-rotary keys (mean only)
+    int32_t n_slots;      // ring depth, a multiple of n_warps
+    int32_t n_warps;      // consumer warps that take tiles (the others leave at once)
+    int32_t slot_bytes;   // bytes of one input tile, rounded up to 128
+    int32_t contiguous;   // rows of a tile are adjacent in global memory
 };
 
-constexpr int kMaxWarps = 8;
+// ------------------------------------------------------------------ PTX wrappers
 
-// code of one element on the fast path (scale in the safe range, reciprocal exact-rounded)
-__device__ __forceinline__ uint32_t code_fast(float x, float m, float s, float y) {
-    const float diff = __fsub_rn(x, m);
-    float q = __fmul_rn(diff, y);
-    float e = __fmaf_rn(-q, s, diff);
-    q = __fmaf_rn(e, y, q);
-    e = __fmaf_rn(-q, s, diff);
-    q = __fmaf_rn(e, y, q);
-    // 1.5 * 2^23: adding it rounds q to an integer (ties to even) in the low mantissa bits
-    const float u = __fadd_rn(q, 12582912.0f);
-    return __float_as_uint(u) & 15u;
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// global -> shared bulk copy; completion (in bytes) is counted on the mbarrier
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
+}
+// shared -> global bulk copy, tracked by the issuing thread's bulk async-group
+__device__ __forceinline__ void bulk_store(void *dst, uint32_t src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// orders this thread's shared-memory writes before later reads by the asynchronous copy engine
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
+// Bounded wait.  Returns false when the limit ran out or another thread of the block gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    for (;;) {
+#pragma unroll 1
+        for (int i = 0; i < 64; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_ns() - t0 > kWaitLimitNs) return false;
+    }
+}
+
+// ------------------------------------------------------------------ arithmetic
 
 // IEEE division; s == 0 marks a constant (or underflowing) channel whose codes are all 0
 __device__ __forceinline__ uint32_t code_slow(float x, float m, float s) {
@@ -66,10 +136,9 @@ __device__ __forceinline__ uint32_t code_slow(float x, float m, float s) {
     return (uint32_t)r;
 }
 
-// element-wise min / max on one 32-bit word of a row fragment (two 16-bit values or one float)
+// element-wise min / max on one 32-bit word of a row (two 16-bit values or one float)
 template <typename T> struct WordOps;
 template <> struct WordOps<__nv_bfloat16> {
-    static constexpr uint32_t kPosInf = 0x7F807F80u, kNegInf = 0xFF80FF80u;
     static __device__ __forceinline__ uint32_t vmin(uint32_t a, uint32_t b) {
         __nv_bfloat162 r = __hmin2(*reinterpret_cast<__nv_bfloat162 *>(&a), *reinterpret_cast<__nv_bfloat162 *>(&b));
         return *reinterpret_cast<uint32_t *>(&r);
@@ -80,7 +149,6 @@ template <> struct WordOps<__nv_bfloat16> {
     }
 };
 template <> struct WordOps<__half> {
-    static constexpr uint32_t kPosInf = 0x7C007C00u, kNegInf = 0xFC00FC00u;
     static __device__ __forceinline__ uint32_t vmin(uint32_t a, uint32_t b) {
         __half2 r = __hmin2(*reinterpret_cast<__half2 *>(&a), *reinterpret_cast<__half2 *>(&b));
         return *reinterpret_cast<uint32_t *>(&r);
@@ -91,7 +159,6 @@ template <> struct WordOps<__half> {
     }
 };
 template <> struct WordOps<float> {
-    static constexpr uint32_t kPosInf = 0x7F800000u, kNegInf = 0xFF800000u;
     static __device__ __forceinline__ uint32_t vmin(uint32_t a, uint32_t b) {
         return __float_as_uint(fminf(__uint_as_float(a), __uint_as_float(b)));
     }
@@ -131,11 +198,8 @@ __device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
 }
 
 // Two adjacent channels at once: x - m, the doubly corrected quotient, the rounding add.  Returns the two
-// floats 1.5*2^23 + code as a pair; `acc` receives x added to the running sums when SUM is set.
-template <bool SUM>
-__device__ __forceinline__ uint64_t code_pair(uint64_t x, uint64_t m, uint64_t neg_s, uint64_t y, uint64_t magic,
-                                              uint64_t &acc) {
-    if constexpr (SUM) acc = add2(acc, x);
+// floats 1.5*2^23 + code as a pair.
+__device__ __forceinline__ uint64_t code_pair(uint64_t x, uint64_t m, uint64_t neg_s, uint64_t y, uint64_t magic) {
     const uint64_t diff = sub2(x, m);
     uint64_t q = mul2(diff, y);
     uint64_t e = fma2(q, neg_s, diff);
@@ -145,284 +209,385 @@ __device__ __forceinline__ uint64_t code_pair(uint64_t x, uint64_t m, uint64_t n
     return add2(q, magic);
 }
 
-// LPR: lanes per token row (d / 8); P: rows a thread owns; EXACT: P * rows-per-pass == G (no ragged last pass).
-// blockDim.x = 32 * warps.  grid = (2 * H, frames, layers): x = kv head * 2 + (0: keys, 1: values).
-template <typename T, int LPR, int P, bool EXACT>
-__global__ void __launch_bounds__(kMaxWarps * 32) quantize_kernel(const QuantParams p) {
-    constexpr int W = 8 * (int)sizeof(T) / 4;  // 32-bit words of one thread's 8 channels: 4 or 8
-    constexpr int RPW = 32 / LPR;              // rows one warp covers per pass
-    constexpr int D = LPR * 8;
-    __shared__ __align__(16) float part_mn[kMaxWarps][D], part_mx[kMaxWarps][D], part_sum[kMaxWarps][D];
-    __shared__ __align__(16) float ch_s[D], ch_y[D], ch_m[D];
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, nwarps = blockDim.x >> 5;
-    const int sub = lane / LPR, cl = lane - sub * LPR;
-    const int rpp = nwarps * RPW;  // rows per pass of the whole block
-    const int rbase = warp * RPW + sub;
-    const int G = p.g.G;
-
-    const int which = blockIdx.x & 1, h = blockIdx.x >> 1, f = blockIdx.y, li = blockIdx.z;
-    const int64_t base = (int64_t)li * p.sl + (int64_t)f * p.sg + (int64_t)h * p.sh + cl * 8;
-    const T *src = reinterpret_cast<const T *>(which ? p.V : p.K) + base;
-    const bool want_sum = !which;              // block-uniform: keys carry the representative key
-    const bool own_sum = want_sum && !p.Ksum;  // sums come from the tile itself
-
-    // ---- load the thread's rows (all requests issued before any use).  A row past the end of a ragged
-    //      last pass re-reads row G-1: harmless for min/max, masked out of sums and stores.
-    Words<W> raw[P];
-    int64_t row_off[P];
+// The C channels of one token row that a lane owns, as 32-bit words read from shared memory.
+template <typename T, int C>
+struct LaneRow {
+    static constexpr int W = C * (int)sizeof(T) / 4;
+    uint32_t w[W];
+    __device__ __forceinline__ void load(const unsigned char *p) {
+        if constexpr (W == 1) {
+            w[0] = *reinterpret_cast<const uint32_t *>(p);
+        } else if constexpr (W == 2) {
+            const uint2 v = *reinterpret_cast<const uint2 *>(p);
+            w[0] = v.x; w[1] = v.y;
+        } else {
 #pragma unroll
-    for (int i = 0; i < P; ++i) {
-        int r = i * rpp + rbase;
-        if constexpr (!EXACT) r = min(r, G - 1);
-        int tok = r;
-        if (p.token_idx) {
-            const int v = p.token_idx[(int64_t)f * G + r];
-            if ((v < 0 || v >= p.n_in) && p.flags) atomicOr(p.flags, STOM_FLAG_BAD_INDEX);
-            tok = min(max(v, 0), p.n_in - 1);
-        }
-        row_off[i] = (int64_t)tok * p.st;
-        raw[i] = load_words<W>(src + row_off[i]);
-    }
-
-    // ---- pass 1: min / max per channel over this thread's rows (two values per word for 16-bit types)
-    uint32_t mnw[W], mxw[W];
-#pragma unroll
-    for (int j = 0; j < W; ++j) mnw[j] = mxw[j] = raw[0].w[j];
-#pragma unroll
-    for (int i = 1; i < P; ++i) {
-#pragma unroll
-        for (int j = 0; j < W; ++j) {
-            mnw[j] = WordOps<T>::vmin(mnw[j], raw[i].w[j]);
-            mxw[j] = WordOps<T>::vmax(mxw[j], raw[i].w[j]);
-        }
-    }
-#pragma unroll
-    for (int o = LPR; o < 32; o <<= 1) {  // rows of the same warp
-#pragma unroll
-        for (int j = 0; j < W; ++j) {
-            mnw[j] = WordOps<T>::vmin(mnw[j], __shfl_xor_sync(0xffffffffu, mnw[j], o));
-            mxw[j] = WordOps<T>::vmax(mxw[j], __shfl_xor_sync(0xffffffffu, mxw[j], o));
-        }
-    }
-    if (sub == 0) {
-        Words<W> a, b;
-#pragma unroll
-        for (int j = 0; j < W; ++j) {
-            a.w[j] = mnw[j];
-            b.w[j] = mxw[j];
-        }
-#pragma unroll
-        for (int j = 0; j < 8; j += 4) {
-            *reinterpret_cast<float4 *>(&part_mn[warp][cl * 8 + j]) =
-                make_float4(elem_of<T, W>(a, j), elem_of<T, W>(a, j + 1), elem_of<T, W>(a, j + 2), elem_of<T, W>(a, j + 3));
-            *reinterpret_cast<float4 *>(&part_mx[warp][cl * 8 + j]) =
-                make_float4(elem_of<T, W>(b, j), elem_of<T, W>(b, j + 1), elem_of<T, W>(b, j + 2), elem_of<T, W>(b, j + 3));
-        }
-    }
-    __syncthreads();
-
-    // ---- owners: thread c finishes the statistics of channel c
-    const int64_t slot = bank_slot(p.g, p.layer_begin + li, p.group_begin + f, h);
-    bool safe = true;
-    for (int c = tid; c < D; c += blockDim.x) {
-        float mn = part_mn[0][c], mx = part_mx[0][c];
-        for (int w = 1; w < nwarps; ++w) {
-            mn = fminf(mn, part_mn[w][c]);
-            mx = fmaxf(mx, part_mx[w][c]);
-        }
-        const float s = __fdiv_rn(__fsub_rn(mx, mn), 15.0f);
-        safe &= (s > 8.673617379884035e-19f) && (s < 1.152921504606847e18f);  // (2^-60, 2^60)
-        ch_s[c] = s;
-        ch_y[c] = __frcp_rn(s);
-        ch_m[c] = mn;
-        (which ? p.scale_v : p.scale_k)[slot * D + c] = s;
-        (which ? p.zero_v : p.zero_k)[slot * D + c] = mn;
-    }
-    safe = __syncthreads_and(safe);
-
-    // ---- pass 2: codes (and, for keys, the channel sums of the rows as a by-product)
-    float s[8], y[8], m[8];
-#pragma unroll
-    for (int j = 0; j < 8; j += 4) {
-        const float4 a = *reinterpret_cast<const float4 *>(&ch_s[cl * 8 + j]);
-        const float4 b = *reinterpret_cast<const float4 *>(&ch_y[cl * 8 + j]);
-        const float4 c = *reinterpret_cast<const float4 *>(&ch_m[cl * 8 + j]);
-        s[j] = a.x; s[j + 1] = a.y; s[j + 2] = a.z; s[j + 3] = a.w;
-        y[j] = b.x; y[j + 1] = b.y; y[j + 2] = b.z; y[j + 3] = b.w;
-        m[j] = c.x; m[j + 1] = c.y; m[j + 2] = c.z; m[j + 3] = c.w;
-    }
-    uint32_t *dst = reinterpret_cast<uint32_t *>((which ? p.codes_v : p.codes_k) + slot * (int64_t)G * p.g.row_bytes) + cl;
-    uint64_t sum2[4];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) sum2[j] = 0ull;  // (+0, +0)
-
-    if (safe) {
-        uint64_t m2[4], ns2[4], y2[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            m2[j] = pack_f2(m[2 * j], m[2 * j + 1]);
-            ns2[j] = pack_f2(-s[2 * j], -s[2 * j + 1]);
-            y2[j] = pack_f2(y[2 * j], y[2 * j + 1]);
-        }
-        const uint64_t magic = pack_f2(12582912.0f, 12582912.0f);  // 1.5 * 2^23: rounds to integer, ties to even
-        // every float 1.5*2^23 + code has the bit pattern 0x4B400000 + code; summing pattern * 16^j over the 8
-        // channels and removing the constant part leaves the 8 nibbles in place (they cannot carry into each other)
-        constexpr uint32_t kBias = 0x4B400000u * 0x11111111u;
-#pragma unroll
-        for (int i = 0; i < P; ++i) {
-            const int r = i * rpp + rbase;
-            const bool valid = EXACT || r < G;
-            uint32_t cw = 0u - kBias;
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                float x0, x1;
-                if constexpr (sizeof(T) == 4) {
-                    x0 = __uint_as_float(raw[i].w[2 * j]);
-                    x1 = __uint_as_float(raw[i].w[2 * j + 1]);
-                } else {
-                    unpack2<T>(raw[i].w[j], x0, x1);
-                }
-                uint64_t x = pack_f2(x0, x1);
-                uint64_t u;
-                if (own_sum) {
-                    if (!EXACT && !valid) x = 0ull;  // a padded row adds (+0, +0) to the sums; its codes are dropped
-                    u = code_pair<true>(x, m2[j], ns2[j], y2[j], magic, sum2[j]);
-                } else {
-                    u = code_pair<false>(x, m2[j], ns2[j], y2[j], magic, sum2[j]);
-                }
-                float u0, u1;
-                unpack_f2(u, u0, u1);
-                cw += __float_as_uint(u0) << (8 * j);
-                cw += __float_as_uint(u1) << (8 * j + 4);
+            for (int i = 0; i < W / 4; ++i) {
+                const uint4 v = *reinterpret_cast<const uint4 *>(p + 16 * i);
+                w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
             }
-            if (valid) dst[(int64_t)r * LPR] = cw;
         }
+    }
+    // channels 2j and 2j+1 as floats (exact)
+    __device__ __forceinline__ void pair(int j, float &a, float &b) const {
+        if constexpr (sizeof(T) == 4) {
+            a = __uint_as_float(w[2 * j]);
+            b = __uint_as_float(w[2 * j + 1]);
+        } else {
+            unpack2<T>(w[j], a, b);
+        }
+    }
+};
+
+template <int C>
+__device__ __forceinline__ void store_floats(float *dst, const float (&v)[C]) {
+    if constexpr (C == 2) {
+        *reinterpret_cast<float2 *>(dst) = make_float2(v[0], v[1]);
     } else {
 #pragma unroll
-        for (int i = 0; i < P; ++i) {
-            const int r = i * rpp + rbase;
-            const bool valid = EXACT || r < G;
-            uint32_t cw = 0;
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const float x = elem_of<T, W>(raw[i], j);
-                cw |= code_slow(x, m[j], s[j]) << (4 * j);
-                if (own_sum && valid) {
-                    float a0, a1;
-                    unpack_f2(sum2[j >> 1], a0, a1);
-                    if (j & 1) a1 += x; else a0 += x;
-                    sum2[j >> 1] = pack_f2(a0, a1);
-                }
-            }
-            if (valid) dst[(int64_t)r * LPR] = cw;
-        }
+        for (int i = 0; i < C; i += 4) *reinterpret_cast<float4 *>(dst + i) = make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]);
     }
-    if (!want_sum) return;  // block-uniform
+}
 
-    // ---- representative key: mean over the G tokens of the keys (or of the pre-rotary keys), |k-bar_h|^2
-    if (!own_sum) {
-        const T *ks = reinterpret_cast<const T *>(p.Ksum) + base;
+
+template <int C>
+__device__ __forceinline__ void store_codes(unsigned char *dst, uint32_t cw) {
+    if constexpr (C == 2) *dst = (unsigned char)cw;
+    else if constexpr (C == 4) *reinterpret_cast<uint16_t *>(dst) = (uint16_t)cw;
+    else *reinterpret_cast<uint32_t *>(dst) = cw;
+}
+
+// Pass 2 on the fast path: the codes of this lane's C channels for all G rows of a tile, written to the staging
+// tile; SUM also adds the rows up (keys: the representative key is their mean).
+template <typename T, int C, bool SUM>
+__device__ __forceinline__ void code_rows(const unsigned char *tile, unsigned char *out_lane, int G,
+                                          const uint64_t (&m2)[C / 2], const uint64_t (&ns2)[C / 2],
+                                          const uint64_t (&y2)[C / 2], uint64_t (&sum2)[C / 2]) {
+    constexpr int ROW_BYTES = 32 * C * (int)sizeof(T), CODE_ROW = 16 * C;
+    const uint64_t magic = pack_f2(12582912.0f, 12582912.0f);  // 1.5 * 2^23: rounds to integer, ties to even
+    // every float 1.5*2^23 + code has the bit pattern 0x4B400000 + code; summing pattern * 16^j over the lane's
+    // channels leaves the nibbles in place in the low 4*C bits (they cannot carry into each other); for C == 8
+    // the constant part wraps into the word and is removed up front
+    constexpr uint32_t kBias = C == 8 ? 0x4B400000u * 0x11111111u : 0u;
+    LaneRow<T, C> row;
+#pragma unroll 5
+    for (int r = 0; r < G; ++r) {
+        row.load(tile + r * ROW_BYTES);
+        uint32_t cw = 0u - kBias;
 #pragma unroll
-        for (int i = 0; i < P; ++i) {
-            const int r = i * rpp + rbase;
-            const Words<W> kr = load_words<W>(ks + row_off[i]);
-            if (EXACT || r < G) {
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    sum2[j] = add2(sum2[j], pack_f2(elem_of<T, W>(kr, 2 * j), elem_of<T, W>(kr, 2 * j + 1)));
-            }
+        for (int j = 0; j < C / 2; ++j) {
+            float x0, x1;
+            row.pair(j, x0, x1);
+            const uint64_t x = pack_f2(x0, x1);
+            if constexpr (SUM) sum2[j] = add2(sum2[j], x);
+            const uint64_t u = code_pair(x, m2[j], ns2[j], y2[j], magic);
+            float u0, u1;
+            unpack_f2(u, u0, u1);
+            cw += __float_as_uint(u0) << (8 * j);
+            cw += __float_as_uint(u1) << (8 * j + 4);
         }
+        store_codes<C>(out_lane + r * CODE_ROW, cw);
     }
-    float sum[8];
-#pragma unroll
-    for (int j = 0; j < 4; ++j) unpack_f2(sum2[j], sum[2 * j], sum[2 * j + 1]);
-#pragma unroll
-    for (int o = LPR; o < 32; o <<= 1) {
-#pragma unroll
-        for (int j = 0; j < 8; ++j) sum[j] += __shfl_xor_sync(0xffffffffu, sum[j], o);
-    }
-    if (sub == 0) {
-#pragma unroll
-        for (int j = 0; j < 8; j += 4)
-            *reinterpret_cast<float4 *>(&part_sum[warp][cl * 8 + j]) = make_float4(sum[j], sum[j + 1], sum[j + 2], sum[j + 3]);
+}
+
+// ------------------------------------------------------------------ tile bookkeeping
+
+struct TileCoord {
+    int kind, h, f, li;
+};
+__device__ __forceinline__ TileCoord tile_coord(uint32_t tau, const QuantParams &p) {
+    TileCoord t;
+    t.kind = (int)(tau % (uint32_t)p.n_kinds);
+    tau /= (uint32_t)p.n_kinds;
+    t.h = (int)(tau % (uint32_t)p.g.H);
+    tau /= (uint32_t)p.g.H;
+    t.f = (int)(tau % (uint32_t)p.F);
+    t.li = (int)(tau / (uint32_t)p.F);
+    return t;
+}
+
+// shared memory: [barriers: full[kMaxSlots], empty[kMaxSlots]] [abort word] [ring of input slots] [code staging]
+constexpr int kBarBytes = 2 * kMaxSlots * 8 + 128;  // barriers, then the abort word; rounded so the ring starts 128-aligned
+
+// C: channels per lane (d / 32).  blockDim.x = kQuantThreads, one block per SM, grid-stride over tiles.
+template <typename T, int C>
+__global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantParams p) {
+    constexpr int D = 32 * C;
+    constexpr int LANE_BYTES = C * (int)sizeof(T);  // bytes of a row that one lane owns
+    constexpr int ROW_BYTES = D * (int)sizeof(T);
+    constexpr int CODE_ROW = D / 2;                 // packed bytes per token row
+    extern __shared__ __align__(128) unsigned char smem[];
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + 2 * kMaxSlots * 8);
+    unsigned char *ring = smem + kBarBytes;
+    const int G = p.g.G, N = p.n_slots;
+    const uint32_t tile_bytes = (uint32_t)G * ROW_BYTES;
+    const uint32_t code_bytes = (uint32_t)G * CODE_ROW;
+    const uint32_t code_slot = (code_bytes + 127u) & ~127u;
+    unsigned char *stage = ring + (size_t)N * p.slot_bytes;  // [n_warps][code_slot]
+    // Tile n of the block goes to ring slot n % N and to consumer warp n % n_warps.  N is a multiple of n_warps, so
+    // a slot is always drained by the same warp, in order: that warp has seen fill k-1 of the slot complete before
+    // it waits for fill k, which is what makes waiting on a one-bit phase parity unambiguous.
+    const uint32_t WA = (uint32_t)p.n_warps;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + kMaxSlots * 8;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < N; ++i) {
+            mbar_init(full0 + 8 * i, 1);
+            mbar_init(empty0 + 8 * i, 1);
+        }
+        abort_flag[0] = 0;  // set by the first thread whose wait ran out
+        abort_flag[1] = 0;  // never set: lets the final drain wait regardless of an abort
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    if (warp == 0) {  // one warp finishes all D channels, so the norm needs no further block barrier
-        float n2 = 0.0f;
-        const float Gf = (float)G;
-#pragma unroll
-        for (int c = lane; c < D; c += 32) {
-            float sm = part_sum[0][c];
-            for (int w = 1; w < nwarps; ++w) sm += part_sum[w][c];
-            const float kb = __fdiv_rn(sm, Gf);
-            p.rep_key[slot * D + c] = kb;
-            n2 = fmaf(kb, kb, n2);
+
+    // tiles of this block: tau = blockIdx.x + n * gridDim.x, n = 0 .. my_count-1
+    const uint32_t my_count = p.n_tiles > blockIdx.x ? (p.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u;
+
+    if (warp == kConsumerWarps) {
+        // =============================================================== producer
+        uint32_t issued = 0;
+        for (uint32_t n = 0; n < my_count; ++n) {
+            const int slot = (int)(n % (uint32_t)N);
+            const uint32_t round = n / (uint32_t)N;
+            bool ok = true;
+            if (round > 0) ok = mbar_wait(empty0 + 8 * slot, (round - 1) & 1u, abort_flag);
+            ok = __all_sync(0xffffffffu, ok && !*abort_flag);  // the whole warp stops together
+            if (!ok) {
+                if (lane == 0) {
+                    if (!*abort_flag && p.flags) atomicOr(p.flags, STOM_FLAG_TIMEOUT);
+                    *abort_flag = 1;
+                }
+                break;
+            }
+            const TileCoord t = tile_coord(blockIdx.x + n * gridDim.x, p);
+            const T *src = reinterpret_cast<const T *>(t.kind == 0 ? p.K : (t.kind == 1 ? p.V : p.Ksum)) +
+                           (int64_t)t.li * p.sl + (int64_t)t.f * p.sg + (int64_t)t.h * p.sh;
+            const uint32_t bar = full0 + 8 * slot;
+            const uint32_t dst = smem_u32(ring + (size_t)slot * p.slot_bytes);
+            if (lane == 0) mbar_expect_tx(bar, tile_bytes);
+            __syncwarp();
+            if (p.contiguous) {
+                if (lane == 0) bulk_load(dst, src, tile_bytes, bar);
+            } else {
+                for (int r = lane; r < G; r += 32) {
+                    int tok = r;
+                    if (p.token_idx) {
+                        const int v = p.token_idx[(int64_t)t.f * G + r];
+                        if ((v < 0 || v >= p.n_in) && p.flags) atomicOr(p.flags, STOM_FLAG_BAD_INDEX);
+                        tok = min(max(v, 0), p.n_in - 1);
+                    }
+                    bulk_load(dst + (uint32_t)r * ROW_BYTES, src + (int64_t)tok * p.st, ROW_BYTES, bar);
+                }
+            }
+            issued = n + 1;
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, o);
-        if (lane == 0) p.rep_norm2[slot] = n2;
+        // nothing may still be landing in this block's shared memory when it exits: on the regular path every
+        // fill has been consumed already and these waits return at once
+        const uint32_t first = issued > (uint32_t)N ? issued - (uint32_t)N : 0u;
+        for (uint32_t n = first; n < issued; ++n)
+            mbar_wait(full0 + 8 * (int)(n % (uint32_t)N), (n / (uint32_t)N) & 1u, abort_flag + 1);
+        return;
     }
+
+    // =================================================================== consumers
+    if ((uint32_t)warp >= WA) return;
+    unsigned char *out = stage + (size_t)warp * code_slot;
+    for (uint32_t n = warp; n < my_count; n += WA) {
+        const int slot = (int)(n % (uint32_t)N);
+        bool ok = mbar_wait(full0 + 8 * slot, (n / (uint32_t)N) & 1u, abort_flag);
+        ok = __all_sync(0xffffffffu, ok && !*abort_flag);  // the whole warp stops together
+        if (!ok) {
+            if (lane == 0) {
+                if (!*abort_flag && p.flags) atomicOr(p.flags, STOM_FLAG_TIMEOUT);
+                *abort_flag = 1;
+            }
+            break;
+        }
+        const TileCoord t = tile_coord(blockIdx.x + n * gridDim.x, p);
+        const unsigned char *tile = ring + (size_t)slot * p.slot_bytes + lane * LANE_BYTES;
+        const int64_t bslot = bank_slot(p.g, p.layer_begin + t.li, p.group_begin + t.f, t.h);
+        const bool is_v = t.kind == 1;
+        const bool want_sum = t.kind == 2 || (t.kind == 0 && p.n_kinds == 2);  // warp-uniform
+
+        uint64_t sum2[C / 2];
+#pragma unroll
+        for (int j = 0; j < C / 2; ++j) sum2[j] = 0ull;  // (+0, +0)
+
+        if (t.kind != 2) {
+            // ---- pass 1: min / max of this lane's channels down the rows
+            LaneRow<T, C> row;
+            row.load(tile);
+            uint32_t mnw[LaneRow<T, C>::W], mxw[LaneRow<T, C>::W];
+#pragma unroll
+            for (int j = 0; j < LaneRow<T, C>::W; ++j) mnw[j] = mxw[j] = row.w[j];
+#pragma unroll 5
+            for (int r = 1; r < G; ++r) {
+                row.load(tile + r * ROW_BYTES);
+#pragma unroll
+                for (int j = 0; j < LaneRow<T, C>::W; ++j) {
+                    mnw[j] = WordOps<T>::vmin(mnw[j], row.w[j]);
+                    mxw[j] = WordOps<T>::vmax(mxw[j], row.w[j]);
+                }
+            }
+            // ---- statistics of the lane's C channels
+            float s[C], m[C], y[C];
+            bool safe = true;
+            {
+                LaneRow<T, C> a, b;
+#pragma unroll
+                for (int j = 0; j < LaneRow<T, C>::W; ++j) {
+                    a.w[j] = mnw[j];
+                    b.w[j] = mxw[j];
+                }
+#pragma unroll
+                for (int j = 0; j < C / 2; ++j) {
+                    float mx0, mx1;
+                    a.pair(j, m[2 * j], m[2 * j + 1]);
+                    b.pair(j, mx0, mx1);
+                    s[2 * j] = __fdiv_rn(__fsub_rn(mx0, m[2 * j]), 15.0f);
+                    s[2 * j + 1] = __fdiv_rn(__fsub_rn(mx1, m[2 * j + 1]), 15.0f);
+                }
+#pragma unroll
+                for (int c = 0; c < C; ++c) {
+                    safe &= (s[c] > 8.673617379884035e-19f) && (s[c] < 1.152921504606847e18f);  // (2^-60, 2^60)
+                    y[c] = __frcp_rn(s[c]);
+                }
+            }
+            store_floats<C>((is_v ? p.scale_v : p.scale_k) + bslot * D + lane * C, s);
+            store_floats<C>((is_v ? p.zero_v : p.zero_k) + bslot * D + lane * C, m);
+            safe = __all_sync(0xffffffffu, safe);
+
+            // the staging tile was handed to a bulk store at the end of this warp's previous tile
+            if (lane == 0) bulk_wait_read<0>();
+            __syncwarp();
+            unsigned char *out_lane = out + lane * (C / 2);
+
+            // ---- pass 2: codes (and, for keys, the channel sums of the rows as a by-product)
+            if (safe) {
+                uint64_t m2[C / 2], ns2[C / 2], y2[C / 2];
+#pragma unroll
+                for (int j = 0; j < C / 2; ++j) {
+                    m2[j] = pack_f2(m[2 * j], m[2 * j + 1]);
+                    ns2[j] = pack_f2(-s[2 * j], -s[2 * j + 1]);
+                    y2[j] = pack_f2(y[2 * j], y[2 * j + 1]);
+                }
+                if (want_sum) code_rows<T, C, true>(tile, out_lane, G, m2, ns2, y2, sum2);
+                else code_rows<T, C, false>(tile, out_lane, G, m2, ns2, y2, sum2);
+            } else {
+#pragma unroll 2
+                for (int r = 0; r < G; ++r) {
+                    row.load(tile + r * ROW_BYTES);
+                    uint32_t cw = 0;
+#pragma unroll
+                    for (int j = 0; j < C / 2; ++j) {
+                        float x0, x1;
+                        row.pair(j, x0, x1);
+                        if (want_sum) sum2[j] = add2(sum2[j], pack_f2(x0, x1));
+                        cw |= code_slow(x0, m[2 * j], s[2 * j]) << (8 * j);
+                        cw |= code_slow(x1, m[2 * j + 1], s[2 * j + 1]) << (8 * j + 4);
+                    }
+                    store_codes<C>(out_lane + r * CODE_ROW, cw);
+                }
+            }
+            // the input slot is free again; the finished code tile leaves with one bulk store
+            fence_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(empty0 + 8 * slot);
+                bulk_store((is_v ? p.codes_v : p.codes_k) + bslot * (int64_t)code_bytes, smem_u32(out), code_bytes);
+                bulk_commit();
+            }
+        } else {
+            // ---- pre-rotary keys: only their mean is wanted
+            LaneRow<T, C> row;
+#pragma unroll 5
+            for (int r = 0; r < G; ++r) {
+                row.load(tile + r * ROW_BYTES);
+#pragma unroll
+                for (int j = 0; j < C / 2; ++j) {
+                    float x0, x1;
+                    row.pair(j, x0, x1);
+                    sum2[j] = add2(sum2[j], pack_f2(x0, x1));
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + 8 * slot);
+        }
+
+        if (want_sum) {
+            // ---- representative key: mean over the G tokens, and |k-bar_h|^2 over the head's d channels
+            float kb[C];
+            const float Gf = (float)G;
+            float n2 = 0.0f;
+#pragma unroll
+            for (int j = 0; j < C / 2; ++j) {
+                float a, b;
+                unpack_f2(sum2[j], a, b);
+                kb[2 * j] = __fdiv_rn(a, Gf);
+                kb[2 * j + 1] = __fdiv_rn(b, Gf);
+            }
+#pragma unroll
+            for (int c = 0; c < C; ++c) n2 = fmaf(kb[c], kb[c], n2);
+            store_floats<C>(p.rep_key + bslot * D + lane * C, kb);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, o);
+            if (lane == 0) p.rep_norm2[bslot] = n2;
+        }
+    }
+    // the staging tiles must stay valid until the copy engine has read them
+    if (lane == 0) bulk_wait_all();
 }
 
-template <typename T, int LPR, int P>
-static void launch_exact(const QuantParams &p, dim3 grid, unsigned block, bool exact, cudaStream_t stream) {
-    if (exact) quantize_kernel<T, LPR, P, true><<<grid, block, 0, stream>>>(p);
-    else quantize_kernel<T, LPR, P, false><<<grid, block, 0, stream>>>(p);
-}
-
-template <typename T, int LPR>
-static int32_t launch_lpr(const QuantParams &p0, int layer_count, cudaStream_t stream) {
-    constexpr int RPW = 32 / LPR;
-    // block shape: the (warps, P) pair that covers G rows with the least padding, P <= 8; ties -> more warps
-    const int G = p0.g.G;
-    int best_w = kMaxWarps, best_p = 8, best_pad = 1 << 30;
-    for (int w = kMaxWarps; w >= 2; --w) {
-        const int P = (G + w * RPW - 1) / (w * RPW);
-        if (P > 8) continue;
-        const int pad = P * w * RPW - G;
-        if (pad < best_pad) {
-            best_pad = pad;
-            best_w = w;
-            best_p = P;
-        }
+template <typename T, int C>
+static int32_t launch_quantize(QuantParams p, cudaStream_t stream) {
+    int dev = 0, sms = 0, smem_max = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) {
+        set_last_cuda_error(e);
+        return STOM_ERR_CUDA;
     }
-    const unsigned block = best_w * 32;
-    const bool exact = best_pad == 0;
-    constexpr int kMaxY = 65535;  // grid.y limit: longer frame ranges are launched in slices
-    for (int f0 = 0; f0 < p0.F; f0 += kMaxY) {
-        QuantParams p = p0;
-        const int nf = p0.F - f0 < kMaxY ? p0.F - f0 : kMaxY;
-        const int64_t shift = (int64_t)f0 * p.sg * (int64_t)sizeof(T);
-        p.K = static_cast<const uint8_t *>(p.K) + shift;
-        p.V = static_cast<const uint8_t *>(p.V) + shift;
-        if (p.Ksum) p.Ksum = static_cast<const uint8_t *>(p.Ksum) + shift;
-        if (p.token_idx) p.token_idx += (int64_t)f0 * G;
-        p.group_begin += f0;
-        p.F = nf;
-        const dim3 grid(2 * p.g.H, nf, layer_count);
-        switch (best_p) {
-        case 1: launch_exact<T, LPR, 1>(p, grid, block, exact, stream); break;
-        case 2: launch_exact<T, LPR, 2>(p, grid, block, exact, stream); break;
-        case 3: launch_exact<T, LPR, 3>(p, grid, block, exact, stream); break;
-        case 4: launch_exact<T, LPR, 4>(p, grid, block, exact, stream); break;
-        case 5: launch_exact<T, LPR, 5>(p, grid, block, exact, stream); break;
-        case 6: launch_exact<T, LPR, 6>(p, grid, block, exact, stream); break;
-        case 7: launch_exact<T, LPR, 7>(p, grid, block, exact, stream); break;
-        default: launch_exact<T, LPR, 8>(p, grid, block, exact, stream); break;
-        }
-        const int32_t rc = finish_launch();
-        if (rc) return rc;
+    const int G = p.g.G, D = 32 * C;
+    const int tile_bytes = G * D * (int)sizeof(T);
+    p.slot_bytes = (tile_bytes + 127) & ~127;
+    const int code_slot = (G * D / 2 + 127) & ~127;
+    // Ring shape: `warps` consumer warps with `depth` slots each.  Two slots per warp (one being read, one
+    // loading) on as many warps as fit; big tiles fall back to one slot per warp; small tiles deepen the ring.
+    const int budget = smem_max - kBarBytes;
+    int depth = 2, warps = budget / (2 * p.slot_bytes + code_slot);
+    if (warps < 4) {
+        depth = 1;
+        warps = budget / (p.slot_bytes + code_slot);
     }
-    return STOM_OK;
+    if (warps > kConsumerWarps) warps = kConsumerWarps;
+    if (warps < 1) return STOM_ERR_SHAPE;
+    while ((depth + 1) * warps <= kMaxSlots && warps * ((depth + 1) * p.slot_bytes + code_slot) <= budget) ++depth;
+    p.n_warps = warps;
+    p.n_slots = depth * warps;
+    const int fixed = kBarBytes + warps * code_slot;
+    const int slots = p.n_slots;
+    const size_t smem = (size_t)fixed + (size_t)slots * p.slot_bytes;
+    e = cudaFuncSetAttribute(quantize_kernel<T, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) {
+        set_last_cuda_error(e);
+        return STOM_ERR_CUDA;
+    }
+    const unsigned grid = p.n_tiles < (uint32_t)sms ? p.n_tiles : (unsigned)sms;
+    quantize_kernel<T, C><<<grid, kQuantThreads, smem, stream>>>(p);
+    return finish_launch();
 }
 
 template <typename T>
-static int32_t launch_for_type(const QuantParams &p, int layer_count, cudaStream_t stream) {
+static int32_t launch_for_type(const QuantParams &p, cudaStream_t stream) {
     switch (p.g.d) {
-    case 64: return launch_lpr<T, 8>(p, layer_count, stream);
-    case 128: return launch_lpr<T, 16>(p, layer_count, stream);
-    case 256: return launch_lpr<T, 32>(p, layer_count, stream);
+    case 64: return launch_quantize<T, 2>(p, stream);
+    case 128: return launch_quantize<T, 4>(p, stream);
+    case 256: return launch_quantize<T, 8>(p, stream);
     default: return STOM_ERR_SHAPE;
     }
 }
@@ -455,7 +620,6 @@ extern "C" int32_t stom_oqm_quantize_frame(const stom_oqm_config *cfg, const sto
         !stride_ok(stride_token, dt))
         return STOM_ERR_ALIGNMENT;
     if (layer_count == 0 || group_count == 0) return STOM_OK;
-    if (layer_count > 65535 || 2 * cfg->n_kv_heads > 65535) return STOM_ERR_SHAPE;
 
     QuantParams p;
     p.K = K; p.V = V; p.Ksum = K_summary; p.token_idx = token_idx;
@@ -464,13 +628,35 @@ extern "C" int32_t stom_oqm_quantize_frame(const stom_oqm_config *cfg, const sto
     p.scale_k = store->scale_k; p.zero_k = store->zero_k; p.scale_v = store->scale_v; p.zero_v = store->zero_v;
     p.rep_key = store->rep_key; p.rep_norm2 = store->rep_norm2;
     p.g = bank_geom(cfg);
-    p.layer_begin = layer_begin; p.group_begin = group_begin; p.F = group_count; p.n_in = tokens_per_frame_in;
+    p.layer_begin = layer_begin; p.group_begin = group_begin; p.n_in = tokens_per_frame_in;
     p.flags = dev_flags;
-    p.n_tiles = (int64_t)layer_count * group_count * cfg->n_kv_heads * 2;
+    p.n_kinds = K_summary ? 3 : 2;
+    p.contiguous = (!token_idx && stride_token == cfg->head_dim) ? 1 : 0;
+    p.n_slots = 0; p.n_warps = 0; p.slot_bytes = 0;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    switch (dt) {
-    case STOM_BF16: return launch_for_type<__nv_bfloat16>(p, layer_count, s);
-    case STOM_FP16: return launch_for_type<__half>(p, layer_count, s);
-    default: return launch_for_type<float>(p, layer_count, s);
+
+    // one launch covers up to 2^30 tiles; longer frame ranges go out in slices
+    const int64_t per_frame = (int64_t)layer_count * cfg->n_kv_heads * p.n_kinds;
+    if (per_frame > (1 << 30)) return STOM_ERR_SHAPE;
+    const int64_t max_frames = (1 << 30) / per_frame;
+    const int eb = elem_bytes(dt);
+    for (int64_t f0 = 0; f0 < group_count; f0 += max_frames) {
+        QuantParams q = p;
+        const int64_t nf = group_count - f0 < max_frames ? group_count - f0 : max_frames;
+        const int64_t shift = f0 * stride_group * eb;
+        q.K = static_cast<const uint8_t *>(K) + shift;
+        q.V = static_cast<const uint8_t *>(V) + shift;
+        if (K_summary) q.Ksum = static_cast<const uint8_t *>(K_summary) + shift;
+        if (token_idx) q.token_idx = token_idx + f0 * cfg->group_tokens;
+        q.group_begin = group_begin + (int32_t)f0;
+        q.F = (int32_t)nf;
+        q.n_tiles = (uint32_t)(per_frame * nf);
+        switch (dt) {
+        case STOM_BF16: rc = launch_for_type<__nv_bfloat16>(q, s); break;
+        case STOM_FP16: rc = launch_for_type<__half>(q, s); break;
+        default: rc = launch_for_type<float>(q, s); break;
+        }
+        if (rc) return rc;
     }
+    return STOM_OK;
 }
