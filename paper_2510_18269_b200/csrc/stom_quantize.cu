@@ -269,10 +269,7 @@ __device__ __forceinline__ void code_rows(const unsigned char *tile, unsigned ch
     // channels leaves the nibbles in place in the low 4*C bits (they cannot carry into each other); for C == 8
     // the constant part wraps into the word and is removed up front
     constexpr uint32_t kBias = C == 8 ? 0x4B400000u * 0x11111111u : 0u;
-    LaneRow<T, C> row;
-#pragma unroll 5
-    for (int r = 0; r < G; ++r) {
-        row.load(tile + r * ROW_BYTES);
+    auto code_word = [&](const LaneRow<T, C> &row) -> uint32_t {
         uint32_t cw = 0u - kBias;
 #pragma unroll
         for (int j = 0; j < C / 2; ++j) {
@@ -286,7 +283,27 @@ __device__ __forceinline__ void code_rows(const unsigned char *tile, unsigned ch
             cw += __float_as_uint(u0) << (8 * j);
             cw += __float_as_uint(u1) << (8 * j + 4);
         }
-        store_codes<C>(out_lane + r * CODE_ROW, cw);
+        return cw;
+    };
+    // Rows go through in batches: all loads of a batch, then its arithmetic, then its stores.  The compiler cannot
+    // prove that the staging tile and the input tile do not overlap, so a load would never move above an earlier
+    // store; batching by hand gives it kBatch * C/2 independent division chains to interleave.
+    constexpr int kBatch = C == 8 ? 3 : 5;
+    int r = 0;
+    for (; r + kBatch <= G; r += kBatch) {
+        LaneRow<T, C> rows[kBatch];
+        uint32_t cw[kBatch];
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) rows[i].load(tile + (r + i) * ROW_BYTES);
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) cw[i] = code_word(rows[i]);
+#pragma unroll
+        for (int i = 0; i < kBatch; ++i) store_codes<C>(out_lane + (r + i) * CODE_ROW, cw[i]);
+    }
+    for (; r < G; ++r) {
+        LaneRow<T, C> row;
+        row.load(tile + r * ROW_BYTES);
+        store_codes<C>(out_lane + r * CODE_ROW, code_word(row));
     }
 }
 
@@ -306,8 +323,18 @@ __device__ __forceinline__ TileCoord tile_coord(uint32_t tau, const QuantParams 
     return t;
 }
 
-// shared memory: [barriers: full[kMaxSlots], empty[kMaxSlots]] [abort word] [ring of input slots] [code staging]
-constexpr int kBarBytes = 2 * kMaxSlots * 8 + 128;  // barriers, then the abort word; rounded so the ring starts 128-aligned
+// What the producer tells the consumer about the tile it put into a ring slot.
+struct SlotInfo {
+    int64_t bslot;  // index of (layer, group, head) in the bank
+    int32_t kind;   // 0 keys, 1 values, 2 pre-rotary keys
+    int32_t pad;
+};
+
+// shared memory: [full[kMaxSlots], empty[kMaxSlots]] [abort words] [SlotInfo[kMaxSlots]] [ring of input slots] [code staging]
+constexpr int kAbortOff = 2 * kMaxSlots * 8;
+constexpr int kInfoOff = 512;
+constexpr int kBarBytes = 1024;
+static_assert(kAbortOff + 8 <= kInfoOff && kInfoOff + kMaxSlots * (int)sizeof(SlotInfo) <= kBarBytes, "header layout");
 
 // C: channels per lane (d / 32).  blockDim.x = kQuantThreads, one block per SM, grid-stride over tiles.
 template <typename T, int C>
@@ -318,7 +345,8 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
     constexpr int CODE_ROW = D / 2;                 // packed bytes per token row
     extern __shared__ __align__(128) unsigned char smem[];
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem);
-    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + 2 * kMaxSlots * 8);
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + kAbortOff);
+    SlotInfo *info = reinterpret_cast<SlotInfo *>(smem + kInfoOff);
     unsigned char *ring = smem + kBarBytes;
     const int G = p.g.G, N = p.n_slots;
     const uint32_t tile_bytes = (uint32_t)G * ROW_BYTES;
@@ -349,41 +377,61 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
 
     if (warp == kConsumerWarps) {
         // =============================================================== producer
+        // Tile coordinates cost a few integer divisions.  One warp doing them tile after tile would cap the block
+        // at about one tile per thousand cycles, so the 32 lanes work out 32 consecutive tiles at once and hand
+        // the results round by shuffle.
         uint32_t issued = 0;
-        for (uint32_t n = 0; n < my_count; ++n) {
-            const int slot = (int)(n % (uint32_t)N);
-            const uint32_t round = n / (uint32_t)N;
-            bool ok = true;
-            if (round > 0) ok = mbar_wait(empty0 + 8 * slot, (round - 1) & 1u, abort_flag);
-            ok = __all_sync(0xffffffffu, ok && !*abort_flag);  // the whole warp stops together
-            if (!ok) {
-                if (lane == 0) {
-                    if (!*abort_flag && p.flags) atomicOr(p.flags, STOM_FLAG_TIMEOUT);
-                    *abort_flag = 1;
-                }
-                break;
-            }
-            const TileCoord t = tile_coord(blockIdx.x + n * gridDim.x, p);
-            const T *src = reinterpret_cast<const T *>(t.kind == 0 ? p.K : (t.kind == 1 ? p.V : p.Ksum)) +
-                           (int64_t)t.li * p.sl + (int64_t)t.f * p.sg + (int64_t)t.h * p.sh;
-            const uint32_t bar = full0 + 8 * slot;
-            const uint32_t dst = smem_u32(ring + (size_t)slot * p.slot_bytes);
-            if (lane == 0) mbar_expect_tx(bar, tile_bytes);
-            __syncwarp();
-            if (p.contiguous) {
-                if (lane == 0) bulk_load(dst, src, tile_bytes, bar);
-            } else {
-                for (int r = lane; r < G; r += 32) {
-                    int tok = r;
-                    if (p.token_idx) {
-                        const int v = p.token_idx[(int64_t)t.f * G + r];
-                        if ((v < 0 || v >= p.n_in) && p.flags) atomicOr(p.flags, STOM_FLAG_BAD_INDEX);
-                        tok = min(max(v, 0), p.n_in - 1);
+        bool stop = false;
+        for (uint32_t n0 = 0; n0 < my_count && !stop; n0 += 32) {
+            const uint32_t mine = n0 + lane < my_count ? n0 + lane : my_count - 1;
+            const TileCoord tl = tile_coord(blockIdx.x + mine * gridDim.x, p);
+            const unsigned long long src_l = reinterpret_cast<unsigned long long>(
+                reinterpret_cast<const T *>(tl.kind == 0 ? p.K : (tl.kind == 1 ? p.V : p.Ksum)) +
+                (int64_t)tl.li * p.sl + (int64_t)tl.f * p.sg + (int64_t)tl.h * p.sh);
+            const long long bslot_l = bank_slot(p.g, p.layer_begin + tl.li, p.group_begin + tl.f, tl.h);
+            const int cnt = (int)(my_count - n0 < 32u ? my_count - n0 : 32u);
+            for (int i = 0; i < cnt; ++i) {
+                const uint32_t n = n0 + i;
+                const int slot = (int)(n % (uint32_t)N);
+                const uint32_t round = n / (uint32_t)N;
+                bool ok = true;
+                if (round > 0) ok = mbar_wait(empty0 + 8 * slot, (round - 1) & 1u, abort_flag);
+                ok = __all_sync(0xffffffffu, ok && !*abort_flag);  // the whole warp stops together
+                if (!ok) {
+                    if (lane == 0) {
+                        if (!*abort_flag && p.flags) atomicOr(p.flags, STOM_FLAG_TIMEOUT);
+                        *abort_flag = 1;
                     }
-                    bulk_load(dst + (uint32_t)r * ROW_BYTES, src + (int64_t)tok * p.st, ROW_BYTES, bar);
+                    stop = true;
+                    break;
                 }
+                const T *src = reinterpret_cast<const T *>(__shfl_sync(0xffffffffu, src_l, i));
+                const long long bslot = __shfl_sync(0xffffffffu, bslot_l, i);
+                const int kind = __shfl_sync(0xffffffffu, tl.kind, i);
+                const int f = __shfl_sync(0xffffffffu, tl.f, i);
+                const uint32_t bar = full0 + 8 * slot;
+                const uint32_t dst = smem_u32(ring + (size_t)slot * p.slot_bytes);
+                if (lane == 0) {
+                    info[slot].bslot = bslot;  // published by the release of the arrive below
+                    info[slot].kind = kind;
+                    mbar_expect_tx(bar, tile_bytes);
+                }
+                __syncwarp();
+                if (p.contiguous) {
+                    if (lane == 0) bulk_load(dst, src, tile_bytes, bar);
+                } else {
+                    for (int r = lane; r < G; r += 32) {
+                        int tok = r;
+                        if (p.token_idx) {
+                            const int v = p.token_idx[(int64_t)f * G + r];
+                            if ((v < 0 || v >= p.n_in) && p.flags) atomicOr(p.flags, STOM_FLAG_BAD_INDEX);
+                            tok = min(max(v, 0), p.n_in - 1);
+                        }
+                        bulk_load(dst + (uint32_t)r * ROW_BYTES, src + (int64_t)tok * p.st, ROW_BYTES, bar);
+                    }
+                }
+                issued = n + 1;
             }
-            issued = n + 1;
         }
         // nothing may still be landing in this block's shared memory when it exits: on the regular path every
         // fill has been consumed already and these waits return at once
@@ -407,17 +455,17 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
             }
             break;
         }
-        const TileCoord t = tile_coord(blockIdx.x + n * gridDim.x, p);
         const unsigned char *tile = ring + (size_t)slot * p.slot_bytes + lane * LANE_BYTES;
-        const int64_t bslot = bank_slot(p.g, p.layer_begin + t.li, p.group_begin + t.f, t.h);
-        const bool is_v = t.kind == 1;
-        const bool want_sum = t.kind == 2 || (t.kind == 0 && p.n_kinds == 2);  // warp-uniform
+        const int64_t bslot = info[slot].bslot;
+        const int kind = info[slot].kind;
+        const bool is_v = kind == 1;
+        const bool want_sum = kind == 2 || (kind == 0 && p.n_kinds == 2);  // warp-uniform
 
         uint64_t sum2[C / 2];
 #pragma unroll
         for (int j = 0; j < C / 2; ++j) sum2[j] = 0ull;  // (+0, +0)
 
-        if (t.kind != 2) {
+        if (kind != 2) {
             // ---- pass 1: min / max of this lane's channels down the rows
             LaneRow<T, C> row;
             row.load(tile);
@@ -461,9 +509,7 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
             store_floats<C>((is_v ? p.zero_v : p.zero_k) + bslot * D + lane * C, m);
             safe = __all_sync(0xffffffffu, safe);
 
-            // the staging tile was handed to a bulk store at the end of this warp's previous tile
-            if (lane == 0) bulk_wait_read<0>();
-            __syncwarp();
+            __syncwarp();  // every lane has finished copying the previous code tile out of the staging tile
             unsigned char *out_lane = out + lane * (C / 2);
 
             // ---- pass 2: codes (and, for keys, the channel sums of the rows as a by-product)
@@ -493,13 +539,15 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
                     store_codes<C>(out_lane + r * CODE_ROW, cw);
                 }
             }
-            // the input slot is free again; the finished code tile leaves with one bulk store
-            fence_async_smem();
+            // the input slot is free again; the finished code tile (contiguous in the bank) leaves in 16-byte pieces
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(empty0 + 8 * slot);
-                bulk_store((is_v ? p.codes_v : p.codes_k) + bslot * (int64_t)code_bytes, smem_u32(out), code_bytes);
-                bulk_commit();
+            if (lane == 0) mbar_arrive(empty0 + 8 * slot);
+            {
+                uint4 *dst = reinterpret_cast<uint4 *>((is_v ? p.codes_v : p.codes_k) + bslot * (int64_t)code_bytes);
+                const uint4 *src = reinterpret_cast<const uint4 *>(out);
+                const int pieces = (int)(code_bytes >> 4);
+#pragma unroll 4
+                for (int i = lane; i < pieces; i += 32) dst[i] = src[i];
             }
         } else {
             // ---- pre-rotary keys: only their mean is wanted
@@ -538,8 +586,6 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
             if (lane == 0) p.rep_norm2[bslot] = n2;
         }
     }
-    // the staging tiles must stay valid until the copy engine has read them
-    if (lane == 0) bulk_wait_all();
 }
 
 template <typename T, int C>
