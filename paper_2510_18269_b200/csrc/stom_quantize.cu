@@ -3,24 +3,27 @@
 //
 // A tile is the G tokens x d channels of one (layer, frame, kv head) of K or
 // of V (12.8 KB at G = 50, d = 128, bf16).  The kernel is persistent: one
-// block per SM, kConsumerWarps consumer warps and one producer warp.
+// block per SM, up to kConsumerWarps consumer warps and one producer warp.
 //
 //   producer  walks the block's tiles in order and, for each, issues bulk
 //             asynchronous copies (cp.async.bulk, completion counted on an
 //             mbarrier) from global memory into the next free slot of a ring
-//             of shared-memory slots; a tile whose rows are contiguous is one
+//             of shared-memory slots that fills the SM's shared memory (18
+//             slots at 12.8 KB); a tile whose rows are contiguous is one
 //             copy, a strided or index-gathered tile is one copy per row.
-//             The ring keeps ~10 tiles per SM in flight, which is what hides
-//             HBM latency; no register is tied up by a load.
-//   consumer  warp w owns every kConsumerWarps-th tile of the block outright.
+//             Whatever is not being read by a consumer is in flight, which
+//             is what hides HBM latency; no register is tied up by a load.
+//   consumer  warp w takes every n_warps-th tile of the block outright.
 //             A lane owns d/32 adjacent channels of ALL G rows, so the
 //             per-channel statistics need no cross-lane traffic at all:
 //               pass 1  packed min / max down the rows (shared memory reads)
 //               stats   s = (max - min)/15, m = min, y = rn(1/s)   -> global
-//               pass 2  codes, two channels per instruction (f32x2), written
-//                       to a shared staging tile; key tiles add up the rows
-//                       for the representative key on the way
-//             and the finished code tile leaves with ONE bulk store.
+//               pass 2  codes, two channels per instruction (f32x2), stored
+//                       straight to the bank (a warp's store covers one
+//                       packed row); key tiles add up the rows for the
+//                       representative key on the way
+//             Sixteen such warps keep the issue slots busy while each one
+//             sits out the fixed latencies of its own division chains.
 //
 // Every wait on an mbarrier is bounded (wall-clock limit); a wait that runs
 // out sets STOM_FLAG_TIMEOUT, tells the rest of the block to stop, and the
@@ -41,9 +44,9 @@
 
 namespace stom {
 
-constexpr int kConsumerWarps = 8;
+constexpr int kConsumerWarps = 16;
 constexpr int kQuantThreads = (kConsumerWarps + 1) * 32;
-constexpr int kMaxSlots = 24;
+constexpr int kMaxSlots = 32;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s: far beyond any legitimate wait
 
 struct QuantParams {
@@ -57,8 +60,8 @@ struct QuantParams {
     uint32_t *flags;
     uint32_t n_tiles;     // layer_count * F * H * n_kinds, below 2^31
     int32_t n_kinds;      // 2: keys, values;  3: keys, values, pre-rotary keys (mean only)
-    int32_t n_slots;      // ring depth, a multiple of n_warps
-    int32_t n_warps;      // consumer warps that take tiles (the others leave at once)
+    int32_t n_slots;      // ring depth
+    int32_t n_warps;      // consumer warps that take tiles, at most n_slots (the others leave at once)
     int32_t slot_bytes;   // bytes of one input tile, rounded up to 128
     int32_t contiguous;   // rows of a tile are adjacent in global memory
 };
@@ -98,20 +101,6 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void *src, uint32_
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
-// shared -> global bulk copy, tracked by the issuing thread's bulk async-group
-__device__ __forceinline__ void bulk_store(void *dst, uint32_t src, uint32_t bytes) {
-    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(src), "r"(bytes)
-                 : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() {
-    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-// orders this thread's shared-memory writes before later reads by the asynchronous copy engine
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
 // Bounded wait.  Returns false when the limit ran out or another thread of the block gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag) {
     if (mbar_try_wait(bar, parity)) return true;
@@ -330,10 +319,10 @@ struct SlotInfo {
     int32_t pad;
 };
 
-// shared memory: [full[kMaxSlots], empty[kMaxSlots]] [abort words] [SlotInfo[kMaxSlots]] [ring of input slots] [code staging]
-constexpr int kAbortOff = 2 * kMaxSlots * 8;
-constexpr int kInfoOff = 512;
-constexpr int kBarBytes = 1024;
+// shared memory: [full[2][kMaxSlots], empty[kMaxSlots]] [abort words] [SlotInfo[kMaxSlots]] [ring of input slots]
+constexpr int kAbortOff = 3 * kMaxSlots * 8;
+constexpr int kInfoOff = 1024;
+constexpr int kBarBytes = 2048;
 static_assert(kAbortOff + 8 <= kInfoOff && kInfoOff + kMaxSlots * (int)sizeof(SlotInfo) <= kBarBytes, "header layout");
 
 // C: channels per lane (d / 32).  blockDim.x = kQuantThreads, one block per SM, grid-stride over tiles.
@@ -351,19 +340,22 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
     const int G = p.g.G, N = p.n_slots;
     const uint32_t tile_bytes = (uint32_t)G * ROW_BYTES;
     const uint32_t code_bytes = (uint32_t)G * CODE_ROW;
-    const uint32_t code_slot = (code_bytes + 127u) & ~127u;
-    unsigned char *stage = ring + (size_t)N * p.slot_bytes;  // [n_warps][code_slot]
-    // Tile n of the block goes to ring slot n % N and to consumer warp n % n_warps.  N is a multiple of n_warps, so
-    // a slot is always drained by the same warp, in order: that warp has seen fill k-1 of the slot complete before
-    // it waits for fill k, which is what makes waiting on a one-bit phase parity unambiguous.
+    // Tile n of the block goes to ring slot n % N and to consumer warp n % n_warps.  A slot has TWO "full" barriers
+    // used by alternate fills: a waiter only tells a barrier's phases apart by one parity bit, and with a single
+    // barrier a warp that runs ahead could take fill k-1 of its slot, still on its way, for fill k.  With two, the
+    // fill it could be confused with is k-2, which lies at least N tiles behind the oldest unfinished tile of the
+    // block once n_warps <= N, so it has long completed.  The producer waits on "empty" phases strictly in order,
+    // so one barrier per slot is enough there.
     const uint32_t WA = (uint32_t)p.n_warps;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const uint32_t full0 = smem_u32(bars), empty0 = full0 + kMaxSlots * 8;
+    const uint32_t full0 = smem_u32(bars), empty0 = full0 + 2 * kMaxSlots * 8;
+    auto full_bar = [&](int slot, uint32_t round) -> uint32_t { return full0 + 8 * ((round & 1u) * kMaxSlots + slot); };
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < N; ++i) {
             mbar_init(full0 + 8 * i, 1);
+            mbar_init(full0 + 8 * (kMaxSlots + i), 1);
             mbar_init(empty0 + 8 * i, 1);
         }
         abort_flag[0] = 0;  // set by the first thread whose wait ran out
@@ -381,6 +373,8 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
         // at about one tile per thousand cycles, so the 32 lanes work out 32 consecutive tiles at once and hand
         // the results round by shuffle.
         uint32_t issued = 0;
+        int slot = 0;
+        uint32_t round = 0;  // fill number of `slot`
         bool stop = false;
         for (uint32_t n0 = 0; n0 < my_count && !stop; n0 += 32) {
             const uint32_t mine = n0 + lane < my_count ? n0 + lane : my_count - 1;
@@ -392,8 +386,6 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
             const int cnt = (int)(my_count - n0 < 32u ? my_count - n0 : 32u);
             for (int i = 0; i < cnt; ++i) {
                 const uint32_t n = n0 + i;
-                const int slot = (int)(n % (uint32_t)N);
-                const uint32_t round = n / (uint32_t)N;
                 bool ok = true;
                 if (round > 0) ok = mbar_wait(empty0 + 8 * slot, (round - 1) & 1u, abort_flag);
                 ok = __all_sync(0xffffffffu, ok && !*abort_flag);  // the whole warp stops together
@@ -409,7 +401,7 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
                 const long long bslot = __shfl_sync(0xffffffffu, bslot_l, i);
                 const int kind = __shfl_sync(0xffffffffu, tl.kind, i);
                 const int f = __shfl_sync(0xffffffffu, tl.f, i);
-                const uint32_t bar = full0 + 8 * slot;
+                const uint32_t bar = full_bar(slot, round);
                 const uint32_t dst = smem_u32(ring + (size_t)slot * p.slot_bytes);
                 if (lane == 0) {
                     info[slot].bslot = bslot;  // published by the release of the arrive below
@@ -431,22 +423,28 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
                     }
                 }
                 issued = n + 1;
+                if (++slot == N) {
+                    slot = 0;
+                    ++round;
+                }
             }
         }
         // nothing may still be landing in this block's shared memory when it exits: on the regular path every
         // fill has been consumed already and these waits return at once
         const uint32_t first = issued > (uint32_t)N ? issued - (uint32_t)N : 0u;
-        for (uint32_t n = first; n < issued; ++n)
-            mbar_wait(full0 + 8 * (int)(n % (uint32_t)N), (n / (uint32_t)N) & 1u, abort_flag + 1);
+        for (uint32_t n = first; n < issued; ++n) {
+            const uint32_t rnd = n / (uint32_t)N;
+            mbar_wait(full_bar((int)(n % (uint32_t)N), rnd), (rnd >> 1) & 1u, abort_flag + 1);
+        }
         return;
     }
 
     // =================================================================== consumers
     if ((uint32_t)warp >= WA) return;
-    unsigned char *out = stage + (size_t)warp * code_slot;
+    int slot = warp;       // n_warps <= N
+    uint32_t round = 0;    // fill number of `slot` that holds tile n
     for (uint32_t n = warp; n < my_count; n += WA) {
-        const int slot = (int)(n % (uint32_t)N);
-        bool ok = mbar_wait(full0 + 8 * slot, (n / (uint32_t)N) & 1u, abort_flag);
+        bool ok = mbar_wait(full_bar(slot, round), (round >> 1) & 1u, abort_flag);
         ok = __all_sync(0xffffffffu, ok && !*abort_flag);  // the whole warp stops together
         if (!ok) {
             if (lane == 0) {
@@ -509,8 +507,7 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
             store_floats<C>((is_v ? p.zero_v : p.zero_k) + bslot * D + lane * C, m);
             safe = __all_sync(0xffffffffu, safe);
 
-            __syncwarp();  // every lane has finished copying the previous code tile out of the staging tile
-            unsigned char *out_lane = out + lane * (C / 2);
+            unsigned char *out_lane = (is_v ? p.codes_v : p.codes_k) + bslot * (int64_t)code_bytes + lane * (C / 2);
 
             // ---- pass 2: codes (and, for keys, the channel sums of the rows as a by-product)
             if (safe) {
@@ -539,16 +536,9 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
                     store_codes<C>(out_lane + r * CODE_ROW, cw);
                 }
             }
-            // the input slot is free again; the finished code tile (contiguous in the bank) leaves in 16-byte pieces
+            // the input slot is free again
             __syncwarp();
             if (lane == 0) mbar_arrive(empty0 + 8 * slot);
-            {
-                uint4 *dst = reinterpret_cast<uint4 *>((is_v ? p.codes_v : p.codes_k) + bslot * (int64_t)code_bytes);
-                const uint4 *src = reinterpret_cast<const uint4 *>(out);
-                const int pieces = (int)(code_bytes >> 4);
-#pragma unroll 4
-                for (int i = lane; i < pieces; i += 32) dst[i] = src[i];
-            }
         } else {
             // ---- pre-rotary keys: only their mean is wanted
             LaneRow<T, C> row;
@@ -585,6 +575,11 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
             for (int o = 16; o > 0; o >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, o);
             if (lane == 0) p.rep_norm2[bslot] = n2;
         }
+        slot += (int)WA;
+        if (slot >= N) {
+            slot -= N;
+            ++round;
+        }
     }
 }
 
@@ -601,22 +596,13 @@ static int32_t launch_quantize(QuantParams p, cudaStream_t stream) {
     const int G = p.g.G, D = 32 * C;
     const int tile_bytes = G * D * (int)sizeof(T);
     p.slot_bytes = (tile_bytes + 127) & ~127;
-    const int code_slot = (G * D / 2 + 127) & ~127;
-    // Ring shape: `warps` consumer warps with `depth` slots each.  Two slots per warp (one being read, one
-    // loading) on as many warps as fit; big tiles fall back to one slot per warp; small tiles deepen the ring.
-    const int budget = smem_max - kBarBytes;
-    int depth = 2, warps = budget / (2 * p.slot_bytes + code_slot);
-    if (warps < 4) {
-        depth = 1;
-        warps = budget / (p.slot_bytes + code_slot);
-    }
-    if (warps > kConsumerWarps) warps = kConsumerWarps;
-    if (warps < 1) return STOM_ERR_SHAPE;
-    while ((depth + 1) * warps <= kMaxSlots && warps * ((depth + 1) * p.slot_bytes + code_slot) <= budget) ++depth;
-    p.n_warps = warps;
-    p.n_slots = depth * warps;
-    const int fixed = kBarBytes + warps * code_slot;
-    const int slots = p.n_slots;
+    // the ring takes all the shared memory there is; consumer warps never outnumber its slots
+    int slots = (smem_max - kBarBytes) / p.slot_bytes;
+    if (slots > kMaxSlots) slots = kMaxSlots;
+    if (slots < 2) return STOM_ERR_SHAPE;
+    p.n_slots = slots;
+    p.n_warps = slots < kConsumerWarps ? slots : kConsumerWarps;
+    const int fixed = kBarBytes;
     const size_t smem = (size_t)fixed + (size_t)slots * p.slot_bytes;
     e = cudaFuncSetAttribute(quantize_kernel<T, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) {
