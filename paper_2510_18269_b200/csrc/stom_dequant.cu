@@ -2,13 +2,19 @@
 // Sec. 3.4: Q_4^{-1} = depack * s + m and KV_active = union of the selected
 // groups; appendix "Cache reconstruction for decoding").
 //
-// One warp owns one item = (layer, selected slot j, kv head, K|V): G rows of
-// d/2 packed bytes in, G rows of d 16-bit values out.  A lane owns 8 adjacent
-// channels: it keeps their 8 (s, m) pairs in registers for the whole group,
-// reads 4 bytes of codes per row and writes one 16-byte vector per row, so a
-// warp's store instruction covers 512 contiguous bytes of the active cache.
-// Output bytes are 3/4 of the traffic; code words of a whole group are
-// requested before the first one is used.
+// One warp owns one unit = half the token rows of (layer, selected slot j, kv
+// head, K|V): up to ceil(G/2) rows of d/2 packed bytes in, as many rows of d
+// 16-bit values out.  A lane owns 8 adjacent channels: it keeps their 8 (s, m)
+// pairs in registers for the whole unit, reads 4 bytes of codes per row and
+// writes one 16-byte vector per row, so a warp's store instruction covers 512
+// contiguous bytes of the active cache.  Output bytes are 3/4 of the traffic.
+// All code words of a unit are requested before the first one is used.
+//
+// A code nibble becomes a float without a conversion instruction: a byte
+// permute drops it into the low mantissa byte of 2^23, and subtracting 2^23
+// leaves the integer.  The subtraction and fmaf(code, s, m) run two channels
+// at a time (f32x2).  The arithmetic per element is exactly fmaf(code, s, m)
+// followed by one rounding to the output type.
 #include "stom_internal.cuh"
 
 namespace stom {
@@ -24,17 +30,39 @@ struct DequantParams {
     BankGeom g;
     int32_t layer_begin, k, n_groups, token_offset, per_head;
     uint32_t *flags;
-    int64_t n_items;
+    int64_t n_units;
 };
 
-template <typename OT>
+__device__ __forceinline__ uint64_t dq_pack(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void dq_unpack(uint64_t v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t dq_fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t dq_sub2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// LPR: lanes per token row (d / 8)
+template <typename OT, int LPR>
 __global__ void __launch_bounds__(kDqWarps * 32) dequant_gather_kernel(const DequantParams p) {
+    constexpr int RPP = 32 / LPR;          // rows one warp pass covers
+    constexpr int kDqMaxRows = 32 / RPP;   // passes that cover half of the largest group (G <= 64)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t item = (int64_t)blockIdx.x * kDqWarps + warp;
-    if (item >= p.n_items) return;
+    const int64_t unit = (int64_t)blockIdx.x * kDqWarps + warp;
+    if (unit >= p.n_units) return;
     const int G = p.g.G, H = p.g.H, d = p.g.d;
-    const int which = (int)(item & 1);
-    int64_t rest = item >> 1;
+    const int half = (int)(unit & 1), which = (int)((unit >> 1) & 1);
+    int64_t rest = unit >> 2;
     const int h = (int)(rest % H);
     rest /= H;
     const int j = (int)(rest % p.k);
@@ -46,52 +74,50 @@ __global__ void __launch_bounds__(kDqWarps * 32) dequant_gather_kernel(const Deq
         return;
     }
     const int64_t slot = bank_slot(p.g, p.layer_begin + li, t, h);
+    const int sub = lane / LPR;       // which row of a warp pass this lane serves
+    const int cl = lane - sub * LPR;  // channel block of this lane
+    const int g_half = (G + 1) >> 1;
+    const int r_begin = half ? g_half : 0, r_end = half ? G : g_half;
 
-    const int lpr = d >> 3;          // lanes per token row (8 channels each)
-    const int rpi = 32 / lpr;        // rows one warp pass covers
-    const int sub = lane / lpr;      // which of those rows this lane serves
-    const int cl = lane - sub * lpr; // channel block of this lane
-
-    float s[8], m[8];
+    // code words of all this lane's rows first, then the statistics
+    const uint32_t *codes = reinterpret_cast<const uint32_t *>((which ? p.codes_v : p.codes_k) +
+                                                               slot * (int64_t)G * p.g.row_bytes) + cl;
+    const int wpr = p.g.row_bytes >> 2;  // 32-bit words per packed row
+    uint32_t w[kDqMaxRows];
+#pragma unroll
+    for (int b = 0; b < kDqMaxRows; ++b) {
+        const int r = r_begin + sub + b * RPP;
+        w[b] = r < r_end ? __ldg(codes + (int64_t)r * wpr) : 0u;
+    }
+    uint64_t s2[4], m2[4];
     {
         const float4 *sp = reinterpret_cast<const float4 *>((which ? p.scale_v : p.scale_k) + slot * d + cl * 8);
         const float4 *mp = reinterpret_cast<const float4 *>((which ? p.zero_v : p.zero_k) + slot * d + cl * 8);
         const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1), m0 = __ldg(mp), m1 = __ldg(mp + 1);
-        s[0] = s0.x; s[1] = s0.y; s[2] = s0.z; s[3] = s0.w; s[4] = s1.x; s[5] = s1.y; s[6] = s1.z; s[7] = s1.w;
-        m[0] = m0.x; m[1] = m0.y; m[2] = m0.z; m[3] = m0.w; m[4] = m1.x; m[5] = m1.y; m[6] = m1.z; m[7] = m1.w;
+        s2[0] = dq_pack(s0.x, s0.y); s2[1] = dq_pack(s0.z, s0.w); s2[2] = dq_pack(s1.x, s1.y); s2[3] = dq_pack(s1.z, s1.w);
+        m2[0] = dq_pack(m0.x, m0.y); m2[1] = dq_pack(m0.z, m0.w); m2[2] = dq_pack(m1.x, m1.y); m2[3] = dq_pack(m1.z, m1.w);
     }
-    const uint32_t *codes = reinterpret_cast<const uint32_t *>((which ? p.codes_v : p.codes_k) +
-                                                               slot * (int64_t)G * p.g.row_bytes) + cl;
-    const int wpr = p.g.row_bytes >> 2;  // 32-bit words per packed row
     OT *out = reinterpret_cast<OT *>(which ? p.va : p.ka) + (int64_t)li * p.sl + (int64_t)h * p.sh +
               ((int64_t)p.token_offset + (int64_t)j * G) * p.st + cl * 8;
-
-    constexpr int kBatch = 8;  // rows whose code words are in flight together, per lane
-    for (int r0 = sub; r0 < G; r0 += rpi * kBatch) {
-        uint32_t w[kBatch];
+    const uint64_t two23 = dq_pack(8388608.0f, 8388608.0f);
 #pragma unroll
-        for (int b = 0; b < kBatch; ++b) {
-            const int r = r0 + b * rpi;
-            if (r < G) w[b] = __ldg(codes + (int64_t)r * wpr);
-        }
+    for (int b = 0; b < kDqMaxRows; ++b) {
+        const int r = r_begin + sub + b * RPP;
+        if (r < r_end) {
+            const uint32_t even = w[b] & 0x0f0f0f0fu;         // byte i: code of channel 2i
+            const uint32_t odd = (w[b] >> 4) & 0x0f0f0f0fu;   // byte i: code of channel 2i+1
+            uint32_t o[4];
 #pragma unroll
-        for (int b = 0; b < kBatch; ++b) {
-            const int r = r0 + b * rpi;
-            if (r < G) {
-                float v[8];
-#pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    // 2^23 + nibble as a float, minus 2^23: exact integer-to-float without a conversion
-                    const float code = __uint_as_float(0x4B000000u | ((w[b] >> (4 * c)) & 15u)) - 8388608.0f;
-                    v[c] = __fmaf_rn(code, s[c], m[c]);
-                }
-                uint4 o;
-                o.x = pack2<OT>(v[0], v[1]);
-                o.y = pack2<OT>(v[2], v[3]);
-                o.z = pack2<OT>(v[4], v[5]);
-                o.w = pack2<OT>(v[6], v[7]);
-                *reinterpret_cast<uint4 *>(out + (int64_t)r * p.st) = o;
+            for (int i = 0; i < 4; ++i) {
+                // 2^23 + code as a float: the code byte goes into the low mantissa byte of 0x4B000000
+                const uint32_t fe = __byte_perm(even, 0x4B000000u, 0x7540u + i);
+                const uint32_t fo = __byte_perm(odd, 0x4B000000u, 0x7540u + i);
+                const uint64_t code = dq_sub2(dq_pack(__uint_as_float(fe), __uint_as_float(fo)), two23);
+                float v0, v1;
+                dq_unpack(dq_fma2(code, s2[i], m2[i]), v0, v1);
+                o[i] = pack2<OT>(v0, v1);
             }
+            *reinterpret_cast<uint4 *>(out + (int64_t)r * p.st) = make_uint4(o[0], o[1], o[2], o[3]);
         }
     }
 }
@@ -129,13 +155,26 @@ extern "C" int32_t stom_oqm_dequant_gather(const stom_oqm_config *cfg, const sto
     p.layer_begin = layer_begin; p.k = k; p.n_groups = n_groups; p.token_offset = token_offset;
     p.per_head = cfg->score_mode == STOM_SCORE_PER_HEAD;
     p.flags = dev_flags;
-    p.n_items = (int64_t)layer_count * k * cfg->n_kv_heads * 2;
-    const int64_t blocks = (p.n_items + kDqWarps - 1) / kDqWarps;
+    p.n_units = (int64_t)layer_count * k * cfg->n_kv_heads * 4;  // x (keys | values) x (first | second half of the rows)
+    const int64_t blocks = (p.n_units + kDqWarps - 1) / kDqWarps;
     if (blocks > 0x7fffffffLL) return STOM_ERR_SHAPE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (out_dtype == STOM_BF16)
-        dequant_gather_kernel<__nv_bfloat16><<<(unsigned)blocks, kDqWarps * 32, 0, s>>>(p);
-    else
-        dequant_gather_kernel<__half><<<(unsigned)blocks, kDqWarps * 32, 0, s>>>(p);
+    const unsigned nb = (unsigned)blocks, nt = kDqWarps * 32;
+    const bool bf = out_dtype == STOM_BF16;
+    switch (cfg->head_dim) {
+    case 64:
+        if (bf) dequant_gather_kernel<__nv_bfloat16, 8><<<nb, nt, 0, s>>>(p);
+        else dequant_gather_kernel<__half, 8><<<nb, nt, 0, s>>>(p);
+        break;
+    case 128:
+        if (bf) dequant_gather_kernel<__nv_bfloat16, 16><<<nb, nt, 0, s>>>(p);
+        else dequant_gather_kernel<__half, 16><<<nb, nt, 0, s>>>(p);
+        break;
+    case 256:
+        if (bf) dequant_gather_kernel<__nv_bfloat16, 32><<<nb, nt, 0, s>>>(p);
+        else dequant_gather_kernel<__half, 32><<<nb, nt, 0, s>>>(p);
+        break;
+    default: return STOM_ERR_SHAPE;
+    }
     return finish_launch();
 }

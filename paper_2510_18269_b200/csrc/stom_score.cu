@@ -24,41 +24,148 @@ struct ScoreParams {
     float *qnorm2;  // workspace: [layer_count][H]
     float *scores;
     BankGeom g;
-    int32_t layer_begin, layer_count, n_groups, T_q, rep, per_head;
+    int32_t layer_begin, layer_count, n_groups, T_q, rep, per_head, groups_per_block;
 };
 
-// grid (H, layer_count), block d threads: thread c owns channel c of kv head h
+constexpr int kEmbedThreads = 256;
+
+// Question embedding of one (layer, kv head): mean over the rep query heads of the GQA block and over the T_q
+// question tokens.  grid (H, layer_count), kEmbedThreads threads.  The rows (rep * T_q of them) are dealt to
+// RG = kEmbedThreads / (d/4) row groups; a thread adds up 4 adjacent channels of its group's rows and shared
+// memory combines the groups.
 template <typename T>
-__global__ void query_embed_kernel(const ScoreParams p) {
-    const int h = blockIdx.x, li = blockIdx.y, c = threadIdx.x, d = p.g.d;
-    const T *q = reinterpret_cast<const T *>(p.Q) + (int64_t)li * p.ql + c;
-    float acc = 0.0f;
-    for (int r = 0; r < p.rep; ++r) {
-        const T *qh = q + (int64_t)(h * p.rep + r) * p.qh;
-        float part = 0.0f;
-        for (int j = 0; j < p.T_q; ++j) part += (float)qh[(int64_t)j * p.qt];
-        acc += part;
+__global__ void __launch_bounds__(kEmbedThreads) query_embed_kernel(const ScoreParams p) {
+    __shared__ float part[kEmbedThreads / 16][256 + 4];  // [row group <= 16][channel <= 256]
+    __shared__ float red[kEmbedThreads / 32];
+    const int h = blockIdx.x, li = blockIdx.y, d = p.g.d;
+    const int lanes_per_row = d >> 2;                 // threads across one row (4 channels each): 16, 32 or 64
+    const int RG = kEmbedThreads / lanes_per_row;     // row groups: 16, 8 or 4
+    const int cq = threadIdx.x % lanes_per_row, rg = threadIdx.x / lanes_per_row;
+    const int rows = p.rep * p.T_q;
+    const T *q = reinterpret_cast<const T *>(p.Q) + (int64_t)li * p.ql + cq * 4;
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    for (int r = rg; r < rows; r += RG) {
+        const int hq = h * p.rep + r / p.T_q, j = r - (r / p.T_q) * p.T_q;
+        const T *src = q + (int64_t)hq * p.qh + (int64_t)j * p.qt;
+        if constexpr (sizeof(T) == 4) {
+            const float4 v = __ldg(reinterpret_cast<const float4 *>(src));
+            a0 += v.x; a1 += v.y; a2 += v.z; a3 += v.w;
+        } else {
+            const uint2 v = __ldg(reinterpret_cast<const uint2 *>(src));
+            float x0, x1, x2, x3;
+            unpack2<T>(v.x, x0, x1);
+            unpack2<T>(v.y, x2, x3);
+            a0 += x0; a1 += x1; a2 += x2; a3 += x3;
+        }
     }
-    const float v = acc / (float)(p.rep * p.T_q);
-    p.qemb[((int64_t)li * p.g.H + h) * d + c] = v;
+    float *mine = &part[rg][cq * 4];
+    mine[0] = a0; mine[1] = a1; mine[2] = a2; mine[3] = a3;
+    __syncthreads();
+    float sq = 0.0f;
+    if (threadIdx.x < d) {
+        const int c = threadIdx.x;
+        float acc = 0.0f;
+        for (int g = 0; g < RG; ++g) acc += part[g][c];
+        const float v = acc / (float)rows;
+        p.qemb[((int64_t)li * p.g.H + h) * d + c] = v;
+        sq = v * v;
+    }
     // |q_h|^2 by block reduction
-    __shared__ float red[8];
-    float sq = v * v;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
-    if ((c & 31) == 0) red[c >> 5] = sq;
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sq;
     __syncthreads();
-    if (c == 0) {
+    if (threadIdx.x == 0) {
         float tot = 0.0f;
-        for (int w = 0; w < (d >> 5); ++w) tot += red[w];
+        for (int w = 0; w < kEmbedThreads / 32; ++w) tot += red[w];
         p.qnorm2[(int64_t)li * p.g.H + h] = tot;
     }
 }
 
 constexpr int kScoreWarps = 8;
-constexpr int kGroupsPerWarp = 4;  // groups a warp scores one after the other per block
+constexpr int kGroupsPerWarp = 2;  // groups a warp scores together
 
-// grid (ceil(n_groups / (kScoreWarps*kGroupsPerWarp)), layer_count)
+// One warp, a strided share of the block's groups [t_begin, t_end) of one layer, kGroupsPerWarp at a time.  The
+// loads of the next pair are issued before the current pair is reduced, so a warp always has 2 pairs of k-bar
+// vectors in flight.  V4: float4 words of the flattened k-bar that one lane covers (H*d / 128).
+template <int V4>
+__device__ __forceinline__ void score_groups_per_layer(const ScoreParams &p, const float *sq, const float *qn, int li,
+                                                       int t_begin, int t_end, int warp, int lane) {
+    const int H = p.g.H, d = p.g.d, l = p.layer_begin + li;
+    float4 q4[V4];
+#pragma unroll
+    for (int i = 0; i < V4; ++i) q4[i] = reinterpret_cast<const float4 *>(sq)[lane + 32 * i];
+    float qq = lane < H ? qn[lane] : 0.0f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) qq += __shfl_xor_sync(0xffffffffu, qq, o);
+    const float qnorm = fmaxf(sqrtf(qq), 1e-12f);
+
+    auto load = [&](int t0, float4 (&kv)[kGroupsPerWarp][V4], float (&kn)[kGroupsPerWarp]) {
+#pragma unroll
+        for (int u = 0; u < kGroupsPerWarp; ++u) {
+            const int t = min(t0 + u, t_end - 1);  // a pair that sticks out re-reads the last group; dropped at the store
+            const int64_t slot = bank_slot(p.g, l, t, 0);
+            const float4 *kb = reinterpret_cast<const float4 *>(p.rep_key + slot * d);
+#pragma unroll
+            for (int i = 0; i < V4; ++i) kv[u][i] = __ldg(kb + lane + 32 * i);
+            kn[u] = lane < H ? __ldg(p.rep_norm2 + slot + lane) : 0.0f;
+        }
+    };
+    const int step = kScoreWarps * kGroupsPerWarp;
+    int t0 = t_begin + warp * kGroupsPerWarp;
+    if (t0 >= t_end) return;
+    float4 cur[kGroupsPerWarp][V4], nxt[kGroupsPerWarp][V4];
+    float kn_cur[kGroupsPerWarp], kn_nxt[kGroupsPerWarp];
+    load(t0, cur, kn_cur);
+    for (; t0 < t_end; t0 += step) {
+        const bool more = t0 + step < t_end;
+        if (more) load(t0 + step, nxt, kn_nxt);
+        float dot[kGroupsPerWarp];
+#pragma unroll
+        for (int u = 0; u < kGroupsPerWarp; ++u) {
+            float a = 0.0f;
+#pragma unroll
+            for (int i = 0; i < V4; ++i) {
+                a = fmaf(cur[u][i].x, q4[i].x, a);
+                a = fmaf(cur[u][i].y, q4[i].y, a);
+                a = fmaf(cur[u][i].z, q4[i].z, a);
+                a = fmaf(cur[u][i].w, q4[i].w, a);
+            }
+            dot[u] = a;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+            for (int u = 0; u < kGroupsPerWarp; ++u) {
+                dot[u] += __shfl_xor_sync(0xffffffffu, dot[u], o);
+                kn_cur[u] += __shfl_xor_sync(0xffffffffu, kn_cur[u], o);
+            }
+        }
+        if (lane < kGroupsPerWarp && t0 + lane < t_end) {
+            float dsel = dot[0], ksel = kn_cur[0];
+#pragma unroll
+            for (int u = 1; u < kGroupsPerWarp; ++u) {
+                if (lane == u) {
+                    dsel = dot[u];
+                    ksel = kn_cur[u];
+                }
+            }
+            p.scores[(int64_t)li * p.n_groups + t0 + lane] = dsel / (qnorm * fmaxf(sqrtf(ksel), 1e-12f));
+        }
+        if (more) {
+#pragma unroll
+            for (int u = 0; u < kGroupsPerWarp; ++u) {
+                kn_cur[u] = kn_nxt[u];
+#pragma unroll
+                for (int i = 0; i < V4; ++i) cur[u][i] = nxt[u][i];
+            }
+        }
+    }
+}
+
+// grid (chunks, layer_count): block x scores groups [x * groups_per_block, (x+1) * groups_per_block) of its layer.
+// V4 > 0: PER_LAYER scoring with H*d == 128 * V4 and H <= 32 (the software-pipelined loop); V4 == 0: everything else.
+template <int V4>
 __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(const ScoreParams p) {
     extern __shared__ __align__(16) float sq[];  // q of this layer: H*d floats, then H norms
     const int li = blockIdx.y, H = p.g.H, d = p.g.d, HD = H * d;
@@ -70,11 +177,14 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(const ScorePara
 
     const int l = p.layer_begin + li;
     const float eps = 1e-12f;
-    const int t0 = (blockIdx.x * kScoreWarps + warp) * kGroupsPerWarp;
+    const int t_begin = blockIdx.x * p.groups_per_block;
+    const int t_end = min(t_begin + p.groups_per_block, p.n_groups);
+    if constexpr (V4 > 0) {
+        score_groups_per_layer<V4>(p, sq, qn, li, t_begin, t_end, warp, lane);
+        return;
+    }
 #pragma unroll 1
-    for (int u = 0; u < kGroupsPerWarp; ++u) {
-        const int t = t0 + u;
-        if (t >= p.n_groups) break;
+    for (int t = t_begin + warp; t < t_end; t += kScoreWarps) {
         const int64_t slot = bank_slot(p.g, l, t, 0);
         const float4 *kb = reinterpret_cast<const float4 *>(p.rep_key + slot * d);
         if (!p.per_head) {
@@ -148,7 +258,9 @@ extern "C" int32_t stom_oqm_score_groups(const stom_oqm_config *cfg, const stom_
     if (q_stride_layer < 0 || q_stride_head < 0 || q_stride_token < 0) return STOM_ERR_INVALID_ARG;
     if (!workspace || !aligned16(workspace) || workspace_bytes < stom_oqm_score_workspace_bytes(cfg, layer_count))
         return STOM_ERR_WORKSPACE;
-    if (reinterpret_cast<uintptr_t>(Q) % elem_bytes(cfg->kv_dtype) || (reinterpret_cast<uintptr_t>(scores) & 3u))
+    if (!aligned16(Q) || (reinterpret_cast<uintptr_t>(scores) & 3u)) return STOM_ERR_ALIGNMENT;
+    if (!stride_ok(q_stride_layer, cfg->kv_dtype) || !stride_ok(q_stride_head, cfg->kv_dtype) ||
+        !stride_ok(q_stride_token, cfg->kv_dtype))
         return STOM_ERR_ALIGNMENT;
     if (layer_count == 0 || n_groups == 0) return STOM_OK;
 
@@ -166,16 +278,33 @@ extern "C" int32_t stom_oqm_score_groups(const stom_oqm_config *cfg, const stom_
 
     dim3 g1(cfg->n_kv_heads, layer_count);
     switch (cfg->kv_dtype) {
-    case STOM_BF16: query_embed_kernel<__nv_bfloat16><<<g1, cfg->head_dim, 0, s>>>(p); break;
-    case STOM_FP16: query_embed_kernel<__half><<<g1, cfg->head_dim, 0, s>>>(p); break;
-    default: query_embed_kernel<float><<<g1, cfg->head_dim, 0, s>>>(p); break;
+    case STOM_BF16: query_embed_kernel<__nv_bfloat16><<<g1, kEmbedThreads, 0, s>>>(p); break;
+    case STOM_FP16: query_embed_kernel<__half><<<g1, kEmbedThreads, 0, s>>>(p); break;
+    default: query_embed_kernel<float><<<g1, kEmbedThreads, 0, s>>>(p); break;
     }
     if ((rc = finish_launch())) return rc;
 
-    const int per_block = kScoreWarps * kGroupsPerWarp;
-    dim3 g2((n_groups + per_block - 1) / per_block, layer_count);
+    // about eight blocks per SM over the whole grid, each with a contiguous run of groups (at least 32)
+    int dev = 0, sms = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) {
+        set_last_cuda_error(e);
+        return STOM_ERR_CUDA;
+    }
+    int chunks = (8 * sms + layer_count - 1) / layer_count;
+    if (chunks > (n_groups + 31) / 32) chunks = (n_groups + 31) / 32;
+    if (chunks < 1) chunks = 1;
+    p.groups_per_block = (n_groups + chunks - 1) / chunks;
+    dim3 g2((n_groups + p.groups_per_block - 1) / p.groups_per_block, layer_count);
     const size_t smem = (size_t)cfg->n_kv_heads * (cfg->head_dim + 1) * sizeof(float);
-    score_kernel<<<g2, kScoreWarps * 32, smem, s>>>(p);
+    const int HD = cfg->n_kv_heads * cfg->head_dim;
+    const bool fast = !p.per_head && cfg->n_kv_heads <= 32;
+    if (fast && HD == 512) score_kernel<4><<<g2, kScoreWarps * 32, smem, s>>>(p);        // 4 kv heads x 128
+    else if (fast && HD == 1024) score_kernel<8><<<g2, kScoreWarps * 32, smem, s>>>(p);  // 8 kv heads x 128
+    else if (fast && HD == 256) score_kernel<2><<<g2, kScoreWarps * 32, smem, s>>>(p);
+    else if (fast && HD == 128) score_kernel<1><<<g2, kScoreWarps * 32, smem, s>>>(p);
+    else score_kernel<0><<<g2, kScoreWarps * 32, smem, s>>>(p);
     return finish_launch();
 }
 

@@ -59,26 +59,55 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkParams p) 
         else return score_key(__ldg(sc + i));
     };
 
-    // ---- radix select of the ksel-th largest key
+    // ---- radix select of the ksel-th largest key: 4 passes of 8 bits.  Scores of one row share their leading bits,
+    //      so a plain histogram would serialise thousands of atomics on a handful of bins: lanes that hit the same bin
+    //      are merged first (match) and one of them adds their count.  The bin in which the running count from the top
+    //      reaches `need` is then found by one warp: a lane owns 8 bins, suffix sums go round by shuffle.
     uint32_t prefix = 0, mask = 0, need = (uint32_t)ksel;
+    const int lane_ = tid & 31;
     for (int shift = 24; shift >= 0; shift -= 8) {
         if (tid < 256) hist[tid] = 0;
         __syncthreads();
-        for (int i = tid; i < n; i += kTopkThreads) {
-            const uint32_t key = key_at(i);
-            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        for (int i0 = 0; i0 < n; i0 += kTopkThreads) {
+            const int i = i0 + tid;
+            uint32_t key = 0;
+            bool in = i < n;
+            if (in) {
+                key = key_at(i);
+                in = (key & mask) == prefix;
+            }
+            const uint32_t live = __ballot_sync(0xffffffffu, in);
+            if (in) {
+                const uint32_t bin = (key >> shift) & 255u;
+                const uint32_t peers = __match_any_sync(live, bin);
+                if (lane_ == __ffs(peers) - 1) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
+            }
         }
         __syncthreads();
-        if (tid == 0) {
-            uint32_t left = need;
-            int b = 255;
-            for (; b > 0; --b) {
-                const uint32_t c = hist[b];
-                if (c >= left) break;
-                left -= c;
+        if (tid < 32) {
+            uint32_t c[8], tot = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                c[j] = hist[tid * 8 + j];
+                tot += c[j];
             }
-            s_prefix = prefix | ((uint32_t)b << shift);
-            s_need = left;
+            uint32_t suf = tot;  // becomes the count in this lane's bins and all higher ones
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t v = __shfl_down_sync(0xffffffffu, suf, o);
+                if (tid + o < 32) suf += v;
+            }
+            const uint32_t above = suf - tot;
+            if (above < need && need <= suf) {  // exactly one lane: 1 <= need <= number of candidates
+                uint32_t left = need - above;
+                int j = 7;
+                for (; j > 0; --j) {
+                    if (c[j] >= left) break;
+                    left -= c[j];
+                }
+                s_prefix = prefix | ((uint32_t)(tid * 8 + j) << shift);
+                s_need = left;
+            }
         }
         __syncthreads();
         prefix = s_prefix;
