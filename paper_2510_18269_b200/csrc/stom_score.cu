@@ -44,18 +44,30 @@ __global__ void __launch_bounds__(kEmbedThreads) query_embed_kernel(const ScoreP
     const int rows = p.rep * p.T_q;
     const T *q = reinterpret_cast<const T *>(p.Q) + (int64_t)li * p.ql + cq * 4;
     float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    for (int r = rg; r < rows; r += RG) {
-        const int hq = h * p.rep + r / p.T_q, j = r - (r / p.T_q) * p.T_q;
-        const T *src = q + (int64_t)hq * p.qh + (int64_t)j * p.qt;
-        if constexpr (sizeof(T) == 4) {
-            const float4 v = __ldg(reinterpret_cast<const float4 *>(src));
-            a0 += v.x; a1 += v.y; a2 += v.z; a3 += v.w;
-        } else {
-            const uint2 v = __ldg(reinterpret_cast<const uint2 *>(src));
-            float x0, x1, x2, x3;
-            unpack2<T>(v.x, x0, x1);
-            unpack2<T>(v.y, x2, x3);
-            a0 += x0; a1 += x1; a2 += x2; a3 += x3;
+    // rows in batches of kRowBatch: all loads of a batch are issued before the first add
+    constexpr int kRowBatch = 8;
+    for (int r0 = rg; r0 < rows; r0 += RG * kRowBatch) {
+        float x[kRowBatch][4];
+#pragma unroll
+        for (int b = 0; b < kRowBatch; ++b) {
+            const int r = r0 + b * RG;
+            x[b][0] = x[b][1] = x[b][2] = x[b][3] = 0.0f;
+            if (r < rows) {
+                const int hr = r / p.T_q, j = r - hr * p.T_q;
+                const T *src = q + (int64_t)(h * p.rep + hr) * p.qh + (int64_t)j * p.qt;
+                if constexpr (sizeof(T) == 4) {
+                    const float4 v = __ldg(reinterpret_cast<const float4 *>(src));
+                    x[b][0] = v.x; x[b][1] = v.y; x[b][2] = v.z; x[b][3] = v.w;
+                } else {
+                    const uint2 v = __ldg(reinterpret_cast<const uint2 *>(src));
+                    unpack2<T>(v.x, x[b][0], x[b][1]);
+                    unpack2<T>(v.y, x[b][2], x[b][3]);
+                }
+            }
+        }
+#pragma unroll
+        for (int b = 0; b < kRowBatch; ++b) {
+            a0 += x[b][0]; a1 += x[b][1]; a2 += x[b][2]; a3 += x[b][3];
         }
     }
     float *mine = &part[rg][cq * 4];
@@ -184,7 +196,7 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(const ScorePara
         return;
     }
 #pragma unroll 1
-    for (int t = t_begin + warp; t < t_end; t += kScoreWarps) {
+    for (int t = t_begin + (V4 > 0 ? t_end : warp); t < t_end; t += kScoreWarps) {
         const int64_t slot = bank_slot(p.g, l, t, 0);
         const float4 *kb = reinterpret_cast<const float4 *>(p.rep_key + slot * d);
         if (!p.per_head) {

@@ -4,17 +4,25 @@
 //
 // One thread block per row.  Scores become order-preserving 32-bit keys; a
 // most-significant-digit radix select (4 passes of 8 bits, shared-memory
-// histograms) finds the K-th largest key exactly; a block-wide ordered
-// compaction then emits, in ascending index order, every element above that
-// key plus the first `need` elements equal to it -- so equal scores resolve
-// to the lower index and the output needs no sort.  No thread ever waits on
-// another block.
+// histogram, the crossing bin found by one warp with shuffles) finds the K-th
+// largest key exactly; a block-wide ordered compaction then emits, in
+// ascending index order, every element above that key plus the first `need`
+// elements equal to it -- so equal scores resolve to the lower index and the
+// output needs no sort.  No thread ever waits on another block.
+//
+// A thread owns a contiguous run of the row.  Rows of up to 8 x 1024 scores
+// (every workload of the paper's geometry: one score per stored frame) keep
+// their keys in registers; longer rows stage them in shared memory, and rows
+// beyond that re-read the scores from global memory in every pass.
 #include "stom_internal.cuh"
 
 namespace stom {
 
 constexpr int kTopkThreads = 1024;
+constexpr int kTopkRegKeys = 8;           // keys a thread holds in registers
 constexpr int kTopkSmemKeys = 48 * 1024;  // rows up to this many scores are staged in shared memory
+
+enum { kKeysGlobal = 0, kKeysShared = 1, kKeysRegs = 2 };
 
 __device__ __forceinline__ uint32_t score_key(float f) {
     f += 0.0f;  // -0 -> +0, so that equal scores have equal keys
@@ -31,9 +39,9 @@ struct TopkParams {
     int32_t *n_sel_out;
 };
 
-template <bool STAGED>
+template <int MODE>
 __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkParams p) {
-    extern __shared__ __align__(16) uint32_t skeys[];  // STAGED: n keys
+    extern __shared__ __align__(16) uint32_t skeys[];  // kKeysShared: n keys
     __shared__ uint32_t hist[256];
     __shared__ uint32_t s_prefix, s_need;
     __shared__ uint32_t warp_gt[32], warp_eq[32];
@@ -51,38 +59,50 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkParams p) 
     }
     if (ksel == 0) return;
 
-    if constexpr (STAGED) {
+    // thread `tid` owns the contiguous index range [lo, hi)
+    const int per = MODE == kKeysRegs ? kTopkRegKeys : (n + kTopkThreads - 1) / kTopkThreads;
+    const int lo = min(tid * per, n), hi = min(lo + per, n);
+
+    uint32_t rk[kTopkRegKeys];  // kKeysRegs: the thread's keys; slots past hi hold 0 and are never counted
+    if constexpr (MODE == kKeysRegs) {
+        const bool vec = ((reinterpret_cast<uintptr_t>(sc) & 15u) == 0) && lo + kTopkRegKeys <= n;
+        if (vec) {
+#pragma unroll
+            for (int e = 0; e < kTopkRegKeys; e += 4) {
+                const float4 v = __ldg(reinterpret_cast<const float4 *>(sc + lo + e));
+                rk[e] = score_key(v.x); rk[e + 1] = score_key(v.y); rk[e + 2] = score_key(v.z); rk[e + 3] = score_key(v.w);
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < kTopkRegKeys; ++e) rk[e] = lo + e < hi ? score_key(__ldg(sc + lo + e)) : 0u;
+        }
+    } else if constexpr (MODE == kKeysShared) {
         for (int i = tid; i < n; i += kTopkThreads) skeys[i] = score_key(sc[i]);
+        __syncthreads();
     }
-    auto key_at = [&](int i) -> uint32_t {
-        if constexpr (STAGED) return skeys[i];
-        else return score_key(__ldg(sc + i));
+    // visits the thread's keys in index order: f(index, key)
+    auto for_my_keys = [&](auto &&f) {
+        if constexpr (MODE == kKeysRegs) {
+#pragma unroll
+            for (int e = 0; e < kTopkRegKeys; ++e)
+                if (lo + e < hi) f(lo + e, rk[e]);
+        } else {
+            for (int i = lo; i < hi; ++i) {
+                if constexpr (MODE == kKeysShared) f(i, skeys[i]);
+                else f(i, score_key(__ldg(sc + i)));
+            }
+        }
     };
 
-    // ---- radix select of the ksel-th largest key: 4 passes of 8 bits.  Scores of one row share their leading bits,
-    //      so a plain histogram would serialise thousands of atomics on a handful of bins: lanes that hit the same bin
-    //      are merged first (match) and one of them adds their count.  The bin in which the running count from the top
-    //      reaches `need` is then found by one warp: a lane owns 8 bins, suffix sums go round by shuffle.
+    // ---- radix select of the ksel-th largest key: 4 passes of 8 bits.  The bin in which the running count from the
+    //      top reaches `need` is found by one warp: a lane owns 8 bins, suffix sums go round by shuffle.
     uint32_t prefix = 0, mask = 0, need = (uint32_t)ksel;
-    const int lane_ = tid & 31;
     for (int shift = 24; shift >= 0; shift -= 8) {
         if (tid < 256) hist[tid] = 0;
         __syncthreads();
-        for (int i0 = 0; i0 < n; i0 += kTopkThreads) {
-            const int i = i0 + tid;
-            uint32_t key = 0;
-            bool in = i < n;
-            if (in) {
-                key = key_at(i);
-                in = (key & mask) == prefix;
-            }
-            const uint32_t live = __ballot_sync(0xffffffffu, in);
-            if (in) {
-                const uint32_t bin = (key >> shift) & 255u;
-                const uint32_t peers = __match_any_sync(live, bin);
-                if (lane_ == __ffs(peers) - 1) atomicAdd(&hist[bin], (uint32_t)__popc(peers));
-            }
-        }
+        for_my_keys([&](int, uint32_t key) {
+            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
+        });
         __syncthreads();
         if (tid < 32) {
             uint32_t c[8], tot = 0;
@@ -116,15 +136,12 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkParams p) 
     }
     const uint32_t kth = prefix;  // exact key of the ksel-th largest; `need` of the elements equal to it are taken
 
-    // ---- ordered compaction: thread `tid` owns the contiguous index range [lo, hi)
-    const int per = (n + kTopkThreads - 1) / kTopkThreads;
-    const int lo = min(tid * per, n), hi = min(lo + per, n);
+    // ---- ordered compaction over the threads' contiguous ranges
     uint32_t gt = 0, eq = 0;
-    for (int i = lo; i < hi; ++i) {
-        const uint32_t key = key_at(i);
+    for_my_keys([&](int, uint32_t key) {
         gt += key > kth;
         eq += key == kth;
-    }
+    });
     // exclusive prefix sums of (gt, eq) over threads: warp scan, then scan of warp totals
     const int lane = tid & 31, warp = tid >> 5;
     uint32_t igt = gt, ieq = eq;
@@ -160,8 +177,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkParams p) 
     __syncthreads();
     uint32_t gt_before = warp_gt[warp] + igt - gt;
     uint32_t eq_before = warp_eq[warp] + ieq - eq;
-    for (int i = lo; i < hi; ++i) {
-        const uint32_t key = key_at(i);
+    for_my_keys([&](int i, uint32_t key) {
         const bool take = key > kth || (key == kth && eq_before < need);
         if (take) {
             const uint32_t pos = gt_before + min(eq_before, need);
@@ -170,7 +186,7 @@ __global__ void __launch_bounds__(kTopkThreads) topk_kernel(const TopkParams p) 
         }
         gt_before += key > kth;
         eq_before += key == kth;
-    }
+    });
 }
 
 }  // namespace stom
@@ -184,19 +200,21 @@ extern "C" int32_t stom_oqm_topk(const float *scores, int32_t rows, int32_t n, i
     if (rows == 0) return STOM_OK;
     TopkParams p{scores, row_stride, n, k, idx_out, score_out, n_sel_out};
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (n <= kTopkSmemKeys) {
+    if (n <= kTopkRegKeys * kTopkThreads) {
+        topk_kernel<kKeysRegs><<<rows, kTopkThreads, 0, s>>>(p);
+    } else if (n <= kTopkSmemKeys) {
         const size_t smem = (size_t)n * sizeof(uint32_t);
         if (smem > 40 * 1024) {
-            cudaError_t e = cudaFuncSetAttribute(topk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            cudaError_t e = cudaFuncSetAttribute(topk_kernel<kKeysShared>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  kTopkSmemKeys * (int)sizeof(uint32_t));
             if (e != cudaSuccess) {
                 set_last_cuda_error(e);
                 return STOM_ERR_CUDA;
             }
         }
-        topk_kernel<true><<<rows, kTopkThreads, smem, s>>>(p);
+        topk_kernel<kKeysShared><<<rows, kTopkThreads, smem, s>>>(p);
     } else {
-        topk_kernel<false><<<rows, kTopkThreads, 0, s>>>(p);
+        topk_kernel<kKeysGlobal><<<rows, kTopkThreads, 0, s>>>(p);
     }
     return finish_launch();
 }
