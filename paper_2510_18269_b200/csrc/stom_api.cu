@@ -1,5 +1,5 @@
 // Host-only part of the C ABI: geometry checks, arena layout, status strings,
-// and the retrieve convenience call that chains score -> top-K -> gather.
+// and the error bookkeeping.
 #include "stom_internal.cuh"
 
 namespace stom {
@@ -106,23 +106,3 @@ extern "C" const char *stom_status_string(int32_t s) {
 }
 
 extern "C" int32_t stom_last_cuda_error(void) { return g_last_cuda_error; }
-
-extern "C" int32_t stom_oqm_retrieve(const stom_oqm_config *cfg, const stom_oqm_store *store,
-                                     int32_t layer_begin, int32_t layer_count, int32_t n_groups,
-                                     const void *Q, int32_t T_q, int64_t q_stride_layer,
-                                     int64_t q_stride_head, int64_t q_stride_token,
-                                     int32_t k, float *scores, int32_t *idx,
-                                     void *k_active, void *v_active, int32_t out_dtype,
-                                     int64_t stride_layer, int64_t stride_head, int64_t stride_token,
-                                     int32_t token_offset, void *workspace, int64_t workspace_bytes,
-                                     uint32_t *dev_flags, void *stream) {
-    int32_t rc = stom_oqm_score_groups(cfg, store, layer_begin, layer_count, n_groups, Q, T_q, q_stride_layer,
-                                       q_stride_head, q_stride_token, scores, workspace, workspace_bytes, stream);
-    if (rc) return rc;
-    const int32_t rows = layer_count * (cfg->score_mode == STOM_SCORE_PER_HEAD ? cfg->n_kv_heads : 1);
-    rc = stom_oqm_topk(scores, rows, n_groups, n_groups, k, idx, nullptr, nullptr, stream);
-    if (rc) return rc;
-    return stom_oqm_dequant_gather(cfg, store, layer_begin, layer_count, idx, k, n_groups, k_active, v_active,
-                                   out_dtype, stride_layer, stride_head, stride_token, token_offset, dev_flags,
-                                   stream);
-}

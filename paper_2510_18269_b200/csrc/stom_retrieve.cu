@@ -1,0 +1,242 @@
+// A2 + A3 in one launch, then A4: retrieval for one question (paper Sec. 3.4:
+// similarity of the decoder state to every stored representative key, TopK,
+// then reconstruction of the selected groups only; appendix "Question-guided
+// single-pass retrieval" and "Cache reconstruction for decoding").
+//
+// The fused kernel runs with about two blocks per SM, each owning a
+// contiguous run of one layer's stored groups:
+//   prologue  the block builds the layer's question embedding q^(l) (mean
+//             over the query heads of each GQA block and over the question
+//             tokens) in shared memory -- Q of one layer is small and comes
+//             from L2 for all but the first block that touches it;
+//   stream    cosine scores of the block's groups (the software-pipelined
+//             loop of the stand-alone scoring kernel), written to `scores`;
+//   select    every block takes a ticket on its layer's counter when its
+//             scores are out; the block that draws the last ticket of a layer
+//             selects that layer's top-K.  Nobody waits for anybody: a block
+//             that is not last simply exits, so selection of early layers
+//             overlaps the streaming of later ones.
+// The layer counters live in the caller's workspace and are zeroed by a
+// memset enqueued ahead of the kernel; the selecting block also puts its
+// counter back to zero.
+#include "stom_score.cuh"
+#include "stom_topk.cuh"
+
+namespace stom {
+
+constexpr int kFusedThreads = kScoreWarps * 32;
+constexpr int kFusedMaxKeys = 10240;  // rows up to this many scores are selected from shared memory
+
+struct RetrieveParams {
+    ScoreParams sp;
+    int32_t k;
+    int32_t *idx;          // [rows][k]
+    uint32_t *counters;    // [layer_count], zero on entry
+    int32_t keys_in_smem;  // the selecting block may stage a row's keys in shared memory
+};
+
+// Question embedding of layer li for all kv heads, into sq[H*d] and qn[H] (shared memory).  A thread owns 8 adjacent
+// channels; the rows of a head (rep * T_q of them) are dealt to RG = kFusedThreads / (d/8) row slots, up to 8 rows of
+// a slot in flight at once; part[RG][d+4] combines the slots.
+template <typename T>
+__device__ __forceinline__ void embed_layer(const ScoreParams &p, int li, float *sq, float *qn, float *part, float *red) {
+    const int d = p.g.d, H = p.g.H, tid = threadIdx.x;
+    const int lanes_per_row = d >> 3;
+    const int RG = kFusedThreads / lanes_per_row;
+    const int cq = tid % lanes_per_row, rs = tid / lanes_per_row;
+    const int rows = p.rep * p.T_q, pitch = d + 4;
+    const T *qbase = reinterpret_cast<const T *>(p.Q) + (int64_t)li * p.ql + cq * 8;
+    constexpr int kRowBatch = 8;
+    for (int h = 0; h < H; ++h) {
+        float acc[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) acc[c] = 0.0f;
+        for (int r0 = rs; r0 < rows; r0 += RG * kRowBatch) {
+            float x[kRowBatch][8];
+#pragma unroll
+            for (int b = 0; b < kRowBatch; ++b) {
+                const int r = r0 + b * RG;
+#pragma unroll
+                for (int c = 0; c < 8; ++c) x[b][c] = 0.0f;
+                if (r < rows) {
+                    const int hr = r / p.T_q, j = r - hr * p.T_q;
+                    const T *src = qbase + (int64_t)(h * p.rep + hr) * p.qh + (int64_t)j * p.qt;
+                    if constexpr (sizeof(T) == 4) {
+                        const float4 v0 = __ldg(reinterpret_cast<const float4 *>(src));
+                        const float4 v1 = __ldg(reinterpret_cast<const float4 *>(src) + 1);
+                        x[b][0] = v0.x; x[b][1] = v0.y; x[b][2] = v0.z; x[b][3] = v0.w;
+                        x[b][4] = v1.x; x[b][5] = v1.y; x[b][6] = v1.z; x[b][7] = v1.w;
+                    } else {
+                        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(src));
+                        unpack2<T>(v.x, x[b][0], x[b][1]);
+                        unpack2<T>(v.y, x[b][2], x[b][3]);
+                        unpack2<T>(v.z, x[b][4], x[b][5]);
+                        unpack2<T>(v.w, x[b][6], x[b][7]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int b = 0; b < kRowBatch; ++b) {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) acc[c] += x[b][c];
+            }
+        }
+        float4 *mine = reinterpret_cast<float4 *>(part + rs * pitch + cq * 8);
+        mine[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+        mine[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+        __syncthreads();
+        float sqv = 0.0f;
+        if (tid < d) {
+            float a = 0.0f;
+            for (int g = 0; g < RG; ++g) a += part[g * pitch + tid];
+            const float v = a / (float)rows;
+            sq[h * d + tid] = v;
+            sqv = v * v;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) sqv += __shfl_xor_sync(0xffffffffu, sqv, o);
+        if ((tid & 31) == 0) red[tid >> 5] = sqv;
+        __syncthreads();
+        if (tid == 0) {
+            float tot = 0.0f;
+            for (int w = 0; w < kFusedThreads / 32; ++w) tot += red[w];
+            qn[h] = tot;
+        }
+        // part and red are rewritten only after the next head's loads and the barrier that follows them
+    }
+    __syncthreads();
+}
+
+// grid (chunks, layer_count), kFusedThreads threads.  Dynamic shared memory: q (H*d floats), norms (H rounded up
+// to 4 floats), then a region used first as the embedding scratch and, in a selecting block, as the key array.
+template <typename T, int V4>
+__global__ void __launch_bounds__(kFusedThreads) retrieve_kernel(const RetrieveParams rp) {
+    extern __shared__ __align__(16) float dyn[];
+    __shared__ float red[kFusedThreads / 32];
+    __shared__ TopkSmem tsm;
+    __shared__ int s_last;
+    const ScoreParams &p = rp.sp;
+    const int li = blockIdx.y, H = p.g.H, HD = H * p.g.d, tid = threadIdx.x;
+    float *sq = dyn, *qn = dyn + HD, *region = qn + ((H + 3) & ~3);
+
+    embed_layer<T>(p, li, sq, qn, region, red);
+
+    const int t_begin = blockIdx.x * p.groups_per_block;
+    const int t_end = min(t_begin + p.groups_per_block, p.n_groups);
+    score_block<V4>(p, sq, qn, li, t_begin, t_end);
+
+    // ---- ticket: the block that completes a layer selects its top-K
+    __threadfence();  // this block's scores are visible device-wide before its ticket is
+    __syncthreads();
+    if (tid == 0) s_last = atomicAdd(&rp.counters[li], 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (tid == 0) rp.counters[li] = 0;  // as found
+    const int n = p.n_groups, rows = p.per_head ? H : 1;
+    uint32_t *skeys = reinterpret_cast<uint32_t *>(region);
+    for (int r = 0; r < rows; ++r) {
+        const int64_t row = (int64_t)li * rows + r;
+        const float *sc = p.scores + row * n;
+        int32_t *out = rp.idx + row * rp.k;
+        if (n <= kTopkRegKeys * kFusedThreads)
+            block_topk<kFusedThreads, kKeysRegs>(sc, n, rp.k, out, nullptr, nullptr, skeys, tsm);
+        else if (rp.keys_in_smem)
+            block_topk<kFusedThreads, kKeysShared>(sc, n, rp.k, out, nullptr, nullptr, skeys, tsm);
+        else
+            block_topk<kFusedThreads, kKeysGlobal>(sc, n, rp.k, out, nullptr, nullptr, skeys, tsm);
+        __syncthreads();  // the scratch is reused by the next row
+    }
+}
+
+template <typename T>
+static void launch_retrieve(const RetrieveParams &rp, dim3 grid, size_t smem, int HD, bool fast, cudaStream_t s) {
+    if (fast && HD == 512) retrieve_kernel<T, 4><<<grid, kFusedThreads, smem, s>>>(rp);        // 4 kv heads x 128
+    else if (fast && HD == 1024) retrieve_kernel<T, 8><<<grid, kFusedThreads, smem, s>>>(rp);  // 8 kv heads x 128
+    else if (fast && HD == 256) retrieve_kernel<T, 2><<<grid, kFusedThreads, smem, s>>>(rp);
+    else if (fast && HD == 128) retrieve_kernel<T, 1><<<grid, kFusedThreads, smem, s>>>(rp);
+    else retrieve_kernel<T, 0><<<grid, kFusedThreads, smem, s>>>(rp);
+}
+
+}  // namespace stom
+
+using namespace stom;
+
+extern "C" int32_t stom_oqm_retrieve(const stom_oqm_config *cfg, const stom_oqm_store *store,
+                                     int32_t layer_begin, int32_t layer_count, int32_t n_groups,
+                                     const void *Q, int32_t T_q, int64_t q_stride_layer,
+                                     int64_t q_stride_head, int64_t q_stride_token,
+                                     int32_t k, float *scores, int32_t *idx,
+                                     void *k_active, void *v_active, int32_t out_dtype,
+                                     int64_t stride_layer, int64_t stride_head, int64_t stride_token,
+                                     int32_t token_offset, void *workspace, int64_t workspace_bytes,
+                                     uint32_t *dev_flags, void *stream) {
+    int32_t rc = check_config(cfg);
+    if (rc) return rc;
+    if ((rc = check_store(store))) return rc;
+    if ((rc = check_layers(cfg, layer_begin, layer_count))) return rc;
+    if (!Q || !scores || !idx || T_q < 1 || n_groups < 0 || k < 1) return STOM_ERR_INVALID_ARG;
+    if (n_groups > cfg->capacity_groups) return STOM_ERR_CAPACITY;
+    if (n_groups > (1 << 24)) return STOM_ERR_SHAPE;
+    if (q_stride_layer < 0 || q_stride_head < 0 || q_stride_token < 0) return STOM_ERR_INVALID_ARG;
+    if (!workspace || !aligned16(workspace) || workspace_bytes < stom_oqm_score_workspace_bytes(cfg, layer_count))
+        return STOM_ERR_WORKSPACE;
+    if (!aligned16(Q) || (reinterpret_cast<uintptr_t>(scores) & 3u) || (reinterpret_cast<uintptr_t>(idx) & 3u))
+        return STOM_ERR_ALIGNMENT;
+    const int dt = cfg->kv_dtype;
+    if (!stride_ok(q_stride_layer, dt) || !stride_ok(q_stride_head, dt) || !stride_ok(q_stride_token, dt))
+        return STOM_ERR_ALIGNMENT;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    if (layer_count > 0 && n_groups > 0) {
+        int dev = 0, sms = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        if (e == cudaSuccess) e = cudaMemsetAsync(workspace, 0, (size_t)layer_count * sizeof(uint32_t), s);
+        if (e != cudaSuccess) {
+            set_last_cuda_error(e);
+            return STOM_ERR_CUDA;
+        }
+        RetrieveParams rp;
+        ScoreParams &p = rp.sp;
+        p.Q = Q; p.ql = q_stride_layer; p.qh = q_stride_head; p.qt = q_stride_token;
+        p.rep_key = store->rep_key; p.rep_norm2 = store->rep_norm2;
+        p.qemb = nullptr; p.qnorm2 = nullptr;
+        p.scores = scores;
+        p.g = bank_geom(cfg);
+        p.layer_begin = layer_begin; p.layer_count = layer_count; p.n_groups = n_groups; p.T_q = T_q;
+        p.rep = cfg->n_q_heads / cfg->n_kv_heads;
+        p.per_head = cfg->score_mode == STOM_SCORE_PER_HEAD;
+        // one wave of about two blocks per SM; a block re-reads its layer's Q, so blocks are kept long
+        int chunks = (2 * sms) / layer_count;
+        if (chunks > (n_groups + 31) / 32) chunks = (n_groups + 31) / 32;
+        if (chunks < 1) chunks = 1;
+        p.groups_per_block = (n_groups + chunks - 1) / chunks;
+        rp.k = k; rp.idx = idx;
+        rp.counters = static_cast<uint32_t *>(workspace);
+        const int H = cfg->n_kv_heads, d = cfg->head_dim, HD = H * d;
+        const int part_floats = (kFusedThreads / (d / 8)) * (d + 4);
+        const size_t fixed = (size_t)HD + ((H + 3) & ~3);
+        int key_words = n_groups > kTopkRegKeys * kFusedThreads && n_groups <= kFusedMaxKeys ? n_groups : 0;
+        if (sizeof(float) * (fixed + key_words) > 48 * 1024) key_words = 0;  // long rows are selected from global memory
+        rp.keys_in_smem = key_words > 0;
+        const size_t smem = sizeof(float) * (fixed + (part_floats > key_words ? part_floats : key_words));
+        if (smem > 48 * 1024) return STOM_ERR_SHAPE;
+        const dim3 grid((n_groups + p.groups_per_block - 1) / p.groups_per_block, layer_count);
+        const bool fast = !p.per_head && H <= 32;
+        switch (dt) {
+        case STOM_BF16: launch_retrieve<__nv_bfloat16>(rp, grid, smem, HD, fast, s); break;
+        case STOM_FP16: launch_retrieve<__half>(rp, grid, smem, HD, fast, s); break;
+        default: launch_retrieve<float>(rp, grid, smem, HD, fast, s); break;
+        }
+        if ((rc = finish_launch())) return rc;
+    } else if (layer_count > 0) {
+        // nothing stored: every slot of idx is unused
+        const int32_t rows = layer_count * (cfg->score_mode == STOM_SCORE_PER_HEAD ? cfg->n_kv_heads : 1);
+        rc = stom_oqm_topk(scores, rows, 0, 0, k, idx, nullptr, nullptr, stream);
+        if (rc) return rc;
+    }
+    return stom_oqm_dequant_gather(cfg, store, layer_begin, layer_count, idx, k, n_groups, k_active, v_active,
+                                   out_dtype, stride_layer, stride_head, stride_token, token_offset, dev_flags,
+                                   stream);
+}

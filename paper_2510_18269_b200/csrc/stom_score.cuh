@@ -1,0 +1,248 @@
+// Device code of A2 (question embedding and cosine scores over the representative keys; paper appendix
+// "Question-guided single-pass retrieval", Sec. 3.4 sim(q, k-bar_i)), shared by the stand-alone scoring kernels and
+// by the fused retrieval kernel.
+#pragma once
+
+#include "stom_internal.cuh"
+
+namespace stom {
+
+struct ScoreParams {
+    const void *Q;
+    int64_t ql, qh, qt;  // element strides of Q: layer, head, token
+    const float *rep_key, *rep_norm2;
+    float *qemb;    // workspace: [layer_count][H][d]
+    float *qnorm2;  // workspace: [layer_count][H]
+    float *scores;
+    BankGeom g;
+    int32_t layer_begin, layer_count, n_groups, T_q, rep, per_head, groups_per_block;
+};
+
+constexpr int kEmbedThreads = 256;
+
+// Question embedding of one (layer, kv head): mean over the rep query heads of the GQA block and over the T_q
+// question tokens.  grid (H, layer_count), kEmbedThreads threads.  The rows (rep * T_q of them) are dealt to
+// RG = kEmbedThreads / (d/4) row groups; a thread adds up 4 adjacent channels of its group's rows and shared
+// memory combines the groups.
+template <typename T>
+__global__ void __launch_bounds__(kEmbedThreads) query_embed_kernel(const ScoreParams p) {
+    __shared__ float part[kEmbedThreads / 16][256 + 4];  // [row group <= 16][channel <= 256]
+    __shared__ float red[kEmbedThreads / 32];
+    const int h = blockIdx.x, li = blockIdx.y, d = p.g.d;
+    const int lanes_per_row = d >> 2;                 // threads across one row (4 channels each): 16, 32 or 64
+    const int RG = kEmbedThreads / lanes_per_row;     // row groups: 16, 8 or 4
+    const int cq = threadIdx.x % lanes_per_row, rg = threadIdx.x / lanes_per_row;
+    const int rows = p.rep * p.T_q;
+    const T *q = reinterpret_cast<const T *>(p.Q) + (int64_t)li * p.ql + cq * 4;
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+    // rows in batches of kRowBatch: all loads of a batch are issued before the first add
+    constexpr int kRowBatch = 8;
+    for (int r0 = rg; r0 < rows; r0 += RG * kRowBatch) {
+        float x[kRowBatch][4];
+#pragma unroll
+        for (int b = 0; b < kRowBatch; ++b) {
+            const int r = r0 + b * RG;
+            x[b][0] = x[b][1] = x[b][2] = x[b][3] = 0.0f;
+            if (r < rows) {
+                const int hr = r / p.T_q, j = r - hr * p.T_q;
+                const T *src = q + (int64_t)(h * p.rep + hr) * p.qh + (int64_t)j * p.qt;
+                if constexpr (sizeof(T) == 4) {
+                    const float4 v = __ldg(reinterpret_cast<const float4 *>(src));
+                    x[b][0] = v.x; x[b][1] = v.y; x[b][2] = v.z; x[b][3] = v.w;
+                } else {
+                    const uint2 v = __ldg(reinterpret_cast<const uint2 *>(src));
+                    unpack2<T>(v.x, x[b][0], x[b][1]);
+                    unpack2<T>(v.y, x[b][2], x[b][3]);
+                }
+            }
+        }
+#pragma unroll
+        for (int b = 0; b < kRowBatch; ++b) {
+            a0 += x[b][0]; a1 += x[b][1]; a2 += x[b][2]; a3 += x[b][3];
+        }
+    }
+    float *mine = &part[rg][cq * 4];
+    mine[0] = a0; mine[1] = a1; mine[2] = a2; mine[3] = a3;
+    __syncthreads();
+    float sq = 0.0f;
+    if (threadIdx.x < d) {
+        const int c = threadIdx.x;
+        float acc = 0.0f;
+        for (int g = 0; g < RG; ++g) acc += part[g][c];
+        const float v = acc / (float)rows;
+        p.qemb[((int64_t)li * p.g.H + h) * d + c] = v;
+        sq = v * v;
+    }
+    // |q_h|^2 by block reduction
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float tot = 0.0f;
+        for (int w = 0; w < kEmbedThreads / 32; ++w) tot += red[w];
+        p.qnorm2[(int64_t)li * p.g.H + h] = tot;
+    }
+}
+
+constexpr int kScoreWarps = 8;
+
+// One warp, a strided share of the block's groups [t_begin, t_end) of one layer, kGroupsPerWarp at a time.  The
+// loads of the next pair are issued before the current pair is reduced, so a warp always has 2 pairs of k-bar
+// vectors in flight.  V4: float4 words of the flattened k-bar that one lane covers (H*d / 128).
+template <int V4>
+__device__ __forceinline__ void score_groups_per_layer(const ScoreParams &p, const float *sq, const float *qn, int li,
+                                                       int t_begin, int t_end, int warp, int lane) {
+    constexpr int kGroupsPerWarp = V4 >= 8 ? 1 : 2;  // groups a warp scores together (register budget)
+    const int H = p.g.H, d = p.g.d, l = p.layer_begin + li;
+    float4 q4[V4];
+#pragma unroll
+    for (int i = 0; i < V4; ++i) q4[i] = reinterpret_cast<const float4 *>(sq)[lane + 32 * i];
+    float qq = lane < H ? qn[lane] : 0.0f;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) qq += __shfl_xor_sync(0xffffffffu, qq, o);
+    const float qnorm = fmaxf(sqrtf(qq), 1e-12f);
+
+    auto load = [&](int t0, float4 (&kv)[kGroupsPerWarp][V4], float (&kn)[kGroupsPerWarp]) {
+#pragma unroll
+        for (int u = 0; u < kGroupsPerWarp; ++u) {
+            const int t = min(t0 + u, t_end - 1);  // a pair that sticks out re-reads the last group; dropped at the store
+            const int64_t slot = bank_slot(p.g, l, t, 0);
+            const float4 *kb = reinterpret_cast<const float4 *>(p.rep_key + slot * d);
+#pragma unroll
+            for (int i = 0; i < V4; ++i) kv[u][i] = __ldg(kb + lane + 32 * i);
+            kn[u] = lane < H ? __ldg(p.rep_norm2 + slot + lane) : 0.0f;
+        }
+    };
+    const int step = kScoreWarps * kGroupsPerWarp;
+    int t0 = t_begin + warp * kGroupsPerWarp;
+    if (t0 >= t_end) return;
+    float4 cur[kGroupsPerWarp][V4], nxt[kGroupsPerWarp][V4];
+    float kn_cur[kGroupsPerWarp], kn_nxt[kGroupsPerWarp];
+    load(t0, cur, kn_cur);
+    for (; t0 < t_end; t0 += step) {
+        const bool more = t0 + step < t_end;
+        if (more) load(t0 + step, nxt, kn_nxt);
+        float dot[kGroupsPerWarp];
+#pragma unroll
+        for (int u = 0; u < kGroupsPerWarp; ++u) {
+            float a = 0.0f;
+#pragma unroll
+            for (int i = 0; i < V4; ++i) {
+                a = fmaf(cur[u][i].x, q4[i].x, a);
+                a = fmaf(cur[u][i].y, q4[i].y, a);
+                a = fmaf(cur[u][i].z, q4[i].z, a);
+                a = fmaf(cur[u][i].w, q4[i].w, a);
+            }
+            dot[u] = a;
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+            for (int u = 0; u < kGroupsPerWarp; ++u) {
+                dot[u] += __shfl_xor_sync(0xffffffffu, dot[u], o);
+                kn_cur[u] += __shfl_xor_sync(0xffffffffu, kn_cur[u], o);
+            }
+        }
+        if (lane < kGroupsPerWarp && t0 + lane < t_end) {
+            float dsel = dot[0], ksel = kn_cur[0];
+#pragma unroll
+            for (int u = 1; u < kGroupsPerWarp; ++u) {
+                if (lane == u) {
+                    dsel = dot[u];
+                    ksel = kn_cur[u];
+                }
+            }
+            p.scores[(int64_t)li * p.n_groups + t0 + lane] = dsel / (qnorm * fmaxf(sqrtf(ksel), 1e-12f));
+        }
+        if (more) {
+#pragma unroll
+            for (int u = 0; u < kGroupsPerWarp; ++u) {
+                kn_cur[u] = kn_nxt[u];
+#pragma unroll
+                for (int i = 0; i < V4; ++i) cur[u][i] = nxt[u][i];
+            }
+        }
+    }
+}
+
+// Scores of groups [t_begin, t_end) of layer li, by one block of kScoreWarps warps.  sq: the layer's question
+// embedding (H*d floats) in shared memory, qn: its H squared norms.
+// V4 > 0: PER_LAYER scoring with H*d == 128 * V4 and H <= 32 (the software-pipelined loop); V4 == 0: everything else.
+template <int V4>
+__device__ __forceinline__ void score_block(const ScoreParams &p, const float *sq, const float *qn, int li, int t_begin,
+                                            int t_end) {
+    const int H = p.g.H, d = p.g.d, HD = H * d;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if constexpr (V4 > 0) {
+        score_groups_per_layer<V4>(p, sq, qn, li, t_begin, t_end, warp, lane);
+        return;
+    }
+    const int l = p.layer_begin + li;
+    const float eps = 1e-12f;
+#pragma unroll 1
+    for (int t = t_begin + (V4 > 0 ? t_end : warp); t < t_end; t += kScoreWarps) {
+        const int64_t slot = bank_slot(p.g, l, t, 0);
+        const float4 *kb = reinterpret_cast<const float4 *>(p.rep_key + slot * d);
+        if (!p.per_head) {
+            float dot = 0.0f;
+            for (int i = lane; i < HD / 4; i += 32) {
+                const float4 a = __ldg(kb + i);
+                const float4 b = reinterpret_cast<const float4 *>(sq)[i];
+                dot = fmaf(a.x, b.x, dot);
+                dot = fmaf(a.y, b.y, dot);
+                dot = fmaf(a.z, b.z, dot);
+                dot = fmaf(a.w, b.w, dot);
+            }
+            float kn = 0.0f, qq = 0.0f;
+            for (int hh = lane; hh < H; hh += 32) {
+                kn += __ldg(p.rep_norm2 + slot + hh);
+                qq += qn[hh];
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                kn += __shfl_xor_sync(0xffffffffu, kn, o);
+                qq += __shfl_xor_sync(0xffffffffu, qq, o);
+            }
+            if (lane == 0)
+                p.scores[(int64_t)li * p.n_groups + t] = dot / (fmaxf(sqrtf(qq), eps) * fmaxf(sqrtf(kn), eps));
+        } else {
+            for (int hh = 0; hh < H; ++hh) {
+                float dot = 0.0f;
+                for (int i = lane; i < d / 4; i += 32) {
+                    const float4 a = __ldg(kb + hh * (d / 4) + i);
+                    const float4 b = reinterpret_cast<const float4 *>(sq)[hh * (d / 4) + i];
+                    dot = fmaf(a.x, b.x, dot);
+                    dot = fmaf(a.y, b.y, dot);
+                    dot = fmaf(a.z, b.z, dot);
+                    dot = fmaf(a.w, b.w, dot);
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
+                if (lane == 0) {
+                    const float kn = __ldg(p.rep_norm2 + slot + hh);
+                    p.scores[((int64_t)li * H + hh) * p.n_groups + t] =
+                        dot / (fmaxf(sqrtf(qn[hh]), eps) * fmaxf(sqrtf(kn), eps));
+                }
+            }
+        }
+    }
+}
+
+
+// grid (chunks, layer_count): block x scores groups [x * groups_per_block, (x+1) * groups_per_block) of its layer
+template <int V4>
+__global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(const ScoreParams p) {
+    extern __shared__ __align__(16) float sq[];  // q of this layer: H*d floats, then H norms
+    const int li = blockIdx.y, H = p.g.H, HD = H * p.g.d;
+    for (int i = threadIdx.x; i < HD; i += blockDim.x) sq[i] = p.qemb[(int64_t)li * HD + i];
+    float *qn = sq + HD;
+    if (threadIdx.x < H) qn[threadIdx.x] = p.qnorm2[(int64_t)li * H + threadIdx.x];
+    __syncthreads();
+    const int t_begin = blockIdx.x * p.groups_per_block;
+    const int t_end = min(t_begin + p.groups_per_block, p.n_groups);
+    score_block<V4>(p, sq, qn, li, t_begin, t_end);
+}
+
+}  // namespace stom

@@ -1,0 +1,108 @@
+"""GPU parity of the fused retrieval call (question embedding + scores + top-K in one launch, then the
+reconstruction) against the CPU oracle, at row lengths that exercise each way the selecting block holds its keys
+(registers, shared memory, global memory), in both scoring modes and for every input type.
+
+The bank is filled with seeded random arrays on both sides (representative keys with their norms, codes, scales,
+offsets), so that long rows do not need a long quantization on the CPU first; the quantizer has its own tests.
+Tolerances are those of tests/_parity.py."""
+import numpy as np
+import pytest
+import torch
+
+import _parity as P
+from paper_2510_18269_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _random_bank(orc, oqm, sh, mode, seed):
+    """The same random bank in an oracle Store (NumPy) and in a device Store."""
+    ocfg, gcfg = P.oracle_cfg(orc, sh, mode), P.gpu_cfg(oqm, sh, mode)
+    ost, gst = orc.Store(ocfg), oqm.Store(gcfg)
+    rng = np.random.default_rng(seed)
+    ost.rep_key[...] = rng.standard_normal(ost.rep_key.shape, dtype=np.float32)
+    # a few groups point along a common direction so that the head of the ranking is not pure noise
+    u = rng.standard_normal((sh.L, 1, sh.H_k, sh.d), dtype=np.float32)
+    pick = rng.choice(sh.T, size=max(1, min(sh.T, sh.k) // 2), replace=False)
+    ost.rep_key[:, pick] = u + 0.3 * ost.rep_key[:, pick]
+    ost.rep_norm2[...] = (ost.rep_key.astype(np.float64) ** 2).sum(-1).astype(np.float32)
+    ost.codes_k[...] = rng.integers(0, 256, ost.codes_k.shape, dtype=np.uint8)
+    ost.codes_v[...] = rng.integers(0, 256, ost.codes_v.shape, dtype=np.uint8)
+    for name in ("scale_k", "scale_v"):
+        getattr(ost, name)[...] = rng.uniform(0.01, 0.5, getattr(ost, name).shape).astype(np.float32)
+    for name in ("zero_k", "zero_v"):
+        getattr(ost, name)[...] = rng.standard_normal(getattr(ost, name).shape, dtype=np.float32)
+    for name in ("codes_k", "codes_v", "scale_k", "zero_k", "scale_v", "zero_v", "rep_key", "rep_norm2"):
+        getattr(gst, name).copy_(torch.from_numpy(getattr(ost, name)))
+    return ocfg, gcfg, ost, gst, u
+
+
+@pytest.mark.parametrize("L,H_q,H_k,d,G,T,T_q,k,mode,dtype", [
+    (2, 28, 4, 128, 4, 7200, 16, 64, 0, "bf16"),   # 7B geometry, keys of the selecting block in shared memory
+    (2, 16, 8, 128, 4, 3600, 5, 64, 0, "bf16"),    # 72B geometry (8 kv heads)
+    (1, 4, 2, 64, 4, 11000, 3, 300, 0, "fp16"),    # row longer than the shared-memory key array
+    (3, 8, 4, 128, 4, 1500, 4, 32, 1, "bf16"),     # one selection per kv head; keys in registers
+    (2, 6, 2, 128, 2, 2500, 2, 2500, 0, "fp32"),   # every stored group selected
+    (1, 2, 1, 256, 4, 40, 1, 64, 0, "bf16"),       # fewer groups stored than asked for
+    (2, 6, 3, 128, 4, 333, 7, 16, 0, "bf16"),      # a head count the pipelined scorer does not cover
+    (2, 6, 3, 128, 4, 333, 7, 16, 1, "fp16"),
+])
+def test_fused_retrieve_matches_oracle(orc, L, H_q, H_k, d, G, T, T_q, k, mode, dtype):
+    from paper_2510_18269_b200 import oqm
+    oqm.lib()
+    sh = synth.Shape("fused", L=L, H_q=H_q, H_k=H_k, d=d, G=G, T=T, T_q=T_q, k=k, dtype=dtype, seed=5)
+    ocfg, gcfg, ost, gst, u = _random_bank(orc, oqm, sh, mode, seed=T + k)
+    rows = L * (H_k if mode else 1)
+    rep = H_q // H_k
+    g = torch.Generator().manual_seed(99)
+    base = torch.from_numpy(u[:, 0]).repeat_interleave(rep, dim=1)[:, :, None, :]
+    Q = (base + 0.5 * torch.randn(L, H_q, T_q, d, generator=g)).to(synth.DTYPES[dtype]).contiguous()
+
+    o_scores = orc.score_groups(ocfg, ost, 0, L, T, P.as_np16(Q), T_q, P.q_strides(sh))
+    o_idx, _, _ = orc.topk(o_scores.reshape(rows, T), k)
+
+    sys_len = 3
+    S = sys_len + k * G + 1
+    ka_flat, ka = P.out_buffers(sh, L, S, torch.bfloat16, "cuda", 3.0)
+    va_flat, va = P.out_buffers(sh, L, S, torch.bfloat16, "cuda", 3.0)
+    scores = torch.full((rows * T + P.GUARD,), -7.0, dtype=torch.float32, device="cuda")
+    idx = torch.full((rows * k + P.GUARD,), -9, dtype=torch.int32, device="cuda")
+    ws = torch.full((oqm.stom_oqm_score_workspace_bytes(gcfg, L),), 0xAB, dtype=torch.uint8, device="cuda")
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for _ in range(2):   # twice: the second call finds the layer counters as the first one left them
+        oqm.stom_oqm_retrieve(gcfg, gst, 0, L, T, Q.cuda(), T_q, P.q_strides(sh), k, scores, idx, ka, va, oqm.BF16,
+                              P.active_strides(sh, S), sys_len, ws, dev_flags=flags)
+    torch.cuda.synchronize()
+    assert int(flags.item()) == 0
+    assert torch.all(scores[rows * T:] == -7.0) and torch.all(idx[rows * k:] == -9), "guard band overwritten"
+    P.compare_scores(scores[:rows * T], o_scores)
+    P.compare_topk(idx[:rows * k], o_idx, o_scores.reshape(rows, T), k)
+
+    # reconstruction: the oracle gathers the groups the GPU selected
+    g_idx = idx[:rows * k].view(rows, k).cpu().numpy().copy()
+    sent = P.as_np16(torch.tensor([3.0], dtype=torch.bfloat16))[0]
+    oka = np.full((L, H_k, S, d), sent, np.uint16)
+    ova = np.full((L, H_k, S, d), sent, np.uint16)
+    assert orc.dequant_gather(ocfg, ost, 0, L, g_idx, k, T, oka, ova, orc.BF16, P.active_strides(sh, S), sys_len) == 0
+    n_el = L * H_k * S * d
+    for flat, o16 in ((ka_flat, oka), (va_flat, ova)):
+        assert torch.all(flat[n_el:] == 3.0), "guard band overwritten"
+        assert np.array_equal(P.as_np16(flat[:n_el]).reshape(o16.shape), o16), "reconstructed cache differs"
+
+
+def test_fused_retrieve_on_an_empty_bank_marks_every_slot_unused(orc):
+    from paper_2510_18269_b200 import oqm
+    sh = synth.Shape("empty", L=2, H_q=4, H_k=2, d=128, G=4, T=8, T_q=2, k=4, seed=1)
+    gcfg = P.gpu_cfg(oqm, sh)
+    gst = oqm.Store(gcfg)
+    Q = synth.queries(sh).cuda()
+    S = sh.k * sh.G
+    _, ka = P.out_buffers(sh, sh.L, S, torch.bfloat16, "cuda", 3.0)
+    _, va = P.out_buffers(sh, sh.L, S, torch.bfloat16, "cuda", 3.0)
+    scores = torch.zeros(sh.L * sh.T, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(sh.L * sh.k, dtype=torch.int32, device="cuda")
+    ws = torch.empty(oqm.stom_oqm_score_workspace_bytes(gcfg, sh.L), dtype=torch.uint8, device="cuda")
+    oqm.stom_oqm_retrieve(gcfg, gst, 0, sh.L, 0, Q, sh.T_q, P.q_strides(sh), sh.k, scores, idx, ka, va, oqm.BF16,
+                          P.active_strides(sh, S), 0, ws)
+    torch.cuda.synchronize()
+    assert torch.all(idx == -1) and torch.all(ka == 3.0) and torch.all(va == 3.0)

@@ -306,5 +306,10 @@ def test_retrieve_convenience_call_matches_the_three_calls(orc, oqm):
                                         P.active_strides(sh, S), 2)
         torch.cuda.synchronize()
         outs.append((sc.clone(), idx.clone(), ka.clone(), va.clone()))
-    for a, b in zip(*outs):
-        assert torch.equal(a, b)
+    # the fused kernel adds the question tokens up in another order: scores agree to the score tolerance (each
+    # side is within 1e-5 of the oracle), the selection up to ties, and the reconstruction exactly for equal indices
+    (sc_a, idx_a, ka_a, va_a), (sc_b, idx_b, ka_b, va_b) = outs
+    assert (sc_a - sc_b).abs().max().item() <= 2e-5
+    P.compare_topk(idx_b, idx_a.view(sh.L, sh.k).cpu().numpy(), sc_a.view(sh.L, sh.T).cpu().numpy(), sh.k)
+    if torch.equal(idx_a, idx_b):
+        assert torch.equal(ka_a, ka_b) and torch.equal(va_a, va_b)
