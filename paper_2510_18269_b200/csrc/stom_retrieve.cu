@@ -8,7 +8,9 @@
 //   prologue  the block builds the layer's question embedding q^(l) (mean
 //             over the query heads of each GQA block and over the question
 //             tokens) in shared memory -- Q of one layer is small and comes
-//             from L2 for all but the first block that touches it;
+//             from L2 for all but the first block that touches it; the rows
+//             of several heads are in flight together, because this step is
+//             all memory latency;
 //   stream    cosine scores of the block's groups (the software-pipelined
 //             loop of the stand-alone scoring kernel), written to `scores`;
 //   select    every block takes a ticket on its layer's counter when its
@@ -35,76 +37,113 @@ struct RetrieveParams {
     int32_t keys_in_smem;  // the selecting block may stage a row's keys in shared memory
 };
 
-// Question embedding of layer li for all kv heads, into sq[H*d] and qn[H] (shared memory).  A thread owns 8 adjacent
-// channels; the rows of a head (rep * T_q of them) are dealt to RG = kFusedThreads / (d/8) row slots, up to 8 rows of
-// a slot in flight at once; part[RG][d+4] combines the slots.
+constexpr int kEmbedHeadGroup = 4;  // kv heads whose rows are in flight together
+
+// Raw 8 channels of one question row as loaded (16 bytes of a 16-bit type, 32 bytes of binary32).
 template <typename T>
-__device__ __forceinline__ void embed_layer(const ScoreParams &p, int li, float *sq, float *qn, float *part, float *red) {
-    const int d = p.g.d, H = p.g.H, tid = threadIdx.x;
+struct QRow {
+    static constexpr int W = 8 * (int)sizeof(T) / 4;
+    uint32_t w[W];
+    __device__ __forceinline__ void load(const T *src) {
+#pragma unroll
+        for (int i = 0; i < W / 4; ++i) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4 *>(src) + i);
+            w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
+        }
+    }
+    __device__ __forceinline__ void add_to(float (&acc)[8]) const {
+        if constexpr (sizeof(T) == 4) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) acc[c] += __uint_as_float(w[c]);
+        } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                float a, b;
+                unpack2<T>(w[c], a, b);
+                acc[2 * c] += a;
+                acc[2 * c + 1] += b;
+            }
+        }
+    }
+};
+
+// Question embedding of layer li for all kv heads, into sq[H*d] and qn[H] (shared memory).  A thread owns 8 adjacent
+// channels; the rows of a head (rep * T_q of them) are dealt to RG = kFusedThreads / (d/8) row slots.  The heads go
+// through in groups of kEmbedHeadGroup: a thread walks its rows of the whole group with kInFlight loads outstanding,
+// whatever head they belong to, so the wait for memory is paid once or twice per group instead of once per head;
+// part[head of the group][RG][d+4] combines the slots.
+template <typename T>
+__device__ __forceinline__ void embed_layer(const ScoreParams &p, int li, float *sq, float *qn, float *part) {
+    constexpr int kInFlight = sizeof(T) == 4 ? 8 : 16;
+    const int d = p.g.d, H = p.g.H, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int lanes_per_row = d >> 3;
     const int RG = kFusedThreads / lanes_per_row;
     const int cq = tid % lanes_per_row, rs = tid / lanes_per_row;
     const int rows = p.rep * p.T_q, pitch = d + 4;
+    const int per_head = (rows + RG - 1) / RG;  // rows of one head that a row slot walks
     const T *qbase = reinterpret_cast<const T *>(p.Q) + (int64_t)li * p.ql + cq * 8;
-    constexpr int kRowBatch = 8;
-    for (int h = 0; h < H; ++h) {
+    for (int h0 = 0; h0 < H; h0 += kEmbedHeadGroup) {
+        const int hg = min(kEmbedHeadGroup, H - h0);
+        const int n_i = hg * per_head;
         float acc[8];
 #pragma unroll
         for (int c = 0; c < 8; ++c) acc[c] = 0.0f;
-        for (int r0 = rs; r0 < rows; r0 += RG * kRowBatch) {
-            float x[kRowBatch][8];
+        int cur = 0;  // head of the group that acc belongs to
+        auto flush = [&](int hh) {
+            float4 *mine = reinterpret_cast<float4 *>(part + (hh * RG + rs) * pitch + cq * 8);
+            mine[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+            mine[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
 #pragma unroll
-            for (int b = 0; b < kRowBatch; ++b) {
-                const int r = r0 + b * RG;
+            for (int c = 0; c < 8; ++c) acc[c] = 0.0f;
+        };
+        for (int i0 = 0; i0 < n_i; i0 += kInFlight) {
+            QRow<T> x[kInFlight];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) x[b][c] = 0.0f;
-                if (r < rows) {
+            for (int b = 0; b < kInFlight; ++b) {
+                const int i = i0 + b;
+                const int hh = i / per_head, r = rs + (i - hh * per_head) * RG;
+#pragma unroll
+                for (int j = 0; j < QRow<T>::W; ++j) x[b].w[j] = 0u;  // +0.0 in every format
+                if (i < n_i && r < rows) {
                     const int hr = r / p.T_q, j = r - hr * p.T_q;
-                    const T *src = qbase + (int64_t)(h * p.rep + hr) * p.qh + (int64_t)j * p.qt;
-                    if constexpr (sizeof(T) == 4) {
-                        const float4 v0 = __ldg(reinterpret_cast<const float4 *>(src));
-                        const float4 v1 = __ldg(reinterpret_cast<const float4 *>(src) + 1);
-                        x[b][0] = v0.x; x[b][1] = v0.y; x[b][2] = v0.z; x[b][3] = v0.w;
-                        x[b][4] = v1.x; x[b][5] = v1.y; x[b][6] = v1.z; x[b][7] = v1.w;
-                    } else {
-                        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(src));
-                        unpack2<T>(v.x, x[b][0], x[b][1]);
-                        unpack2<T>(v.y, x[b][2], x[b][3]);
-                        unpack2<T>(v.z, x[b][4], x[b][5]);
-                        unpack2<T>(v.w, x[b][6], x[b][7]);
-                    }
+                    x[b].load(qbase + (int64_t)((h0 + hh) * p.rep + hr) * p.qh + (int64_t)j * p.qt);
                 }
             }
 #pragma unroll
-            for (int b = 0; b < kRowBatch; ++b) {
-#pragma unroll
-                for (int c = 0; c < 8; ++c) acc[c] += x[b][c];
+            for (int b = 0; b < kInFlight; ++b) {
+                const int i = i0 + b;
+                if (i < n_i) {
+                    const int hh = i / per_head;
+                    if (hh != cur) {
+                        flush(cur);
+                        cur = hh;
+                    }
+                    x[b].add_to(acc);
+                }
             }
         }
-        float4 *mine = reinterpret_cast<float4 *>(part + rs * pitch + cq * 8);
-        mine[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
-        mine[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+        flush(cur);
         __syncthreads();
-        float sqv = 0.0f;
-        if (tid < d) {
+        for (int e = tid; e < hg * d; e += kFusedThreads) {
+            const int hh = e / d, c = e - hh * d;
             float a = 0.0f;
-            for (int g = 0; g < RG; ++g) a += part[g * pitch + tid];
-            const float v = a / (float)rows;
-            sq[h * d + tid] = v;
-            sqv = v * v;
+            for (int g = 0; g < RG; ++g) a += part[(hh * RG + g) * pitch + c];
+            sq[(h0 + hh) * d + c] = a / (float)rows;
         }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) sqv += __shfl_xor_sync(0xffffffffu, sqv, o);
-        if ((tid & 31) == 0) red[tid >> 5] = sqv;
         __syncthreads();
-        if (tid == 0) {
-            float tot = 0.0f;
-            for (int w = 0; w < kFusedThreads / 32; ++w) tot += red[w];
-            qn[h] = tot;
+        for (int hh = warp; hh < hg; hh += kFusedThreads / 32) {  // |q_h|^2: one warp per head
+            float n2 = 0.0f;
+            for (int c = lane; c < d; c += 32) {
+                const float v = sq[(h0 + hh) * d + c];
+                n2 = fmaf(v, v, n2);
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, o);
+            if (lane == 0) qn[h0 + hh] = n2;
         }
-        // part and red are rewritten only after the next head's loads and the barrier that follows them
+        // part is rewritten by the next group only after that group's loads; the barrier below orders it for all
+        __syncthreads();
     }
-    __syncthreads();
 }
 
 // grid (chunks, layer_count), kFusedThreads threads.  Dynamic shared memory: q (H*d floats), norms (H rounded up
@@ -112,14 +151,13 @@ __device__ __forceinline__ void embed_layer(const ScoreParams &p, int li, float 
 template <typename T, int V4>
 __global__ void __launch_bounds__(kFusedThreads) retrieve_kernel(const RetrieveParams rp) {
     extern __shared__ __align__(16) float dyn[];
-    __shared__ float red[kFusedThreads / 32];
     __shared__ TopkSmem tsm;
     __shared__ int s_last;
     const ScoreParams &p = rp.sp;
     const int li = blockIdx.y, H = p.g.H, HD = H * p.g.d, tid = threadIdx.x;
     float *sq = dyn, *qn = dyn + HD, *region = qn + ((H + 3) & ~3);
 
-    embed_layer<T>(p, li, sq, qn, region, red);
+    embed_layer<T>(p, li, sq, qn, region);
 
     const int t_begin = blockIdx.x * p.groups_per_block;
     const int t_end = min(t_begin + p.groups_per_block, p.n_groups);
@@ -215,7 +253,7 @@ extern "C" int32_t stom_oqm_retrieve(const stom_oqm_config *cfg, const stom_oqm_
         rp.k = k; rp.idx = idx;
         rp.counters = static_cast<uint32_t *>(workspace);
         const int H = cfg->n_kv_heads, d = cfg->head_dim, HD = H * d;
-        const int part_floats = (kFusedThreads / (d / 8)) * (d + 4);
+        const int part_floats = (H < kEmbedHeadGroup ? H : kEmbedHeadGroup) * (kFusedThreads / (d / 8)) * (d + 4);
         const size_t fixed = (size_t)HD + ((H + 3) & ~3);
         int key_words = n_groups > kTopkRegKeys * kFusedThreads && n_groups <= kFusedMaxKeys ? n_groups : 0;
         if (sizeof(float) * (fixed + key_words) > 48 * 1024) key_words = 0;  // long rows are selected from global memory
