@@ -40,9 +40,12 @@ FALLBACK_HBM_GBS = 6650.0
 # dram bytes per unit of work measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum) on a reduced
 # case of the same kernel and scaled by the units one launch processes; see profiles/*.md.  None = not captured.
 NCU_TRAFFIC_PER_UNIT = {
-    "quantize_kernel": 133150.0,    # bytes per (layer, frame): 545.4 MB over 4 x 1024 units
-    "dequant_gather_kernel": None,  # bytes per (layer, selected group): the capture's writes stayed in L2, not usable
-    "score_kernel": 2070.0,         # bytes per (layer, stored group): 8.48 MB over 4 x 1024 units
+    "quantize_kernel": 137448.0,        # bytes per (layer, frame): 3.941 GB over 28 x 1024 units
+    # bytes per (layer, selected group): 186.3 MB over 28 x 64 units; of the 183.5 MB the kernel writes only
+    # 125.7 MB had left L2 when it ended (the rest is written back later), so this undercounts by design
+    "dequant_gather_kernel": 103985.0,
+    "score_kernel": 2066.0,             # bytes per (layer, stored group): 59.25 MB over 28 x 1024 units
+    "retrieve_kernel": 2178.0,          # bytes per (layer, stored group): 62.46 MB over 28 x 1024 units (Q re-read per block)
 }
 
 
@@ -325,6 +328,20 @@ def run_ours(args, sh):
     q_ms, sc_ms, tk_ms, ga_ms, r_ms = (sdist.max_over_ranks(x) for x in (q_ms, sc_ms, tk_ms, ga_ms, r_ms))
     assert int(flags.item()) == 0, "a kernel flagged a bad index or a wait that ran out"
 
+    # Writes alone run at about 60 % of the copy rate on this part, so a kernel whose traffic is 3/4 writes (the
+    # gather) is bounded by the write rate, not by `peak`: measure it here with a plain 1 GiB fill.
+    wbuf = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+    w_ms = []
+    for i in range(6):
+        a, b = ev(), ev()
+        a.record()
+        wbuf.fill_(i)
+        b.record()
+        torch.cuda.synchronize()
+        w_ms.append(a.elapsed_time(b))
+    write_gbs = (1 << 30) / (min(w_ms[1:]) * 1e-3) / 1e9
+    del wbuf
+
     rbytes = bytes_score(sh, sh.T) + bytes_topk(sh, sh.T) + bytes_gather(sh, sh.k)
     value = world * rbytes / (r_ms * 1e-3) / 1e9
     qbytes = bytes_quantize(sh, sh.T)
@@ -341,6 +358,10 @@ def run_ours(args, sh):
         roof("dequant_gather_kernel", bytes_gather(sh, sh.k), ga_ms, 1, sh.L * sh.k),
         roof("score_kernel", bytes_score(sh, sh.T), sc_ms, 1, sh.L * sh.T),
     ]
+    # the gather writes 2*H_k*G*d*2 bytes per selected group: its floor is those bytes at the measured fill rate
+    gw = 2 * sh.H_k * sh.G * sh.d * 2 * sh.k * sh.L
+    roofs[1].update({"write_bytes_per_launch": gw, "measured_fill_GBps": write_gbs,
+                     "write_bound_us": gw / write_gbs / 1e3, "frac_of_write_bound": (gw / write_gbs / 1e6) / ga_ms})
     out = {
         "metric": "OQM retrieve+dequant throughput", "value": value, "unit": "GB/s", "n_gpus": world,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,

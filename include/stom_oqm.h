@@ -278,6 +278,44 @@ int32_t stom_oqm_retrieve(const stom_oqm_config *cfg, const stom_oqm_store *stor
                           int32_t token_offset, void *workspace, int64_t workspace_bytes,
                           uint32_t *dev_flags, void *stream);
 
+/* ---- A5: decode attention over [system tokens || selected groups] without
+ *      materialising the cache (Sec. 3.4: decoding attends to the bounded
+ *      active kv; appendix "Cache reconstruction for decoding": the per-layer
+ *      indices are reused for every decode step) ---------------------------
+ *
+ * For every layer of the range and every query head h_q (kv head h = h_q /
+ * (H_q/H_k)):  out[l][h_q][:] = softmax_t(softmax_scale * <q[l][h_q], K_t>) V_t
+ * over the tokens t of  [the sys_len system tokens of (l, h)] followed by [the
+ * G tokens of every selected group idx[..][j] >= 0, j < k], where a group's K
+ * and V rows are fmaf(code, s, m) of the bank (binary32, not rounded to a
+ * 16-bit type on the way).  Accumulation is binary32; the output is rounded
+ * once to cache_dtype.
+ * idx: as for stom_oqm_dequant_gather (PER_LAYER [layer_count][k]; PER_HEAD
+ *   [layer_count][H_k][k]); -1 entries are skipped, other out-of-range entries
+ *   are skipped and flagged.  k may be 0 if sys_len > 0.
+ * q_dec (cfg->kv_dtype): element (l, h_q, c) at (l-layer_begin)*q_stride_layer
+ *   + h_q*q_stride_head + c.
+ * k_sys, v_sys (cache_dtype = STOM_BF16 | STOM_FP16; may be NULL if sys_len == 0):
+ *   element (l, h, tok, c) at (l-layer_begin)*sys_stride_layer + h*sys_stride_head
+ *   + tok*sys_stride_token + c -- the first sys_len tokens of the active cache.
+ * out (cache_dtype): element (l, h_q, c) at (l-layer_begin)*out_stride_layer +
+ *   h_q*out_stride_head + c.
+ * workspace: DEVICE, 256-byte aligned, stom_oqm_attend_workspace_bytes() bytes;
+ *   holds the partial results of the blocks that share a (layer, kv head).
+ * Errors: INVALID_ARG, SHAPE, UNSUPPORTED, ALIGNMENT, CAPACITY, WORKSPACE, CUDA.
+ */
+int64_t stom_oqm_attend_workspace_bytes(const stom_oqm_config *cfg, int32_t layer_count, int32_t k,
+                                        int32_t sys_len);
+int32_t stom_oqm_attend(const stom_oqm_config *cfg, const stom_oqm_store *store,
+                        int32_t layer_begin, int32_t layer_count,
+                        const int32_t *idx, int32_t k, int32_t n_groups,
+                        const void *q_dec, int64_t q_stride_layer, int64_t q_stride_head,
+                        const void *k_sys, const void *v_sys, int32_t cache_dtype,
+                        int64_t sys_stride_layer, int64_t sys_stride_head, int64_t sys_stride_token,
+                        int32_t sys_len, float softmax_scale,
+                        void *out, int64_t out_stride_layer, int64_t out_stride_head,
+                        void *workspace, int64_t workspace_bytes, uint32_t *dev_flags, void *stream);
+
 /* ---- the same path driven from HOST memory -----------------------------
  * These two calls take HOST input/output buffers (pinned memory makes the
  * copies asynchronous), stage them through caller-provided DEVICE scratch with

@@ -1,0 +1,403 @@
+// A5: decode attention of one new query token over [system tokens || the
+// selected groups], dequantizing the groups on the fly (paper Sec. 3.4:
+// decoding attends to the bounded active kv, KV_active = union of the
+// dequantized selected groups plus the full-precision system tokens; appendix
+// "Cache reconstruction for decoding": the per-layer indices are reused for
+// every decode step).  Nothing is materialised: a decode step reads the
+// packed codes and their (s, m) -- a quarter of the bytes of the bf16 cache --
+// instead of writing that cache once and re-reading it every step.
+//
+// Work unit: a segment = one selected group (G <= 64 tokens) or a run of up to
+// 64 system tokens.  A block of 8 warps takes 8 consecutive segments of one
+// (layer, kv head) and all the query heads of that kv head's GQA block (in
+// chunks of 8); warp w owns segment w:
+//   phase 1  scores: a lane owns 8 adjacent channels, d/8 lanes share a token;
+//            K is rebuilt as fmaf(code, s, m) in registers, dotted with the
+//            query heads, reduced by shuffles, scores land in shared memory
+//   phase 2  block-local softmax statistics per query head (max, sum) in the
+//            base-2 domain (the scores carry softmax_scale * log2(e))
+//   phase 3  weighted sum of V, rebuilt the same way, per warp; the warps'
+//            sums are combined through shared memory
+// and writes (max, sum, weighted sum) per query head to the workspace.  The
+// block that draws the last ticket of its (layer, kv head) merges the partial
+// results of all its blocks and writes the output row.  Nobody waits.
+#include "stom_internal.cuh"
+
+namespace stom {
+
+constexpr int kAtWarps = 8;
+constexpr int kAtThreads = kAtWarps * 32;
+constexpr int kAtSegTokens = 64;  // token slots per segment (G <= 64)
+constexpr int kAtHeads = 8;       // query heads handled together
+
+struct AttendParams {
+    const int32_t *idx;
+    const uint8_t *codes_k, *codes_v;
+    const float *scale_k, *zero_k, *scale_v, *zero_v;
+    const void *q;
+    int64_t q_sl, q_sh;  // element strides of q_dec: layer, query head
+    const void *ksys, *vsys;
+    int64_t s_sl, s_sh, s_st;  // element strides of the system-token cache: layer, kv head, token
+    void *out;
+    int64_t o_sl, o_sh;  // element strides of out: layer, query head
+    float *part;         // [layer][H][blocks][rep][d + 2]
+    uint32_t *counters;  // [layer][H]
+    BankGeom g;
+    int32_t layer_begin, k, n_groups, per_head, rep, sys_len, n_sys_seg, n_seg;
+    float scale_log2e;
+    uint32_t *flags;
+};
+
+// 2^23 + code as a float for the code byte i of `bytes` (see the dequantize-gather kernel), minus 2^23
+__device__ __forceinline__ float code_float(uint32_t bytes, int i) {
+    return __uint_as_float(__byte_perm(bytes, 0x4B000000u, 0x7540u + i)) - 8388608.0f;
+}
+
+// QT: type of q_dec; CT: type of the system-token cache and of the output; LPR: lanes per token (d / 8)
+template <typename QT, typename CT, int LPR>
+__global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p) {
+    constexpr int D = LPR * 8;
+    constexpr int TPW = 32 / LPR;  // tokens one warp pass covers
+    constexpr int kSlots = kAtWarps * kAtSegTokens;
+    constexpr int kBuf = (32 * 1024) / (kAtHeads * D * 4) < kAtWarps ? (32 * 1024) / (kAtHeads * D * 4) : kAtWarps;
+    __shared__ __align__(16) float buf[8192];  // phases 1-3: scores [kAtHeads][kSlots]; then warp sums [kBuf][kAtHeads][D]
+    __shared__ __align__(16) float qf[kAtHeads][D];
+    __shared__ float blk_max[kAtHeads], blk_sum[kAtHeads];
+    __shared__ int s_last;
+    static_assert(kAtHeads * kSlots <= 8192 && kBuf * kAtHeads * D <= 8192, "shared buffer");
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int sub = lane / LPR, cl = lane - sub * LPR;
+    const int bx = blockIdx.x, h = blockIdx.y, li = blockIdx.z;
+    const int G = p.g.G, H = p.g.H;
+    const int seg = bx * kAtWarps + warp;  // this warp's segment of (li, h)
+    float(*sc)[kSlots] = reinterpret_cast<float(*)[kSlots]>(buf);
+
+    // ---- what the warp's segment is
+    int n_tok = 0;          // tokens in the segment
+    int sys_begin = -1;     // >= 0: a run of system tokens starting here
+    int64_t slot = 0;       // bank slot of a group segment
+    if (seg < p.n_sys_seg) {
+        sys_begin = seg * kAtSegTokens;
+        n_tok = min(kAtSegTokens, p.sys_len - sys_begin);
+    } else if (seg < p.n_seg) {
+        const int j = seg - p.n_sys_seg;
+        const int t = p.per_head ? p.idx[((int64_t)li * H + h) * p.k + j] : p.idx[(int64_t)li * p.k + j];
+        if (t >= 0 && t < p.n_groups) {
+            n_tok = G;
+            slot = bank_slot(p.g, p.layer_begin + li, t, h);
+        } else if (t != -1 && p.flags && lane == 0) {
+            atomicOr(p.flags, STOM_FLAG_BAD_INDEX);
+        }
+    }
+    const int wpr = p.g.row_bytes >> 2;  // 32-bit words per packed row
+    const CT *ksys = reinterpret_cast<const CT *>(p.ksys) + (int64_t)li * p.s_sl + (int64_t)h * p.s_sh + cl * 8;
+    const CT *vsys = reinterpret_cast<const CT *>(p.vsys) + (int64_t)li * p.s_sl + (int64_t)h * p.s_sh + cl * 8;
+
+    // 8 channels of one token as floats: a system token is read as stored, a group token is rebuilt from its code word
+    auto token8 = [&](bool keys, int g, const float (&s)[8], const float (&m)[8], float (&x)[8]) {
+        if (sys_begin >= 0) {
+            const uint4 v = __ldg(reinterpret_cast<const uint4 *>((keys ? ksys : vsys) + (int64_t)(sys_begin + g) * p.s_st));
+            unpack2<CT>(v.x, x[0], x[1]);
+            unpack2<CT>(v.y, x[2], x[3]);
+            unpack2<CT>(v.z, x[4], x[5]);
+            unpack2<CT>(v.w, x[6], x[7]);
+        } else {
+            const uint32_t *codes = reinterpret_cast<const uint32_t *>((keys ? p.codes_k : p.codes_v) +
+                                                                       slot * (int64_t)G * p.g.row_bytes) + cl;
+            const uint32_t w = __ldg(codes + (int64_t)g * wpr);
+            const uint32_t even = w & 0x0f0f0f0fu, odd = (w >> 4) & 0x0f0f0f0fu;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                x[2 * i] = __fmaf_rn(code_float(even, i), s[2 * i], m[2 * i]);
+                x[2 * i + 1] = __fmaf_rn(code_float(odd, i), s[2 * i + 1], m[2 * i + 1]);
+            }
+        }
+    };
+    auto load_stats = [&](bool keys, float (&s)[8], float (&m)[8]) {
+        if (sys_begin >= 0 || n_tok == 0) return;
+        const float4 *sp = reinterpret_cast<const float4 *>((keys ? p.scale_k : p.scale_v) + slot * D + cl * 8);
+        const float4 *mp = reinterpret_cast<const float4 *>((keys ? p.zero_k : p.zero_v) + slot * D + cl * 8);
+        const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1), m0 = __ldg(mp), m1 = __ldg(mp + 1);
+        s[0] = s0.x; s[1] = s0.y; s[2] = s0.z; s[3] = s0.w; s[4] = s1.x; s[5] = s1.y; s[6] = s1.z; s[7] = s1.w;
+        m[0] = m0.x; m[1] = m0.y; m[2] = m0.z; m[3] = m0.w; m[4] = m1.x; m[5] = m1.y; m[6] = m1.z; m[7] = m1.w;
+    };
+
+    const int n_blocks = gridDim.x;
+    for (int h0 = 0; h0 < p.rep; h0 += kAtHeads) {  // query heads of this kv head, kAtHeads at a time
+        const int nh = min(kAtHeads, p.rep - h0);
+        // ---- the query rows, scaled so that exp2 can be used
+        for (int e = tid; e < kAtHeads * D; e += kAtThreads) {
+            const int hh = e / D, c = e - hh * D;
+            float v = 0.0f;
+            if (hh < nh) {
+                const QT *q = reinterpret_cast<const QT *>(p.q) + (int64_t)li * p.q_sl + (int64_t)(h * p.rep + h0 + hh) * p.q_sh;
+                v = (float)q[c] * p.scale_log2e;
+            }
+            qf[hh][c] = v;
+        }
+        __syncthreads();
+
+        // ---- phase 1: scores of the warp's segment
+        {
+            float s[8], m[8];
+            load_stats(true, s, m);
+            float q8[kAtHeads][8];
+#pragma unroll
+            for (int hh = 0; hh < kAtHeads; ++hh) {
+                const float4 a = *reinterpret_cast<const float4 *>(&qf[hh][cl * 8]);
+                const float4 b = *reinterpret_cast<const float4 *>(&qf[hh][cl * 8 + 4]);
+                q8[hh][0] = a.x; q8[hh][1] = a.y; q8[hh][2] = a.z; q8[hh][3] = a.w;
+                q8[hh][4] = b.x; q8[hh][5] = b.y; q8[hh][6] = b.z; q8[hh][7] = b.w;
+            }
+            for (int g0 = 0; g0 < kAtSegTokens; g0 += TPW) {
+                const int g = g0 + sub;
+                float dot[kAtHeads];
+#pragma unroll
+                for (int hh = 0; hh < kAtHeads; ++hh) dot[hh] = 0.0f;
+                if (g0 < n_tok) {  // warp-uniform
+                    float x[8];
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) x[c] = 0.0f;
+                    if (g < n_tok) token8(true, g, s, m, x);
+#pragma unroll
+                    for (int hh = 0; hh < kAtHeads; ++hh) {
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) dot[hh] = fmaf(x[c], q8[hh][c], dot[hh]);
+                    }
+#pragma unroll
+                    for (int o = LPR / 2; o > 0; o >>= 1) {
+#pragma unroll
+                        for (int hh = 0; hh < kAtHeads; ++hh) dot[hh] += __shfl_xor_sync(0xffffffffu, dot[hh], o);
+                    }
+                }
+                // lane cl of the token's lanes files the score of query head cl
+                if (cl < kAtHeads) {
+                    float mine = dot[0];
+#pragma unroll
+                    for (int hh = 1; hh < kAtHeads; ++hh)
+                        if (cl == hh) mine = dot[hh];
+                    sc[cl][warp * kAtSegTokens + g] = g < n_tok ? mine : -INFINITY;
+                }
+            }
+        }
+        __syncthreads();
+
+        // ---- phase 2: the block's softmax statistics; scores become weights in place
+        if (warp < kAtHeads) {
+            float mx = -INFINITY;
+            for (int i = lane; i < kSlots; i += 32) mx = fmaxf(mx, sc[warp][i]);
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            float sum = 0.0f;
+            for (int i = lane; i < kSlots; i += 32) {
+                const float v = sc[warp][i];
+                const float w = v == -INFINITY ? 0.0f : exp2f(v - mx);
+                sc[warp][i] = w;
+                sum += w;
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+            if (lane == 0) {
+                blk_max[warp] = mx;
+                blk_sum[warp] = sum;
+            }
+        }
+        __syncthreads();
+
+        // ---- phase 3: weighted sum of the values of the warp's segment
+        float acc[kAtHeads][8];
+#pragma unroll
+        for (int hh = 0; hh < kAtHeads; ++hh)
+#pragma unroll
+            for (int c = 0; c < 8; ++c) acc[hh][c] = 0.0f;
+        {
+            float s[8], m[8];
+            load_stats(false, s, m);
+            for (int g0 = 0; g0 < n_tok; g0 += TPW) {
+                const int g = g0 + sub;
+                if (g < n_tok) {
+                    float x[8];
+                    token8(false, g, s, m, x);
+#pragma unroll
+                    for (int hh = 0; hh < kAtHeads; ++hh) {
+                        const float w = sc[hh][warp * kAtSegTokens + g];
+#pragma unroll
+                        for (int c = 0; c < 8; ++c) acc[hh][c] = fmaf(w, x[c], acc[hh][c]);
+                    }
+                }
+            }
+            // the token slots of a warp pass hold different tokens of the same channels
+#pragma unroll
+            for (int o = LPR; o < 32; o <<= 1) {
+#pragma unroll
+                for (int hh = 0; hh < kAtHeads; ++hh)
+#pragma unroll
+                    for (int c = 0; c < 8; ++c) acc[hh][c] += __shfl_xor_sync(0xffffffffu, acc[hh][c], o);
+            }
+        }
+        __syncthreads();  // every warp is done with the weights; the buffer now takes the warps' sums
+        float tot[kAtHeads * D / kAtThreads];
+#pragma unroll
+        for (int e = 0; e < kAtHeads * D / kAtThreads; ++e) tot[e] = 0.0f;
+        for (int r = 0; r < kAtWarps; r += kBuf) {
+            if (warp >= r && warp < r + kBuf && sub == 0) {
+                float *dst = buf + (size_t)(warp - r) * kAtHeads * D + cl * 8;
+#pragma unroll
+                for (int hh = 0; hh < kAtHeads; ++hh) {
+                    *reinterpret_cast<float4 *>(dst + hh * D) = make_float4(acc[hh][0], acc[hh][1], acc[hh][2], acc[hh][3]);
+                    *reinterpret_cast<float4 *>(dst + hh * D + 4) = make_float4(acc[hh][4], acc[hh][5], acc[hh][6], acc[hh][7]);
+                }
+            }
+            __syncthreads();
+#pragma unroll
+            for (int e = 0; e < kAtHeads * D / kAtThreads; ++e) {
+                const int i = e * kAtThreads + tid;  // (head, channel) pair
+                for (int w = 0; w < kBuf && r + w < kAtWarps; ++w) tot[e] += buf[(size_t)w * kAtHeads * D + i];
+            }
+            __syncthreads();
+        }
+        // ---- partial result of this block: (max, sum, weighted sum) per query head
+#pragma unroll
+        for (int e = 0; e < kAtHeads * D / kAtThreads; ++e) {
+            const int i = e * kAtThreads + tid, hh = i / D, c = i - hh * D;
+            if (hh < nh) {
+                float *rec = p.part + ((((int64_t)li * H + h) * n_blocks + bx) * p.rep + h0 + hh) * (D + 2);
+                rec[2 + c] = tot[e];
+                if (c == 0) {
+                    rec[0] = blk_max[hh];
+                    rec[1] = blk_sum[hh];
+                }
+            }
+        }
+        __syncthreads();  // qf, buf and the statistics are rewritten by the next chunk of heads
+    }
+
+    // ---- ticket: the block that completes (layer, kv head) merges the partial results
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = atomicAdd(&p.counters[li * H + h], 1u) == (unsigned)n_blocks - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (tid == 0) p.counters[li * H + h] = 0;  // as found
+    for (int e = tid; e < p.rep * D; e += kAtThreads) {
+        const int hq = e / D, c = e - hq * D;
+        const float *rec0 = p.part + (((int64_t)li * H + h) * n_blocks * p.rep + hq) * (D + 2);
+        const int64_t step = (int64_t)p.rep * (D + 2);
+        float mx = -INFINITY;
+        for (int b = 0; b < n_blocks; ++b) mx = fmaxf(mx, __ldcg(rec0 + b * step));
+        float num = 0.0f, den = 0.0f;
+        for (int b = 0; b < n_blocks; ++b) {
+            const float mb = __ldcg(rec0 + b * step);
+            if (mb == -INFINITY) continue;
+            const float w = exp2f(mb - mx);
+            den = fmaf(__ldcg(rec0 + b * step + 1), w, den);
+            num = fmaf(__ldcg(rec0 + b * step + 2 + c), w, num);
+        }
+        const float o = den > 0.0f ? num / den : 0.0f;
+        CT *out = reinterpret_cast<CT *>(p.out) + (int64_t)li * p.o_sl + (int64_t)(h * p.rep + hq) * p.o_sh;
+        out[c] = (CT)o;
+    }
+}
+
+static int attend_segments(const stom_oqm_config *cfg, int32_t k, int32_t sys_len, int *n_sys_seg) {
+    (void)cfg;
+    *n_sys_seg = (sys_len + kAtSegTokens - 1) / kAtSegTokens;
+    return *n_sys_seg + k;
+}
+
+template <typename QT, typename CT>
+static int32_t launch_attend(const AttendParams &p, dim3 grid, cudaStream_t s) {
+    switch (p.g.d) {
+    case 64: attend_kernel<QT, CT, 8><<<grid, kAtThreads, 0, s>>>(p); break;
+    case 128: attend_kernel<QT, CT, 16><<<grid, kAtThreads, 0, s>>>(p); break;
+    case 256: attend_kernel<QT, CT, 32><<<grid, kAtThreads, 0, s>>>(p); break;
+    default: return STOM_ERR_SHAPE;
+    }
+    return finish_launch();
+}
+
+}  // namespace stom
+
+using namespace stom;
+
+extern "C" int64_t stom_oqm_attend_workspace_bytes(const stom_oqm_config *cfg, int32_t layer_count, int32_t k,
+                                                   int32_t sys_len) {
+    if (check_config(cfg) || layer_count < 0 || k < 0 || sys_len < 0) return STOM_ERR_INVALID_ARG;
+    int n_sys_seg = 0;
+    const int n_seg = attend_segments(cfg, k, sys_len, &n_sys_seg);
+    const int64_t blocks = (n_seg + kAtWarps - 1) / kAtWarps;
+    const int64_t counters = ((int64_t)layer_count * cfg->n_kv_heads * 4 + 255) / 256 * 256;
+    const int64_t part = (int64_t)layer_count * cfg->n_kv_heads * blocks * (cfg->n_q_heads / cfg->n_kv_heads) *
+                         (cfg->head_dim + 2) * 4;
+    return counters + (part + 255) / 256 * 256;
+}
+
+extern "C" int32_t stom_oqm_attend(const stom_oqm_config *cfg, const stom_oqm_store *store,
+                                   int32_t layer_begin, int32_t layer_count,
+                                   const int32_t *idx, int32_t k, int32_t n_groups,
+                                   const void *q_dec, int64_t q_stride_layer, int64_t q_stride_head,
+                                   const void *k_sys, const void *v_sys, int32_t cache_dtype,
+                                   int64_t sys_stride_layer, int64_t sys_stride_head, int64_t sys_stride_token,
+                                   int32_t sys_len, float softmax_scale,
+                                   void *out, int64_t out_stride_layer, int64_t out_stride_head,
+                                   void *workspace, int64_t workspace_bytes, uint32_t *dev_flags, void *stream) {
+    int32_t rc = check_config(cfg);
+    if (rc) return rc;
+    if ((rc = check_store(store))) return rc;
+    if ((rc = check_layers(cfg, layer_begin, layer_count))) return rc;
+    if (!q_dec || !out || k < 0 || n_groups < 0 || sys_len < 0 || (k > 0 && !idx)) return STOM_ERR_INVALID_ARG;
+    if (k + sys_len < 1) return STOM_ERR_INVALID_ARG;
+    if (sys_len > 0 && (!k_sys || !v_sys)) return STOM_ERR_INVALID_ARG;
+    if (n_groups > cfg->capacity_groups) return STOM_ERR_CAPACITY;
+    if (cache_dtype != STOM_BF16 && cache_dtype != STOM_FP16) return STOM_ERR_UNSUPPORTED;
+    if (q_stride_layer < 0 || q_stride_head < cfg->head_dim || out_stride_layer < 0 || out_stride_head < cfg->head_dim ||
+        sys_stride_layer < 0 || sys_stride_head < 0 || (sys_len > 0 && sys_stride_token < cfg->head_dim))
+        return STOM_ERR_INVALID_ARG;
+    if ((idx && (reinterpret_cast<uintptr_t>(idx) & 3u)) || (reinterpret_cast<uintptr_t>(q_dec) & 3u) ||
+        (reinterpret_cast<uintptr_t>(out) & 1u))
+        return STOM_ERR_ALIGNMENT;
+    if (sys_len > 0 && (!aligned16(k_sys) || !aligned16(v_sys) || !stride_ok(sys_stride_layer, cache_dtype) ||
+                        !stride_ok(sys_stride_head, cache_dtype) || !stride_ok(sys_stride_token, cache_dtype)))
+        return STOM_ERR_ALIGNMENT;
+    const int64_t need = stom_oqm_attend_workspace_bytes(cfg, layer_count, k, sys_len);
+    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need) return STOM_ERR_WORKSPACE;
+    if (layer_count == 0) return STOM_OK;
+
+    AttendParams p;
+    p.idx = idx;
+    p.codes_k = store->codes_k; p.codes_v = store->codes_v;
+    p.scale_k = store->scale_k; p.zero_k = store->zero_k; p.scale_v = store->scale_v; p.zero_v = store->zero_v;
+    p.q = q_dec; p.q_sl = q_stride_layer; p.q_sh = q_stride_head;
+    p.ksys = k_sys; p.vsys = v_sys; p.s_sl = sys_stride_layer; p.s_sh = sys_stride_head; p.s_st = sys_stride_token;
+    p.out = out; p.o_sl = out_stride_layer; p.o_sh = out_stride_head;
+    const int64_t counters = ((int64_t)layer_count * cfg->n_kv_heads * 4 + 255) / 256 * 256;
+    p.counters = static_cast<uint32_t *>(workspace);
+    p.part = reinterpret_cast<float *>(static_cast<uint8_t *>(workspace) + counters);
+    p.g = bank_geom(cfg);
+    p.layer_begin = layer_begin; p.k = k; p.n_groups = n_groups;
+    p.per_head = cfg->score_mode == STOM_SCORE_PER_HEAD;
+    p.rep = cfg->n_q_heads / cfg->n_kv_heads;
+    p.sys_len = sys_len;
+    p.n_seg = attend_segments(cfg, k, sys_len, &p.n_sys_seg);
+    p.scale_log2e = softmax_scale * 1.4426950408889634f;
+    p.flags = dev_flags;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, (size_t)layer_count * cfg->n_kv_heads * sizeof(uint32_t), s);
+    if (e != cudaSuccess) {
+        set_last_cuda_error(e);
+        return STOM_ERR_CUDA;
+    }
+    if (layer_count > 65535 || cfg->n_kv_heads > 65535) return STOM_ERR_SHAPE;
+    const dim3 grid((p.n_seg + kAtWarps - 1) / kAtWarps, cfg->n_kv_heads, layer_count);
+    const bool bf = cache_dtype == STOM_BF16;
+    switch (cfg->kv_dtype) {
+    case STOM_BF16:
+        return bf ? launch_attend<__nv_bfloat16, __nv_bfloat16>(p, grid, s) : launch_attend<__nv_bfloat16, __half>(p, grid, s);
+    case STOM_FP16:
+        return bf ? launch_attend<__half, __nv_bfloat16>(p, grid, s) : launch_attend<__half, __half>(p, grid, s);
+    default:
+        return bf ? launch_attend<float, __nv_bfloat16>(p, grid, s) : launch_attend<float, __half>(p, grid, s);
+    }
+}

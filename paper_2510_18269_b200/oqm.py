@@ -27,7 +27,7 @@ EXPORTS = (
     "stom_oqm_topk", "stom_oqm_dequant_gather", "stom_oqm_retrieve",
     "stom_oqm_quantize_host_scratch_bytes", "stom_oqm_quantize_frame_host",
     "stom_oqm_retrieve_host_scratch_bytes", "stom_oqm_retrieve_host",
-    "stom_oqm_score_groups_noalloc",
+    "stom_oqm_score_groups_noalloc", "stom_oqm_attend_workspace_bytes", "stom_oqm_attend",
 )
 
 
@@ -72,6 +72,7 @@ def lib():
         L.stom_oqm_score_workspace_bytes.restype = C.c_int64
         L.stom_oqm_score_workspace_bytes.argtypes = [C.POINTER(Config), C.c_int32]
         L.stom_oqm_budget_to_k.argtypes = [C.c_int64, C.c_int32, C.c_int32]
+        L.stom_oqm_attend_workspace_bytes.restype = C.c_int64
         L.stom_oqm_quantize_host_scratch_bytes.restype = C.c_int64
         L.stom_oqm_retrieve_host_scratch_bytes.restype = C.c_int64
         for name in EXPORTS:
@@ -221,6 +222,24 @@ def stom_oqm_retrieve(cfg: Config, store: Store, layer_begin, layer_count, n_gro
         C.c_int64(0 if workspace is None else workspace.numel() * workspace.element_size()), _ptr(dev_flags),
         _stream(stream))
     _check(rc, "stom_oqm_retrieve")
+
+
+def stom_oqm_attend_workspace_bytes(cfg: Config, layer_count: int, k: int, sys_len: int) -> int:
+    return int(lib().stom_oqm_attend_workspace_bytes(C.byref(cfg), C.c_int32(layer_count), C.c_int32(k),
+                                                     C.c_int32(sys_len)))
+
+
+def stom_oqm_attend(cfg: Config, store: Store, layer_begin, layer_count, idx, k, n_groups, q_dec, q_strides,
+                    k_sys, v_sys, cache_dtype, sys_strides, sys_len, softmax_scale, out, out_strides, workspace,
+                    dev_flags=None, stream=None):
+    """q_strides = (layer, head); sys_strides = (layer, head, token); out_strides = (layer, head), all in elements."""
+    rc = lib().stom_oqm_attend(
+        C.byref(cfg), C.byref(store.desc), C.c_int32(layer_begin), C.c_int32(layer_count), _ptr(idx), C.c_int32(k),
+        C.c_int32(n_groups), _ptr(q_dec), C.c_int64(q_strides[0]), C.c_int64(q_strides[1]), _ptr(k_sys), _ptr(v_sys),
+        C.c_int32(cache_dtype), C.c_int64(sys_strides[0]), C.c_int64(sys_strides[1]), C.c_int64(sys_strides[2]),
+        C.c_int32(sys_len), C.c_float(softmax_scale), _ptr(out), C.c_int64(out_strides[0]), C.c_int64(out_strides[1]),
+        _ptr(workspace), C.c_int64(workspace.numel() * workspace.element_size()), _ptr(dev_flags), _stream(stream))
+    _check(rc, "stom_oqm_attend")
 
 
 # ---------------------------------------------------------------- host-buffer entry points

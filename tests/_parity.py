@@ -119,3 +119,25 @@ def as_np16(t: torch.Tensor) -> np.ndarray:
 
 def f32_of(orc, arr: np.ndarray, dtype: str) -> np.ndarray:
     return arr if dtype == "fp32" else orc.to_f32(arr, dt_code(dtype))
+
+
+def random_bank(orc, oqm, sh, mode, seed):
+    """The same random bank in an oracle Store (NumPy) and in a device Store."""
+    ocfg, gcfg = oracle_cfg(orc, sh, mode), gpu_cfg(oqm, sh, mode)
+    ost, gst = orc.Store(ocfg), oqm.Store(gcfg)
+    rng = np.random.default_rng(seed)
+    ost.rep_key[...] = rng.standard_normal(ost.rep_key.shape, dtype=np.float32)
+    # a few groups point along a common direction so that the head of the ranking is not pure noise
+    u = rng.standard_normal((sh.L, 1, sh.H_k, sh.d), dtype=np.float32)
+    pick = rng.choice(sh.T, size=max(1, min(sh.T, sh.k) // 2), replace=False)
+    ost.rep_key[:, pick] = u + 0.3 * ost.rep_key[:, pick]
+    ost.rep_norm2[...] = (ost.rep_key.astype(np.float64) ** 2).sum(-1).astype(np.float32)
+    ost.codes_k[...] = rng.integers(0, 256, ost.codes_k.shape, dtype=np.uint8)
+    ost.codes_v[...] = rng.integers(0, 256, ost.codes_v.shape, dtype=np.uint8)
+    for name in ("scale_k", "scale_v"):
+        getattr(ost, name)[...] = rng.uniform(0.01, 0.5, getattr(ost, name).shape).astype(np.float32)
+    for name in ("zero_k", "zero_v"):
+        getattr(ost, name)[...] = rng.standard_normal(getattr(ost, name).shape, dtype=np.float32)
+    for name in ("codes_k", "codes_v", "scale_k", "zero_k", "scale_v", "zero_v", "rep_key", "rep_norm2"):
+        getattr(gst, name).copy_(torch.from_numpy(getattr(ost, name)))
+    return ocfg, gcfg, ost, gst, u

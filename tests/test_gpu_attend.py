@@ -1,0 +1,100 @@
+"""GPU parity of the decode attention that dequantizes the selected groups on the fly (stom_oqm_attend) against the
+CPU oracle: the oracle reconstructs the active cache (system tokens followed by the selected groups, rounded to
+bf16 as a materialised cache holds them) and runs plain softmax attention over it in binary64.
+
+Tolerance: 2e-2 absolute on the 16-bit output (the benchmark definition's figure for attention outputs), widened to
+one unit in the last place of bfloat16 (2^-7 relative) where an output exceeds 2 in magnitude: there the spacing of
+the output type itself is above 2e-2, and two correctly rounded results of nearby sums may land one step apart.
+The kernel works from the unrounded reconstruction fmaf(code, s, m) and accumulates in binary32."""
+import numpy as np
+import pytest
+import torch
+
+import _parity as P
+from paper_2510_18269_b200 import synth
+
+pytestmark = pytest.mark.gpu
+TOL = 2e-2
+
+
+def _selection(rng, rows, T, k, n_sel):
+    """[rows][k] ascending group ids, the last k - n_sel slots unused (-1), as the top-K call leaves them."""
+    idx = np.full((rows, k), -1, np.int32)
+    for r in range(rows):
+        idx[r, :n_sel] = np.sort(rng.choice(T, size=n_sel, replace=False))
+    return idx
+
+
+@pytest.mark.parametrize("L,H_q,H_k,d,G,T,k,n_sel,sys_len,mode,dtype,cache", [
+    (2, 28, 4, 128, 50, 200, 64, 64, 37, 0, "bf16", "bf16"),   # 7B geometry
+    (1, 16, 2, 128, 50, 90, 24, 24, 5, 0, "bf16", "bf16"),     # 8 query heads per kv head (72B ratio)
+    (2, 8, 4, 64, 16, 70, 9, 9, 130, 0, "fp16", "fp16"),       # three runs of system tokens, d = 64
+    (1, 4, 2, 256, 64, 30, 10, 10, 3, 0, "bf16", "bf16"),      # d = 256, full 64-token groups
+    (2, 8, 4, 128, 50, 120, 16, 16, 20, 1, "bf16", "bf16"),    # one selection per kv head
+    (1, 8, 4, 128, 50, 60, 20, 13, 8, 0, "bf16", "bf16"),      # fewer groups stored than slots: trailing -1
+    (1, 12, 1, 128, 7, 40, 11, 11, 0, 0, "fp32", "bf16"),      # 12 query heads on one kv head; no system tokens
+    (1, 4, 4, 128, 50, 10, 8, 0, 70, 0, "bf16", "bf16"),       # nothing selected: system tokens only
+])
+def test_attend_matches_oracle(orc, L, H_q, H_k, d, G, T, k, n_sel, sys_len, mode, dtype, cache):
+    from paper_2510_18269_b200 import oqm
+    oqm.lib()
+    sh = synth.Shape("attend", L=L, H_q=H_q, H_k=H_k, d=d, G=G, T=T, T_q=1, k=k, dtype=dtype, seed=3)
+    ocfg, gcfg, ost, gst, _ = P.random_bank(orc, oqm, sh, mode, seed=17 * k + sys_len)
+    rng = np.random.default_rng(5 + k)
+    rows = L * (H_k if mode else 1)
+    idx = _selection(rng, rows, T, k, n_sel)
+
+    cdt = torch.bfloat16 if cache == "bf16" else torch.float16
+    ccode = P.dt_code(cache)
+    g = torch.Generator().manual_seed(21)
+    q = torch.randn(L, H_q, d, generator=g).to(synth.DTYPES[dtype]).contiguous()
+    S = sys_len + k * G
+    k_act = torch.randn(L, H_k, S, d, generator=g).to(cdt).contiguous()     # system tokens in front, rest overwritten
+    v_act = torch.randn(L, H_k, S, d, generator=g).to(cdt).contiguous()
+
+    # oracle: materialise the cache, then plain attention over its first sys_len + n_sel*G tokens
+    oka, ova = P.as_np16(k_act).copy(), P.as_np16(v_act).copy()
+    assert orc.dequant_gather(ocfg, ost, 0, L, idx, k, T, oka, ova, ccode, P.active_strides(sh, S), sys_len) == 0
+    n_tok = sys_len + n_sel * G
+    scale = 1.0 / np.sqrt(d)
+    qn = P.as_np16(q)
+    want = np.stack([orc.to_f32(orc.attend(H_q, H_k, d, qn[l], P.dt_code(dtype), oka[l], ova[l], ccode, S * d, d,
+                                           n_tok, scale, out_dtype=ccode), ccode) for l in range(L)])
+
+    ws = torch.empty(oqm.stom_oqm_attend_workspace_bytes(gcfg, L, k, sys_len) + 256, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 256:]
+    out_flat = torch.full((L * H_q * d + P.GUARD,), 3.0, dtype=cdt, device="cuda")
+    out = out_flat[:L * H_q * d].view(L, H_q, d)
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ks, vs = k_act.cuda(), v_act.cuda()
+    for _ in range(2):   # twice: the second call finds the counters as the first one left them
+        oqm.stom_oqm_attend(gcfg, gst, 0, L, torch.from_numpy(idx).cuda(), k, T, q.cuda(), (H_q * d, d), ks, vs, ccode,
+                            P.active_strides(sh, S), sys_len, float(scale), out, (H_q * d, d), ws, dev_flags=flags)
+    torch.cuda.synchronize()
+    assert int(flags.item()) == 0
+    assert torch.all(out_flat[L * H_q * d:] == 3.0), "guard band overwritten"
+    got = orc.to_f32(P.as_np16(out), ccode)
+    err = np.abs(got - want)
+    tol = np.maximum(TOL, 2.0 ** -7 * np.abs(want))
+    assert np.isfinite(got).all() and np.all(err <= tol), f"attention output differs by {err.max()}"
+    assert err.mean() <= 0.2 * TOL, f"mean error {err.mean()} is too close to the tolerance to be rounding noise"
+    assert np.abs(want).max() > 0.05, "degenerate case: outputs too small to mean anything"
+
+
+def test_attend_flags_bad_indices_and_skips_them(orc):
+    from paper_2510_18269_b200 import oqm
+    sh = synth.Shape("attend-bad", L=1, H_q=4, H_k=2, d=128, G=8, T=12, T_q=1, k=4, seed=3)
+    ocfg, gcfg, ost, gst, _ = P.random_bank(orc, oqm, sh, 0, seed=9)
+    q = torch.randn(1, 4, 128).to(torch.bfloat16).cuda()
+    ws = torch.empty(oqm.stom_oqm_attend_workspace_bytes(gcfg, 1, 4, 0) + 256, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 256:]
+    outs = []
+    for idx in ([1, 5, 99, -1], [1, 5, -1, -1]):   # 99 is out of range: skipped and flagged
+        out = torch.zeros(1, 4, 128, dtype=torch.bfloat16, device="cuda")
+        flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+        oqm.stom_oqm_attend(gcfg, gst, 0, 1, torch.tensor([idx], dtype=torch.int32).cuda(), 4, 12, q, (512, 128), None,
+                            None, oqm.BF16, (0, 0, 128), 0, 0.088, out, (512, 128), ws, dev_flags=flags)
+        torch.cuda.synchronize()
+        outs.append((out.clone(), int(flags.item())))
+    assert outs[0][1] == oqm.FLAG_BAD_INDEX and outs[1][1] == 0
+    assert torch.equal(outs[0][0], outs[1][0])

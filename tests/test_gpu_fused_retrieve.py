@@ -15,28 +15,6 @@ from paper_2510_18269_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-def _random_bank(orc, oqm, sh, mode, seed):
-    """The same random bank in an oracle Store (NumPy) and in a device Store."""
-    ocfg, gcfg = P.oracle_cfg(orc, sh, mode), P.gpu_cfg(oqm, sh, mode)
-    ost, gst = orc.Store(ocfg), oqm.Store(gcfg)
-    rng = np.random.default_rng(seed)
-    ost.rep_key[...] = rng.standard_normal(ost.rep_key.shape, dtype=np.float32)
-    # a few groups point along a common direction so that the head of the ranking is not pure noise
-    u = rng.standard_normal((sh.L, 1, sh.H_k, sh.d), dtype=np.float32)
-    pick = rng.choice(sh.T, size=max(1, min(sh.T, sh.k) // 2), replace=False)
-    ost.rep_key[:, pick] = u + 0.3 * ost.rep_key[:, pick]
-    ost.rep_norm2[...] = (ost.rep_key.astype(np.float64) ** 2).sum(-1).astype(np.float32)
-    ost.codes_k[...] = rng.integers(0, 256, ost.codes_k.shape, dtype=np.uint8)
-    ost.codes_v[...] = rng.integers(0, 256, ost.codes_v.shape, dtype=np.uint8)
-    for name in ("scale_k", "scale_v"):
-        getattr(ost, name)[...] = rng.uniform(0.01, 0.5, getattr(ost, name).shape).astype(np.float32)
-    for name in ("zero_k", "zero_v"):
-        getattr(ost, name)[...] = rng.standard_normal(getattr(ost, name).shape, dtype=np.float32)
-    for name in ("codes_k", "codes_v", "scale_k", "zero_k", "scale_v", "zero_v", "rep_key", "rep_norm2"):
-        getattr(gst, name).copy_(torch.from_numpy(getattr(ost, name)))
-    return ocfg, gcfg, ost, gst, u
-
-
 @pytest.mark.parametrize("L,H_q,H_k,d,G,T,T_q,k,mode,dtype", [
     (2, 28, 4, 128, 4, 7200, 16, 64, 0, "bf16"),   # 7B geometry, keys of the selecting block in shared memory
     (2, 16, 8, 128, 4, 3600, 5, 64, 0, "bf16"),    # 72B geometry (8 kv heads)
@@ -51,7 +29,7 @@ def test_fused_retrieve_matches_oracle(orc, L, H_q, H_k, d, G, T, T_q, k, mode, 
     from paper_2510_18269_b200 import oqm
     oqm.lib()
     sh = synth.Shape("fused", L=L, H_q=H_q, H_k=H_k, d=d, G=G, T=T, T_q=T_q, k=k, dtype=dtype, seed=5)
-    ocfg, gcfg, ost, gst, u = _random_bank(orc, oqm, sh, mode, seed=T + k)
+    ocfg, gcfg, ost, gst, u = P.random_bank(orc, oqm, sh, mode, seed=T + k)
     rows = L * (H_k if mode else 1)
     rep = H_q // H_k
     g = torch.Generator().manual_seed(99)
