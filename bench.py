@@ -58,7 +58,7 @@ def parse():
     ap.add_argument("--config", default="C3")
     ap.add_argument("--frames-per-call", type=int, default=0, help="0: the whole stream in one quantize call")
     ap.add_argument("--e2e-steps", type=int, default=2)
-    ap.add_argument("--cpu-sample-frames", type=int, default=256)
+    ap.add_argument("--cpu-sample-frames", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--layers", type=int, default=0, help="override L (reduced case for profiler captures)")
