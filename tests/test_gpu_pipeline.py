@@ -1,0 +1,96 @@
+"""The streaming interleave end to end, CUDA library against the oracle driven by the same call sequence: frames of
+196 tokens arrive one at a time, 50 of them are kept by a seeded mask, quantized and appended; every few frames a
+question is scored against what has been stored so far, the top groups are selected and reconstructed behind the
+system tokens, and one decode step attends over the result.  Checked at every question: scores, selection, the
+reconstructed cache (bit for bit), the size of the active cache (system tokens + K*G with K = min(k, stored groups),
+whatever the stream length), and the attention output; at the end: the whole bank."""
+import dataclasses
+
+import numpy as np
+import torch
+
+import pytest
+
+import _parity as P
+from paper_2510_18269_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+
+def test_streaming_interleave_matches_oracle(orc):
+    from paper_2510_18269_b200 import oqm
+    oqm.lib()
+    sh = dataclasses.replace(synth.C4, L=2, H_q=8, H_k=4, T=40, T_q=5, k=8, name="C4-small")
+    every, sys_len = 6, 11
+    K, V = synth.kv_stream(sh)                                       # [L][T][H_k][196][d]
+    keep = synth.keep_mask(sh, 0, sh.T)                              # [T][50]
+    ocfg, gcfg = P.oracle_cfg(orc, sh), P.gpu_cfg(oqm, sh)
+    ost, gst = orc.Store(ocfg), oqm.Store(gcfg)
+    Kd, Vd, keep_d = K.cuda(), V.cuda(), keep.cuda()
+    kn, vn = P.as_np16(K), P.as_np16(V)
+    strides = P.contiguous_strides(sh, sh.N_in)
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    S = sys_len + sh.k * sh.G
+    gen = torch.Generator().manual_seed(8)
+    sys_k = torch.randn(sh.L, sh.H_k, sys_len, sh.d, generator=gen).to(torch.bfloat16)
+    sys_v = torch.randn(sh.L, sh.H_k, sys_len, sh.d, generator=gen).to(torch.bfloat16)
+    ws = torch.empty(oqm.stom_oqm_score_workspace_bytes(gcfg, sh.L), dtype=torch.uint8, device="cuda")
+    aws = torch.empty(oqm.stom_oqm_attend_workspace_bytes(gcfg, sh.L, sh.k, sys_len) + 256, dtype=torch.uint8, device="cuda")
+    aws = aws[(-aws.data_ptr()) % 256:]
+    n_questions = 0
+    for f in range(sh.T):
+        # ---- ingest one frame (all layers in one call)
+        off = f * strides[1]
+        oqm.stom_oqm_quantize_frame(gcfg, gst, 0, sh.L, f, 1, Kd.view(-1)[off:], Vd.view(-1)[off:], strides,
+                                    token_idx=keep_d[f:f + 1], tokens_per_frame_in=sh.N_in, dev_flags=flags)
+        assert orc.quantize_frame(ocfg, ost, 0, sh.L, f, 1, kn.reshape(-1)[off:], vn.reshape(-1)[off:], strides,
+                                  token_idx=keep[f:f + 1].numpy(), tokens_per_frame_in=sh.N_in) == 0
+        if (f + 1) % every:
+            continue
+        # ---- a question over the f + 1 groups stored so far
+        n_questions += 1
+        n = f + 1
+        qsh = dataclasses.replace(sh, seed=sh.seed + n)
+        Q = synth.queries(qsh)
+        o_scores = orc.score_groups(ocfg, ost, 0, sh.L, n, P.as_np16(Q), sh.T_q, P.q_strides(sh))
+        o_idx, _, o_nsel = orc.topk(o_scores.reshape(sh.L, n), sh.k)
+        ka = torch.zeros(sh.L, sh.H_k, S, sh.d, dtype=torch.bfloat16)
+        va = torch.zeros_like(ka)
+        ka[:, :, :sys_len], va[:, :, :sys_len] = sys_k, sys_v
+        oka, ova = P.as_np16(ka).copy(), P.as_np16(va).copy()
+        ka, va = ka.cuda(), va.cuda()
+        scores = torch.empty(sh.L, n, dtype=torch.float32, device="cuda")
+        idx = torch.empty(sh.L, sh.k, dtype=torch.int32, device="cuda")
+        oqm.stom_oqm_retrieve(gcfg, gst, 0, sh.L, n, Q.cuda(), sh.T_q, P.q_strides(sh), sh.k, scores, idx, ka, va,
+                              oqm.BF16, P.active_strides(sh, S), sys_len, ws, dev_flags=flags)
+        torch.cuda.synchronize()
+        P.compare_scores(scores, o_scores)
+        P.compare_topk(idx, o_idx, o_scores.reshape(sh.L, n), sh.k)
+        K_sel = min(sh.k, n)
+        assert np.all(o_nsel == K_sel)
+        g_idx = idx.cpu().numpy().copy()
+        assert np.all(g_idx[:, :K_sel] >= 0) and np.all(g_idx[:, K_sel:] == -1)
+        assert orc.dequant_gather(ocfg, ost, 0, sh.L, g_idx, sh.k, n, oka, ova, orc.BF16, P.active_strides(sh, S),
+                                  sys_len) == 0
+        assert np.array_equal(P.as_np16(ka), oka) and np.array_equal(P.as_np16(va), ova)
+        # the active cache never exceeds the system tokens plus K groups, however long the stream is
+        n_active = sys_len + K_sel * sh.G
+        assert n_active <= S and torch.all(ka[:, :, n_active:] == 0)
+        # ---- one decode step over [system tokens || selected groups]
+        q_dec = torch.randn(sh.L, sh.H_q, sh.d, generator=gen).to(torch.bfloat16)
+        out = torch.zeros(sh.L, sh.H_q, sh.d, dtype=torch.bfloat16, device="cuda")
+        scale = 1.0 / np.sqrt(sh.d)
+        oqm.stom_oqm_attend(gcfg, gst, 0, sh.L, idx, sh.k, n, q_dec.cuda(), (sh.H_q * sh.d, sh.d), ka, va, oqm.BF16,
+                            P.active_strides(sh, S), sys_len, float(scale), out, (sh.H_q * sh.d, sh.d), aws,
+                            dev_flags=flags)
+        torch.cuda.synchronize()
+        qn = P.as_np16(q_dec)
+        want = np.stack([orc.to_f32(orc.attend(sh.H_q, sh.H_k, sh.d, qn[l], orc.BF16, oka[l], ova[l], orc.BF16,
+                                               S * sh.d, sh.d, n_active, scale, out_dtype=orc.BF16), orc.BF16)
+                         for l in range(sh.L)])
+        got = orc.to_f32(P.as_np16(out), orc.BF16)
+        assert np.all(np.abs(got - want) <= np.maximum(2e-2, 2.0 ** -7 * np.abs(want)))
+    assert n_questions == sh.T // every and int(flags.item()) == 0
+    Kkept = orc.to_f32(kn, P.dt_code(sh.dtype)).transpose(0, 1, 2, 3, 4)
+    Kkept = np.stack([Kkept[:, f][:, :, keep[f].numpy()] for f in range(sh.T)], axis=1)      # [L][T][H][G][d]
+    P.compare_store(gst, ost, Kkept)
