@@ -61,6 +61,7 @@ def parse():
     ap.add_argument("--cpu-sample-frames", type=int, default=1024)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--query-every", type=int, default=60, help="C4: frames between questions")
     ap.add_argument("--layers", type=int, default=0, help="override L (reduced case for profiler captures)")
     ap.add_argument("--frames", type=int, default=0, help="override T (reduced case for profiler captures)")
     return ap.parse_args()
@@ -176,6 +177,12 @@ def oracle_sample(sh, K_cpu, V_cpu, Q_cpu, frames, threads=0):
             "cores": orc.host_cores()}
 
 
+def cpu_sample_frames(args, sh):
+    """Frames of the CPU sample: --cpu-sample-frames at the 7B geometry, fewer for wider models (same bytes)."""
+    f = args.cpu_sample_frames * (28 * 4) // (sh.L * sh.H_k)
+    return max(16, min(sh.T, f))
+
+
 def cpu_inputs(sh, frames):
     """The first `frames` frames of every layer, generated on the CPU with the same recipe."""
     import dataclasses
@@ -194,7 +201,7 @@ def run_reference(args, sh):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    frames = args.cpu_sample_frames
+    frames = cpu_sample_frames(args, sh)
     K, V, Q = cpu_inputs(sh, frames)
     for _ in range(min(args.warmup, 1)):
         oracle_sample(sh, K, V, Q, min(frames, 16))
@@ -392,7 +399,7 @@ def run_ours(args, sh):
         out["e2e"] = run_e2e(args, sh, cfg, store, K, V, Q, dev, world, sdist, rbytes)
     # ---- the oracle on this machine's host cores, rank 0 only, single-GPU runs only
     if not args.no_cpu_baseline and rank == 0 and world == 1:
-        frames = args.cpu_sample_frames
+        frames = cpu_sample_frames(args, sh)
         Kc, Vc, Qc = cpu_inputs(sh, frames)
         info = oracle_sample(sh, Kc, Vc, Qc, frames)
         k = info["k"]
@@ -459,10 +466,110 @@ def run_e2e(args, sh, cfg, store, K, V, Q, dev, world, sdist, rbytes):
     }
 
 
+def run_stream(args, sh):
+    """The streaming interleave (C4): frames of N_in tokens arrive one at a time, G of them are kept by a seeded mask and
+    quantized on arrival (all layers in one call); every `--query-every` frames a question runs retrieval over what is
+    stored so far and one decode-attention step over [system tokens || selected groups].  Reports latencies."""
+    import torch
+    from paper_2510_18269_b200 import oqm, synth
+    import dataclasses
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    oqm.lib()
+    cfg = oqm.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, sh.T, 4, oqm.dtype_code(synth.DTYPES[sh.dtype]))
+    store = oqm.Store(cfg, device=dev, zero=False)
+    pool = 32                                    # distinct synthetic frames, cycled (5.6 MB of K and of V per frame)
+    psh = dataclasses.replace(sh, T=pool)
+    K, V = synth.kv_stream(psh, dev)             # [L][pool][H_k][N_in][d]
+    keep = synth.keep_mask(sh, 0, sh.T).to(dev)  # [T][G]
+    strides = (pool * sh.H_k * sh.N_in * sh.d, sh.H_k * sh.N_in * sh.d, sh.N_in * sh.d, sh.d)
+    qs = (sh.H_q * sh.T_q * sh.d, sh.T_q * sh.d, sh.d)
+    sys_len = 32
+    S = sys_len + sh.k * sh.G
+    act = (sh.H_k * S * sh.d, S * sh.d, sh.d)
+    Q = synth.queries(sh, dev)
+    q_dec = torch.randn(sh.L, sh.H_q, sh.d, device=dev).to(torch.bfloat16)
+    ka = torch.randn(sh.L, sh.H_k, S, sh.d, device=dev).to(torch.bfloat16)
+    va = torch.randn(sh.L, sh.H_k, S, sh.d, device=dev).to(torch.bfloat16)
+    scores = torch.empty(sh.L, sh.T, dtype=torch.float32, device=dev)
+    idx = torch.empty(sh.L, sh.k, dtype=torch.int32, device=dev)
+    out = torch.empty(sh.L, sh.H_q, sh.d, dtype=torch.bfloat16, device=dev)
+    ws = torch.empty(oqm.stom_oqm_score_workspace_bytes(cfg, sh.L), dtype=torch.uint8, device=dev)
+    aws = torch.empty(oqm.stom_oqm_attend_workspace_bytes(cfg, sh.L, sh.k, sys_len) + 256, dtype=torch.uint8, device=dev)
+    aws = aws[(-aws.data_ptr()) % 256:]
+    flags = torch.zeros(1, dtype=torch.int32, device=dev)
+    scale = float(sh.d) ** -0.5
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def ingest(f):
+        off = (f % pool) * strides[1]
+        oqm.stom_oqm_quantize_frame(cfg, store, 0, sh.L, f, 1, K.view(-1)[off:], V.view(-1)[off:], strides,
+                                    token_idx=keep[f:f + 1], tokens_per_frame_in=sh.N_in, dev_flags=flags)
+
+    def question(n):
+        sc = scores.view(-1)[:sh.L * n].view(sh.L, n)
+        oqm.stom_oqm_retrieve(cfg, store, 0, sh.L, n, Q, sh.T_q, qs, sh.k, sc, idx, ka, va, oqm.BF16, act, sys_len, ws,
+                              dev_flags=flags)
+
+    def decode(n):
+        oqm.stom_oqm_attend(cfg, store, 0, sh.L, idx, sh.k, n, q_dec, (sh.H_q * sh.d, sh.d), ka, va, oqm.BF16, act,
+                            sys_len, scale, out, (sh.H_q * sh.d, sh.d), aws, dev_flags=flags)
+
+    for f in range(8):                           # warm-up (slots are rewritten by the timed pass)
+        ingest(f)
+    question(8)
+    decode(8)
+    torch.cuda.synchronize()
+    ing, qry, dec = [], [], []
+    every = args.query_every
+    t0 = time.perf_counter()
+    for f in range(sh.T):
+        a, b = ev(), ev()
+        a.record(); ingest(f); b.record()
+        ing.append((a, b))
+        if (f + 1) % every == 0:
+            a, b, c = ev(), ev(), ev()
+            a.record(); question(f + 1); b.record(); decode(f + 1); c.record()
+            qry.append((a, b)); dec.append((b, c))
+        if f % 256 == 255:
+            torch.cuda.synchronize()             # bounds the number of events in flight
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    assert int(flags.item()) == 0
+
+    def stats(pairs):
+        v = sorted(x.elapsed_time(y) * 1e3 for x, y in pairs)
+        return {"p50_us": v[len(v) // 2], "p99_us": v[min(len(v) - 1, int(0.99 * len(v)))], "mean_us": statistics.mean(v),
+                "max_us": v[-1], "n": len(v)}
+
+    i_st, q_st, d_st = stats(ing), stats(qry), stats(dec)
+    frame_bytes = sh.L * (2 * sh.H_k * sh.G * sh.d * 2 + 2 * sh.H_k * sh.G * sh.d // 2 + 5 * sh.H_k * sh.d * 4 + sh.H_k * 4)
+    print(json.dumps({
+        "metric": "per-query OQM latency (score + top-k + dequant-gather + decode attention), streaming interleave",
+        "value": q_st["p50_us"] + d_st["p50_us"], "unit": "us", "n_gpus": 1, "steps": sh.T, "warmup": 8,
+        "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": sh.name, "L": sh.L, "H_q": sh.H_q, "H_k": sh.H_k, "d": sh.d, "tokens_per_frame": sh.N_in,
+                   "kept_per_frame": sh.G, "frames": sh.T, "query_every": every, "T_q": sh.T_q, "k": sh.k,
+                   "system_tokens": sys_len, "frame_pool": pool},
+        "per_frame_ingest": dict(i_st, algorithmic_bytes=frame_bytes),
+        "per_query_retrieve": q_st, "per_decode_step_attend_all_layers": d_st,
+        "wall_s_including_python": wall,
+        "note": "CUDA-event times of single calls issued from Python one after the other; latencies, not bandwidths",
+    }))
+
+
 def main():
     args = parse()
     from paper_2510_18269_b200 import synth
     sh = synth.CONFIGS[args.config]
+    if args.config == "C4" and args.impl == "ours":
+        if args.frames:
+            import dataclasses
+            sh = dataclasses.replace(sh, T=args.frames)
+        run_stream(args, sh)
+        return
     if args.layers or args.frames:
         import dataclasses
         sh = dataclasses.replace(sh, L=args.layers or sh.L, T=args.frames or sh.T,

@@ -94,28 +94,74 @@ __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p
     const CT *ksys = reinterpret_cast<const CT *>(p.ksys) + (int64_t)li * p.s_sl + (int64_t)h * p.s_sh + cl * 8;
     const CT *vsys = reinterpret_cast<const CT *>(p.vsys) + (int64_t)li * p.s_sl + (int64_t)h * p.s_sh + cl * 8;
 
-    // 8 channels of one token as floats: a system token is read as stored, a group token is rebuilt from its code word
-    auto token8 = [&](bool keys, int g, const float (&s)[8], const float (&m)[8], float (&x)[8]) {
-        if (sys_begin >= 0) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4 *>((keys ? ksys : vsys) + (int64_t)(sys_begin + g) * p.s_st));
-            unpack2<CT>(v.x, x[0], x[1]);
-            unpack2<CT>(v.y, x[2], x[3]);
-            unpack2<CT>(v.z, x[4], x[5]);
-            unpack2<CT>(v.w, x[6], x[7]);
+    // Tokens go through in batches whose loads are all issued before the first use (a decode step is pure latency):
+    // 16 passes of group tokens (one code word per lane and pass) or 4 passes of system tokens (16 bytes per lane).
+    constexpr int kRaw = 16;
+    const bool is_sys = sys_begin >= 0;
+    const int batch_passes = is_sys ? kRaw / 4 : kRaw;
+    auto load_batch = [&](bool keys, int g0, uint32_t (&raw)[kRaw]) {
+        if (is_sys) {
+            const CT *base = keys ? ksys : vsys;
+#pragma unroll
+            for (int b = 0; b < kRaw / 4; ++b) {
+                const int g = g0 + b * TPW + sub;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (g < n_tok) v = __ldg(reinterpret_cast<const uint4 *>(base + (int64_t)(sys_begin + g) * p.s_st));
+                raw[4 * b] = v.x; raw[4 * b + 1] = v.y; raw[4 * b + 2] = v.z; raw[4 * b + 3] = v.w;
+            }
         } else {
             const uint32_t *codes = reinterpret_cast<const uint32_t *>((keys ? p.codes_k : p.codes_v) +
                                                                        slot * (int64_t)G * p.g.row_bytes) + cl;
-            const uint32_t w = __ldg(codes + (int64_t)g * wpr);
-            const uint32_t even = w & 0x0f0f0f0fu, odd = (w >> 4) & 0x0f0f0f0fu;
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                x[2 * i] = __fmaf_rn(code_float(even, i), s[2 * i], m[2 * i]);
-                x[2 * i + 1] = __fmaf_rn(code_float(odd, i), s[2 * i + 1], m[2 * i + 1]);
+            for (int b = 0; b < kRaw; ++b) {
+                const int g = g0 + b * TPW + sub;
+                raw[b] = g < n_tok ? __ldg(codes + (int64_t)g * wpr) : 0u;
+            }
+        }
+    };
+    // 8 channels of the token of pass b of a batch as floats: a system token as stored, a group token rebuilt
+    auto sys8 = [&](const uint32_t (&raw)[kRaw], int b, float (&x)[8]) {
+        unpack2<CT>(raw[4 * b], x[0], x[1]);
+        unpack2<CT>(raw[4 * b + 1], x[2], x[3]);
+        unpack2<CT>(raw[4 * b + 2], x[4], x[5]);
+        unpack2<CT>(raw[4 * b + 3], x[6], x[7]);
+    };
+    auto group8 = [&](uint32_t w, const float (&s)[8], const float (&m)[8], float (&x)[8]) {
+        const uint32_t even = w & 0x0f0f0f0fu, odd = (w >> 4) & 0x0f0f0f0fu;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            x[2 * i] = __fmaf_rn(code_float(even, i), s[2 * i], m[2 * i]);
+            x[2 * i + 1] = __fmaf_rn(code_float(odd, i), s[2 * i + 1], m[2 * i + 1]);
+        }
+    };
+    // runs f(g, x) for every token of the warp's segment, keys or values
+    auto for_tokens = [&](bool keys, const float (&s)[8], const float (&m)[8], auto &&f) {
+        for (int g0 = 0; g0 < n_tok; g0 += TPW * batch_passes) {
+            uint32_t raw[kRaw];
+            load_batch(keys, g0, raw);
+            if (is_sys) {
+#pragma unroll
+                for (int b = 0; b < kRaw / 4; ++b) {
+                    if (g0 + b * TPW < n_tok) {  // warp-uniform
+                        float x[8];
+                        sys8(raw, b, x);
+                        f(g0 + b * TPW + sub, x);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int b = 0; b < kRaw; ++b) {
+                    if (g0 + b * TPW < n_tok) {  // warp-uniform
+                        float x[8];
+                        group8(raw[b], s, m, x);
+                        f(g0 + b * TPW + sub, x);
+                    }
+                }
             }
         }
     };
     auto load_stats = [&](bool keys, float (&s)[8], float (&m)[8]) {
-        if (sys_begin >= 0 || n_tok == 0) return;
+        if (is_sys || n_tok == 0) return;
         const float4 *sp = reinterpret_cast<const float4 *>((keys ? p.scale_k : p.scale_v) + slot * D + cl * 8);
         const float4 *mp = reinterpret_cast<const float4 *>((keys ? p.zero_k : p.zero_v) + slot * D + cl * 8);
         const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1), m0 = __ldg(mp), m1 = __ldg(mp + 1);
@@ -150,36 +196,32 @@ __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p
                 q8[hh][0] = a.x; q8[hh][1] = a.y; q8[hh][2] = a.z; q8[hh][3] = a.w;
                 q8[hh][4] = b.x; q8[hh][5] = b.y; q8[hh][6] = b.z; q8[hh][7] = b.w;
             }
-            for (int g0 = 0; g0 < kAtSegTokens; g0 += TPW) {
-                const int g = g0 + sub;
+            // slots without a token score -inf
+            for (int e = lane; e < kAtHeads * kAtSegTokens; e += 32)
+                sc[e / kAtSegTokens][warp * kAtSegTokens + (e % kAtSegTokens)] = -INFINITY;
+            __syncwarp();
+            for_tokens(true, s, m, [&](int g, const float (&x)[8]) {
                 float dot[kAtHeads];
 #pragma unroll
-                for (int hh = 0; hh < kAtHeads; ++hh) dot[hh] = 0.0f;
-                if (g0 < n_tok) {  // warp-uniform
-                    float x[8];
+                for (int hh = 0; hh < kAtHeads; ++hh) {
+                    dot[hh] = 0.0f;
 #pragma unroll
-                    for (int c = 0; c < 8; ++c) x[c] = 0.0f;
-                    if (g < n_tok) token8(true, g, s, m, x);
+                    for (int c = 0; c < 8; ++c) dot[hh] = fmaf(x[c], q8[hh][c], dot[hh]);
+                }
 #pragma unroll
-                    for (int hh = 0; hh < kAtHeads; ++hh) {
+                for (int o = LPR / 2; o > 0; o >>= 1) {
 #pragma unroll
-                        for (int c = 0; c < 8; ++c) dot[hh] = fmaf(x[c], q8[hh][c], dot[hh]);
-                    }
-#pragma unroll
-                    for (int o = LPR / 2; o > 0; o >>= 1) {
-#pragma unroll
-                        for (int hh = 0; hh < kAtHeads; ++hh) dot[hh] += __shfl_xor_sync(0xffffffffu, dot[hh], o);
-                    }
+                    for (int hh = 0; hh < kAtHeads; ++hh) dot[hh] += __shfl_xor_sync(0xffffffffu, dot[hh], o);
                 }
                 // lane cl of the token's lanes files the score of query head cl
-                if (cl < kAtHeads) {
+                if (cl < kAtHeads && g < n_tok) {
                     float mine = dot[0];
 #pragma unroll
                     for (int hh = 1; hh < kAtHeads; ++hh)
                         if (cl == hh) mine = dot[hh];
-                    sc[cl][warp * kAtSegTokens + g] = g < n_tok ? mine : -INFINITY;
+                    sc[cl][warp * kAtSegTokens + g] = mine;
                 }
-            }
+            });
         }
         __syncthreads();
 
@@ -214,11 +256,8 @@ __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p
         {
             float s[8], m[8];
             load_stats(false, s, m);
-            for (int g0 = 0; g0 < n_tok; g0 += TPW) {
-                const int g = g0 + sub;
+            for_tokens(false, s, m, [&](int g, const float (&x)[8]) {
                 if (g < n_tok) {
-                    float x[8];
-                    token8(false, g, s, m, x);
 #pragma unroll
                     for (int hh = 0; hh < kAtHeads; ++hh) {
                         const float w = sc[hh][warp * kAtSegTokens + g];
@@ -226,7 +265,7 @@ __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p
                         for (int c = 0; c < 8; ++c) acc[hh][c] = fmaf(w, x[c], acc[hh][c]);
                     }
                 }
-            }
+            });
             // the token slots of a warp pass hold different tokens of the same channels
 #pragma unroll
             for (int o = LPR; o < 32; o <<= 1) {
@@ -281,23 +320,35 @@ __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p
     if (!s_last) return;
     __threadfence();
     if (tid == 0) p.counters[li * H + h] = 0;  // as found
-    for (int e = tid; e < p.rep * D; e += kAtThreads) {
-        const int hq = e / D, c = e - hq * D;
+    // one warp per query head: lanes first share out the blocks (max, then the sum of the weighted sums of
+    // weights), then the channels, with the loads of several blocks in flight
+    for (int hq = warp; hq < p.rep; hq += kAtWarps) {
         const float *rec0 = p.part + (((int64_t)li * H + h) * n_blocks * p.rep + hq) * (D + 2);
         const int64_t step = (int64_t)p.rep * (D + 2);
         float mx = -INFINITY;
-        for (int b = 0; b < n_blocks; ++b) mx = fmaxf(mx, __ldcg(rec0 + b * step));
-        float num = 0.0f, den = 0.0f;
+        for (int b = lane; b < n_blocks; b += 32) mx = fmaxf(mx, __ldcg(rec0 + b * step));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float den = 0.0f;
+        for (int b = lane; b < n_blocks; b += 32) {
+            const float mb = __ldcg(rec0 + b * step);
+            if (mb != -INFINITY) den = fmaf(__ldcg(rec0 + b * step + 1), exp2f(mb - mx), den);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+        float num[D / 32];
+#pragma unroll
+        for (int i = 0; i < D / 32; ++i) num[i] = 0.0f;
+#pragma unroll 4
         for (int b = 0; b < n_blocks; ++b) {
             const float mb = __ldcg(rec0 + b * step);
-            if (mb == -INFINITY) continue;
-            const float w = exp2f(mb - mx);
-            den = fmaf(__ldcg(rec0 + b * step + 1), w, den);
-            num = fmaf(__ldcg(rec0 + b * step + 2 + c), w, num);
+            const float w = mb == -INFINITY ? 0.0f : exp2f(mb - mx);
+#pragma unroll
+            for (int i = 0; i < D / 32; ++i) num[i] = fmaf(__ldcg(rec0 + b * step + 2 + lane + 32 * i), w, num[i]);
         }
-        const float o = den > 0.0f ? num / den : 0.0f;
         CT *out = reinterpret_cast<CT *>(p.out) + (int64_t)li * p.o_sl + (int64_t)(h * p.rep + hq) * p.o_sh;
-        out[c] = (CT)o;
+#pragma unroll
+        for (int i = 0; i < D / 32; ++i) out[lane + 32 * i] = (CT)(den > 0.0f ? num[i] / den : 0.0f);
     }
 }
 
