@@ -40,12 +40,13 @@ FALLBACK_HBM_GBS = 6650.0
 # dram bytes per unit of work measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum) on a reduced
 # case of the same kernel and scaled by the units one launch processes; see profiles/*.md.  None = not captured.
 NCU_TRAFFIC_PER_UNIT = {
-    "quantize_kernel": 137448.0,        # bytes per (layer, frame): 3.941 GB over 28 x 1024 units
+    # all figures are per kv head of the unit named (the captures ran the 4-head 7B geometry)
+    "quantize_kernel": 137448.0 / 4,    # bytes per (layer, frame): 3.941 GB over 28 x 1024 units
     # bytes per (layer, selected group): 186.3 MB over 28 x 64 units; of the 183.5 MB the kernel writes only
     # 125.7 MB had left L2 when it ended (the rest is written back later), so this undercounts by design
-    "dequant_gather_kernel": 103985.0,
-    "score_kernel": 2066.0,             # bytes per (layer, stored group): 59.25 MB over 28 x 1024 units
-    "retrieve_kernel": 2178.0,          # bytes per (layer, stored group): 62.46 MB over 28 x 1024 units (Q re-read per block)
+    "dequant_gather_kernel": 103985.0 / 4,
+    "score_kernel": 2066.0 / 4,         # bytes per (layer, stored group): 59.25 MB over 28 x 1024 units
+    "retrieve_kernel": 2178.0 / 4,      # bytes per (layer, stored group): 62.46 MB over 28 x 1024 units (Q re-read per block)
 }
 
 
@@ -357,7 +358,7 @@ def run_ours(args, sh):
         a = nbytes / launches / (ms / launches * 1e-3) / 1e9
         tpu = NCU_TRAFFIC_PER_UNIT.get(name)
         return {"kernel": name, "bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s", "frac": a / peak,
-                "traffic": None if tpu is None else tpu * unit_count / launches, "peak_source": peak_src,
+                "traffic": None if tpu is None else tpu * sh.H_k * unit_count / launches, "peak_source": peak_src,
                 "algorithmic_bytes_per_launch": nbytes / launches, "ms_per_launch": ms / launches}
 
     roofs = [

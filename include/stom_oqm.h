@@ -72,7 +72,7 @@ typedef struct stom_oqm_config {
     int32_t head_dim;        /* d: 32, 64, 128 or 256                           */
     int32_t group_tokens;    /* G, tokens per group (frame); 1..64              */
     int32_t capacity_groups; /* groups the bank can hold per layer              */
-    int32_t bits;            /* 4                                               */
+    int32_t bits;            /* 4 (the paper's setting) or 2 (its ablation)     */
     int32_t kv_dtype;        /* STOM_BF16 | STOM_FP16 | STOM_FP32: type of K, V, Q inputs */
     int32_t score_mode;      /* STOM_SCORE_PER_LAYER | STOM_SCORE_PER_HEAD      */
 } stom_oqm_config;
@@ -80,8 +80,9 @@ typedef struct stom_oqm_config {
 /*
  * The memory bank M_t (Sec. 3.4): device arrays, all caller-owned, each
  * indexed [layer][group][kv head]... with `capacity_groups` groups per layer.
- *   codes_*   [L][cap][H_k][G][d/2]  uint8: two 4-bit codes per byte along
- *             the channel axis, even channel in the low nibble
+ *   codes_*   [L][cap][H_k][G][d*bits/8]  uint8: 8/bits codes per byte along
+ *             the channel axis, lowest channel in the lowest bits (bits = 4:
+ *             two per byte, even channel in the low nibble)
  *   scale_*   [L][cap][H_k][d] float: s = (max - min)/15 over the G tokens
  *   zero_*    [L][cap][H_k][d] float: m = min over the G tokens
  *   rep_key   [L][cap][H_k][d] float: mean of the group's keys (k-bar)
@@ -144,6 +145,8 @@ int32_t stom_last_cuda_error(void);
  *     m = min_g x,  s = (max_g x - m)/15,
  *     code = clamp(rne((x - m)/s), 0, 15)   (binary32, true division;
  *                                            s == 0 -> every code 0)
+ * (with cfg->bits == 2, the variant of the paper's ablation table: 3 in place
+ * of 15, four codes per byte)
  * for K and for V, and for K also k-bar[c] = mean_g and |k-bar_h|^2.  Results
  * go to bank slot group_begin + f of layer l.  Older groups are never read.
  *

@@ -12,13 +12,13 @@ int32_t check_config(const stom_oqm_config *c) {
     if (!c) return STOM_ERR_INVALID_ARG;
     if (c->n_layers < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1 || c->capacity_groups < 1) return STOM_ERR_INVALID_ARG;
     if (c->n_q_heads % c->n_kv_heads) return STOM_ERR_SHAPE;
-    if (c->bits != 4) return STOM_ERR_UNSUPPORTED;
+    if (c->bits != 4 && c->bits != 2) return STOM_ERR_UNSUPPORTED;
     if (c->kv_dtype != STOM_BF16 && c->kv_dtype != STOM_FP16 && c->kv_dtype != STOM_FP32) return STOM_ERR_UNSUPPORTED;
     if (c->score_mode != STOM_SCORE_PER_LAYER && c->score_mode != STOM_SCORE_PER_HEAD) return STOM_ERR_UNSUPPORTED;
     if (c->head_dim != 64 && c->head_dim != 128 && c->head_dim != 256) return STOM_ERR_SHAPE;
     if (c->group_tokens < 1 || c->group_tokens > 64) return STOM_ERR_SHAPE;
     // one (group, head) block of codes must keep 16-byte alignment for vector stores
-    if (((int64_t)c->group_tokens * c->head_dim / 2) % 16) return STOM_ERR_SHAPE;
+    if (((int64_t)c->group_tokens * c->head_dim * c->bits / 8) % 16) return STOM_ERR_SHAPE;
     return STOM_OK;
 }
 

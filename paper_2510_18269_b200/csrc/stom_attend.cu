@@ -48,13 +48,9 @@ struct AttendParams {
     uint32_t *flags;
 };
 
-// 2^23 + code as a float for the code byte i of `bytes` (see the dequantize-gather kernel), minus 2^23
-__device__ __forceinline__ float code_float(uint32_t bytes, int i) {
-    return __uint_as_float(__byte_perm(bytes, 0x4B000000u, 0x7540u + i)) - 8388608.0f;
-}
-
-// QT: type of q_dec; CT: type of the system-token cache and of the output; LPR: lanes per token (d / 8)
-template <typename QT, typename CT, int LPR>
+// QT: type of q_dec; CT: type of the system-token cache and of the output; LPR: lanes per token (d / 8);
+// BITS: width of a code
+template <typename QT, typename CT, int LPR, int BITS>
 __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p) {
     constexpr int D = LPR * 8;
     constexpr int TPW = 32 / LPR;  // tokens one warp pass covers
@@ -90,7 +86,6 @@ __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p
             atomicOr(p.flags, STOM_FLAG_BAD_INDEX);
         }
     }
-    const int wpr = p.g.row_bytes >> 2;  // 32-bit words per packed row
     const CT *ksys = reinterpret_cast<const CT *>(p.ksys) + (int64_t)li * p.s_sl + (int64_t)h * p.s_sh + cl * 8;
     const CT *vsys = reinterpret_cast<const CT *>(p.vsys) + (int64_t)li * p.s_sl + (int64_t)h * p.s_sh + cl * 8;
 
@@ -110,12 +105,11 @@ __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p
                 raw[4 * b] = v.x; raw[4 * b + 1] = v.y; raw[4 * b + 2] = v.z; raw[4 * b + 3] = v.w;
             }
         } else {
-            const uint32_t *codes = reinterpret_cast<const uint32_t *>((keys ? p.codes_k : p.codes_v) +
-                                                                       slot * (int64_t)G * p.g.row_bytes) + cl;
+            const uint8_t *codes = (keys ? p.codes_k : p.codes_v) + slot * (int64_t)G * p.g.row_bytes;
 #pragma unroll
             for (int b = 0; b < kRaw; ++b) {
                 const int g = g0 + b * TPW + sub;
-                raw[b] = g < n_tok ? __ldg(codes + (int64_t)g * wpr) : 0u;
+                raw[b] = g < n_tok ? load_codes8<BITS>(codes + (int64_t)g * p.g.row_bytes, cl) : 0u;
             }
         }
     };
@@ -127,12 +121,10 @@ __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p
         unpack2<CT>(raw[4 * b + 3], x[6], x[7]);
     };
     auto group8 = [&](uint32_t w, const float (&s)[8], const float (&m)[8], float (&x)[8]) {
-        const uint32_t even = w & 0x0f0f0f0fu, odd = (w >> 4) & 0x0f0f0f0fu;
+        uint32_t f[8];
+        code_floats8<BITS>(w, f);
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            x[2 * i] = __fmaf_rn(code_float(even, i), s[2 * i], m[2 * i]);
-            x[2 * i + 1] = __fmaf_rn(code_float(odd, i), s[2 * i + 1], m[2 * i + 1]);
-        }
+        for (int c = 0; c < 8; ++c) x[c] = __fmaf_rn(__uint_as_float(f[c]) - 8388608.0f, s[c], m[c]);
     };
     // runs f(g, x) for every token of the warp's segment, keys or values
     auto for_tokens = [&](bool keys, const float (&s)[8], const float (&m)[8], auto &&f) {
@@ -360,10 +352,20 @@ static int attend_segments(const stom_oqm_config *cfg, int32_t k, int32_t sys_le
 
 template <typename QT, typename CT>
 static int32_t launch_attend(const AttendParams &p, dim3 grid, cudaStream_t s) {
+    const bool b4 = p.g.row_bytes * 2 == p.g.d;  // 4-bit codes: d/2 bytes per row
     switch (p.g.d) {
-    case 64: attend_kernel<QT, CT, 8><<<grid, kAtThreads, 0, s>>>(p); break;
-    case 128: attend_kernel<QT, CT, 16><<<grid, kAtThreads, 0, s>>>(p); break;
-    case 256: attend_kernel<QT, CT, 32><<<grid, kAtThreads, 0, s>>>(p); break;
+    case 64:
+        if (b4) attend_kernel<QT, CT, 8, 4><<<grid, kAtThreads, 0, s>>>(p);
+        else attend_kernel<QT, CT, 8, 2><<<grid, kAtThreads, 0, s>>>(p);
+        break;
+    case 128:
+        if (b4) attend_kernel<QT, CT, 16, 4><<<grid, kAtThreads, 0, s>>>(p);
+        else attend_kernel<QT, CT, 16, 2><<<grid, kAtThreads, 0, s>>>(p);
+        break;
+    case 256:
+        if (b4) attend_kernel<QT, CT, 32, 4><<<grid, kAtThreads, 0, s>>>(p);
+        else attend_kernel<QT, CT, 32, 2><<<grid, kAtThreads, 0, s>>>(p);
+        break;
     default: return STOM_ERR_SHAPE;
     }
     return finish_launch();

@@ -52,8 +52,8 @@ __device__ __forceinline__ uint64_t dq_sub2(uint64_t a, uint64_t b) {
     return d;
 }
 
-// LPR: lanes per token row (d / 8)
-template <typename OT, int LPR>
+// LPR: lanes per token row (d / 8); BITS: width of a code
+template <typename OT, int LPR, int BITS>
 __global__ void __launch_bounds__(kDqWarps * 32) dequant_gather_kernel(const DequantParams p) {
     constexpr int RPP = 32 / LPR;          // rows one warp pass covers
     constexpr int kDqMaxRows = 32 / RPP;   // passes that cover half of the largest group (G <= 64)
@@ -80,14 +80,12 @@ __global__ void __launch_bounds__(kDqWarps * 32) dequant_gather_kernel(const Deq
     const int r_begin = half ? g_half : 0, r_end = half ? G : g_half;
 
     // code words of all this lane's rows first, then the statistics
-    const uint32_t *codes = reinterpret_cast<const uint32_t *>((which ? p.codes_v : p.codes_k) +
-                                                               slot * (int64_t)G * p.g.row_bytes) + cl;
-    const int wpr = p.g.row_bytes >> 2;  // 32-bit words per packed row
+    const uint8_t *codes = (which ? p.codes_v : p.codes_k) + slot * (int64_t)G * p.g.row_bytes;
     uint32_t w[kDqMaxRows];
 #pragma unroll
     for (int b = 0; b < kDqMaxRows; ++b) {
         const int r = r_begin + sub + b * RPP;
-        w[b] = r < r_end ? __ldg(codes + (int64_t)r * wpr) : 0u;
+        w[b] = r < r_end ? load_codes8<BITS>(codes + (int64_t)r * p.g.row_bytes, cl) : 0u;
     }
     uint64_t s2[4], m2[4];
     {
@@ -104,15 +102,11 @@ __global__ void __launch_bounds__(kDqWarps * 32) dequant_gather_kernel(const Deq
     for (int b = 0; b < kDqMaxRows; ++b) {
         const int r = r_begin + sub + b * RPP;
         if (r < r_end) {
-            const uint32_t even = w[b] & 0x0f0f0f0fu;         // byte i: code of channel 2i
-            const uint32_t odd = (w[b] >> 4) & 0x0f0f0f0fu;   // byte i: code of channel 2i+1
-            uint32_t o[4];
+            uint32_t f[8], o[4];
+            code_floats8<BITS>(w[b], f);
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                // 2^23 + code as a float: the code byte goes into the low mantissa byte of 0x4B000000
-                const uint32_t fe = __byte_perm(even, 0x4B000000u, 0x7540u + i);
-                const uint32_t fo = __byte_perm(odd, 0x4B000000u, 0x7540u + i);
-                const uint64_t code = dq_sub2(dq_pack(__uint_as_float(fe), __uint_as_float(fo)), two23);
+                const uint64_t code = dq_sub2(dq_pack(__uint_as_float(f[2 * i]), __uint_as_float(f[2 * i + 1])), two23);
                 float v0, v1;
                 dq_unpack(dq_fma2(code, s2[i], m2[i]), v0, v1);
                 o[i] = pack2<OT>(v0, v1);
@@ -161,20 +155,22 @@ extern "C" int32_t stom_oqm_dequant_gather(const stom_oqm_config *cfg, const sto
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const unsigned nb = (unsigned)blocks, nt = kDqWarps * 32;
     const bool bf = out_dtype == STOM_BF16;
+#define STOM_DQ_LAUNCH(LPR_)                                                                             \
+    do {                                                                                             \
+        if (cfg->bits == 4) {                                                                        \
+            if (bf) dequant_gather_kernel<__nv_bfloat16, LPR_, 4><<<nb, nt, 0, s>>>(p);              \
+            else dequant_gather_kernel<__half, LPR_, 4><<<nb, nt, 0, s>>>(p);                        \
+        } else {                                                                                     \
+            if (bf) dequant_gather_kernel<__nv_bfloat16, LPR_, 2><<<nb, nt, 0, s>>>(p);              \
+            else dequant_gather_kernel<__half, LPR_, 2><<<nb, nt, 0, s>>>(p);                        \
+        }                                                                                            \
+    } while (0)
     switch (cfg->head_dim) {
-    case 64:
-        if (bf) dequant_gather_kernel<__nv_bfloat16, 8><<<nb, nt, 0, s>>>(p);
-        else dequant_gather_kernel<__half, 8><<<nb, nt, 0, s>>>(p);
-        break;
-    case 128:
-        if (bf) dequant_gather_kernel<__nv_bfloat16, 16><<<nb, nt, 0, s>>>(p);
-        else dequant_gather_kernel<__half, 16><<<nb, nt, 0, s>>>(p);
-        break;
-    case 256:
-        if (bf) dequant_gather_kernel<__nv_bfloat16, 32><<<nb, nt, 0, s>>>(p);
-        else dequant_gather_kernel<__half, 32><<<nb, nt, 0, s>>>(p);
-        break;
+    case 64: STOM_DQ_LAUNCH(8); break;
+    case 128: STOM_DQ_LAUNCH(16); break;
+    case 256: STOM_DQ_LAUNCH(32); break;
     default: return STOM_ERR_SHAPE;
     }
+#undef STOM_DQ_LAUNCH
     return finish_launch();
 }

@@ -89,6 +89,35 @@ __device__ __forceinline__ uint32_t pack2<__half>(float a, float b) {
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
+// The codes of 8 adjacent channels (32 bits at 4 bits per code, 16 bits at 2), each as the bit pattern of the float
+// 2^23 + code: a byte permute drops the code into the low mantissa byte of 0x4B000000, so that subtracting 2^23
+// leaves the integer without a conversion instruction.  Channel c sits in bits [BITS*c, BITS*c + BITS).
+template <int BITS>
+__device__ __forceinline__ void code_floats8(uint32_t w, uint32_t (&f)[8]) {
+    if constexpr (BITS == 4) {
+        const uint32_t even = w & 0x0f0f0f0fu;        // byte i: code of channel 2i
+        const uint32_t odd = (w >> 4) & 0x0f0f0f0fu;  // byte i: code of channel 2i+1
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            f[2 * i] = __byte_perm(even, 0x4B000000u, 0x7540u + i);
+            f[2 * i + 1] = __byte_perm(odd, 0x4B000000u, 0x7540u + i);
+        }
+    } else {
+        uint32_t t[4];  // t[j], byte b: code of channel 4b + j
+#pragma unroll
+        for (int j = 0; j < 4; ++j) t[j] = (w >> (2 * j)) & 0x0303u;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) f[c] = __byte_perm(t[c & 3], 0x4B000000u, 0x7540u + (c >> 2));
+    }
+}
+
+// The packed codes of 8 adjacent channels of one row: p points at the row, cl is the 8-channel block.
+template <int BITS>
+__device__ __forceinline__ uint32_t load_codes8(const uint8_t *row, int cl) {
+    if constexpr (BITS == 4) return __ldg(reinterpret_cast<const uint32_t *>(row) + cl);
+    else return __ldg(reinterpret_cast<const uint16_t *>(row) + cl);
+}
+
 // W consecutive 32-bit words from global memory through the read-only path.
 template <int W>
 struct Words {

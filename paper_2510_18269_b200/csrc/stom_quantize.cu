@@ -117,11 +117,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 // ------------------------------------------------------------------ arithmetic
 
 // IEEE division; s == 0 marks a constant (or underflowing) channel whose codes are all 0
-__device__ __forceinline__ uint32_t code_slow(float x, float m, float s) {
+__device__ __forceinline__ uint32_t code_slow(float x, float m, float s, float levels) {
     if (s == 0.0f) return 0u;
     const float t = __fdiv_rn(__fsub_rn(x, m), s);
     float r = rintf(t);
-    r = fminf(fmaxf(r, 0.0f), 15.0f);
+    r = fminf(fmaxf(r, 0.0f), levels);
     return (uint32_t)r;
 }
 
@@ -239,25 +239,35 @@ __device__ __forceinline__ void store_floats(float *dst, const float (&v)[C]) {
 }
 
 
-template <int C>
-__device__ __forceinline__ void store_codes(unsigned char *dst, uint32_t cw) {
-    if constexpr (C == 2) *dst = (unsigned char)cw;
-    else if constexpr (C == 4) *reinterpret_cast<uint16_t *>(dst) = (uint16_t)cw;
-    else *reinterpret_cast<uint32_t *>(dst) = cw;
+// The C * BITS code bits of one row that a lane produced go to dst = row start + byte offset of the lane.  With
+// 2 channels of 2 bits a lane has only half a byte: the even lane takes its neighbour's half and stores for both.
+template <int C, int BITS>
+__device__ __forceinline__ void store_codes(unsigned char *dst, uint32_t cw, int lane) {
+    constexpr int NB = C * BITS;
+    if constexpr (NB == 4) {
+        const uint32_t hi = __shfl_down_sync(0xffffffffu, cw, 1);
+        if (!(lane & 1)) *dst = (unsigned char)((cw & 15u) | (hi << 4));
+    } else if constexpr (NB == 8) {
+        *dst = (unsigned char)cw;
+    } else if constexpr (NB == 16) {
+        *reinterpret_cast<uint16_t *>(dst) = (uint16_t)cw;
+    } else {
+        *reinterpret_cast<uint32_t *>(dst) = cw;
+    }
 }
 
 // Pass 2 on the fast path: the codes of this lane's C channels for all G rows of a tile, written to the staging
 // tile; SUM also adds the rows up (keys: the representative key is their mean).
-template <typename T, int C, bool SUM>
-__device__ __forceinline__ void code_rows(const unsigned char *tile, unsigned char *out_lane, int G,
+template <typename T, int C, int BITS, bool SUM>
+__device__ __forceinline__ void code_rows(const unsigned char *tile, unsigned char *out_lane, int G, int lane,
                                           const uint64_t (&m2)[C / 2], const uint64_t (&ns2)[C / 2],
                                           const uint64_t (&y2)[C / 2], uint64_t (&sum2)[C / 2]) {
-    constexpr int ROW_BYTES = 32 * C * (int)sizeof(T), CODE_ROW = 16 * C;
+    constexpr int ROW_BYTES = 32 * C * (int)sizeof(T), CODE_ROW = 4 * C * BITS;
     const uint64_t magic = pack_f2(12582912.0f, 12582912.0f);  // 1.5 * 2^23: rounds to integer, ties to even
-    // every float 1.5*2^23 + code has the bit pattern 0x4B400000 + code; summing pattern * 16^j over the lane's
-    // channels leaves the nibbles in place in the low 4*C bits (they cannot carry into each other); for C == 8
-    // the constant part wraps into the word and is removed up front
-    constexpr uint32_t kBias = C == 8 ? 0x4B400000u * 0x11111111u : 0u;
+    // every float 1.5*2^23 + code has the bit pattern 0x4B400000 + code; summing pattern << (BITS * channel) over
+    // the lane's channels leaves the codes in place in the low BITS*C bits (they cannot carry into each other);
+    // only with 8 channels of 4 bits does the constant part wrap into the word, and it is removed up front
+    constexpr uint32_t kBias = (C == 8 && BITS == 4) ? 0x4B400000u * 0x11111111u : 0u;
     auto code_word = [&](const LaneRow<T, C> &row) -> uint32_t {
         uint32_t cw = 0u - kBias;
 #pragma unroll
@@ -269,8 +279,8 @@ __device__ __forceinline__ void code_rows(const unsigned char *tile, unsigned ch
             const uint64_t u = code_pair(x, m2[j], ns2[j], y2[j], magic);
             float u0, u1;
             unpack_f2(u, u0, u1);
-            cw += __float_as_uint(u0) << (8 * j);
-            cw += __float_as_uint(u1) << (8 * j + 4);
+            cw += __float_as_uint(u0) << (2 * BITS * j);
+            cw += __float_as_uint(u1) << (2 * BITS * j + BITS);
         }
         return cw;
     };
@@ -287,12 +297,12 @@ __device__ __forceinline__ void code_rows(const unsigned char *tile, unsigned ch
 #pragma unroll
         for (int i = 0; i < kBatch; ++i) cw[i] = code_word(rows[i]);
 #pragma unroll
-        for (int i = 0; i < kBatch; ++i) store_codes<C>(out_lane + (r + i) * CODE_ROW, cw[i]);
+        for (int i = 0; i < kBatch; ++i) store_codes<C, BITS>(out_lane + (r + i) * CODE_ROW, cw[i], lane);
     }
     for (; r < G; ++r) {
         LaneRow<T, C> row;
         row.load(tile + r * ROW_BYTES);
-        store_codes<C>(out_lane + r * CODE_ROW, code_word(row));
+        store_codes<C, BITS>(out_lane + r * CODE_ROW, code_word(row), lane);
     }
 }
 
@@ -326,12 +336,13 @@ constexpr int kBarBytes = 2048;
 static_assert(kAbortOff + 8 <= kInfoOff && kInfoOff + kMaxSlots * (int)sizeof(SlotInfo) <= kBarBytes, "header layout");
 
 // C: channels per lane (d / 32).  blockDim.x = kQuantThreads, one block per SM, grid-stride over tiles.
-template <typename T, int C>
+template <typename T, int C, int BITS>
 __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantParams p) {
+    constexpr float kLevels = (float)((1 << BITS) - 1);  // 15 levels above the offset at 4 bits, 3 at 2 bits
     constexpr int D = 32 * C;
     constexpr int LANE_BYTES = C * (int)sizeof(T);  // bytes of a row that one lane owns
     constexpr int ROW_BYTES = D * (int)sizeof(T);
-    constexpr int CODE_ROW = D / 2;                 // packed bytes per token row
+    constexpr int CODE_ROW = D * BITS / 8;          // packed bytes per token row
     extern __shared__ __align__(128) unsigned char smem[];
     uint64_t *bars = reinterpret_cast<uint64_t *>(smem);
     volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + kAbortOff);
@@ -494,8 +505,8 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
                     float mx0, mx1;
                     a.pair(j, m[2 * j], m[2 * j + 1]);
                     b.pair(j, mx0, mx1);
-                    s[2 * j] = __fdiv_rn(__fsub_rn(mx0, m[2 * j]), 15.0f);
-                    s[2 * j + 1] = __fdiv_rn(__fsub_rn(mx1, m[2 * j + 1]), 15.0f);
+                    s[2 * j] = __fdiv_rn(__fsub_rn(mx0, m[2 * j]), kLevels);
+                    s[2 * j + 1] = __fdiv_rn(__fsub_rn(mx1, m[2 * j + 1]), kLevels);
                 }
 #pragma unroll
                 for (int c = 0; c < C; ++c) {
@@ -507,7 +518,7 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
             store_floats<C>((is_v ? p.zero_v : p.zero_k) + bslot * D + lane * C, m);
             safe = __all_sync(0xffffffffu, safe);
 
-            unsigned char *out_lane = (is_v ? p.codes_v : p.codes_k) + bslot * (int64_t)code_bytes + lane * (C / 2);
+            unsigned char *out_lane = (is_v ? p.codes_v : p.codes_k) + bslot * (int64_t)code_bytes + lane * C * BITS / 8;
 
             // ---- pass 2: codes (and, for keys, the channel sums of the rows as a by-product)
             if (safe) {
@@ -518,8 +529,8 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
                     ns2[j] = pack_f2(-s[2 * j], -s[2 * j + 1]);
                     y2[j] = pack_f2(y[2 * j], y[2 * j + 1]);
                 }
-                if (want_sum) code_rows<T, C, true>(tile, out_lane, G, m2, ns2, y2, sum2);
-                else code_rows<T, C, false>(tile, out_lane, G, m2, ns2, y2, sum2);
+                if (want_sum) code_rows<T, C, BITS, true>(tile, out_lane, G, lane, m2, ns2, y2, sum2);
+                else code_rows<T, C, BITS, false>(tile, out_lane, G, lane, m2, ns2, y2, sum2);
             } else {
 #pragma unroll 2
                 for (int r = 0; r < G; ++r) {
@@ -530,10 +541,10 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
                         float x0, x1;
                         row.pair(j, x0, x1);
                         if (want_sum) sum2[j] = add2(sum2[j], pack_f2(x0, x1));
-                        cw |= code_slow(x0, m[2 * j], s[2 * j]) << (8 * j);
-                        cw |= code_slow(x1, m[2 * j + 1], s[2 * j + 1]) << (8 * j + 4);
+                        cw |= code_slow(x0, m[2 * j], s[2 * j], kLevels) << (2 * BITS * j);
+                        cw |= code_slow(x1, m[2 * j + 1], s[2 * j + 1], kLevels) << (2 * BITS * j + BITS);
                     }
-                    store_codes<C>(out_lane + r * CODE_ROW, cw);
+                    store_codes<C, BITS>(out_lane + r * CODE_ROW, cw, lane);
                 }
             }
             // the input slot is free again
@@ -583,7 +594,7 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
     }
 }
 
-template <typename T, int C>
+template <typename T, int C, int BITS>
 static int32_t launch_quantize(QuantParams p, cudaStream_t stream) {
     int dev = 0, sms = 0, smem_max = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -604,22 +615,22 @@ static int32_t launch_quantize(QuantParams p, cudaStream_t stream) {
     p.n_warps = slots < kConsumerWarps ? slots : kConsumerWarps;
     const int fixed = kBarBytes;
     const size_t smem = (size_t)fixed + (size_t)slots * p.slot_bytes;
-    e = cudaFuncSetAttribute(quantize_kernel<T, C>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(quantize_kernel<T, C, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) {
         set_last_cuda_error(e);
         return STOM_ERR_CUDA;
     }
     const unsigned grid = p.n_tiles < (uint32_t)sms ? p.n_tiles : (unsigned)sms;
-    quantize_kernel<T, C><<<grid, kQuantThreads, smem, stream>>>(p);
+    quantize_kernel<T, C, BITS><<<grid, kQuantThreads, smem, stream>>>(p);
     return finish_launch();
 }
 
 template <typename T>
-static int32_t launch_for_type(const QuantParams &p, cudaStream_t stream) {
+static int32_t launch_for_type(const QuantParams &p, int bits, cudaStream_t stream) {
     switch (p.g.d) {
-    case 64: return launch_quantize<T, 2>(p, stream);
-    case 128: return launch_quantize<T, 4>(p, stream);
-    case 256: return launch_quantize<T, 8>(p, stream);
+    case 64: return bits == 4 ? launch_quantize<T, 2, 4>(p, stream) : launch_quantize<T, 2, 2>(p, stream);
+    case 128: return bits == 4 ? launch_quantize<T, 4, 4>(p, stream) : launch_quantize<T, 4, 2>(p, stream);
+    case 256: return bits == 4 ? launch_quantize<T, 8, 4>(p, stream) : launch_quantize<T, 8, 2>(p, stream);
     default: return STOM_ERR_SHAPE;
     }
 }
@@ -684,9 +695,9 @@ extern "C" int32_t stom_oqm_quantize_frame(const stom_oqm_config *cfg, const sto
         q.F = (int32_t)nf;
         q.n_tiles = (uint32_t)(per_frame * nf);
         switch (dt) {
-        case STOM_BF16: rc = launch_for_type<__nv_bfloat16>(q, s); break;
-        case STOM_FP16: rc = launch_for_type<__half>(q, s); break;
-        default: rc = launch_for_type<float>(q, s); break;
+        case STOM_BF16: rc = launch_for_type<__nv_bfloat16>(q, cfg->bits, s); break;
+        case STOM_FP16: rc = launch_for_type<__half>(q, cfg->bits, s); break;
+        default: rc = launch_for_type<float>(q, cfg->bits, s); break;
         }
         if (rc) return rc;
     }

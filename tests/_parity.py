@@ -36,12 +36,17 @@ def q_strides(sh):
     return (sh.H_q * sh.T_q * sh.d, sh.T_q * sh.d, sh.d)
 
 
+def bits_of(sh) -> int:
+    """Width of a code for this workload: 4 unless the shape asks for the 2-bit variant."""
+    return int(sh.extra.get("bits", 4))
+
+
 def oracle_cfg(orc, sh, mode=0, cap=None):
-    return orc.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, cap or sh.T, 4, dt_code(sh.dtype), mode)
+    return orc.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, cap or sh.T, bits_of(sh), dt_code(sh.dtype), mode)
 
 
 def gpu_cfg(oqm, sh, mode=0, cap=None):
-    return oqm.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, cap or sh.T, 4, dt_code(sh.dtype), mode)
+    return oqm.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, cap or sh.T, bits_of(sh), dt_code(sh.dtype), mode)
 
 
 def compare_store(gst, ost, K_f32, groups=None, layers=None):

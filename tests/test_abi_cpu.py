@@ -56,7 +56,7 @@ def test_budget_to_k_matches_paper_example(oqm):
 
 
 @pytest.mark.parametrize("kw,code", [
-    (dict(head_dim=96), -2), (dict(group_tokens=0), -2), (dict(group_tokens=65), -2), (dict(bits=2), -6),
+    (dict(head_dim=96), -2), (dict(group_tokens=0), -2), (dict(group_tokens=65), -2), (dict(bits=3), -6),
     (dict(n_q_heads=7), -2), (dict(kv_dtype=5), -6), (dict(n_layers=0), -1), (dict(score_mode=3), -6),
 ])
 def test_config_validation(oqm, kw, code):

@@ -36,9 +36,23 @@ def _selection(rng, rows, T, k, n_sel):
     (1, 4, 4, 128, 50, 10, 8, 0, 70, 0, "bf16", "bf16"),       # nothing selected: system tokens only
 ])
 def test_attend_matches_oracle(orc, L, H_q, H_k, d, G, T, k, n_sel, sys_len, mode, dtype, cache):
+    _check_attend(orc, L, H_q, H_k, d, G, T, k, n_sel, sys_len, mode, dtype, cache, bits=4)
+
+
+@pytest.mark.parametrize("L,H_q,H_k,d,G,T,k,n_sel,sys_len,mode,dtype,cache", [
+    (2, 28, 4, 128, 50, 100, 16, 16, 9, 0, "bf16", "bf16"),
+    (1, 4, 2, 64, 16, 40, 5, 4, 70, 1, "fp16", "fp16"),
+    (1, 8, 1, 256, 8, 20, 6, 6, 0, 0, "bf16", "bf16"),
+])
+def test_attend_two_bit_codes(orc, L, H_q, H_k, d, G, T, k, n_sel, sys_len, mode, dtype, cache):
+    _check_attend(orc, L, H_q, H_k, d, G, T, k, n_sel, sys_len, mode, dtype, cache, bits=2)
+
+
+def _check_attend(orc, L, H_q, H_k, d, G, T, k, n_sel, sys_len, mode, dtype, cache, bits):
     from paper_2510_18269_b200 import oqm
     oqm.lib()
-    sh = synth.Shape("attend", L=L, H_q=H_q, H_k=H_k, d=d, G=G, T=T, T_q=1, k=k, dtype=dtype, seed=3)
+    sh = synth.Shape("attend", L=L, H_q=H_q, H_k=H_k, d=d, G=G, T=T, T_q=1, k=k, dtype=dtype, seed=3,
+                     extra={"bits": bits})
     ocfg, gcfg, ost, gst, _ = P.random_bank(orc, oqm, sh, mode, seed=17 * k + sys_len)
     rng = np.random.default_rng(5 + k)
     rows = L * (H_k if mode else 1)

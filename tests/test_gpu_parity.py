@@ -151,6 +151,16 @@ def test_shape_sweep_bf16(orc, oqm, G, d, H_k, H_q):
     _full_path(orc, oqm, sh)
 
 
+@pytest.mark.parametrize("G,d,H_k,H_q,dtype", [
+    (50, 128, 4, 28, "bf16"), (16, 64, 1, 2, "bf16"), (49, 64, 2, 4, "fp16"), (7, 256, 8, 8, "bf16"),
+    (64, 128, 2, 6, "fp32"), (1, 64, 1, 1, "bf16"), (51, 256, 1, 3, "fp16")])
+def test_two_bit_codes(orc, oqm, G, d, H_k, H_q, dtype):
+    """The 2-bit variant of the paper's ablation: three levels above the offset, four codes per byte."""
+    sh = synth.Shape("two-bit", L=2, H_q=H_q, H_k=H_k, d=d, G=G, T=29, T_q=2, k=6, dtype=dtype, seed=300 + G + d,
+                     extra={"bits": 2})
+    _full_path(orc, oqm, sh)
+
+
 @pytest.mark.parametrize("dtype,G", [("fp32", 16), ("fp32", 50), ("fp16", 50), ("fp16", 7)])
 def test_input_dtypes(orc, oqm, dtype, G):
     sh = synth.Shape("dtype", L=2, H_q=8, H_k=4, d=128, G=G, T=21, T_q=2, k=4, dtype=dtype, seed=7)
