@@ -260,7 +260,7 @@ def run_ours(args, sh):
     idx = torch.empty(sh.L, sh.k, dtype=torch.int32, device=dev)
     ka = torch.empty(sh.L, sh.H_k, S, sh.d, dtype=torch.bfloat16, device=dev)
     va = torch.empty_like(ka)
-    ws = torch.empty(oqm.stom_oqm_score_workspace_bytes(cfg, sh.L), dtype=torch.uint8, device=dev)
+    ws = torch.empty(oqm.stom_oqm_retrieve_workspace_bytes(cfg, sh.L, sh.T, sh.k), dtype=torch.uint8, device=dev)
     flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
     flags = torch.zeros(1, dtype=torch.int32, device=dev)
     fpc = args.frames_per_call or sh.T
@@ -495,7 +495,7 @@ def run_stream(args, sh):
     scores = torch.empty(sh.L, sh.T, dtype=torch.float32, device=dev)
     idx = torch.empty(sh.L, sh.k, dtype=torch.int32, device=dev)
     out = torch.empty(sh.L, sh.H_q, sh.d, dtype=torch.bfloat16, device=dev)
-    ws = torch.empty(oqm.stom_oqm_score_workspace_bytes(cfg, sh.L), dtype=torch.uint8, device=dev)
+    ws = torch.empty(oqm.stom_oqm_retrieve_workspace_bytes(cfg, sh.L, sh.T, sh.k), dtype=torch.uint8, device=dev)
     aws = torch.empty(oqm.stom_oqm_attend_workspace_bytes(cfg, sh.L, sh.k, sys_len) + 256, dtype=torch.uint8, device=dev)
     aws = aws[(-aws.data_ptr()) % 256:]
     flags = torch.zeros(1, dtype=torch.int32, device=dev)

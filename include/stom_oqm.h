@@ -270,7 +270,13 @@ int32_t stom_oqm_dequant_gather(const stom_oqm_config *cfg, const stom_oqm_store
  *      reconstruction, once per question) ---------------------------------
  * Same arguments as the three calls above; scores, idx are caller buffers that
  * receive the intermediate results ([rows][n_groups] and [rows][k]).
+ * workspace: at least stom_oqm_score_workspace_bytes() bytes, 16-byte aligned.
+ * With stom_oqm_retrieve_workspace_bytes() bytes, 256-byte aligned, the
+ * selection runs in two levels (every block pre-selects in its own run of
+ * groups), which shortens the call; the results are the same.
  */
+int64_t stom_oqm_retrieve_workspace_bytes(const stom_oqm_config *cfg, int32_t layer_count,
+                                          int32_t n_groups, int32_t k);
 int32_t stom_oqm_retrieve(const stom_oqm_config *cfg, const stom_oqm_store *store,
                           int32_t layer_begin, int32_t layer_count, int32_t n_groups,
                           const void *Q, int32_t T_q, int64_t q_stride_layer,

@@ -67,7 +67,7 @@ RetrieveScratch retrieve_scratch(const stom_oqm_config *cfg, int32_t layer_count
     r.off_q = off; off += up256(r.bytes_q);
     r.off_scores = off; off += up256(rows * (int64_t)n_groups * 4);
     r.off_idx = off; off += up256(r.bytes_idx);
-    r.off_ws = off; off += up256(stom_oqm_score_workspace_bytes(cfg, layer_count));
+    r.off_ws = off; off += up256(stom_oqm_retrieve_workspace_bytes(cfg, layer_count, n_groups, k));
     r.off_ka = off; off += up256(r.bytes_act);
     r.off_va = off; off += up256(r.bytes_act);
     r.total = off;
@@ -104,7 +104,7 @@ extern "C" int32_t stom_oqm_retrieve_host(const stom_oqm_config *cfg, const stom
                            (int64_t)cfg->n_q_heads * T_q * d, (int64_t)T_q * d, d, k,
                            reinterpret_cast<float *>(b + r.off_scores), reinterpret_cast<int32_t *>(b + r.off_idx),
                            b + r.off_ka, b + r.off_va, out_dtype, (int64_t)cfg->n_kv_heads * S * d, S * d, d, 0,
-                           b + r.off_ws, up256(stom_oqm_score_workspace_bytes(cfg, layer_count)), dev_flags, stream);
+                           b + r.off_ws, up256(stom_oqm_retrieve_workspace_bytes(cfg, layer_count, n_groups, k)), dev_flags, stream);
     if (rc) return rc;
     if ((rc = copy_async(idx_host, b + r.off_idx, r.bytes_idx, cudaMemcpyDeviceToHost, s))) return rc;
     if (k_active_host) {

@@ -16,8 +16,12 @@
 //   select    every block takes a ticket on its layer's counter when its
 //             scores are out; the block that draws the last ticket of a layer
 //             selects that layer's top-K.  Nobody waits for anybody: a block
-//             that is not last simply exits, so selection of early layers
-//             overlaps the streaming of later ones.
+//             that is not last simply exits.  With enough workspace the
+//             selection has two levels: each block first selects the top-K of
+//             its own run (all blocks in parallel, a few keys per thread), and
+//             the completing block only selects among chunks * K candidates,
+//             which are in ascending index order, so ties still go to the
+//             lower index and the result is the same set.
 // The layer counters live in the caller's workspace and are zeroed by a
 // memset enqueued ahead of the kernel; the selecting block also puts its
 // counter back to zero.
@@ -35,7 +39,14 @@ struct RetrieveParams {
     int32_t *idx;          // [rows][k]
     uint32_t *counters;    // [layer_count], zero on entry
     int32_t keys_in_smem;  // the selecting block may stage a row's keys in shared memory
+    // two-level selection (0: off): every block first selects the top-K of its own run of groups, the block
+    // that completes the layer then selects among those candidates only
+    int32_t two_level;
+    int32_t *cand_idx;     // [layer_count][chunks][k] positions inside the block's run, ascending; unused -1
+    float *cand_score;     // [layer_count][chunks][k] their scores; unused -inf
 };
+
+constexpr int kTwoLevelMaxK = 256;  // the selecting block keeps the chosen candidate positions in shared memory
 
 constexpr int kEmbedHeadGroup = 4;  // kv heads whose rows are in flight together
 
@@ -163,16 +174,45 @@ __global__ void __launch_bounds__(kFusedThreads) retrieve_kernel(const RetrieveP
     const int t_end = min(t_begin + p.groups_per_block, p.n_groups);
     score_block<V4>(p, sq, qn, li, t_begin, t_end);
 
+    uint32_t *skeys = reinterpret_cast<uint32_t *>(region);
+    const int n = p.n_groups, chunks = gridDim.x;
+    if (rp.two_level) {
+        // ---- level 1: the candidates of this block's run
+        __syncthreads();  // the run's scores are out (all warps of this block)
+        const int64_t cbase = ((int64_t)li * chunks + blockIdx.x) * rp.k;
+        const int len = t_end - t_begin;
+        block_topk<kFusedThreads, kKeysRegs>(p.scores + (int64_t)li * n + t_begin, len, rp.k, rp.cand_idx + cbase,
+                                             rp.cand_score + cbase, nullptr, skeys, tsm);
+        for (int j = min(rp.k, len) + tid; j < rp.k; j += kFusedThreads) rp.cand_score[cbase + j] = -INFINITY;
+    }
+
     // ---- ticket: the block that completes a layer selects its top-K
-    __threadfence();  // this block's scores are visible device-wide before its ticket is
+    __threadfence();  // this block's scores (and candidates) are visible device-wide before its ticket is
     __syncthreads();
     if (tid == 0) s_last = atomicAdd(&rp.counters[li], 1u) == gridDim.x - 1;
     __syncthreads();
     if (!s_last) return;
     __threadfence();
     if (tid == 0) rp.counters[li] = 0;  // as found
-    const int n = p.n_groups, rows = p.per_head ? H : 1;
-    uint32_t *skeys = reinterpret_cast<uint32_t *>(region);
+    if (rp.two_level) {
+        // ---- level 2: among chunks * k candidates, kept in ascending index order
+        __shared__ int32_t pos[kTwoLevelMaxK];
+        const int ksel = min(rp.k, n);
+        const int64_t cbase = (int64_t)li * chunks * rp.k;
+        block_topk<kFusedThreads, kKeysRegs>(rp.cand_score + cbase, chunks * rp.k, ksel, pos, nullptr, nullptr, skeys, tsm);
+        __syncthreads();
+        int32_t *out = rp.idx + (int64_t)li * rp.k;
+        for (int j = tid; j < rp.k; j += kFusedThreads) {
+            int32_t g = -1;
+            if (j < ksel) {
+                const int c = pos[j] / rp.k;
+                g = c * p.groups_per_block + __ldcg(rp.cand_idx + cbase + pos[j]);
+            }
+            out[j] = g;
+        }
+        return;
+    }
+    const int rows = p.per_head ? H : 1;
     for (int r = 0; r < rows; ++r) {
         const int64_t row = (int64_t)li * rows + r;
         const float *sc = p.scores + row * n;
@@ -199,6 +239,26 @@ static void launch_retrieve(const RetrieveParams &rp, dim3 grid, size_t smem, in
 }  // namespace stom
 
 using namespace stom;
+
+// chunks the fused kernel cuts a layer into on a device with `sms` multiprocessors
+static int retrieve_chunks(int sms, int layer_count, int n_groups) {
+    int chunks = (2 * sms) / layer_count;
+    if (chunks > (n_groups + 31) / 32) chunks = (n_groups + 31) / 32;
+    return chunks < 1 ? 1 : chunks;
+}
+
+static int64_t up256(int64_t x) { return (x + 255) / 256 * 256; }
+
+extern "C" int64_t stom_oqm_retrieve_workspace_bytes(const stom_oqm_config *cfg, int32_t layer_count,
+                                                     int32_t n_groups, int32_t k) {
+    if (check_config(cfg) || layer_count < 0 || n_groups < 0 || k < 1) return STOM_ERR_INVALID_ARG;
+    const int64_t base = stom_oqm_score_workspace_bytes(cfg, layer_count);
+    if (layer_count == 0 || k > kTwoLevelMaxK) return base;
+    // sized for any device of up to 256 multiprocessors
+    const int64_t chunks = retrieve_chunks(256, layer_count, n_groups);
+    const int64_t two = up256((int64_t)layer_count * 4) + 2 * up256((int64_t)layer_count * chunks * k * 4);
+    return two > base ? two : base;
+}
 
 extern "C" int32_t stom_oqm_retrieve(const stom_oqm_config *cfg, const stom_oqm_store *store,
                                      int32_t layer_begin, int32_t layer_count, int32_t n_groups,
@@ -246,12 +306,21 @@ extern "C" int32_t stom_oqm_retrieve(const stom_oqm_config *cfg, const stom_oqm_
         p.rep = cfg->n_q_heads / cfg->n_kv_heads;
         p.per_head = cfg->score_mode == STOM_SCORE_PER_HEAD;
         // one wave of about two blocks per SM; a block re-reads its layer's Q, so blocks are kept long
-        int chunks = (2 * sms) / layer_count;
-        if (chunks > (n_groups + 31) / 32) chunks = (n_groups + 31) / 32;
-        if (chunks < 1) chunks = 1;
+        int chunks = retrieve_chunks(sms, layer_count, n_groups);
         p.groups_per_block = (n_groups + chunks - 1) / chunks;
+        chunks = (n_groups + p.groups_per_block - 1) / p.groups_per_block;
         rp.k = k; rp.idx = idx;
         rp.counters = static_cast<uint32_t *>(workspace);
+        // two-level selection when it pays (several runs per layer, K well below a run) and the workspace has room
+        const int64_t off_ci = up256((int64_t)layer_count * 4);
+        const int64_t off_cs = off_ci + up256((int64_t)layer_count * chunks * k * 4);
+        const int64_t need2 = off_cs + up256((int64_t)layer_count * chunks * k * 4);
+        rp.two_level = !p.per_head && chunks >= 2 && k <= kTwoLevelMaxK && 2 * k <= p.groups_per_block &&
+                       p.groups_per_block <= kTopkRegKeys * kFusedThreads &&
+                       (int64_t)chunks * k <= kTopkRegKeys * kFusedThreads && workspace_bytes >= need2 &&
+                       (reinterpret_cast<uintptr_t>(workspace) & 255u) == 0;
+        rp.cand_idx = reinterpret_cast<int32_t *>(static_cast<uint8_t *>(workspace) + off_ci);
+        rp.cand_score = reinterpret_cast<float *>(static_cast<uint8_t *>(workspace) + off_cs);
         const int H = cfg->n_kv_heads, d = cfg->head_dim, HD = H * d;
         const int part_floats = (H < kEmbedHeadGroup ? H : kEmbedHeadGroup) * (kFusedThreads / (d / 8)) * (d + 4);
         const size_t fixed = (size_t)HD + ((H + 3) & ~3);

@@ -28,6 +28,7 @@ EXPORTS = (
     "stom_oqm_quantize_host_scratch_bytes", "stom_oqm_quantize_frame_host",
     "stom_oqm_retrieve_host_scratch_bytes", "stom_oqm_retrieve_host",
     "stom_oqm_score_groups_noalloc", "stom_oqm_attend_workspace_bytes", "stom_oqm_attend",
+    "stom_oqm_retrieve_workspace_bytes",
 )
 
 
@@ -73,6 +74,7 @@ def lib():
         L.stom_oqm_score_workspace_bytes.argtypes = [C.POINTER(Config), C.c_int32]
         L.stom_oqm_budget_to_k.argtypes = [C.c_int64, C.c_int32, C.c_int32]
         L.stom_oqm_attend_workspace_bytes.restype = C.c_int64
+        L.stom_oqm_retrieve_workspace_bytes.restype = C.c_int64
         L.stom_oqm_quantize_host_scratch_bytes.restype = C.c_int64
         L.stom_oqm_retrieve_host_scratch_bytes.restype = C.c_int64
         for name in EXPORTS:
@@ -207,6 +209,11 @@ def stom_oqm_dequant_gather(cfg: Config, store: Store, layer_begin, layer_count,
         C.c_int32(k), C.c_int32(n_groups), _ptr(k_active), _ptr(v_active), C.c_int32(out_dtype),
         C.c_int64(sl), C.c_int64(sh), C.c_int64(st), C.c_int32(token_offset), _ptr(dev_flags), _stream(stream))
     _check(rc, "stom_oqm_dequant_gather")
+
+
+def stom_oqm_retrieve_workspace_bytes(cfg: Config, layer_count: int, n_groups: int, k: int) -> int:
+    return int(lib().stom_oqm_retrieve_workspace_bytes(C.byref(cfg), C.c_int32(layer_count), C.c_int32(n_groups),
+                                                       C.c_int32(k)))
 
 
 def stom_oqm_retrieve(cfg: Config, store: Store, layer_begin, layer_count, n_groups, Q, T_q, q_strides, k,

@@ -40,7 +40,7 @@ def test_c3_full_stream_one_layer_in_full_and_samples_elsewhere(orc):
     idx = torch.empty(sh.L, sh.k, dtype=torch.int32, device=dev)
     ka = torch.empty(sh.L, sh.H_k, S, sh.d, dtype=torch.bfloat16, device=dev)
     va = torch.empty_like(ka)
-    ws = torch.empty(oqm.stom_oqm_score_workspace_bytes(gcfg, sh.L), dtype=torch.uint8, device=dev)
+    ws = torch.empty(oqm.stom_oqm_retrieve_workspace_bytes(gcfg, sh.L, sh.T, sh.k), dtype=torch.uint8, device=dev)
     oqm.stom_oqm_retrieve(gcfg, gst, 0, sh.L, sh.T, Q, sh.T_q, P.q_strides(sh), sh.k, scores, idx, ka, va, oqm.BF16,
                           P.active_strides(sh, S), sys_len, ws, dev_flags=flags)
     torch.cuda.synchronize()

@@ -25,7 +25,8 @@ pytestmark = pytest.mark.gpu
     (2, 6, 3, 128, 4, 333, 7, 16, 0, "bf16"),      # a head count the pipelined scorer does not cover
     (2, 6, 3, 128, 4, 333, 7, 16, 1, "fp16"),
 ])
-def test_fused_retrieve_matches_oracle(orc, L, H_q, H_k, d, G, T, T_q, k, mode, dtype):
+@pytest.mark.parametrize("two_level_ws", [False, True])
+def test_fused_retrieve_matches_oracle(orc, L, H_q, H_k, d, G, T, T_q, k, mode, dtype, two_level_ws):
     from paper_2510_18269_b200 import oqm
     oqm.lib()
     sh = synth.Shape("fused", L=L, H_q=H_q, H_k=H_k, d=d, G=G, T=T, T_q=T_q, k=k, dtype=dtype, seed=5)
@@ -45,7 +46,10 @@ def test_fused_retrieve_matches_oracle(orc, L, H_q, H_k, d, G, T, T_q, k, mode, 
     va_flat, va = P.out_buffers(sh, L, S, torch.bfloat16, "cuda", 3.0)
     scores = torch.full((rows * T + P.GUARD,), -7.0, dtype=torch.float32, device="cuda")
     idx = torch.full((rows * k + P.GUARD,), -9, dtype=torch.int32, device="cuda")
-    ws = torch.full((oqm.stom_oqm_score_workspace_bytes(gcfg, L),), 0xAB, dtype=torch.uint8, device="cuda")
+    # the small workspace keeps the selection in the completing block; the large one lets every block pre-select
+    nbytes = oqm.stom_oqm_retrieve_workspace_bytes(gcfg, L, T, k) if two_level_ws else oqm.stom_oqm_score_workspace_bytes(gcfg, L)
+    ws = torch.full((nbytes + 256,), 0xAB, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 256:]
     flags = torch.zeros(1, dtype=torch.int32, device="cuda")
     for _ in range(2):   # twice: the second call finds the layer counters as the first one left them
         oqm.stom_oqm_retrieve(gcfg, gst, 0, L, T, Q.cuda(), T_q, P.q_strides(sh), k, scores, idx, ka, va, oqm.BF16,

@@ -34,7 +34,7 @@ def test_streaming_interleave_matches_oracle(orc):
     gen = torch.Generator().manual_seed(8)
     sys_k = torch.randn(sh.L, sh.H_k, sys_len, sh.d, generator=gen).to(torch.bfloat16)
     sys_v = torch.randn(sh.L, sh.H_k, sys_len, sh.d, generator=gen).to(torch.bfloat16)
-    ws = torch.empty(oqm.stom_oqm_score_workspace_bytes(gcfg, sh.L), dtype=torch.uint8, device="cuda")
+    ws = torch.empty(oqm.stom_oqm_retrieve_workspace_bytes(gcfg, sh.L, sh.T, sh.k), dtype=torch.uint8, device="cuda")
     aws = torch.empty(oqm.stom_oqm_attend_workspace_bytes(gcfg, sh.L, sh.k, sys_len) + 256, dtype=torch.uint8, device="cuda")
     aws = aws[(-aws.data_ptr()) % 256:]
     n_questions = 0
