@@ -68,6 +68,7 @@ __global__ void __launch_bounds__(kDqWarps * 32) dequant_gather_kernel(const Deq
     const int j = (int)(rest % p.k);
     const int li = (int)(rest / p.k);
 
+    grid_dependency_wait();  // idx may come from the kernel just ahead in the stream
     const int t = p.per_head ? p.idx[((int64_t)li * H + h) * p.k + j] : p.idx[(int64_t)li * p.k + j];
     if (t < 0 || t >= p.n_groups) {
         if (t != -1 && p.flags && lane == 0) atomicOr(p.flags, STOM_FLAG_BAD_INDEX);
@@ -126,6 +127,15 @@ extern "C" int32_t stom_oqm_dequant_gather(const stom_oqm_config *cfg, const sto
                                            void *k_active, void *v_active, int32_t out_dtype,
                                            int64_t stride_layer, int64_t stride_head, int64_t stride_token,
                                            int32_t token_offset, uint32_t *dev_flags, void *stream) {
+    return dequant_gather_launch(cfg, store, layer_begin, layer_count, idx, k, n_groups, k_active, v_active, out_dtype,
+                                 stride_layer, stride_head, stride_token, token_offset, dev_flags, stream, false);
+}
+
+int32_t stom::dequant_gather_launch(const stom_oqm_config *cfg, const stom_oqm_store *store, int32_t layer_begin,
+                                    int32_t layer_count, const int32_t *idx, int32_t k, int32_t n_groups,
+                                    void *k_active, void *v_active, int32_t out_dtype, int64_t stride_layer,
+                                    int64_t stride_head, int64_t stride_token, int32_t token_offset,
+                                    uint32_t *dev_flags, void *stream, bool after_producer) {
     int32_t rc = check_config(cfg);
     if (rc) return rc;
     if ((rc = check_store(store))) return rc;
@@ -155,15 +165,21 @@ extern "C" int32_t stom_oqm_dequant_gather(const stom_oqm_config *cfg, const sto
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const unsigned nb = (unsigned)blocks, nt = kDqWarps * 32;
     const bool bf = out_dtype == STOM_BF16;
-#define STOM_DQ_LAUNCH(LPR_)                                                                             \
-    do {                                                                                             \
-        if (cfg->bits == 4) {                                                                        \
-            if (bf) dequant_gather_kernel<__nv_bfloat16, LPR_, 4><<<nb, nt, 0, s>>>(p);              \
-            else dequant_gather_kernel<__half, LPR_, 4><<<nb, nt, 0, s>>>(p);                        \
-        } else {                                                                                     \
-            if (bf) dequant_gather_kernel<__nv_bfloat16, LPR_, 2><<<nb, nt, 0, s>>>(p);              \
-            else dequant_gather_kernel<__half, LPR_, 2><<<nb, nt, 0, s>>>(p);                        \
-        }                                                                                            \
+    cudaError_t le = cudaSuccess;
+#define STOM_DQ_KERNEL(OT_, LPR_, BITS_)                                                               \
+    do {                                                                                               \
+        if (after_producer) le = launch_after_producer(dequant_gather_kernel<OT_, LPR_, BITS_>, dim3(nb), dim3(nt), 0, s, p); \
+        else dequant_gather_kernel<OT_, LPR_, BITS_><<<nb, nt, 0, s>>>(p);                             \
+    } while (0)
+#define STOM_DQ_LAUNCH(LPR_)                                                                           \
+    do {                                                                                               \
+        if (cfg->bits == 4) {                                                                          \
+            if (bf) STOM_DQ_KERNEL(__nv_bfloat16, LPR_, 4);                                            \
+            else STOM_DQ_KERNEL(__half, LPR_, 4);                                                      \
+        } else {                                                                                       \
+            if (bf) STOM_DQ_KERNEL(__nv_bfloat16, LPR_, 2);                                            \
+            else STOM_DQ_KERNEL(__half, LPR_, 2);                                                      \
+        }                                                                                              \
     } while (0)
     switch (cfg->head_dim) {
     case 64: STOM_DQ_LAUNCH(8); break;
@@ -171,6 +187,11 @@ extern "C" int32_t stom_oqm_dequant_gather(const stom_oqm_config *cfg, const sto
     case 256: STOM_DQ_LAUNCH(32); break;
     default: return STOM_ERR_SHAPE;
     }
+#undef STOM_DQ_KERNEL
 #undef STOM_DQ_LAUNCH
+    if (le != cudaSuccess) {
+        set_last_cuda_error(le);
+        return STOM_ERR_CUDA;
+    }
     return finish_launch();
 }

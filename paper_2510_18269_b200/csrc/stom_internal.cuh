@@ -47,9 +47,40 @@ inline BankGeom bank_geom(const stom_oqm_config *c) {
     return BankGeom{c->n_kv_heads, c->group_tokens, c->head_dim, c->capacity_groups, c->head_dim * c->bits / 8};
 }
 
+// A2+A3 -> A4 inside one retrieval: same checks and launch as stom_oqm_dequant_gather; `after_producer` launches the
+// kernel with programmatic stream serialization, so that its blocks may be scheduled while the kernel ahead of it in
+// the stream (which wrote idx) is still draining -- the kernel itself waits for that grid before it reads idx.
+int32_t dequant_gather_launch(const stom_oqm_config *cfg, const stom_oqm_store *store, int32_t layer_begin,
+                              int32_t layer_count, const int32_t *idx, int32_t k, int32_t n_groups, void *k_active,
+                              void *v_active, int32_t out_dtype, int64_t stride_layer, int64_t stride_head,
+                              int64_t stride_token, int32_t token_offset, uint32_t *dev_flags, void *stream,
+                              bool after_producer);
+
 // ---------------------------------------------------------------- device
 
 #ifdef __CUDACC__
+
+// Programmatic dependent launch (sm_90+).  grid_dependency_wait: returns once the grids this one depends on have
+// completed and their writes are visible (at once if the launch had no programmatic dependency).
+// grid_launch_dependents: lets a dependent grid start being scheduled from here on.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Launches `kernel` so that it may overlap the tail of the kernel ahead of it in the stream.
+template <typename P>
+inline cudaError_t launch_after_producer(void (*kernel)(P), dim3 grid, dim3 block, size_t smem, cudaStream_t s, const P &p) {
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = grid;
+    lc.blockDim = block;
+    lc.dynamicSmemBytes = smem;
+    lc.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = at;
+    lc.numAttrs = 1;
+    return cudaLaunchKernelEx(&lc, kernel, p);
+}
 
 // Index of (layer, group, head) in the [L][cap][H] lattice every bank array shares.
 __device__ __forceinline__ int64_t bank_slot(const BankGeom &g, int l, int t, int h) {

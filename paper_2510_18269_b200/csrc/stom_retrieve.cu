@@ -168,6 +168,7 @@ __global__ void __launch_bounds__(kFusedThreads) retrieve_kernel(const RetrieveP
     const int li = blockIdx.y, H = p.g.H, HD = H * p.g.d, tid = threadIdx.x;
     float *sq = dyn, *qn = dyn + HD, *region = qn + ((H + 3) & ~3);
 
+    grid_launch_dependents();  // the gather that follows may be scheduled as this grid drains; it waits before it reads idx
     embed_layer<T>(p, li, sq, qn, region);
 
     const int t_begin = blockIdx.x * p.groups_per_block;
@@ -343,7 +344,7 @@ extern "C" int32_t stom_oqm_retrieve(const stom_oqm_config *cfg, const stom_oqm_
         rc = stom_oqm_topk(scores, rows, 0, 0, k, idx, nullptr, nullptr, stream);
         if (rc) return rc;
     }
-    return stom_oqm_dequant_gather(cfg, store, layer_begin, layer_count, idx, k, n_groups, k_active, v_active,
-                                   out_dtype, stride_layer, stride_head, stride_token, token_offset, dev_flags,
-                                   stream);
+    return dequant_gather_launch(cfg, store, layer_begin, layer_count, idx, k, n_groups, k_active, v_active, out_dtype,
+                                 stride_layer, stride_head, stride_token, token_offset, dev_flags, stream,
+                                 layer_count > 0 && n_groups > 0);
 }
