@@ -7,13 +7,15 @@
 // packed codes and their (s, m) -- a quarter of the bytes of the bf16 cache --
 // instead of writing that cache once and re-reading it every step.
 //
-// Work unit: a segment = one selected group (G <= 64 tokens) or a run of up to
-// 64 system tokens.  A block of 8 warps takes 8 consecutive segments of one
-// (layer, kv head) and all the query heads of that kv head's GQA block (in
-// chunks of 8); warp w owns segment w:
+// Work unit: a segment = up to 32 consecutive tokens of one selected group (a
+// group of 50 tokens is two segments) or of the system tokens.  A block of 8
+// warps takes 8 consecutive segments of one (layer, kv head) and all the query
+// heads of that kv head's GQA block (in chunks of 8); warp w owns segment w:
 //   phase 1  scores: a lane owns 8 adjacent channels, d/8 lanes share a token;
-//            K is rebuilt as fmaf(code, s, m) in registers, dotted with the
-//            query heads, reduced by shuffles, scores land in shared memory
+//            the code words of the whole segment are requested at once, K is
+//            rebuilt as fmaf(code, s, m) in registers, dotted with the query
+//            heads, and the 8 partial dot products of a lane are summed across
+//            the token's lanes by a reduce-scatter (8 shuffles, not 32)
 //   phase 2  block-local softmax statistics per query head (max, sum) in the
 //            base-2 domain (the scores carry softmax_scale * log2(e))
 //   phase 3  weighted sum of V, rebuilt the same way, per warp; the warps'
@@ -21,13 +23,14 @@
 // and writes (max, sum, weighted sum) per query head to the workspace.  The
 // block that draws the last ticket of its (layer, kv head) merges the partial
 // results of all its blocks and writes the output row.  Nobody waits.
+// A decode step is latency, not bandwidth: 2.2 MB per layer at the 7B geometry.
 #include "stom_internal.cuh"
 
 namespace stom {
 
 constexpr int kAtWarps = 8;
 constexpr int kAtThreads = kAtWarps * 32;
-constexpr int kAtSegTokens = 64;  // token slots per segment (G <= 64)
+constexpr int kAtSegTokens = 32;  // token slots per segment
 constexpr int kAtHeads = 8;       // query heads handled together
 
 struct AttendParams {
@@ -43,7 +46,7 @@ struct AttendParams {
     float *part;         // [layer][H][blocks][rep][d + 2]
     uint32_t *counters;  // [layer][H]
     BankGeom g;
-    int32_t layer_begin, k, n_groups, per_head, rep, sys_len, n_sys_seg, n_seg;
+    int32_t layer_begin, k, n_groups, per_head, rep, sys_len, n_sys_seg, n_seg, segs_per_group;
     float scale_log2e;
     uint32_t *flags;
 };
@@ -71,85 +74,80 @@ __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p
 
     // ---- what the warp's segment is
     int n_tok = 0;          // tokens in the segment
-    int sys_begin = -1;     // >= 0: a run of system tokens starting here
+    int tok0 = 0;           // first token of the segment inside its group / inside the system tokens
+    bool is_sys = false;
     int64_t slot = 0;       // bank slot of a group segment
     if (seg < p.n_sys_seg) {
-        sys_begin = seg * kAtSegTokens;
-        n_tok = min(kAtSegTokens, p.sys_len - sys_begin);
+        is_sys = true;
+        tok0 = seg * kAtSegTokens;
+        n_tok = min(kAtSegTokens, p.sys_len - tok0);
     } else if (seg < p.n_seg) {
-        const int j = seg - p.n_sys_seg;
+        const int sg = seg - p.n_sys_seg;
+        const int j = sg / p.segs_per_group;
+        tok0 = (sg - j * p.segs_per_group) * kAtSegTokens;
         const int t = p.per_head ? p.idx[((int64_t)li * H + h) * p.k + j] : p.idx[(int64_t)li * p.k + j];
         if (t >= 0 && t < p.n_groups) {
-            n_tok = G;
+            n_tok = min(kAtSegTokens, G - tok0);
             slot = bank_slot(p.g, p.layer_begin + li, t, h);
-        } else if (t != -1 && p.flags && lane == 0) {
+        } else if (t != -1 && p.flags && lane == 0 && tok0 == 0) {
             atomicOr(p.flags, STOM_FLAG_BAD_INDEX);
         }
     }
     const CT *ksys = reinterpret_cast<const CT *>(p.ksys) + (int64_t)li * p.s_sl + (int64_t)h * p.s_sh + cl * 8;
     const CT *vsys = reinterpret_cast<const CT *>(p.vsys) + (int64_t)li * p.s_sl + (int64_t)h * p.s_sh + cl * 8;
 
-    // Tokens go through in batches whose loads are all issued before the first use (a decode step is pure latency):
-    // 16 passes of group tokens (one code word per lane and pass) or 4 passes of system tokens (16 bytes per lane).
-    constexpr int kRaw = 16;
-    const bool is_sys = sys_begin >= 0;
-    const int batch_passes = is_sys ? kRaw / 4 : kRaw;
-    auto load_batch = [&](bool keys, int g0, uint32_t (&raw)[kRaw]) {
+    // All loads of a segment (16 passes of group tokens: one code word per lane and pass) or of a quarter of it (4
+    // passes of system tokens: 16 bytes per lane and pass) are issued at once -- a decode step is pure latency -- and
+    // parked in a per-warp staging area; the passes then run in a ROLLED loop.  Unrolling them instead made the
+    // kernel several thousand instructions long, executed once per warp, and instruction fetch became the bottleneck.
+    constexpr int kStageWords = 16;
+    uint32_t *stage = reinterpret_cast<uint32_t *>(buf) + kAtHeads * kSlots + warp * kStageWords * 32 + lane;
+    static_assert(kAtHeads * kSlots + kAtWarps * kStageWords * 32 <= 8192, "shared buffer");
+    const int n_pass = (n_tok + TPW - 1) / TPW;
+    const int batch_passes = is_sys ? kStageWords / 4 : kStageWords;
+    auto load_batch = [&](bool keys, int p0) {
         if (is_sys) {
             const CT *base = keys ? ksys : vsys;
 #pragma unroll
-            for (int b = 0; b < kRaw / 4; ++b) {
-                const int g = g0 + b * TPW + sub;
+            for (int b = 0; b < kStageWords / 4; ++b) {
+                const int g = (p0 + b) * TPW + sub;
                 uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (g < n_tok) v = __ldg(reinterpret_cast<const uint4 *>(base + (int64_t)(sys_begin + g) * p.s_st));
-                raw[4 * b] = v.x; raw[4 * b + 1] = v.y; raw[4 * b + 2] = v.z; raw[4 * b + 3] = v.w;
+                if (g < n_tok) v = __ldg(reinterpret_cast<const uint4 *>(base + (int64_t)(tok0 + g) * p.s_st));
+                stage[(4 * b) * 32] = v.x; stage[(4 * b + 1) * 32] = v.y;
+                stage[(4 * b + 2) * 32] = v.z; stage[(4 * b + 3) * 32] = v.w;
             }
         } else {
             const uint8_t *codes = (keys ? p.codes_k : p.codes_v) + slot * (int64_t)G * p.g.row_bytes;
 #pragma unroll
-            for (int b = 0; b < kRaw; ++b) {
-                const int g = g0 + b * TPW + sub;
-                raw[b] = g < n_tok ? load_codes8<BITS>(codes + (int64_t)g * p.g.row_bytes, cl) : 0u;
+            for (int b = 0; b < kStageWords; ++b) {
+                const int g = (p0 + b) * TPW + sub;
+                stage[b * 32] = g < n_tok ? load_codes8<BITS>(codes + (int64_t)(tok0 + g) * p.g.row_bytes, cl) : 0u;
             }
         }
     };
-    // 8 channels of the token of pass b of a batch as floats: a system token as stored, a group token rebuilt
-    auto sys8 = [&](const uint32_t (&raw)[kRaw], int b, float (&x)[8]) {
-        unpack2<CT>(raw[4 * b], x[0], x[1]);
-        unpack2<CT>(raw[4 * b + 1], x[2], x[3]);
-        unpack2<CT>(raw[4 * b + 2], x[4], x[5]);
-        unpack2<CT>(raw[4 * b + 3], x[6], x[7]);
-    };
-    auto group8 = [&](uint32_t w, const float (&s)[8], const float (&m)[8], float (&x)[8]) {
-        uint32_t f[8];
-        code_floats8<BITS>(w, f);
-#pragma unroll
-        for (int c = 0; c < 8; ++c) x[c] = __fmaf_rn(__uint_as_float(f[c]) - 8388608.0f, s[c], m[c]);
-    };
-    // runs f(g, x) for every token of the warp's segment, keys or values
+    // runs f(g, x) for every token of the warp's segment (x: 8 channels as floats), keys or values
     auto for_tokens = [&](bool keys, const float (&s)[8], const float (&m)[8], auto &&f) {
-        for (int g0 = 0; g0 < n_tok; g0 += TPW * batch_passes) {
-            uint32_t raw[kRaw];
-            load_batch(keys, g0, raw);
-            if (is_sys) {
+        for (int p0 = 0; p0 < n_pass; p0 += batch_passes) {
+            load_batch(keys, p0);
+            __syncwarp();
+            const int nb = min(batch_passes, n_pass - p0);
+#pragma unroll 1
+            for (int b = 0; b < nb; ++b) {
+                float x[8];
+                if (is_sys) {
+                    unpack2<CT>(stage[(4 * b) * 32], x[0], x[1]);
+                    unpack2<CT>(stage[(4 * b + 1) * 32], x[2], x[3]);
+                    unpack2<CT>(stage[(4 * b + 2) * 32], x[4], x[5]);
+                    unpack2<CT>(stage[(4 * b + 3) * 32], x[6], x[7]);
+                } else {
+                    uint32_t fbits[8];
+                    code_floats8<BITS>(stage[b * 32], fbits);
 #pragma unroll
-                for (int b = 0; b < kRaw / 4; ++b) {
-                    if (g0 + b * TPW < n_tok) {  // warp-uniform
-                        float x[8];
-                        sys8(raw, b, x);
-                        f(g0 + b * TPW + sub, x);
-                    }
+                    for (int c = 0; c < 8; ++c) x[c] = __fmaf_rn(__uint_as_float(fbits[c]) - 8388608.0f, s[c], m[c]);
                 }
-            } else {
-#pragma unroll
-                for (int b = 0; b < kRaw; ++b) {
-                    if (g0 + b * TPW < n_tok) {  // warp-uniform
-                        float x[8];
-                        group8(raw[b], s, m, x);
-                        f(g0 + b * TPW + sub, x);
-                    }
-                }
+                f((p0 + b) * TPW + sub, x);
             }
+            __syncwarp();
         }
     };
     auto load_stats = [&](bool keys, float (&s)[8], float (&m)[8]) {
@@ -200,17 +198,26 @@ __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p
 #pragma unroll
                     for (int c = 0; c < 8; ++c) dot[hh] = fmaf(x[c], q8[hh][c], dot[hh]);
                 }
+                // reduce-scatter over the token's lanes: each step halves the heads a lane still carries, so that lane
+                // cl ends with the full sum of query head cl & 7 (8 channel blocks cover 3 steps; wider rows add plain steps)
+                float v4[4], v2[2], mine;
 #pragma unroll
-                for (int o = LPR / 2; o > 0; o >>= 1) {
-#pragma unroll
-                    for (int hh = 0; hh < kAtHeads; ++hh) dot[hh] += __shfl_xor_sync(0xffffffffu, dot[hh], o);
+                for (int i = 0; i < 4; ++i) {
+                    const float keep = (cl & 4) ? dot[4 + i] : dot[i], give = (cl & 4) ? dot[i] : dot[4 + i];
+                    v4[i] = keep + __shfl_xor_sync(0xffffffffu, give, 4);
                 }
-                // lane cl of the token's lanes files the score of query head cl
-                if (cl < kAtHeads && g < n_tok) {
-                    float mine = dot[0];
 #pragma unroll
-                    for (int hh = 1; hh < kAtHeads; ++hh)
-                        if (cl == hh) mine = dot[hh];
+                for (int i = 0; i < 2; ++i) {
+                    const float keep = (cl & 2) ? v4[2 + i] : v4[i], give = (cl & 2) ? v4[i] : v4[2 + i];
+                    v2[i] = keep + __shfl_xor_sync(0xffffffffu, give, 2);
+                }
+                {
+                    const float keep = (cl & 1) ? v2[1] : v2[0], give = (cl & 1) ? v2[0] : v2[1];
+                    mine = keep + __shfl_xor_sync(0xffffffffu, give, 1);
+                }
+#pragma unroll
+                for (int o = 8; o < LPR; o <<= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
+                if (cl < kAtHeads && g < n_tok) {
                     sc[cl][warp * kAtSegTokens + g] = mine;
                 }
             });
@@ -317,37 +324,45 @@ __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p
     for (int hq = warp; hq < p.rep; hq += kAtWarps) {
         const float *rec0 = p.part + (((int64_t)li * H + h) * n_blocks * p.rep + hq) * (D + 2);
         const int64_t step = (int64_t)p.rep * (D + 2);
+        // lanes share out the blocks 32 at a time: their maxima and sums are loaded once, the weight of a block is
+        // then handed round by shuffle while every lane adds up its own channels, 8 blocks' loads in flight
         float mx = -INFINITY;
         for (int b = lane; b < n_blocks; b += 32) mx = fmaxf(mx, __ldcg(rec0 + b * step));
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         float den = 0.0f;
-        for (int b = lane; b < n_blocks; b += 32) {
-            const float mb = __ldcg(rec0 + b * step);
-            if (mb != -INFINITY) den = fmaf(__ldcg(rec0 + b * step + 1), exp2f(mb - mx), den);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
         float num[D / 32];
 #pragma unroll
         for (int i = 0; i < D / 32; ++i) num[i] = 0.0f;
-#pragma unroll 4
-        for (int b = 0; b < n_blocks; ++b) {
-            const float mb = __ldcg(rec0 + b * step);
-            const float w = mb == -INFINITY ? 0.0f : exp2f(mb - mx);
+        for (int b0 = 0; b0 < n_blocks; b0 += 32) {
+            float w_mine = 0.0f;
+            if (b0 + lane < n_blocks) {
+                const float mb = __ldcg(rec0 + (b0 + lane) * step);
+                if (mb != -INFINITY) {
+                    w_mine = exp2f(mb - mx);
+                    den = fmaf(__ldcg(rec0 + (b0 + lane) * step + 1), w_mine, den);
+                }
+            }
+            const int nb = min(32, n_blocks - b0);
+#pragma unroll 8
+            for (int j = 0; j < nb; ++j) {
+                const float w = __shfl_sync(0xffffffffu, w_mine, j);
 #pragma unroll
-            for (int i = 0; i < D / 32; ++i) num[i] = fmaf(__ldcg(rec0 + b * step + 2 + lane + 32 * i), w, num[i]);
+                for (int i = 0; i < D / 32; ++i) num[i] = fmaf(__ldcg(rec0 + (b0 + j) * step + 2 + lane + 32 * i), w, num[i]);
+            }
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
         CT *out = reinterpret_cast<CT *>(p.out) + (int64_t)li * p.o_sl + (int64_t)(h * p.rep + hq) * p.o_sh;
 #pragma unroll
         for (int i = 0; i < D / 32; ++i) out[lane + 32 * i] = (CT)(den > 0.0f ? num[i] / den : 0.0f);
     }
 }
 
-static int attend_segments(const stom_oqm_config *cfg, int32_t k, int32_t sys_len, int *n_sys_seg) {
-    (void)cfg;
+static int attend_segments(const stom_oqm_config *cfg, int32_t k, int32_t sys_len, int *n_sys_seg, int *segs_per_group) {
     *n_sys_seg = (sys_len + kAtSegTokens - 1) / kAtSegTokens;
-    return *n_sys_seg + k;
+    *segs_per_group = (cfg->group_tokens + kAtSegTokens - 1) / kAtSegTokens;
+    return *n_sys_seg + k * *segs_per_group;
 }
 
 template <typename QT, typename CT>
@@ -378,8 +393,8 @@ using namespace stom;
 extern "C" int64_t stom_oqm_attend_workspace_bytes(const stom_oqm_config *cfg, int32_t layer_count, int32_t k,
                                                    int32_t sys_len) {
     if (check_config(cfg) || layer_count < 0 || k < 0 || sys_len < 0) return STOM_ERR_INVALID_ARG;
-    int n_sys_seg = 0;
-    const int n_seg = attend_segments(cfg, k, sys_len, &n_sys_seg);
+    int n_sys_seg = 0, spg = 0;
+    const int n_seg = attend_segments(cfg, k, sys_len, &n_sys_seg, &spg);
     const int64_t blocks = (n_seg + kAtWarps - 1) / kAtWarps;
     const int64_t counters = ((int64_t)layer_count * cfg->n_kv_heads * 4 + 255) / 256 * 256;
     const int64_t part = (int64_t)layer_count * cfg->n_kv_heads * blocks * (cfg->n_q_heads / cfg->n_kv_heads) *
@@ -433,7 +448,7 @@ extern "C" int32_t stom_oqm_attend(const stom_oqm_config *cfg, const stom_oqm_st
     p.per_head = cfg->score_mode == STOM_SCORE_PER_HEAD;
     p.rep = cfg->n_q_heads / cfg->n_kv_heads;
     p.sys_len = sys_len;
-    p.n_seg = attend_segments(cfg, k, sys_len, &p.n_sys_seg);
+    p.n_seg = attend_segments(cfg, k, sys_len, &p.n_sys_seg, &p.segs_per_group);
     p.scale_log2e = softmax_scale * 1.4426950408889634f;
     p.flags = dev_flags;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
