@@ -94,3 +94,59 @@ def test_streaming_interleave_matches_oracle(orc):
     Kkept = orc.to_f32(kn, P.dt_code(sh.dtype)).transpose(0, 1, 2, 3, 4)
     Kkept = np.stack([Kkept[:, f][:, :, keep[f].numpy()] for f in range(sh.T)], axis=1)      # [L][T][H][G][d]
     P.compare_store(gst, ost, Kkept)
+
+
+def test_question_sequence_replays_from_a_cuda_graph(orc):
+    """The per-question sequence (fused retrieval, gather, one decode-attention step) captured once into a CUDA graph
+    and replayed: same selection, same reconstructed cache, same attention output as the direct calls, also after
+    the bank has grown and the question changed between replays (the graph reads the same buffers)."""
+    from paper_2510_18269_b200 import oqm
+    oqm.lib()
+    sh = synth.Shape("graph", L=3, H_q=8, H_k=4, d=128, G=50, T=120, T_q=4, k=8, seed=77)
+    ocfg, gcfg, ost, gst, _ = P.random_bank(orc, oqm, sh, 0, seed=5)
+    sys_len = 6
+    S = sys_len + sh.k * sh.G
+    dev = "cuda"
+    Q = synth.queries(sh).cuda()
+    q_dec = torch.randn(sh.L, sh.H_q, sh.d, generator=torch.Generator().manual_seed(3)).to(torch.bfloat16).cuda()
+    scores = torch.zeros(sh.L, sh.T, dtype=torch.float32, device=dev)
+    idx = torch.zeros(sh.L, sh.k, dtype=torch.int32, device=dev)
+    ka = torch.randn(sh.L, sh.H_k, S, sh.d, generator=torch.Generator().manual_seed(4)).to(torch.bfloat16).cuda()
+    va = ka.clone()
+    out = torch.zeros(sh.L, sh.H_q, sh.d, dtype=torch.bfloat16, device=dev)
+    ws = torch.empty(oqm.stom_oqm_retrieve_workspace_bytes(gcfg, sh.L, sh.T, sh.k), dtype=torch.uint8, device=dev)
+    aws = torch.empty(oqm.stom_oqm_attend_workspace_bytes(gcfg, sh.L, sh.k, sys_len) + 256, dtype=torch.uint8, device=dev)
+    aws = aws[(-aws.data_ptr()) % 256:]
+    flags = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def question():
+        oqm.stom_oqm_retrieve(gcfg, gst, 0, sh.L, sh.T, Q, sh.T_q, P.q_strides(sh), sh.k, scores, idx, ka, va, oqm.BF16,
+                              P.active_strides(sh, S), sys_len, ws, dev_flags=flags)
+        oqm.stom_oqm_attend(gcfg, gst, 0, sh.L, idx, sh.k, sh.T, q_dec, (sh.H_q * sh.d, sh.d), ka, va, oqm.BF16,
+                            P.active_strides(sh, S), sys_len, float(sh.d) ** -0.5, out, (sh.H_q * sh.d, sh.d), aws,
+                            dev_flags=flags)
+
+    # warm up on a side stream (first use of each kernel), then capture
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        question()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        question()
+    for trial in range(2):
+        if trial == 1:   # another question against a changed bank, through the same buffers
+            Q.copy_(synth.queries(dataclasses.replace(sh, seed=78)).cuda())
+            gst.rep_key[:, 5:9].mul_(-1.0)
+        idx.fill_(-7); out.zero_(); scores.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        got = (scores.clone(), idx.clone(), ka.clone(), va.clone(), out.clone())
+        idx.fill_(-7); out.zero_(); scores.zero_()
+        question()
+        torch.cuda.synchronize()
+        for a, b in zip(got, (scores, idx, ka, va, out)):
+            assert torch.equal(a, b)
+    assert int(flags.item()) == 0
