@@ -22,54 +22,72 @@ constexpr int kEmbedThreads = 256;
 
 // Question embedding of one (layer, kv head): mean over the rep query heads of the GQA block and over the T_q
 // question tokens.  grid (H, layer_count), kEmbedThreads threads.  The rows (rep * T_q of them) are dealt to
-// RG = kEmbedThreads / (d/4) row groups; a thread adds up 4 adjacent channels of its group's rows and shared
-// memory combines the groups.
+// RG = kEmbedThreads / (d/8) row groups; a thread adds up 8 adjacent channels (16-byte loads) of its group's rows,
+// up to 16 rows in flight at once -- the kernel is a few memory round trips and nothing else -- and shared memory
+// combines the groups.
 template <typename T>
 __global__ void __launch_bounds__(kEmbedThreads) query_embed_kernel(const ScoreParams p) {
-    __shared__ float part[kEmbedThreads / 16][256 + 4];  // [row group <= 16][channel <= 256]
+    __shared__ __align__(16) float part[kEmbedThreads / 8][256 + 4];  // [row group <= 32][channel <= 256]
     __shared__ float red[kEmbedThreads / 32];
     const int h = blockIdx.x, li = blockIdx.y, d = p.g.d;
-    const int lanes_per_row = d >> 2;                 // threads across one row (4 channels each): 16, 32 or 64
-    const int RG = kEmbedThreads / lanes_per_row;     // row groups: 16, 8 or 4
+    const int lanes_per_row = d >> 3;                 // threads across one row (8 channels each): 8, 16 or 32
+    const int RG = kEmbedThreads / lanes_per_row;     // row groups: 32, 16 or 8
     const int cq = threadIdx.x % lanes_per_row, rg = threadIdx.x / lanes_per_row;
     const int rows = p.rep * p.T_q;
-    const T *q = reinterpret_cast<const T *>(p.Q) + (int64_t)li * p.ql + cq * 4;
-    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
-    // rows in batches of kRowBatch: all loads of a batch are issued before the first add
-    constexpr int kRowBatch = 8;
+    const T *q = reinterpret_cast<const T *>(p.Q) + (int64_t)li * p.ql + (int64_t)h * p.rep * p.qh + cq * 8;
+    float acc[8];
+#pragma unroll
+    for (int c = 0; c < 8; ++c) acc[c] = 0.0f;
+    constexpr int kRowBatch = sizeof(T) == 4 ? 8 : 16;
+    constexpr int W = 8 * (int)sizeof(T) / 4;  // 32-bit words of a thread's 8 channels
+    // (hr, j): query head inside the block and token of the thread's current row, stepped without a division
+    int hr = rg / p.T_q, j = rg - hr * p.T_q;
     for (int r0 = rg; r0 < rows; r0 += RG * kRowBatch) {
-        float x[kRowBatch][4];
+        uint32_t x[kRowBatch][W];
 #pragma unroll
         for (int b = 0; b < kRowBatch; ++b) {
-            const int r = r0 + b * RG;
-            x[b][0] = x[b][1] = x[b][2] = x[b][3] = 0.0f;
-            if (r < rows) {
-                const int hr = r / p.T_q, j = r - hr * p.T_q;
-                const T *src = q + (int64_t)(h * p.rep + hr) * p.qh + (int64_t)j * p.qt;
-                if constexpr (sizeof(T) == 4) {
-                    const float4 v = __ldg(reinterpret_cast<const float4 *>(src));
-                    x[b][0] = v.x; x[b][1] = v.y; x[b][2] = v.z; x[b][3] = v.w;
-                } else {
-                    const uint2 v = __ldg(reinterpret_cast<const uint2 *>(src));
-                    unpack2<T>(v.x, x[b][0], x[b][1]);
-                    unpack2<T>(v.y, x[b][2], x[b][3]);
+#pragma unroll
+            for (int i = 0; i < W; ++i) x[b][i] = 0u;  // +0.0 in every format
+            if (r0 + b * RG < rows) {
+                const uint4 *src = reinterpret_cast<const uint4 *>(q + (int64_t)hr * p.qh + (int64_t)j * p.qt);
+#pragma unroll
+                for (int i = 0; i < W / 4; ++i) {
+                    const uint4 v = __ldg(src + i);
+                    x[b][4 * i] = v.x; x[b][4 * i + 1] = v.y; x[b][4 * i + 2] = v.z; x[b][4 * i + 3] = v.w;
                 }
+            }
+            j += RG;
+            while (j >= p.T_q) {
+                j -= p.T_q;
+                ++hr;
             }
         }
 #pragma unroll
         for (int b = 0; b < kRowBatch; ++b) {
-            a0 += x[b][0]; a1 += x[b][1]; a2 += x[b][2]; a3 += x[b][3];
+            if constexpr (sizeof(T) == 4) {
+#pragma unroll
+                for (int c = 0; c < 8; ++c) acc[c] += __uint_as_float(x[b][c]);
+            } else {
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    float lo, hi;
+                    unpack2<T>(x[b][c], lo, hi);
+                    acc[2 * c] += lo;
+                    acc[2 * c + 1] += hi;
+                }
+            }
         }
     }
-    float *mine = &part[rg][cq * 4];
-    mine[0] = a0; mine[1] = a1; mine[2] = a2; mine[3] = a3;
+    float4 *mine = reinterpret_cast<float4 *>(&part[rg][cq * 8]);
+    mine[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    mine[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
     __syncthreads();
     float sq = 0.0f;
     if (threadIdx.x < d) {
         const int c = threadIdx.x;
-        float acc = 0.0f;
-        for (int g = 0; g < RG; ++g) acc += part[g][c];
-        const float v = acc / (float)rows;
+        float a = 0.0f;
+        for (int g = 0; g < RG; ++g) a += part[g][c];
+        const float v = a / (float)rows;
         p.qemb[((int64_t)li * p.g.H + h) * d + c] = v;
         sq = v * v;
     }
