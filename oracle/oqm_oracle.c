@@ -35,7 +35,16 @@
  *   - inverse map: fmaf(code, s, m), then one rounding to the output type;
  *   - GQA: query head h_q belongs to kv head h_q / (H_q / H_k);
  *   - zero norms: each norm is clamped below by 1e-12 (score becomes 0);
- *   - ties in top-K: the lower group index wins.
+ *   - ties in top-K: the lower group index wins;
+ *   - 16-bit metadata (meta_dtype = fp16 or bf16; Sec. 4.1 runs the model in
+ *     FP16, the (s_t, m_t) equation fixes no storage type): the offset is the
+ *     largest 16-bit value <= the channel minimum, the scale the smallest
+ *     16-bit value >= fl32((max - m) / levels), and the codes are taken
+ *     against THOSE two numbers, so that every code stays in range and the
+ *     reconstruction error stays <= s/2 for the stored s; the representative
+ *     key is rounded to nearest-even and its norm is the norm of the rounded
+ *     vector.  The bank arrays here stay binary32 and hold values that are
+ *     exactly representable in the 16-bit type.
  *
  * Pin status: every exported function is pinned by tests that do not call it
  * to produce their own expectation (closed forms, invariants, brute force,
@@ -70,6 +79,7 @@ typedef struct {
     int32_t bits;            /* 4 or 2 */
     int32_t kv_dtype;        /* ORC_BF16 | ORC_FP16 | ORC_FP32 */
     int32_t score_mode;      /* ORC_PER_LAYER | ORC_PER_HEAD */
+    int32_t meta_dtype;      /* type s, m and k-bar are stored in: ORC_FP32 (default reading) | ORC_FP16 | ORC_BF16 */
 } orc_config;
 
 /* Arrays of the memory bank, all indexed [layer][group][kv head]... */
@@ -161,6 +171,43 @@ void orc_convert_from_f32(const float *src, int dtype, int64_t n, void *dst) {
     }
 }
 
+/* Nearest-even rounding of a binary32 to the type `dtype`, returned as binary32. */
+float orc_round_nearest(float x, int dtype) {
+    if (dtype == ORC_BF16) return orc_bf16_to_f32(orc_f32_to_bf16(x));
+    if (dtype == ORC_FP16) return orc_f16_to_f32(orc_f32_to_f16(x));
+    return x;
+}
+
+/* The neighbour of the 16-bit pattern h one step towards -inf (dir < 0) or
+ * +inf (dir > 0) on the number line.  Both formats are sign-magnitude, so a
+ * step away from zero adds one to the pattern and a step towards zero takes
+ * one off; stepping down from +0 lands on the smallest negative subnormal. */
+static uint16_t step16(uint16_t h, int dir) {
+    int negative = (h & 0x8000u) != 0;
+    if ((h & 0x7fffu) == 0) return dir > 0 ? (uint16_t)0x0001u : (uint16_t)0x8001u;
+    if ((dir > 0) == !negative) return (uint16_t)(h + 1u); /* away from zero */
+    return (uint16_t)(h - 1u);                               /* towards zero   */
+}
+
+static float f32_of16(uint16_t h, int dtype) { return dtype == ORC_BF16 ? orc_bf16_to_f32(h) : orc_f16_to_f32(h); }
+static uint16_t to16(float x, int dtype) { return dtype == ORC_BF16 ? orc_f32_to_bf16(x) : orc_f32_to_f16(x); }
+
+/* Largest value of the type that is <= x (x finite and inside the type's range). */
+float orc_round_down(float x, int dtype) {
+    if (dtype == ORC_FP32) return x;
+    uint16_t h = to16(x, dtype);
+    if (f32_of16(h, dtype) > x) h = step16(h, -1);
+    return f32_of16(h, dtype);
+}
+
+/* Smallest value of the type that is >= x. */
+float orc_round_up(float x, int dtype) {
+    if (dtype == ORC_FP32) return x;
+    uint16_t h = to16(x, dtype);
+    if (f32_of16(h, dtype) < x) h = step16(h, +1);
+    return f32_of16(h, dtype);
+}
+
 /* ------------------------------------------------------------------ */
 /* O1  group quantizer (Sec. 3.4, Q_4 and the (s_t, m_t) equation)     */
 /* ------------------------------------------------------------------ */
@@ -172,7 +219,7 @@ static int levels_of(int bits) { return (1 << bits) - 1; } /* 15 for 4-bit, 3 fo
  * head and per channel across the G tokens.  codes is [H][G][d] with one
  * code per byte (not yet packed); s and m are [H][d].
  */
-void orc_quantize_group(const float *X, int H, int G, int d, int bits,
+void orc_quantize_group(const float *X, int H, int G, int d, int bits, int meta_dtype,
                         uint8_t *codes, float *s, float *m) {
     const float nlev = (float)levels_of(bits);
     for (int h = 0; h < H; ++h) {
@@ -184,8 +231,9 @@ void orc_quantize_group(const float *X, int H, int G, int d, int bits,
                 if (x < mn) mn = x;
                 if (x > mx) mx = x;
             }
+            mn = orc_round_down(mn, meta_dtype); /* the stored offset; unchanged for binary32 metadata */
             float range = mx - mn;
-            float sc = range / nlev;
+            float sc = orc_round_up(range / nlev, meta_dtype);
             s[h * d + c] = sc;
             m[h * d + c] = mn;
             for (int g = 0; g < G; ++g) {
@@ -231,13 +279,13 @@ float orc_dequant_value(int code, float s, float m) { return fmaf((float)code, s
 /*     memory": k_t = (1/G) sum_{i in G_t} K_i)                         */
 /* ------------------------------------------------------------------ */
 
-void orc_rep_key(const float *K, int H, int G, int d, float *rep, float *norm2) {
+void orc_rep_key(const float *K, int H, int G, int d, int meta_dtype, float *rep, float *norm2) {
     for (int h = 0; h < H; ++h) {
         double n2 = 0.0;
         for (int c = 0; c < d; ++c) {
             double acc = 0.0;
             for (int g = 0; g < G; ++g) acc += (double)K[((int64_t)h * G + g) * d + c];
-            float kb = (float)(acc / (double)G);
+            float kb = orc_round_nearest((float)(acc / (double)G), meta_dtype);
             rep[h * d + c] = kb;
             n2 += (double)kb * (double)kb;
         }
@@ -269,6 +317,7 @@ static int check_cfg(const orc_config *c) {
     if ((c->head_dim * c->bits) % 8) return 0;
     if (c->kv_dtype < 0 || c->kv_dtype > 2) return 0;
     if (c->score_mode < 0 || c->score_mode > 1) return 0;
+    if (c->meta_dtype < 0 || c->meta_dtype > 2) return 0;
     return 1;
 }
 
@@ -331,12 +380,12 @@ int32_t orc_quantize_frame(const orc_config *cfg, const orc_store *st,
                 }
             float *s = (which ? st->scale_v : st->scale_k) + meta_off(cfg, l, t, 0);
             float *m = (which ? st->zero_v : st->zero_k) + meta_off(cfg, l, t, 0);
-            orc_quantize_group(X, H, G, d, cfg->bits, codes, s, m);
+            orc_quantize_group(X, H, G, d, cfg->bits, cfg->meta_dtype, codes, s, m);
             uint8_t *dst = (which ? st->codes_v : st->codes_k) + codes_off(cfg, l, t, 0);
             for (int64_t r = 0; r < (int64_t)H * G; ++r)
                 orc_pack_row(codes + r * d, d, cfg->bits, dst + r * code_row_bytes(cfg));
             if (!which)
-                orc_rep_key(Ks, H, G, d, st->rep_key + meta_off(cfg, l, t, 0),
+                orc_rep_key(Ks, H, G, d, cfg->meta_dtype, st->rep_key + meta_off(cfg, l, t, 0),
                             st->rep_norm2 + norm_off(cfg, l, t, 0));
         }
         free(X); free(Ks); free(codes);
@@ -593,7 +642,8 @@ double orc_fp16_kv_bytes(int32_t L, int64_t frames, int32_t N, int32_t H_kv, int
 /* bytes this store really holds for `groups` groups per layer, metadata included */
 double orc_store_bytes(const orc_config *c, int64_t groups, int32_t with_metadata) {
     double per_head_codes = 2.0 * c->group_tokens * (double)code_row_bytes(c); /* K and V */
-    double per_head_meta = 4.0 * c->head_dim * 4.0 /* sK mK sV mV */ + c->head_dim * 4.0 /* k-bar */ + 4.0;
+    double eb = c->meta_dtype == ORC_FP32 ? 4.0 : 2.0; /* bytes of one stored s, m or k-bar value */
+    double per_head_meta = 4.0 * c->head_dim * eb /* sK mK sV mV */ + c->head_dim * eb /* k-bar */ + 4.0 /* norm */;
     double per = per_head_codes + (with_metadata ? per_head_meta : 0.0);
     return per * c->n_kv_heads * (double)groups * c->n_layers;
 }

@@ -37,7 +37,7 @@ def build(force: bool = False) -> Path:
 class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "n_q_heads", "n_kv_heads", "head_dim", "group_tokens",
-        "capacity_groups", "bits", "kv_dtype", "score_mode")]
+        "capacity_groups", "bits", "kv_dtype", "score_mode", "meta_dtype")]
 
 
 class _Store(C.Structure):
@@ -62,6 +62,9 @@ def lib():
         L.orc_f32_to_bf16.argtypes = [C.c_float]
         L.orc_f32_to_f16.restype = C.c_uint16
         L.orc_f32_to_f16.argtypes = [C.c_float]
+        for name in ("orc_round_nearest", "orc_round_down", "orc_round_up"):
+            getattr(L, name).restype = C.c_float
+            getattr(L, name).argtypes = [C.c_float, C.c_int]
         L.orc_dequant_value.restype = C.c_float
         L.orc_dequant_value.argtypes = [C.c_int, C.c_float, C.c_float]
         L.orc_paper_ratio.restype = C.c_double
@@ -86,13 +89,14 @@ def _p(a):
 
 
 def make_config(n_layers, n_q_heads, n_kv_heads, head_dim, group_tokens, capacity_groups,
-                bits=4, kv_dtype=BF16, score_mode=PER_LAYER) -> Config:
+                bits=4, kv_dtype=BF16, score_mode=PER_LAYER, meta_dtype=FP32) -> Config:
     return Config(n_layers, n_q_heads, n_kv_heads, head_dim, group_tokens, capacity_groups,
-                  bits, kv_dtype, score_mode)
+                  bits, kv_dtype, score_mode, meta_dtype)
 
 
 class Store:
-    """Host-side memory bank: plain NumPy arrays, zero-initialised."""
+    """Host-side memory bank: plain NumPy arrays, zero-initialised.  s, m and k-bar are float32 arrays whatever
+    cfg.meta_dtype says: with 16-bit metadata they hold values that are exactly representable in that type."""
 
     def __init__(self, cfg: Config):
         L, T, H, G, d = cfg.n_layers, cfg.capacity_groups, cfg.n_kv_heads, cfg.group_tokens, cfg.head_dim
@@ -131,14 +135,27 @@ def from_f32(a: np.ndarray, dtype: int) -> np.ndarray:
 
 # ---------------------------------------------------------------- pieces
 
-def quantize_group(X: np.ndarray, bits: int = 4):
+def round_nearest(x: float, dtype: int) -> float:
+    return float(lib().orc_round_nearest(C.c_float(x), dtype))
+
+
+def round_down(x: float, dtype: int) -> float:
+    return float(lib().orc_round_down(C.c_float(x), dtype))
+
+
+def round_up(x: float, dtype: int) -> float:
+    return float(lib().orc_round_up(C.c_float(x), dtype))
+
+
+def quantize_group(X: np.ndarray, bits: int = 4, meta_dtype: int = FP32):
     """X [H][G][d] float32 -> (codes [H][G][d] uint8 unpacked, s [H][d], m [H][d])."""
     X = np.ascontiguousarray(X, np.float32)
     H, G, d = X.shape
     codes = np.empty((H, G, d), np.uint8)
     s = np.empty((H, d), np.float32)
     m = np.empty((H, d), np.float32)
-    lib().orc_quantize_group(_p(X), C.c_int(H), C.c_int(G), C.c_int(d), C.c_int(bits), _p(codes), _p(s), _p(m))
+    lib().orc_quantize_group(_p(X), C.c_int(H), C.c_int(G), C.c_int(d), C.c_int(bits), C.c_int(meta_dtype),
+                             _p(codes), _p(s), _p(m))
     return codes, s, m
 
 
@@ -160,13 +177,13 @@ def dequant_value(code: int, s: float, m: float) -> float:
     return float(lib().orc_dequant_value(int(code), C.c_float(s), C.c_float(m)))
 
 
-def rep_key(K: np.ndarray):
+def rep_key(K: np.ndarray, meta_dtype: int = FP32):
     """K [H][G][d] float32 -> (k-bar [H][d] float32, |k-bar_h|^2 [H] float32)."""
     K = np.ascontiguousarray(K, np.float32)
     H, G, d = K.shape
     rep = np.empty((H, d), np.float32)
     n2 = np.empty((H,), np.float32)
-    lib().orc_rep_key(_p(K), C.c_int(H), C.c_int(G), C.c_int(d), _p(rep), _p(n2))
+    lib().orc_rep_key(_p(K), C.c_int(H), C.c_int(G), C.c_int(d), C.c_int(meta_dtype), _p(rep), _p(n2))
     return rep, n2
 
 

@@ -206,6 +206,139 @@ def test_rep_key_is_numpy_mean_over_tokens(orc):
     np.testing.assert_allclose(n2, [140.0, 140.0])
 
 
+# ------------------------------------------------------------------ 16-bit metadata (storage reading of s, m, k-bar)
+
+def _values16(dtype_name):
+    """Every finite value of a 16-bit format, ascending, as float64 (built from bit patterns with torch, not with
+    the oracle)."""
+    bits = torch.arange(65536, dtype=torch.int32).to(torch.int16)
+    t = bits.view(torch.float16 if dtype_name == "fp16" else torch.bfloat16).to(torch.float64)
+    v = t[torch.isfinite(t)].numpy()
+    return np.unique(v)  # sorted; +0 and -0 collapse
+
+
+@pytest.mark.parametrize("dtype_name", ["fp16", "bf16"])
+def test_directed_rounding_brackets_every_input(orc, dtype_name):
+    """round_down(x) is the largest representable value <= x and round_up(x) the smallest >= x: checked against the
+    sorted table of all values of the format (searchsorted), at representable points, midpoints and random points."""
+    dt = orc.FP16 if dtype_name == "fp16" else orc.BF16
+    table = _values16(dtype_name)
+    rng = np.random.default_rng(41)
+    lim = 6.0e4 if dtype_name == "fp16" else 1.0e30
+    pts = np.concatenate([
+        rng.choice(table[np.abs(table) < lim], 300),                                      # representable
+        rng.standard_normal(300) * 3.0, rng.standard_normal(200) * 1e-3, rng.standard_normal(100) * 1e3,
+        rng.standard_normal(100) * 1e-7,                                                  # fp16 subnormal range
+        np.array([0.0, 1e-30, -1e-30, 1.0, -1.0, 0.1, -0.1]),
+    ]).astype(np.float32)
+    mids = ((table[1:] + table[:-1]) / 2.0)
+    mids = mids[np.abs(mids) < lim]
+    pts = np.concatenate([pts, rng.choice(mids, 300).astype(np.float32)])
+    for x in pts:
+        x = float(x)
+        lo = table[np.searchsorted(table, x, side="right") - 1]
+        hi = table[np.searchsorted(table, x, side="left")]
+        assert orc.round_down(x, dt) == lo, x
+        assert orc.round_up(x, dt) == hi, x
+        assert orc.round_down(x, orc.FP32) == x and orc.round_up(x, orc.FP32) == x
+    # nearest-even agrees with torch's conversion
+    t = torch.from_numpy(pts)
+    want = t.to(torch.float16 if dtype_name == "fp16" else torch.bfloat16).to(torch.float32).numpy()
+    got = np.array([orc.round_nearest(float(x), dt) for x in pts], np.float32)
+    np.testing.assert_array_equal(got, want)
+
+
+@pytest.mark.parametrize("dtype_name", ["fp16", "bf16"])
+@pytest.mark.parametrize("bits", [4, 2])
+def test_quantizer_with_16bit_metadata_keeps_codes_in_range_and_the_error_bound(orc, dtype_name, bits):
+    dt = orc.FP16 if dtype_name == "fp16" else orc.BF16
+    tdt = torch.float16 if dtype_name == "fp16" else torch.bfloat16
+    table = _values16(dtype_name)
+    rng = np.random.default_rng(43)
+    X = _group(rng, H=3, G=50, d=64)
+    X[1, :, 5] = 0.375           # a constant channel
+    X[2, :, 7] += 100.0          # a channel whose offset is far from zero: m loses bits in 16-bit storage
+    codes, s, m = orc.quantize_group(X, bits, dt)
+    nlev = (1 << bits) - 1
+    # stored values are representable
+    for a in (s, m):
+        np.testing.assert_array_equal(torch.from_numpy(a).to(tdt).to(torch.float32).numpy(), a)
+    mn, mx = X.min(axis=1).astype(np.float64), X.max(axis=1).astype(np.float64)
+    m64, s64 = m.astype(np.float64), s.astype(np.float64)
+    # m is the largest representable value <= min
+    assert np.all(m64 <= mn)
+    nxt = table[np.searchsorted(table, m64.ravel(), side="right")].reshape(m.shape)
+    assert np.all(nxt > mn)
+    # s covers the range from the STORED offset (so the top code never overshoots) and is minimal up to one step
+    assert np.all(m64 + nlev * s64 >= mx * (1 - 2.0 ** -23) - 1e-30)
+    prev = table[np.maximum(np.searchsorted(table, s64.ravel(), side="left") - 1, 0)].reshape(s.shape)
+    need = ((mx - m64) / nlev)
+    assert np.all((prev < need * (1 + 2.0 ** -22)) | (s64 == 0))
+    assert s[1, 5] == 0 and np.all(codes[1, :, 5] == 0) and m[1, 5] == np.float32(0.375)
+    # codes in range, nearest level of the stored (s, m), error <= s/2
+    assert codes.max() <= nlev
+    xhat = m64[:, None, :] + codes.astype(np.float64) * s64[:, None, :]
+    err = np.abs(X.astype(np.float64) - xhat)
+    assert np.all(err <= s64[:, None, :] * (0.5 + 2.0 ** -18) + 2.0 ** -22 * np.abs(X))
+    lv = np.arange(nlev + 1, dtype=np.float64)
+    dist = np.abs(X.astype(np.float64)[..., None] - (m64[:, None, :, None] + lv * s64[:, None, :, None]))
+    chosen = np.take_along_axis(dist, codes[..., None].astype(np.int64), axis=-1)[..., 0]
+    assert np.all(chosen <= dist.min(axis=-1) + 2.0 ** -20 * np.maximum(1.0, np.abs(X)))
+    # inputs that are already 16-bit values of the same type keep their minimum exactly
+    X16 = torch.from_numpy(X).to(tdt).to(torch.float32).numpy()
+    _, _, m16 = orc.quantize_group(X16, bits, dt)
+    np.testing.assert_array_equal(m16, X16.min(axis=1))
+
+
+@pytest.mark.parametrize("dtype_name", ["fp16", "bf16"])
+def test_rep_key_with_16bit_metadata_is_the_rounded_mean(orc, dtype_name):
+    dt = orc.FP16 if dtype_name == "fp16" else orc.BF16
+    tdt = torch.float16 if dtype_name == "fp16" else torch.bfloat16
+    rng = np.random.default_rng(47)
+    K = _group(rng, H=4, G=50, d=128)
+    rep, n2 = orc.rep_key(K, dt)
+    mean = torch.from_numpy(K.astype(np.float64).mean(axis=1))
+    lo = mean.to(torch.float32).to(tdt).to(torch.float64).numpy()
+    # the mean passes through binary32 first; allow the neighbouring 16-bit value only where that matters
+    step = np.abs(lo) * (2.0 ** -10 if dtype_name == "fp16" else 2.0 ** -7) + 1e-12
+    assert np.all(np.abs(rep.astype(np.float64) - lo) <= step)
+    assert np.mean(rep.astype(np.float64) == lo) > 0.999
+    np.testing.assert_array_equal(torch.from_numpy(rep).to(tdt).to(torch.float32).numpy(), rep)   # representable
+    np.testing.assert_allclose(n2, (rep.astype(np.float64) ** 2).sum(axis=1), rtol=1e-6)           # norm of the STORED key
+
+
+def test_store_bytes_with_16bit_metadata(orc):
+    """Per (group, kv head) at G = 50, d = 128: 6400 bytes of codes, 5 x 128 metadata values, one norm."""
+    for dt, eb in ((orc.FP32, 4), (orc.FP16, 2), (orc.BF16, 2)):
+        cfg = orc.make_config(1, 1, 1, 128, 50, 1, meta_dtype=dt)
+        assert orc.store_bytes(cfg, 1, True) == 6400 + 5 * 128 * eb + 4
+        assert orc.store_bytes(cfg, 1, False) == 6400
+    full = 2 * 50 * 128 * 2  # the same group in 16-bit K and V
+    assert abs(full / (orc.store_bytes(orc.make_config(1, 1, 1, 128, 50, 1, meta_dtype=orc.FP16), 1, True) - 4) - 10 / 3) < 1e-9
+
+
+def test_quantize_frame_with_16bit_metadata_matches_the_group_functions(orc):
+    """The frame-level call applies the same reading to every (layer, group, head) and to the representative key."""
+    rng = np.random.default_rng(53)
+    L, T, H, G, d = 2, 3, 2, 5, 32
+    cfg = orc.make_config(L, 4, H, d, G, T, kv_dtype=orc.FP32, meta_dtype=orc.BF16)
+    st = orc.Store(cfg)
+    K = rng.standard_normal((L, T, H, G, d)).astype(np.float32)
+    V = rng.standard_normal((L, T, H, G, d)).astype(np.float32)
+    assert orc.quantize_frame(cfg, st, 0, L, 0, T, K, V, (T * H * G * d, H * G * d, G * d, d)) == 0
+    for l in range(L):
+        for t in range(T):
+            _, s, m = orc.quantize_group(V[l, t], 4, orc.BF16)
+            np.testing.assert_array_equal(st.scale_v[l, t], s)
+            np.testing.assert_array_equal(st.zero_v[l, t], m)
+            rep, n2 = orc.rep_key(K[l, t], orc.BF16)
+            np.testing.assert_array_equal(st.rep_key[l, t], rep)
+            np.testing.assert_array_equal(st.rep_norm2[l, t], n2)
+    f32 = orc.Store(orc.make_config(L, 4, H, d, G, T, kv_dtype=orc.FP32))
+    orc.quantize_frame(f32.cfg, f32, 0, L, 0, T, K, V, (T * H * G * d, H * G * d, G * d, d))
+    assert np.all(st.zero_v <= f32.zero_v) and np.all(st.scale_v >= f32.scale_v)
+
+
 # ------------------------------------------------------------------ O3 / O4 query embedding, scores
 
 def test_query_embedding_gqa_blocks_and_token_mean(orc):
