@@ -65,19 +65,34 @@ def parse():
     ap.add_argument("--query-every", type=int, default=60, help="C4: frames between questions")
     ap.add_argument("--layers", type=int, default=0, help="override L (reduced case for profiler captures)")
     ap.add_argument("--frames", type=int, default=0, help="override T (reduced case for profiler captures)")
+    ap.add_argument("--meta", default="fp32", choices=["fp32", "fp16", "bf16"],
+                    help="type the bank keeps s, m and k-bar in (fp32: the default reading; 16-bit: the compact variant)")
     return ap.parse_args()
 
 
 # ---------------------------------------------------------------- byte accounting (algorithmic bytes)
 
+META_CODE = {"bf16": 0, "fp16": 1, "fp32": 2}
+
+
+def meta_of(sh) -> str:
+    return str(sh.extra.get("meta", "fp32"))
+
+
+def meta_bytes(sh) -> int:
+    """Bytes of one stored s, m or k-bar value."""
+    return 4 if meta_of(sh) == "fp32" else 2
+
+
 def bytes_quantize(sh, frames):
     e = 4 if sh.dtype == "fp32" else 2
-    per = 2 * sh.H_k * sh.G * sh.d * e + 2 * sh.H_k * sh.G * sh.d // 2 + 4 * sh.H_k * sh.d * 4 + sh.H_k * sh.d * 4 + sh.H_k * 4
+    mb = meta_bytes(sh)
+    per = 2 * sh.H_k * sh.G * sh.d * e + 2 * sh.H_k * sh.G * sh.d // 2 + 4 * sh.H_k * sh.d * mb + sh.H_k * sh.d * mb + sh.H_k * 4
     return per * frames * sh.L
 
 
 def bytes_score(sh, groups):
-    return (sh.H_k * sh.d * 4 + sh.H_k * 4 + 4) * groups * sh.L + sh.L * sh.H_q * sh.T_q * sh.d * 2
+    return (sh.H_k * sh.d * meta_bytes(sh) + sh.H_k * 4 + 4) * groups * sh.L + sh.L * sh.H_q * sh.T_q * sh.d * 2
 
 
 def bytes_topk(sh, groups):
@@ -85,7 +100,7 @@ def bytes_topk(sh, groups):
 
 
 def bytes_gather(sh, k):
-    per = 2 * sh.H_k * sh.G * sh.d // 2 + 4 * sh.H_k * sh.d * 4 + 2 * sh.H_k * sh.G * sh.d * 2
+    per = 2 * sh.H_k * sh.G * sh.d // 2 + 4 * sh.H_k * sh.d * meta_bytes(sh) + 2 * sh.H_k * sh.G * sh.d * 2
     return per * k * sh.L
 
 
@@ -158,7 +173,8 @@ def oracle_sample(sh, K_cpu, V_cpu, Q_cpu, frames, threads=0):
     from paper_2510_18269_b200 import synth
     import numpy as np
     k = min(sh.k, frames)
-    cfg = orc.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, frames, 4, {"bf16": 0, "fp16": 1, "fp32": 2}[sh.dtype])
+    cfg = orc.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, frames, 4, {"bf16": 0, "fp16": 1, "fp32": 2}[sh.dtype],
+                          meta_dtype=META_CODE[meta_of(sh)])
     st = orc.Store(cfg)
     kn, vn, qn = synth.as_u16(K_cpu), synth.as_u16(V_cpu), synth.as_u16(Q_cpu)
     strides = (frames * sh.H_k * sh.G * sh.d, sh.H_k * sh.G * sh.d, sh.G * sh.d, sh.d)
@@ -247,7 +263,8 @@ def run_ours(args, sh):
     # independent streams per rank (weak scaling: every GPU serves its own video stream)
     import dataclasses
     sh = dataclasses.replace(sh, seed=sh.seed + 17 * rank)
-    cfg = oqm.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, sh.T, 4, oqm.dtype_code(synth.DTYPES[sh.dtype]))
+    cfg = oqm.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, sh.T, 4, oqm.dtype_code(synth.DTYPES[sh.dtype]),
+                          meta_dtype=META_CODE[meta_of(sh)])
     store = oqm.Store(cfg, device=dev, zero=False)
     K, V = synth.kv_stream(sh, dev)
     Q = synth.queries(sh, dev)
@@ -356,7 +373,7 @@ def run_ours(args, sh):
 
     def roof(name, nbytes, ms, launches, unit_count):
         a = nbytes / launches / (ms / launches * 1e-3) / 1e9
-        tpu = NCU_TRAFFIC_PER_UNIT.get(name)
+        tpu = NCU_TRAFFIC_PER_UNIT.get(name) if meta_of(sh) == "fp32" else None  # captured with binary32 metadata only
         return {"kernel": name, "bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s", "frac": a / peak,
                 "traffic": None if tpu is None else tpu * sh.H_k * unit_count / launches, "peak_source": peak_src,
                 "algorithmic_bytes_per_launch": nbytes / launches, "ms_per_launch": ms / launches}
@@ -375,7 +392,7 @@ def run_ours(args, sh):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": total_ms / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": sh.name, "L": sh.L, "H_q": sh.H_q, "H_k": sh.H_k, "d": sh.d, "G": sh.G, "T": sh.T,
-                   "T_q": sh.T_q, "k": sh.k, "kv_dtype": sh.dtype, "frames_per_quantize_call": fpc,
+                   "T_q": sh.T_q, "k": sh.k, "kv_dtype": sh.dtype, "meta_dtype": meta_of(sh), "frames_per_quantize_call": fpc,
                    "l2": "inputs 20.6 GB >> L2; 512 MB flush between quantize and retrieve",
                    "multi_gpu": "independent stream per rank, no collective"},
         "submetrics": {
@@ -477,7 +494,8 @@ def run_stream(args, sh):
     torch.cuda.set_device(0)
     dev = torch.device("cuda", 0)
     oqm.lib()
-    cfg = oqm.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, sh.T, 4, oqm.dtype_code(synth.DTYPES[sh.dtype]))
+    cfg = oqm.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, sh.T, 4, oqm.dtype_code(synth.DTYPES[sh.dtype]),
+                          meta_dtype=META_CODE[meta_of(sh)])
     store = oqm.Store(cfg, device=dev, zero=False)
     pool = 32                                    # distinct synthetic frames, cycled (5.6 MB of K and of V per frame)
     psh = dataclasses.replace(sh, T=pool)
@@ -565,6 +583,9 @@ def main():
     args = parse()
     from paper_2510_18269_b200 import synth
     sh = synth.CONFIGS[args.config]
+    if args.meta != "fp32":
+        import dataclasses
+        sh = dataclasses.replace(sh, extra={**sh.extra, "meta": args.meta}, name=f"{sh.name}-meta-{args.meta}")
     if args.config == "C4" and args.impl == "ours":
         if args.frames:
             import dataclasses

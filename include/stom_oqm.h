@@ -75,6 +75,8 @@ typedef struct stom_oqm_config {
     int32_t bits;            /* 4 (the paper's setting) or 2 (its ablation)     */
     int32_t kv_dtype;        /* STOM_BF16 | STOM_FP16 | STOM_FP32: type of K, V, Q inputs */
     int32_t score_mode;      /* STOM_SCORE_PER_LAYER | STOM_SCORE_PER_HEAD      */
+    int32_t meta_dtype;      /* type the bank keeps s, m and k-bar in: STOM_FP32 (the (s_t, m_t) equation taken
+                                in binary32), or STOM_FP16 / STOM_BF16 (half the metadata bytes; see below)   */
 } stom_oqm_config;
 
 /*
@@ -83,21 +85,28 @@ typedef struct stom_oqm_config {
  *   codes_*   [L][cap][H_k][G][d*bits/8]  uint8: 8/bits codes per byte along
  *             the channel axis, lowest channel in the lowest bits (bits = 4:
  *             two per byte, even channel in the low nibble)
- *   scale_*   [L][cap][H_k][d] float: s = (max - min)/15 over the G tokens
- *   zero_*    [L][cap][H_k][d] float: m = min over the G tokens
- *   rep_key   [L][cap][H_k][d] float: mean of the group's keys (k-bar)
- *   rep_norm2 [L][cap][H_k]    float: squared L2 norm of k-bar per head
+ *   scale_*   [L][cap][H_k][d] meta_dtype: s = (max - min)/15 over the G tokens
+ *   zero_*    [L][cap][H_k][d] meta_dtype: m = min over the G tokens
+ *   rep_key   [L][cap][H_k][d] meta_dtype: mean of the group's keys (k-bar)
+ *   rep_norm2 [L][cap][H_k]    float: squared L2 norm of the STORED k-bar per head
+ * With 16-bit metadata (the paper fixes no storage type for the (s_t, m_t) of
+ * Sec. 3.4; its experiments run in FP16, Sec. 4.1) the stored offset is the
+ * largest 16-bit value <= the channel minimum, the stored scale the smallest
+ * 16-bit value >= fl32((max - m)/levels) for that stored m, and the codes are
+ * taken against the stored pair: every code stays in range and the
+ * reconstruction error stays <= s/2 of the stored s.  k-bar is rounded to
+ * nearest-even.  Inputs must then lie inside the 16-bit type's finite range.
  * System-prompt tokens are not part of the bank; they stay in full precision
  * in the caller's active cache.
  */
 typedef struct stom_oqm_store {
     uint8_t *codes_k;
     uint8_t *codes_v;
-    float *scale_k;
-    float *zero_k;
-    float *scale_v;
-    float *zero_v;
-    float *rep_key;
+    void *scale_k; /* elements of cfg.meta_dtype, like the next four */
+    void *zero_k;
+    void *scale_v;
+    void *zero_v;
+    void *rep_key;
     float *rep_norm2;
 } stom_oqm_store;
 

@@ -15,6 +15,7 @@ int32_t check_config(const stom_oqm_config *c) {
     if (c->bits != 4 && c->bits != 2) return STOM_ERR_UNSUPPORTED;
     if (c->kv_dtype != STOM_BF16 && c->kv_dtype != STOM_FP16 && c->kv_dtype != STOM_FP32) return STOM_ERR_UNSUPPORTED;
     if (c->score_mode != STOM_SCORE_PER_LAYER && c->score_mode != STOM_SCORE_PER_HEAD) return STOM_ERR_UNSUPPORTED;
+    if (c->meta_dtype != STOM_BF16 && c->meta_dtype != STOM_FP16 && c->meta_dtype != STOM_FP32) return STOM_ERR_UNSUPPORTED;
     if (c->head_dim != 64 && c->head_dim != 128 && c->head_dim != 256) return STOM_ERR_SHAPE;
     if (c->group_tokens < 1 || c->group_tokens > 64) return STOM_ERR_SHAPE;
     // one (group, head) block of codes must keep 16-byte alignment for vector stores
@@ -50,7 +51,7 @@ extern "C" int32_t stom_oqm_store_layout(const stom_oqm_config *cfg, stom_oqm_la
     if (!out) return STOM_ERR_INVALID_ARG;
     const int64_t slots = (int64_t)cfg->n_layers * cfg->capacity_groups * cfg->n_kv_heads;
     out->bytes_codes = slots * cfg->group_tokens * (cfg->head_dim * cfg->bits / 8);
-    out->bytes_meta = slots * cfg->head_dim * 4;
+    out->bytes_meta = slots * cfg->head_dim * elem_bytes(cfg->meta_dtype);
     out->bytes_norm2 = slots * 4;
     int64_t off = 0;
     out->off_codes_k = off; off = round_up(off + out->bytes_codes, 256);
@@ -74,11 +75,11 @@ extern "C" int32_t stom_oqm_store_bind(const stom_oqm_config *cfg, void *arena, 
     uint8_t *b = static_cast<uint8_t *>(arena);
     out->codes_k = b + lay.off_codes_k;
     out->codes_v = b + lay.off_codes_v;
-    out->scale_k = reinterpret_cast<float *>(b + lay.off_scale_k);
-    out->zero_k = reinterpret_cast<float *>(b + lay.off_zero_k);
-    out->scale_v = reinterpret_cast<float *>(b + lay.off_scale_v);
-    out->zero_v = reinterpret_cast<float *>(b + lay.off_zero_v);
-    out->rep_key = reinterpret_cast<float *>(b + lay.off_rep_key);
+    out->scale_k = b + lay.off_scale_k;
+    out->zero_k = b + lay.off_zero_k;
+    out->scale_v = b + lay.off_scale_v;
+    out->zero_v = b + lay.off_zero_v;
+    out->rep_key = b + lay.off_rep_key;
     out->rep_norm2 = reinterpret_cast<float *>(b + lay.off_rep_norm2);
     return STOM_OK;
 }

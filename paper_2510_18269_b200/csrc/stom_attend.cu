@@ -36,7 +36,7 @@ constexpr int kAtHeads = 8;       // query heads handled together
 struct AttendParams {
     const int32_t *idx;
     const uint8_t *codes_k, *codes_v;
-    const float *scale_k, *zero_k, *scale_v, *zero_v;
+    const void *scale_k, *zero_k, *scale_v, *zero_v;  // elements of g.meta_dtype
     const void *q;
     int64_t q_sl, q_sh;  // element strides of q_dec: layer, query head
     const void *ksys, *vsys;
@@ -152,11 +152,7 @@ __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p
     };
     auto load_stats = [&](bool keys, float (&s)[8], float (&m)[8]) {
         if (is_sys || n_tok == 0) return;
-        const float4 *sp = reinterpret_cast<const float4 *>((keys ? p.scale_k : p.scale_v) + slot * D + cl * 8);
-        const float4 *mp = reinterpret_cast<const float4 *>((keys ? p.zero_k : p.zero_v) + slot * D + cl * 8);
-        const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1), m0 = __ldg(mp), m1 = __ldg(mp + 1);
-        s[0] = s0.x; s[1] = s0.y; s[2] = s0.z; s[3] = s0.w; s[4] = s1.x; s[5] = s1.y; s[6] = s1.z; s[7] = s1.w;
-        m[0] = m0.x; m[1] = m0.y; m[2] = m0.z; m[3] = m0.w; m[4] = m1.x; m[5] = m1.y; m[6] = m1.z; m[7] = m1.w;
+        load_scale_zero8(keys ? p.scale_k : p.scale_v, keys ? p.zero_k : p.zero_v, slot * D + cl * 8, p.g.meta_dtype, s, m);
     };
 
     const int n_blocks = gridDim.x;

@@ -24,7 +24,7 @@ constexpr int kDqWarps = 4;
 struct DequantParams {
     const int32_t *idx;
     const uint8_t *codes_k, *codes_v;
-    const float *scale_k, *zero_k, *scale_v, *zero_v;
+    const void *scale_k, *zero_k, *scale_v, *zero_v;  // elements of g.meta_dtype
     void *ka, *va;
     int64_t sl, sh, st;  // element strides of the active cache: layer, head, token
     BankGeom g;
@@ -90,11 +90,14 @@ __global__ void __launch_bounds__(kDqWarps * 32) dequant_gather_kernel(const Deq
     }
     uint64_t s2[4], m2[4];
     {
-        const float4 *sp = reinterpret_cast<const float4 *>((which ? p.scale_v : p.scale_k) + slot * d + cl * 8);
-        const float4 *mp = reinterpret_cast<const float4 *>((which ? p.zero_v : p.zero_k) + slot * d + cl * 8);
-        const float4 s0 = __ldg(sp), s1 = __ldg(sp + 1), m0 = __ldg(mp), m1 = __ldg(mp + 1);
-        s2[0] = dq_pack(s0.x, s0.y); s2[1] = dq_pack(s0.z, s0.w); s2[2] = dq_pack(s1.x, s1.y); s2[3] = dq_pack(s1.z, s1.w);
-        m2[0] = dq_pack(m0.x, m0.y); m2[1] = dq_pack(m0.z, m0.w); m2[2] = dq_pack(m1.x, m1.y); m2[3] = dq_pack(m1.z, m1.w);
+        float sf[8], mf[8];
+        load_scale_zero8(which ? p.scale_v : p.scale_k, which ? p.zero_v : p.zero_k, slot * d + cl * 8, p.g.meta_dtype,
+                         sf, mf);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            s2[i] = dq_pack(sf[2 * i], sf[2 * i + 1]);
+            m2[i] = dq_pack(mf[2 * i], mf[2 * i + 1]);
+        }
     }
     OT *out = reinterpret_cast<OT *>(which ? p.va : p.ka) + (int64_t)li * p.sl + (int64_t)h * p.sh +
               ((int64_t)p.token_offset + (int64_t)j * G) * p.st + cl * 8;

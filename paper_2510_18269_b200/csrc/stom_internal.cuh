@@ -40,11 +40,13 @@ struct BankGeom {
     int32_t G;        // tokens per group
     int32_t d;        // head dim
     int32_t cap;      // groups per layer
-    int32_t row_bytes;  // packed bytes per token row = d/2
+    int32_t row_bytes;  // packed bytes per token row = d * bits / 8
+    int32_t meta_dtype;  // STOM_FP32 | STOM_FP16 | STOM_BF16: element type of the s, m and k-bar arrays
 };
 
 inline BankGeom bank_geom(const stom_oqm_config *c) {
-    return BankGeom{c->n_kv_heads, c->group_tokens, c->head_dim, c->capacity_groups, c->head_dim * c->bits / 8};
+    return BankGeom{c->n_kv_heads, c->group_tokens, c->head_dim, c->capacity_groups, c->head_dim * c->bits / 8,
+                    c->meta_dtype};
 }
 
 // A2+A3 -> A4 inside one retrieval: same checks and launch as stom_oqm_dequant_gather; `after_producer` launches the
@@ -118,6 +120,39 @@ template <>
 __device__ __forceinline__ uint32_t pack2<__half>(float a, float b) {
     __half2 v = __floats2half2_rn(a, b);
     return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// Eight adjacent values of a bank array of s, m or k-bar (element type MT), starting at element `at` (a multiple of
+// 8), as floats.
+template <typename MT>
+__device__ __forceinline__ void load_meta8(const void *base, int64_t at, float (&f)[8]) {
+    if constexpr (sizeof(MT) == 4) {
+        const float4 *p = reinterpret_cast<const float4 *>(static_cast<const float *>(base) + at);
+        const float4 a = __ldg(p), b = __ldg(p + 1);
+        f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+    } else {
+        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(static_cast<const MT *>(base) + at));
+        unpack2<MT>(v.x, f[0], f[1]);
+        unpack2<MT>(v.y, f[2], f[3]);
+        unpack2<MT>(v.z, f[4], f[5]);
+        unpack2<MT>(v.w, f[6], f[7]);
+    }
+}
+
+// A (scale, offset) pair of 8 channels with the element type known only at run time: one warp-uniform branch around
+// both loads, so that they are in flight together.  Used where the load happens once per unit of work.
+__device__ __forceinline__ void load_scale_zero8(const void *scale, const void *zero, int64_t at, int meta_dtype,
+                                                 float (&s)[8], float (&m)[8]) {
+    if (meta_dtype == STOM_FP32) {
+        load_meta8<float>(scale, at, s);
+        load_meta8<float>(zero, at, m);
+    } else if (meta_dtype == STOM_BF16) {
+        load_meta8<__nv_bfloat16>(scale, at, s);
+        load_meta8<__nv_bfloat16>(zero, at, m);
+    } else {
+        load_meta8<__half>(scale, at, s);
+        load_meta8<__half>(zero, at, m);
+    }
 }
 
 // The codes of 8 adjacent channels (32 bits at 4 bits per code, 16 bits at 2), each as the bit pattern of the float

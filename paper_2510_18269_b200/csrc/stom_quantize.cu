@@ -54,7 +54,8 @@ struct QuantParams {
     const int32_t *token_idx;
     int64_t sl, sg, sh, st;  // element strides: layer, group(frame), head, token
     uint8_t *codes_k, *codes_v;
-    float *scale_k, *zero_k, *scale_v, *zero_v, *rep_key, *rep_norm2;
+    void *scale_k, *zero_k, *scale_v, *zero_v, *rep_key;  // elements of g.meta_dtype
+    float *rep_norm2;
     BankGeom g;
     int32_t layer_begin, group_begin, F, n_in;
     uint32_t *flags;
@@ -238,6 +239,45 @@ __device__ __forceinline__ void store_floats(float *dst, const float (&v)[C]) {
     }
 }
 
+// ---- 16-bit metadata.  The stored offset must not exceed the channel minimum and the stored scale must reach the
+// channel maximum from it, so the offset rounds towards -inf and the scale towards +inf; the codes are then taken
+// against the stored pair.  bfloat16 is the upper half of a binary32: truncation rounds towards zero, one step more
+// on the side that needs it.  binary16 has conversion instructions with both directed modes.
+__device__ __forceinline__ float meta_round_down(float x, int meta_dtype) {
+    if (meta_dtype == STOM_BF16) {
+        const uint32_t u = __float_as_uint(x);
+        return __uint_as_float((u & 0xffff0000u) + (((u & 0xffffu) != 0u && (u >> 31)) ? 0x10000u : 0u));
+    }
+    return __half2float(__float2half_rd(x));
+}
+__device__ __forceinline__ float meta_round_up(float x, int meta_dtype) {
+    if (meta_dtype == STOM_BF16) {
+        const uint32_t u = __float_as_uint(x);
+        return __uint_as_float((u & 0xffff0000u) + (((u & 0xffffu) != 0u && !(u >> 31)) ? 0x10000u : 0u));
+    }
+    return __half2float(__float2half_ru(x));
+}
+__device__ __forceinline__ float meta_round_nearest(float x, int meta_dtype) {
+    return meta_dtype == STOM_BF16 ? __bfloat162float(__float2bfloat16_rn(x)) : __half2float(__float2half_rn(x));
+}
+
+// C adjacent metadata values to element `at` of a bank array of type meta_dtype; for the 16-bit types the values are
+// already representable, so the conversion is exact.
+template <int C>
+__device__ __forceinline__ void store_meta(void *base, int64_t at, int meta_dtype, const float (&v)[C]) {
+    if (meta_dtype == STOM_FP32) {
+        store_floats<C>(static_cast<float *>(base) + at, v);
+        return;
+    }
+    uint32_t w[C / 2];
+#pragma unroll
+    for (int i = 0; i < C / 2; ++i)
+        w[i] = meta_dtype == STOM_BF16 ? pack2<__nv_bfloat16>(v[2 * i], v[2 * i + 1]) : pack2<__half>(v[2 * i], v[2 * i + 1]);
+    uint16_t *dst = static_cast<uint16_t *>(base) + at;
+    if constexpr (C == 2) *reinterpret_cast<uint32_t *>(dst) = w[0];
+    else if constexpr (C == 4) *reinterpret_cast<uint2 *>(dst) = make_uint2(w[0], w[1]);
+    else *reinterpret_cast<uint4 *>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+}
 
 // The C * BITS code bits of one row that a lane produced go to dst = row start + byte offset of the lane.  With
 // 2 channels of 2 bits a lane has only half a byte: the even lane takes its neighbour's half and stores for both.
@@ -336,7 +376,8 @@ constexpr int kBarBytes = 2048;
 static_assert(kAbortOff + 8 <= kInfoOff && kInfoOff + kMaxSlots * (int)sizeof(SlotInfo) <= kBarBytes, "header layout");
 
 // C: channels per lane (d / 32).  blockDim.x = kQuantThreads, one block per SM, grid-stride over tiles.
-template <typename T, int C, int BITS>
+// MD: type the bank keeps s, m and k-bar in (STOM_FP32 | STOM_FP16 | STOM_BF16)
+template <typename T, int C, int BITS, int MD>
 __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantParams p) {
     constexpr float kLevels = (float)((1 << BITS) - 1);  // 15 levels above the offset at 4 bits, 3 at 2 bits
     constexpr int D = 32 * C;
@@ -468,6 +509,7 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
         const int64_t bslot = info[slot].bslot;
         const int kind = info[slot].kind;
         const bool is_v = kind == 1;
+        constexpr int md = MD;
         const bool want_sum = kind == 2 || (kind == 0 && p.n_kinds == 2);  // warp-uniform
 
         uint64_t sum2[C / 2];
@@ -505,8 +547,16 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
                     float mx0, mx1;
                     a.pair(j, m[2 * j], m[2 * j + 1]);
                     b.pair(j, mx0, mx1);
+                    if (md != STOM_FP32) {  // warp-uniform
+                        m[2 * j] = meta_round_down(m[2 * j], md);
+                        m[2 * j + 1] = meta_round_down(m[2 * j + 1], md);
+                    }
                     s[2 * j] = __fdiv_rn(__fsub_rn(mx0, m[2 * j]), kLevels);
                     s[2 * j + 1] = __fdiv_rn(__fsub_rn(mx1, m[2 * j + 1]), kLevels);
+                    if (md != STOM_FP32) {
+                        s[2 * j] = meta_round_up(s[2 * j], md);
+                        s[2 * j + 1] = meta_round_up(s[2 * j + 1], md);
+                    }
                 }
 #pragma unroll
                 for (int c = 0; c < C; ++c) {
@@ -514,8 +564,8 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
                     y[c] = __frcp_rn(s[c]);
                 }
             }
-            store_floats<C>((is_v ? p.scale_v : p.scale_k) + bslot * D + lane * C, s);
-            store_floats<C>((is_v ? p.zero_v : p.zero_k) + bslot * D + lane * C, m);
+            store_meta<C>(is_v ? p.scale_v : p.scale_k, bslot * D + lane * C, md, s);
+            store_meta<C>(is_v ? p.zero_v : p.zero_k, bslot * D + lane * C, md, m);
             safe = __all_sync(0xffffffffu, safe);
 
             unsigned char *out_lane = (is_v ? p.codes_v : p.codes_k) + bslot * (int64_t)code_bytes + lane * C * BITS / 8;
@@ -578,10 +628,14 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
                 unpack_f2(sum2[j], a, b);
                 kb[2 * j] = __fdiv_rn(a, Gf);
                 kb[2 * j + 1] = __fdiv_rn(b, Gf);
+                if (md != STOM_FP32) {  // the norm below is the norm of the stored key
+                    kb[2 * j] = meta_round_nearest(kb[2 * j], md);
+                    kb[2 * j + 1] = meta_round_nearest(kb[2 * j + 1], md);
+                }
             }
 #pragma unroll
             for (int c = 0; c < C; ++c) n2 = fmaf(kb[c], kb[c], n2);
-            store_floats<C>(p.rep_key + bslot * D + lane * C, kb);
+            store_meta<C>(p.rep_key, bslot * D + lane * C, md, kb);
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, o);
             if (lane == 0) p.rep_norm2[bslot] = n2;
@@ -594,7 +648,7 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
     }
 }
 
-template <typename T, int C, int BITS>
+template <typename T, int C, int BITS, int MD>
 static int32_t launch_quantize(QuantParams p, cudaStream_t stream) {
     int dev = 0, sms = 0, smem_max = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -615,22 +669,31 @@ static int32_t launch_quantize(QuantParams p, cudaStream_t stream) {
     p.n_warps = slots < kConsumerWarps ? slots : kConsumerWarps;
     const int fixed = kBarBytes;
     const size_t smem = (size_t)fixed + (size_t)slots * p.slot_bytes;
-    e = cudaFuncSetAttribute(quantize_kernel<T, C, BITS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(quantize_kernel<T, C, BITS, MD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) {
         set_last_cuda_error(e);
         return STOM_ERR_CUDA;
     }
     const unsigned grid = p.n_tiles < (uint32_t)sms ? p.n_tiles : (unsigned)sms;
-    quantize_kernel<T, C, BITS><<<grid, kQuantThreads, smem, stream>>>(p);
+    quantize_kernel<T, C, BITS, MD><<<grid, kQuantThreads, smem, stream>>>(p);
     return finish_launch();
+}
+
+template <typename T, int C, int BITS>
+static int32_t launch_for_meta(const QuantParams &p, cudaStream_t stream) {
+    switch (p.g.meta_dtype) {
+    case STOM_BF16: return launch_quantize<T, C, BITS, STOM_BF16>(p, stream);
+    case STOM_FP16: return launch_quantize<T, C, BITS, STOM_FP16>(p, stream);
+    default: return launch_quantize<T, C, BITS, STOM_FP32>(p, stream);
+    }
 }
 
 template <typename T>
 static int32_t launch_for_type(const QuantParams &p, int bits, cudaStream_t stream) {
     switch (p.g.d) {
-    case 64: return bits == 4 ? launch_quantize<T, 2, 4>(p, stream) : launch_quantize<T, 2, 2>(p, stream);
-    case 128: return bits == 4 ? launch_quantize<T, 4, 4>(p, stream) : launch_quantize<T, 4, 2>(p, stream);
-    case 256: return bits == 4 ? launch_quantize<T, 8, 4>(p, stream) : launch_quantize<T, 8, 2>(p, stream);
+    case 64: return bits == 4 ? launch_for_meta<T, 2, 4>(p, stream) : launch_for_meta<T, 2, 2>(p, stream);
+    case 128: return bits == 4 ? launch_for_meta<T, 4, 4>(p, stream) : launch_for_meta<T, 4, 2>(p, stream);
+    case 256: return bits == 4 ? launch_for_meta<T, 8, 4>(p, stream) : launch_for_meta<T, 8, 2>(p, stream);
     default: return STOM_ERR_SHAPE;
     }
 }

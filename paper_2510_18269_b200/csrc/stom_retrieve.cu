@@ -159,7 +159,7 @@ __device__ __forceinline__ void embed_layer(const ScoreParams &p, int li, float 
 
 // grid (chunks, layer_count), kFusedThreads threads.  Dynamic shared memory: q (H*d floats), norms (H rounded up
 // to 4 floats), then a region used first as the embedding scratch and, in a selecting block, as the key array.
-template <typename T, int V4>
+template <typename T, int V4, typename KT>
 __global__ void __launch_bounds__(kFusedThreads) retrieve_kernel(const RetrieveParams rp) {
     extern __shared__ __align__(16) float dyn[];
     __shared__ TopkSmem tsm;
@@ -173,7 +173,7 @@ __global__ void __launch_bounds__(kFusedThreads) retrieve_kernel(const RetrieveP
 
     const int t_begin = blockIdx.x * p.groups_per_block;
     const int t_end = min(t_begin + p.groups_per_block, p.n_groups);
-    score_block<V4>(p, sq, qn, li, t_begin, t_end);
+    score_block<V4, KT>(p, sq, qn, li, t_begin, t_end);
 
     uint32_t *skeys = reinterpret_cast<uint32_t *>(region);
     const int n = p.n_groups, chunks = gridDim.x;
@@ -228,13 +228,27 @@ __global__ void __launch_bounds__(kFusedThreads) retrieve_kernel(const RetrieveP
     }
 }
 
+template <typename T, typename KT>
+static void launch_retrieve_kt(const RetrieveParams &rp, dim3 grid, size_t smem, int v4, cudaStream_t s) {
+    switch (v4) {
+    case 4: retrieve_kernel<T, 4, KT><<<grid, kFusedThreads, smem, s>>>(rp); break;  // 4 kv heads x 128
+    case 8: retrieve_kernel<T, 8, KT><<<grid, kFusedThreads, smem, s>>>(rp); break;  // 8 kv heads x 128
+    case 2: retrieve_kernel<T, 2, KT><<<grid, kFusedThreads, smem, s>>>(rp); break;
+    case 1:
+        if constexpr (sizeof(KT) == 4) {
+            retrieve_kernel<T, 1, KT><<<grid, kFusedThreads, smem, s>>>(rp);
+            break;
+        }
+    default: retrieve_kernel<T, 0, KT><<<grid, kFusedThreads, smem, s>>>(rp); break;
+    }
+}
+
 template <typename T>
 static void launch_retrieve(const RetrieveParams &rp, dim3 grid, size_t smem, int HD, bool fast, cudaStream_t s) {
-    if (fast && HD == 512) retrieve_kernel<T, 4><<<grid, kFusedThreads, smem, s>>>(rp);        // 4 kv heads x 128
-    else if (fast && HD == 1024) retrieve_kernel<T, 8><<<grid, kFusedThreads, smem, s>>>(rp);  // 8 kv heads x 128
-    else if (fast && HD == 256) retrieve_kernel<T, 2><<<grid, kFusedThreads, smem, s>>>(rp);
-    else if (fast && HD == 128) retrieve_kernel<T, 1><<<grid, kFusedThreads, smem, s>>>(rp);
-    else retrieve_kernel<T, 0><<<grid, kFusedThreads, smem, s>>>(rp);
+    const int md = rp.sp.g.meta_dtype, v4 = score_fast_v4(HD, fast, md);
+    if (md == STOM_BF16) launch_retrieve_kt<T, __nv_bfloat16>(rp, grid, smem, v4, s);
+    else if (md == STOM_FP16) launch_retrieve_kt<T, __half>(rp, grid, smem, v4, s);
+    else launch_retrieve_kt<T, float>(rp, grid, smem, v4, s);
 }
 
 }  // namespace stom

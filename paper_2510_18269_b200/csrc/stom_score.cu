@@ -79,11 +79,24 @@ extern "C" int32_t stom_oqm_score_groups(const stom_oqm_config *cfg, const stom_
     const size_t smem = (size_t)cfg->n_kv_heads * (cfg->head_dim + 1) * sizeof(float);
     const int HD = cfg->n_kv_heads * cfg->head_dim;
     const bool fast = !p.per_head && cfg->n_kv_heads <= 32;
-    if (fast && HD == 512) score_kernel<4><<<g2, kScoreWarps * 32, smem, s>>>(p);        // 4 kv heads x 128
-    else if (fast && HD == 1024) score_kernel<8><<<g2, kScoreWarps * 32, smem, s>>>(p);  // 8 kv heads x 128
-    else if (fast && HD == 256) score_kernel<2><<<g2, kScoreWarps * 32, smem, s>>>(p);
-    else if (fast && HD == 128) score_kernel<1><<<g2, kScoreWarps * 32, smem, s>>>(p);
-    else score_kernel<0><<<g2, kScoreWarps * 32, smem, s>>>(p);
+#define STOM_SCORE_LAUNCH(KT_)                                                                       \
+    switch (score_fast_v4(HD, fast, cfg->meta_dtype)) {                                             \
+    case 4: score_kernel<4, KT_><<<g2, kScoreWarps * 32, smem, s>>>(p); break; /* 4 kv heads x 128 */ \
+    case 8: score_kernel<8, KT_><<<g2, kScoreWarps * 32, smem, s>>>(p); break; /* 8 kv heads x 128 */ \
+    case 2: score_kernel<2, KT_><<<g2, kScoreWarps * 32, smem, s>>>(p); break;                      \
+    case 1:                                                                                         \
+        if constexpr (sizeof(KT_) == 4) {                                                           \
+            score_kernel<1, KT_><<<g2, kScoreWarps * 32, smem, s>>>(p);                             \
+            break;                                                                                  \
+        }                                                                                           \
+    default: score_kernel<0, KT_><<<g2, kScoreWarps * 32, smem, s>>>(p); break;                     \
+    }
+    switch (cfg->meta_dtype) {
+    case STOM_BF16: STOM_SCORE_LAUNCH(__nv_bfloat16) break;
+    case STOM_FP16: STOM_SCORE_LAUNCH(__half) break;
+    default: STOM_SCORE_LAUNCH(float) break;
+    }
+#undef STOM_SCORE_LAUNCH
     return finish_launch();
 }
 

@@ -10,7 +10,8 @@ namespace stom {
 struct ScoreParams {
     const void *Q;
     int64_t ql, qh, qt;  // element strides of Q: layer, head, token
-    const float *rep_key, *rep_norm2;
+    const void *rep_key;  // elements of g.meta_dtype
+    const float *rep_norm2;
     float *qemb;    // workspace: [layer_count][H][d]
     float *qnorm2;  // workspace: [layer_count][H]
     float *scores;
@@ -106,36 +107,47 @@ __global__ void __launch_bounds__(kEmbedThreads) query_embed_kernel(const ScoreP
 constexpr int kScoreWarps = 8;
 
 // One warp, a strided share of the block's groups [t_begin, t_end) of one layer, kGroupsPerWarp at a time.  The
-// loads of the next pair are issued before the current pair is reduced, so a warp always has 2 pairs of k-bar
-// vectors in flight.  V4: float4 words of the flattened k-bar that one lane covers (H*d / 128).
-template <int V4>
+// loads of the next batch are issued before the current batch is reduced, so a warp always has 2 batches of k-bar
+// vectors in flight.  V4: the flattened k-bar has H*d = 128 * V4 channels; KT: the type it is stored in.  A lane
+// covers NV 16-byte vectors of each k-bar: vector i of a lane holds channels [(lane + 32 i) * E, ... + E).
+template <int V4, typename KT>
 __device__ __forceinline__ void score_groups_per_layer(const ScoreParams &p, const float *sq, const float *qn, int li,
                                                        int t_begin, int t_end, int warp, int lane) {
-    constexpr int kGroupsPerWarp = V4 >= 8 ? 1 : 2;  // groups a warp scores together (register budget)
+    constexpr int E = 16 / (int)sizeof(KT);  // channels per 16-byte vector
+    constexpr int NV = V4 * 4 / E;           // vectors of one k-bar per lane
+    static_assert(NV >= 1 && NV * E == V4 * 4, "k-bar must fill whole 16-byte vectors across the warp");
+    // groups a warp scores together (register budget: about 8 vectors per batch)
+    constexpr int kGroupsPerWarp = sizeof(KT) == 4 ? (V4 >= 8 ? 1 : 2) : (NV >= 4 ? 2 : 4);
     const int H = p.g.H, d = p.g.d, l = p.layer_begin + li;
-    float4 q4[V4];
+    float q[NV][E];
 #pragma unroll
-    for (int i = 0; i < V4; ++i) q4[i] = reinterpret_cast<const float4 *>(sq)[lane + 32 * i];
+    for (int i = 0; i < NV; ++i) {
+#pragma unroll
+        for (int e = 0; e < E; e += 4) {
+            const float4 v = reinterpret_cast<const float4 *>(sq)[((lane + 32 * i) * E + e) >> 2];
+            q[i][e] = v.x; q[i][e + 1] = v.y; q[i][e + 2] = v.z; q[i][e + 3] = v.w;
+        }
+    }
     float qq = lane < H ? qn[lane] : 0.0f;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) qq += __shfl_xor_sync(0xffffffffu, qq, o);
     const float qnorm = fmaxf(sqrtf(qq), 1e-12f);
 
-    auto load = [&](int t0, float4 (&kv)[kGroupsPerWarp][V4], float (&kn)[kGroupsPerWarp]) {
+    auto load = [&](int t0, uint4 (&kv)[kGroupsPerWarp][NV], float (&kn)[kGroupsPerWarp]) {
 #pragma unroll
         for (int u = 0; u < kGroupsPerWarp; ++u) {
-            const int t = min(t0 + u, t_end - 1);  // a pair that sticks out re-reads the last group; dropped at the store
+            const int t = min(t0 + u, t_end - 1);  // a batch that sticks out re-reads the last group; dropped at the store
             const int64_t slot = bank_slot(p.g, l, t, 0);
-            const float4 *kb = reinterpret_cast<const float4 *>(p.rep_key + slot * d);
+            const uint4 *kb = reinterpret_cast<const uint4 *>(static_cast<const KT *>(p.rep_key) + slot * d);
 #pragma unroll
-            for (int i = 0; i < V4; ++i) kv[u][i] = __ldg(kb + lane + 32 * i);
+            for (int i = 0; i < NV; ++i) kv[u][i] = __ldg(kb + lane + 32 * i);
             kn[u] = lane < H ? __ldg(p.rep_norm2 + slot + lane) : 0.0f;
         }
     };
     const int step = kScoreWarps * kGroupsPerWarp;
     int t0 = t_begin + warp * kGroupsPerWarp;
     if (t0 >= t_end) return;
-    float4 cur[kGroupsPerWarp][V4], nxt[kGroupsPerWarp][V4];
+    uint4 cur[kGroupsPerWarp][NV], nxt[kGroupsPerWarp][NV];
     float kn_cur[kGroupsPerWarp], kn_nxt[kGroupsPerWarp];
     load(t0, cur, kn_cur);
     for (; t0 < t_end; t0 += step) {
@@ -146,11 +158,20 @@ __device__ __forceinline__ void score_groups_per_layer(const ScoreParams &p, con
         for (int u = 0; u < kGroupsPerWarp; ++u) {
             float a = 0.0f;
 #pragma unroll
-            for (int i = 0; i < V4; ++i) {
-                a = fmaf(cur[u][i].x, q4[i].x, a);
-                a = fmaf(cur[u][i].y, q4[i].y, a);
-                a = fmaf(cur[u][i].z, q4[i].z, a);
-                a = fmaf(cur[u][i].w, q4[i].w, a);
+            for (int i = 0; i < NV; ++i) {
+                const uint32_t w[4] = {cur[u][i].x, cur[u][i].y, cur[u][i].z, cur[u][i].w};
+                if constexpr (sizeof(KT) == 4) {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) a = fmaf(__uint_as_float(w[e]), q[i][e], a);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        float lo, hi;
+                        unpack2<KT>(w[e], lo, hi);
+                        a = fmaf(lo, q[i][2 * e], a);
+                        a = fmaf(hi, q[i][2 * e + 1], a);
+                    }
+                }
             }
             dot[u] = a;
         }
@@ -178,22 +199,33 @@ __device__ __forceinline__ void score_groups_per_layer(const ScoreParams &p, con
             for (int u = 0; u < kGroupsPerWarp; ++u) {
                 kn_cur[u] = kn_nxt[u];
 #pragma unroll
-                for (int i = 0; i < V4; ++i) cur[u][i] = nxt[u][i];
+                for (int i = 0; i < NV; ++i) cur[u][i] = nxt[u][i];
             }
         }
     }
 }
 
+// Dot product of 8 adjacent channels of a stored k-bar (element `at` of the bank array) with 8 floats of q.
+template <typename KT>
+__device__ __forceinline__ float dot8(const void *rep_key, int64_t at, const float *q, float acc) {
+    float k[8];
+    load_meta8<KT>(rep_key, at, k);
+    const float4 a = reinterpret_cast<const float4 *>(q)[0], b = reinterpret_cast<const float4 *>(q)[1];
+    acc = fmaf(k[0], a.x, acc); acc = fmaf(k[1], a.y, acc); acc = fmaf(k[2], a.z, acc); acc = fmaf(k[3], a.w, acc);
+    acc = fmaf(k[4], b.x, acc); acc = fmaf(k[5], b.y, acc); acc = fmaf(k[6], b.z, acc); acc = fmaf(k[7], b.w, acc);
+    return acc;
+}
+
 // Scores of groups [t_begin, t_end) of layer li, by one block of kScoreWarps warps.  sq: the layer's question
 // embedding (H*d floats) in shared memory, qn: its H squared norms.
 // V4 > 0: PER_LAYER scoring with H*d == 128 * V4 and H <= 32 (the software-pipelined loop); V4 == 0: everything else.
-template <int V4>
+template <int V4, typename KT>
 __device__ __forceinline__ void score_block(const ScoreParams &p, const float *sq, const float *qn, int li, int t_begin,
                                             int t_end) {
     const int H = p.g.H, d = p.g.d, HD = H * d;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if constexpr (V4 > 0) {
-        score_groups_per_layer<V4>(p, sq, qn, li, t_begin, t_end, warp, lane);
+        score_groups_per_layer<V4, KT>(p, sq, qn, li, t_begin, t_end, warp, lane);
         return;
     }
     const int l = p.layer_begin + li;
@@ -201,17 +233,9 @@ __device__ __forceinline__ void score_block(const ScoreParams &p, const float *s
 #pragma unroll 1
     for (int t = t_begin + (V4 > 0 ? t_end : warp); t < t_end; t += kScoreWarps) {
         const int64_t slot = bank_slot(p.g, l, t, 0);
-        const float4 *kb = reinterpret_cast<const float4 *>(p.rep_key + slot * d);
         if (!p.per_head) {
             float dot = 0.0f;
-            for (int i = lane; i < HD / 4; i += 32) {
-                const float4 a = __ldg(kb + i);
-                const float4 b = reinterpret_cast<const float4 *>(sq)[i];
-                dot = fmaf(a.x, b.x, dot);
-                dot = fmaf(a.y, b.y, dot);
-                dot = fmaf(a.z, b.z, dot);
-                dot = fmaf(a.w, b.w, dot);
-            }
+            for (int i = lane; i < HD / 8; i += 32) dot = dot8<KT>(p.rep_key, slot * d + i * 8, sq + i * 8, dot);
             float kn = 0.0f, qq = 0.0f;
             for (int hh = lane; hh < H; hh += 32) {
                 kn += __ldg(p.rep_norm2 + slot + hh);
@@ -228,14 +252,8 @@ __device__ __forceinline__ void score_block(const ScoreParams &p, const float *s
         } else {
             for (int hh = 0; hh < H; ++hh) {
                 float dot = 0.0f;
-                for (int i = lane; i < d / 4; i += 32) {
-                    const float4 a = __ldg(kb + hh * (d / 4) + i);
-                    const float4 b = reinterpret_cast<const float4 *>(sq)[hh * (d / 4) + i];
-                    dot = fmaf(a.x, b.x, dot);
-                    dot = fmaf(a.y, b.y, dot);
-                    dot = fmaf(a.z, b.z, dot);
-                    dot = fmaf(a.w, b.w, dot);
-                }
+                for (int i = lane; i < d / 8; i += 32)
+                    dot = dot8<KT>(p.rep_key, slot * d + hh * d + i * 8, sq + hh * d + i * 8, dot);
 #pragma unroll
                 for (int o = 16; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
                 if (lane == 0) {
@@ -250,7 +268,7 @@ __device__ __forceinline__ void score_block(const ScoreParams &p, const float *s
 
 
 // grid (chunks, layer_count): block x scores groups [x * groups_per_block, (x+1) * groups_per_block) of its layer
-template <int V4>
+template <int V4, typename KT>
 __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(const ScoreParams p) {
     extern __shared__ __align__(16) float sq[];  // q of this layer: H*d floats, then H norms
     const int li = blockIdx.y, H = p.g.H, HD = H * p.g.d;
@@ -260,7 +278,16 @@ __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(const ScorePara
     __syncthreads();
     const int t_begin = blockIdx.x * p.groups_per_block;
     const int t_end = min(t_begin + p.groups_per_block, p.n_groups);
-    score_block<V4>(p, sq, qn, li, t_begin, t_end);
+    score_block<V4, KT>(p, sq, qn, li, t_begin, t_end);
+}
+
+// The fast scoring loop exists for H*d = 128 * V4 with V4 in {1, 2, 4, 8}; a 16-bit k-bar needs H*d to be a multiple
+// of 256.  Returns the V4 to instantiate, 0 for the general loop.
+inline int score_fast_v4(int HD, bool fast, int meta_dtype) {
+    if (!fast) return 0;
+    if (HD != 128 && HD != 256 && HD != 512 && HD != 1024) return 0;
+    if (meta_dtype != STOM_FP32 && HD == 128) return 0;
+    return HD / 128;
 }
 
 }  // namespace stom

@@ -35,7 +35,7 @@ EXPORTS = (
 class Config(C.Structure):
     _fields_ = [(n, C.c_int32) for n in (
         "n_layers", "n_q_heads", "n_kv_heads", "head_dim", "group_tokens",
-        "capacity_groups", "bits", "kv_dtype", "score_mode")]
+        "capacity_groups", "bits", "kv_dtype", "score_mode", "meta_dtype")]
 
 
 class StoreDesc(C.Structure):
@@ -100,9 +100,9 @@ def _check(rc: int, where: str):
 
 
 def make_config(n_layers, n_q_heads, n_kv_heads, head_dim, group_tokens, capacity_groups,
-                bits=4, kv_dtype=BF16, score_mode=PER_LAYER) -> Config:
+                bits=4, kv_dtype=BF16, score_mode=PER_LAYER, meta_dtype=FP32) -> Config:
     return Config(n_layers, n_q_heads, n_kv_heads, head_dim, group_tokens, capacity_groups,
-                  bits, kv_dtype, score_mode)
+                  bits, kv_dtype, score_mode, meta_dtype)
 
 
 def dtype_code(t: torch.dtype) -> int:
@@ -144,11 +144,12 @@ class Store:
 
         self.codes_k = view(lay.off_codes_k, lay.bytes_codes, torch.uint8, (L, T, H, G, d * cfg.bits // 8))
         self.codes_v = view(lay.off_codes_v, lay.bytes_codes, torch.uint8, (L, T, H, G, d * cfg.bits // 8))
-        self.scale_k = view(lay.off_scale_k, lay.bytes_meta, torch.float32, (L, T, H, d))
-        self.zero_k = view(lay.off_zero_k, lay.bytes_meta, torch.float32, (L, T, H, d))
-        self.scale_v = view(lay.off_scale_v, lay.bytes_meta, torch.float32, (L, T, H, d))
-        self.zero_v = view(lay.off_zero_v, lay.bytes_meta, torch.float32, (L, T, H, d))
-        self.rep_key = view(lay.off_rep_key, lay.bytes_meta, torch.float32, (L, T, H, d))
+        mt = _TORCH_DTYPE[cfg.meta_dtype]  # element type of s, m and k-bar
+        self.scale_k = view(lay.off_scale_k, lay.bytes_meta, mt, (L, T, H, d))
+        self.zero_k = view(lay.off_zero_k, lay.bytes_meta, mt, (L, T, H, d))
+        self.scale_v = view(lay.off_scale_v, lay.bytes_meta, mt, (L, T, H, d))
+        self.zero_v = view(lay.off_zero_v, lay.bytes_meta, mt, (L, T, H, d))
+        self.rep_key = view(lay.off_rep_key, lay.bytes_meta, mt, (L, T, H, d))
         self.rep_norm2 = view(lay.off_rep_norm2, lay.bytes_norm2, torch.float32, (L, T, H))
 
 

@@ -47,6 +47,11 @@ def test_store_layout_and_bind(oqm):
     assert oqm.lib().stom_oqm_store_bind(C.byref(cfg), C.c_void_p(base), C.byref(desc)) == 0
     assert desc.codes_k == base and desc.rep_norm2 == base + lay.off_rep_norm2
     assert oqm.lib().stom_oqm_store_bind(C.byref(cfg), C.c_void_p(base + 8), C.byref(desc)) == -3   # alignment
+    # 16-bit metadata halves the five metadata arrays and nothing else
+    for meta in (oqm.FP16, oqm.BF16):
+        lay16 = oqm.stom_oqm_store_layout(oqm.make_config(28, 28, 4, 128, 50, 7200, meta_dtype=meta))
+        assert lay16.bytes_meta * 2 == lay.bytes_meta and lay16.bytes_codes == lay.bytes_codes
+        assert lay16.bytes_norm2 == lay.bytes_norm2 and lay16.bytes_total < lay.bytes_total
 
 
 def test_budget_to_k_matches_paper_example(oqm):
@@ -58,6 +63,7 @@ def test_budget_to_k_matches_paper_example(oqm):
 @pytest.mark.parametrize("kw,code", [
     (dict(head_dim=96), -2), (dict(group_tokens=0), -2), (dict(group_tokens=65), -2), (dict(bits=3), -6),
     (dict(n_q_heads=7), -2), (dict(kv_dtype=5), -6), (dict(n_layers=0), -1), (dict(score_mode=3), -6),
+    (dict(meta_dtype=3), -6), (dict(meta_dtype=-1), -6),
 ])
 def test_config_validation(oqm, kw, code):
     args = dict(n_layers=2, n_q_heads=8, n_kv_heads=4, head_dim=128, group_tokens=50, capacity_groups=10)

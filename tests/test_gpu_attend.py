@@ -48,11 +48,21 @@ def test_attend_two_bit_codes(orc, L, H_q, H_k, d, G, T, k, n_sel, sys_len, mode
     _check_attend(orc, L, H_q, H_k, d, G, T, k, n_sel, sys_len, mode, dtype, cache, bits=2)
 
 
-def _check_attend(orc, L, H_q, H_k, d, G, T, k, n_sel, sys_len, mode, dtype, cache, bits):
+@pytest.mark.parametrize("L,H_q,H_k,d,G,T,k,n_sel,sys_len,mode,dtype,cache,meta,bits", [
+    (2, 28, 4, 128, 50, 100, 16, 16, 9, 0, "bf16", "bf16", "bf16", 4),
+    (2, 28, 4, 128, 50, 100, 16, 16, 9, 0, "bf16", "bf16", "fp16", 4),
+    (1, 4, 2, 64, 16, 40, 5, 4, 70, 1, "fp16", "fp16", "fp16", 2),
+    (1, 8, 1, 256, 8, 20, 6, 6, 0, 0, "fp32", "bf16", "bf16", 4),
+])
+def test_attend_sixteen_bit_metadata(orc, L, H_q, H_k, d, G, T, k, n_sel, sys_len, mode, dtype, cache, meta, bits):
+    _check_attend(orc, L, H_q, H_k, d, G, T, k, n_sel, sys_len, mode, dtype, cache, bits=bits, meta=meta)
+
+
+def _check_attend(orc, L, H_q, H_k, d, G, T, k, n_sel, sys_len, mode, dtype, cache, bits, meta="fp32"):
     from paper_2510_18269_b200 import oqm
     oqm.lib()
     sh = synth.Shape("attend", L=L, H_q=H_q, H_k=H_k, d=d, G=G, T=T, T_q=1, k=k, dtype=dtype, seed=3,
-                     extra={"bits": bits})
+                     extra={"bits": bits, "meta": meta})
     ocfg, gcfg, ost, gst, _ = P.random_bank(orc, oqm, sh, mode, seed=17 * k + sys_len)
     rng = np.random.default_rng(5 + k)
     rows = L * (H_k if mode else 1)
