@@ -133,6 +133,31 @@ def compare_topk(g_idx: torch.Tensor, o_idx: np.ndarray, o_scores_rows: np.ndarr
     return exact_rows
 
 
+def compare_active(g16: np.ndarray, o16: np.ndarray, g_idx: np.ndarray, o_idx: np.ndarray, sys_len: int, G: int,
+                   per_head: bool = False, min_same: float = 0.9):
+    """Active caches [L][H][S][d] as 16-bit patterns: the library's (built from ITS selection g_idx) against the
+    oracle's (built from the oracle's selection o_idx; nothing the library produced is fed to the oracle).  Slot j of
+    a ranking row lands in tokens [sys_len + j*G, sys_len + (j+1)*G) and depends on idx[row][j] alone, so the slots
+    where both sides selected the same group are compared bit for bit; they differ only behind a tie at the K-th
+    score.  The system tokens in front and whatever lies behind the last slot must be identical.  Returns the rows
+    whose selections agree completely."""
+    L, H, S, d = o16.shape
+    rows, k = o_idx.shape
+    g_idx = g_idx.reshape(rows, k)
+    same = g_idx == o_idx
+    assert same.mean() >= min_same, f"only {same.mean():.3f} of the slots hold the same group on both sides"
+    gr = g16.reshape(rows, -1, S, d) if per_head else g16.reshape(rows, H, S, d)
+    orr = o16.reshape(gr.shape)
+    assert np.array_equal(gr[:, :, :sys_len], orr[:, :, :sys_len]), "system tokens differ"
+    assert np.array_equal(gr[:, :, sys_len + k * G:], orr[:, :, sys_len + k * G:]), "tokens behind the last slot differ"
+    for r in range(rows):
+        for j in range(k):
+            if same[r, j]:
+                a, b = sys_len + j * G, sys_len + (j + 1) * G
+                assert np.array_equal(gr[r, :, a:b], orr[r, :, a:b]), f"row {r} slot {j}: reconstructed group differs"
+    return same.all(axis=1)
+
+
 def out_buffers(sh, layer_count, S_tokens, torch_dtype, device, sentinel):
     """Active cache [layer_count][H_k][S_tokens][d] with a guard band after it, filled with a sentinel."""
     n = layer_count * sh.H_k * S_tokens * sh.d

@@ -76,11 +76,11 @@ def test_c3_full_stream_one_layer_in_full_and_samples_elsewhere(orc):
     P.compare_scores(scores[lf], o_scores.reshape(-1))
     o_idx, _, _ = orc.topk(o_scores.reshape(1, sh.T), sh.k)
     P.compare_topk(idx[lf:lf + 1], o_idx, o_scores.reshape(1, sh.T), sh.k)
-    g_idx = ix_all[lf:lf + 1].copy()
     oka = np.zeros((1, sh.H_k, S, sh.d), np.uint16)
     ova = np.zeros_like(oka)
-    assert orc.dequant_gather(ocfg, ost, 0, 1, g_idx, sh.k, sh.T, oka, ova, orc.BF16, P.active_strides(sh, S), 0) == 0
-    assert np.array_equal(P.as_np16(ka[lf]), oka[0]) and np.array_equal(P.as_np16(va[lf]), ova[0])
+    assert orc.dequant_gather(ocfg, ost, 0, 1, o_idx, sh.k, sh.T, oka, ova, orc.BF16, P.active_strides(sh, S), 0) == 0
+    P.compare_active(P.as_np16(ka[lf])[None], oka, ix_all[lf:lf + 1], o_idx, 0, sh.G)
+    P.compare_active(P.as_np16(va[lf])[None], ova, ix_all[lf:lf + 1], o_idx, 0, sh.G)
 
     # ---- sampled (layer, frame) units of the other layers, first and last frames included
     rng = np.random.default_rng(0)
