@@ -23,6 +23,11 @@
  *     single-pass retrieval" (the q^(l) equation and the K = min(..) equation)
  *   - active cache ............................ Sec. 3.4, the KV_active
  *     equation; appendix "Cache reconstruction for decoding"
+ *   - CTR: temporal similarity, static/dynamic split, budget split, dynamic
+ *     selection ............................... Sec. 3.3, the s_t^(i) equation,
+ *     the (S_t, D_t) equation, the (k_s, k_d) equation and the TopK half of
+ *     the (G_d, G_s) equation.  The Merge half (density-based clustering of
+ *     the static tokens) is not restated: the paper gives no definition of it
  *   - storage accounting ...................... Sec. 3.1 memory-growth
  *     equation and its footnote; Sec. 3.2 ratio 4N/G; ablation table "Ratio"
  *
@@ -36,6 +41,11 @@
  *   - GQA: query head h_q belongs to kv head h_q / (H_q / H_k);
  *   - zero norms: each norm is clamped below by 1e-12 (score becomes 0);
  *   - ties in top-K: the lower group index wins;
+ *   - CTR: the first frame of a stream has no predecessor, so none of its
+ *     tokens is static (similarity -inf); a zero feature vector has
+ *     similarity 0 (norms clamped below by 1e-12, as for the scores); ties in
+ *     the saliency TopK go to the lower token index and the selection is
+ *     returned in ascending token order;
  *   - 16-bit metadata (meta_dtype = fp16 or bf16; Sec. 4.1 runs the model in
  *     FP16, the (s_t, m_t) equation fixes no storage type): the offset is the
  *     largest 16-bit value <= the channel minimum, the scale the smallest
@@ -621,6 +631,94 @@ int32_t orc_attend(int32_t H_q, int32_t H_k, int32_t d, const void *q_dec, int32
         for (int c = 0; c < d; ++c) store_out(out, (int64_t)hq * d + c, out_dtype, (float)(acc[c] / den));
     }
     free(p); free(acc);
+    return ORC_OK;
+}
+
+/* ------------------------------------------------------------------ */
+/* CTR (Sec. 3.3): temporal similarity, static / dynamic split, budget, */
+/*     saliency selection of the dynamic tokens                         */
+/* ------------------------------------------------------------------ */
+
+/*
+ * s_t^(i) = F_t^(i) . F_{t-1}^(i) / (|F_t^(i)| |F_{t-1}^(i)|)  for the frames t of one call.
+ * F: element (t, i, c) at t*stride_frame + i*stride_token + c, T frames of N tokens of D channels.
+ * prev (nullable): the features of the frame before F[0], [N][D] with the same token stride -- the state the
+ * method carries from call to call; without it frame 0 has no predecessor and gets -inf.
+ * sim: [T][N] binary32 (the binary64 result rounded once).
+ */
+int32_t orc_ctr_similarity(const void *F, const void *prev, int dtype, int32_t T, int32_t N, int32_t D,
+                           int64_t stride_frame, int64_t stride_token, float *sim) {
+    if (!F || !sim || T < 0 || N < 1 || D < 1) return ORC_ERR_ARG;
+    for (int t = 0; t < T; ++t)
+        for (int i = 0; i < N; ++i) {
+            const void *a_base = F, *b_base = F;
+            int64_t a0 = (int64_t)t * stride_frame + (int64_t)i * stride_token, b0;
+            if (t == 0) {
+                if (!prev) { sim[(int64_t)t * N + i] = -INFINITY; continue; }
+                b_base = prev;
+                b0 = (int64_t)i * stride_token;
+            } else {
+                b0 = (int64_t)(t - 1) * stride_frame + (int64_t)i * stride_token;
+            }
+            double dot = 0.0, na = 0.0, nb = 0.0;
+            for (int c = 0; c < D; ++c) {
+                double a = (double)load_elem(a_base, a0 + c, dtype), b = (double)load_elem(b_base, b0 + c, dtype);
+                dot += a * b;
+                na += a * a;
+                nb += b * b;
+            }
+            double da = sqrt(na), db = sqrt(nb);
+            if (da < 1e-12) da = 1e-12;
+            if (db < 1e-12) db = 1e-12;
+            sim[(int64_t)t * N + i] = (float)(dot / (da * db));
+        }
+    return ORC_OK;
+}
+
+/*
+ * Per frame: S_t = {i : s_t^(i) > tau_c}, D_t the rest; k_s = floor(G |S_t| / N), k_d = G - k_s;
+ * G_d = the k_d dynamic tokens of largest saliency alpha.
+ * static_idx [T][N]: S_t ascending, then -1.  dyn_idx [T][G]: G_d ascending, then -1.
+ * k_s, k_d: [T].  (The k_s tokens that Merge would add are not produced here.)
+ */
+int32_t orc_ctr_select(const float *sim, const float *alpha, int32_t T, int32_t N, int32_t G, float tau_c,
+                       int32_t *k_s, int32_t *k_d, int32_t *static_idx, int32_t *dyn_idx) {
+    if (!sim || !alpha || !k_s || !k_d || !static_idx || !dyn_idx || T < 0 || N < 1 || G < 1 || G > N) return ORC_ERR_ARG;
+    int32_t *dyn = (int32_t *)malloc(sizeof(int32_t) * (size_t)N);
+    uint8_t *taken = (uint8_t *)malloc((size_t)N);
+    if (!dyn || !taken) { free(dyn); free(taken); return ORC_ERR_ARG; }
+    for (int t = 0; t < T; ++t) {
+        const float *s = sim + (int64_t)t * N, *a = alpha + (int64_t)t * N;
+        int ns = 0, nd = 0;
+        for (int i = 0; i < N; ++i) {
+            if (s[i] > tau_c) static_idx[(int64_t)t * N + ns++] = i;
+            else dyn[nd++] = i;
+        }
+        for (int i = ns; i < N; ++i) static_idx[(int64_t)t * N + i] = -1;
+        const int ks = (int)(((int64_t)G * ns) / N), kd = G - ks;
+        k_s[t] = ks;
+        k_d[t] = kd;
+        /* kd times: the not yet taken dynamic token of largest alpha, the lowest index among equals */
+        memset(taken, 0, (size_t)N);
+        int got = 0;
+        for (int r = 0; r < kd && r < nd; ++r) {
+            int best = -1;
+            for (int j = 0; j < nd; ++j) {
+                int i = dyn[j];
+                if (taken[i]) continue;
+                if (best < 0 || a[i] > a[best]) best = i; /* dyn is ascending: equal alpha keeps the earlier one */
+            }
+            taken[best] = 1;
+            ++got;
+        }
+        int w = 0;
+        for (int i = 0; i < N; ++i)
+            if (taken[i]) dyn_idx[(int64_t)t * G + w++] = i;
+        for (; w < G; ++w) dyn_idx[(int64_t)t * G + w] = -1;
+        (void)got;
+    }
+    free(dyn);
+    free(taken);
     return ORC_OK;
 }
 

@@ -78,7 +78,8 @@ def lib():
         L.orc_budget_to_k.restype = C.c_int32
         L.orc_budget_to_k.argtypes = [C.c_int64, C.c_int32, C.c_int32]
         L.orc_max_threads.restype = C.c_int32
-        for name in ("orc_quantize_frame", "orc_score_groups", "orc_topk", "orc_dequant_gather", "orc_attend"):
+        for name in ("orc_quantize_frame", "orc_score_groups", "orc_topk", "orc_dequant_gather", "orc_attend",
+                     "orc_ctr_similarity", "orc_ctr_select"):
             getattr(L, name).restype = C.c_int32
         _lib = L
     return _lib
@@ -264,6 +265,37 @@ def attend(H_q, H_k, d, q_dec, q_dtype, k_cache, v_cache, kv_dtype, stride_head,
     if rc:
         raise ValueError(f"orc_attend -> {rc}")
     return out
+
+
+# ---------------------------------------------------------------- CTR (specified steps only)
+
+def ctr_similarity(F: np.ndarray, dtype: int, prev: np.ndarray | None = None) -> np.ndarray:
+    """F [T][N][D] (contiguous; uint16 patterns for the 16-bit types), prev [N][D] or None -> sim [T][N] float32."""
+    F = np.ascontiguousarray(F)
+    T, N, D = F.shape
+    if prev is not None:
+        prev = np.ascontiguousarray(prev)
+        assert prev.shape == (N, D) and prev.dtype == F.dtype
+    sim = np.empty((T, N), np.float32)
+    rc = lib().orc_ctr_similarity(_p(F), _p(prev), C.c_int(dtype), C.c_int32(T), C.c_int32(N), C.c_int32(D),
+                                  C.c_int64(N * D), C.c_int64(D), _p(sim))
+    if rc:
+        raise ValueError(f"orc_ctr_similarity -> {rc}")
+    return sim
+
+
+def ctr_select(sim: np.ndarray, alpha: np.ndarray, G: int, tau_c: float):
+    """sim, alpha [T][N] float32 -> (k_s [T], k_d [T], static_idx [T][N], dyn_idx [T][G]), int32, -1 padded."""
+    sim = np.ascontiguousarray(sim, np.float32)
+    alpha = np.ascontiguousarray(alpha, np.float32)
+    T, N = sim.shape
+    ks, kd = np.empty(T, np.int32), np.empty(T, np.int32)
+    sidx, didx = np.empty((T, N), np.int32), np.empty((T, G), np.int32)
+    rc = lib().orc_ctr_select(_p(sim), _p(alpha), C.c_int32(T), C.c_int32(N), C.c_int32(G), C.c_float(tau_c),
+                              _p(ks), _p(kd), _p(sidx), _p(didx))
+    if rc:
+        raise ValueError(f"orc_ctr_select -> {rc}")
+    return ks, kd, sidx, didx
 
 
 # ---------------------------------------------------------------- accounting

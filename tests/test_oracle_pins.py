@@ -577,6 +577,66 @@ def test_accounting_matches_paper(orc):
     assert per_head_real == 6400 + 2048 + 512 + 4
 
 
+# ------------------------------------------------------------------ CTR: similarity, split, budget, dynamic selection
+
+def test_ctr_similarity_closed_forms_and_library(orc):
+    rng = np.random.default_rng(61)
+    T, N, D = 5, 7, 24
+    F = rng.standard_normal((T, N, D)).astype(np.float32)
+    F[2] = F[1]                      # a frame that repeats its predecessor: similarity exactly 1
+    F[3, :, :] = -2.5 * F[2]         # negated and rescaled: exactly -1, whatever the scale
+    F[4, 0] = 0.0                    # a zero vector: 0 by the norm clamp
+    F[4, 1, :12], F[4, 1, 12:] = F[3, 1, 12:], -F[3, 1, :12]   # (b, -a) against (a, b): orthogonal
+    sim = orc.ctr_similarity(F, orc.FP32)
+    assert np.all(np.isneginf(sim[0]))                        # no predecessor
+    np.testing.assert_allclose(sim[2], 1.0, atol=1e-7)
+    np.testing.assert_allclose(sim[3], -1.0, atol=1e-7)
+    assert sim[4, 0] == 0.0 and abs(sim[4, 1]) < 1e-7
+    # library routine, token by token
+    want = torch.nn.functional.cosine_similarity(torch.from_numpy(F[1:]).double(), torch.from_numpy(F[:-1]).double(), dim=-1)
+    np.testing.assert_allclose(sim[1], want[0].numpy(), atol=1e-6)
+    assert abs(sim[4, 3] - float(want[3, 3])) < 1e-6
+    # positions do not mix: changing token 5 of frame 1 moves s_1^(5) and s_2^(5) only
+    F2 = F.copy()
+    F2[1, 5] = rng.standard_normal(D)
+    sim2 = orc.ctr_similarity(F2, orc.FP32)
+    changed = sim2 != sim
+    assert changed[1, 5] and changed[2, 5] and changed.sum() == 2
+    # the carried state: scoring frames 2.. with frame 1 as `prev` equals the tail of the whole-stream result
+    tail = orc.ctr_similarity(F[2:], orc.FP32, prev=F[1])
+    np.testing.assert_array_equal(tail, sim[2:])
+    # 16-bit inputs are read exactly
+    Fb = torch.from_numpy(F).to(torch.bfloat16)
+    sb = orc.ctr_similarity(Fb.view(torch.int16).numpy().view(np.uint16), orc.BF16)
+    np.testing.assert_array_equal(sb, orc.ctr_similarity(Fb.to(torch.float32).numpy(), orc.FP32))
+
+
+def test_ctr_select_split_budget_and_saliency_topk(orc):
+    rng = np.random.default_rng(67)
+    T, N, G, tau = 40, 196, 50, 0.9
+    sim = rng.uniform(0.5, 1.0, (T, N)).astype(np.float32)
+    sim[0] = -np.inf                     # first frame: everything dynamic
+    sim[1] = 0.99                        # everything static
+    sim[2, :98], sim[2, 98:] = 0.95, 0.2  # half and half: k_s = floor(50 * 98 / 196) = 25
+    sim[3, :10] = np.float32(tau)        # exactly on the threshold: NOT static (strict inequality)
+    sim[3, 10:] = 0.0
+    alpha = rng.uniform(0, 1, (T, N)).astype(np.float32)
+    alpha[4, ::2] = 0.5                  # many equal saliencies: ties go to the lower index
+    ks, kd, sidx, didx = orc.ctr_select(sim, alpha, G, tau)
+    assert ks[0] == 0 and kd[0] == G and ks[1] == G and kd[1] == 0 and ks[2] == 25 and kd[2] == 25 and ks[3] == 0
+    for t in range(T):
+        S = np.flatnonzero(sim[t] > np.float32(tau))
+        Dm = np.setdiff1d(np.arange(N), S)
+        assert np.array_equal(sidx[t, :len(S)], S) and np.all(sidx[t, len(S):] == -1)
+        assert ks[t] == (G * len(S)) // N and ks[t] + kd[t] == G
+        assert ks[t] <= len(S) and kd[t] <= max(len(Dm), 0) or len(Dm) == 0
+        # brute force with a library sort: descending saliency, ascending index among equals
+        order = Dm[np.lexsort((Dm, -alpha[t, Dm].astype(np.float64)))]
+        want = np.sort(order[:kd[t]])
+        assert np.array_equal(didx[t, :len(want)], want) and np.all(didx[t, len(want):] == -1)
+        assert len(want) == kd[t]
+
+
 # ------------------------------------------------------------------ whole path on the tiny workload
 
 def test_tiny_workload_retrieves_planted_groups_and_bounds_active_cache(orc):
