@@ -29,6 +29,7 @@ EXPORTS = (
     "stom_oqm_retrieve_host_scratch_bytes", "stom_oqm_retrieve_host",
     "stom_oqm_score_groups_noalloc", "stom_oqm_attend_workspace_bytes", "stom_oqm_attend",
     "stom_oqm_retrieve_workspace_bytes",
+    "stom_ctr_similarity", "stom_ctr_select", "stom_ctr_reduce",
 )
 
 
@@ -286,3 +287,27 @@ def stom_oqm_retrieve_host(cfg: Config, store: Store, layer_begin, layer_count, 
         C.c_int32(out_dtype), _ptr(scratch), C.c_int64(scratch.numel() * scratch.element_size()), _ptr(dev_flags),
         _stream(stream))
     _check(rc, "stom_oqm_retrieve_host")
+
+
+# ---------------------------------------------------------------- CTR (include/stom_ctr.h)
+
+def stom_ctr_similarity(F, prev, T, N, D, strides, sim, stream=None):
+    """F: device tensor of T x N x D features (strides = (frame, token) in elements); prev: [N][D] or None."""
+    sf, st = strides
+    _check(lib().stom_ctr_similarity(_ptr(F), _ptr(prev), C.c_int32(dtype_code(F.dtype)), C.c_int32(T), C.c_int32(N),
+                                     C.c_int32(D), C.c_int64(sf), C.c_int64(st), _ptr(sim), _stream(stream)),
+           "stom_ctr_similarity")
+
+
+def stom_ctr_select(sim, alpha, T, N, G, tau_c, k_s, k_d, static_idx, dyn_idx, stream=None):
+    _check(lib().stom_ctr_select(_ptr(sim), _ptr(alpha), C.c_int32(T), C.c_int32(N), C.c_int32(G), C.c_float(tau_c),
+                                 _ptr(k_s), _ptr(k_d), _ptr(static_idx), _ptr(dyn_idx), _stream(stream)),
+           "stom_ctr_select")
+
+
+def stom_ctr_reduce(F, prev, T, N, D, strides, alpha, G, tau_c, sim, k_s, k_d, static_idx, dyn_idx, stream=None):
+    sf, st = strides
+    _check(lib().stom_ctr_reduce(_ptr(F), _ptr(prev), C.c_int32(dtype_code(F.dtype)), C.c_int32(T), C.c_int32(N),
+                                 C.c_int32(D), C.c_int64(sf), C.c_int64(st), _ptr(alpha), C.c_int32(G),
+                                 C.c_float(tau_c), _ptr(sim), _ptr(k_s), _ptr(k_d), _ptr(static_idx), _ptr(dyn_idx),
+                                 _stream(stream)), "stom_ctr_reduce")

@@ -149,6 +149,38 @@ def keep_mask(shape: Shape, frame_begin: int, frame_count: int) -> torch.Tensor:
     return torch.stack(rows).to(torch.int32)
 
 
+def ctr_stream(T: int, N: int, D: int, seed: int, device="cpu", dtype: str = "bf16", frame_chunk: int = 256):
+    """Vision-encoder features and saliency for the CTR steps: F [T][N][D] in the storage dtype, alpha [T][N] float32.
+
+    A fixed scene (one base vector per patch position) seen by a camera that does not move: most positions repeat
+    their base vector with a little noise (cosine similarity to the previous frame around 0.99: static); a block of
+    adjacent positions that wanders over the frame is redrawn every frame (similarity around 0: dynamic); one
+    position in eight drifts with noise chosen so that its similarity falls on both sides of 0.9.  The saliency is
+    uniform noise, raised where the content changes.  No arithmetic of the method is done here.
+    """
+    dt = DTYPES[dtype]
+    g0 = _gen(seed * 9973 + 1, device)
+    base = torch.randn(N, D, generator=g0, device=device)
+    drift = (torch.arange(N, device=device) % 8) == 3
+    F = torch.empty(T, N, D, dtype=dt, device=device)
+    alpha = torch.empty(T, N, dtype=torch.float32, device=device)
+    width = max(1, N // 6)
+    for f0 in range(0, T, frame_chunk):
+        n = min(frame_chunk, T - f0)
+        g = _gen(seed * 9973 + 7 + f0, device)
+        noise = torch.randn(n, N, D, generator=g, device=device)
+        x = base[None] + 0.1 * noise
+        x[:, drift] = base[None, drift] + 0.33 * noise[:, drift]
+        start = (torch.arange(f0, f0 + n, device=device) * 5) % max(1, N - width)          # [n]
+        pos = torch.arange(N, device=device)[None, :]
+        moving = (pos >= start[:, None]) & (pos < start[:, None] + width)                   # [n][N]
+        x = torch.where(moving[:, :, None], 1.5 * noise, x)
+        a = torch.rand(n, N, generator=g, device=device) * 0.6 + 0.4 * moving.float()
+        F[f0:f0 + n] = x.to(dt)
+        alpha[f0:f0 + n] = a.clamp_(0.0, 1.0)
+    return F, alpha
+
+
 def as_u16(t: torch.Tensor):
     """NumPy view for the oracle: uint16 bit patterns for bf16/fp16, float32 unchanged."""
     t = t.detach().cpu().contiguous()

@@ -19,7 +19,7 @@ def oqm():
 
 
 def declared_symbols():
-    text = (ROOT / "include" / "stom_oqm.h").read_text()
+    text = "".join(h.read_text() for h in sorted((ROOT / "include").glob("*.h")))
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
     return sorted(set(re.findall(r"\b(stom_[a-z0-9_]+)\s*\(", text)))
 
@@ -28,6 +28,7 @@ def test_library_exports_every_declared_symbol(oqm):
     names = declared_symbols()
     assert "stom_oqm_quantize_frame" in names and "stom_oqm_dequant_gather" in names
     assert "stom_oqm_score_groups" in names and "stom_oqm_topk" in names
+    assert "stom_ctr_similarity" in names and "stom_ctr_select" in names and "stom_ctr_reduce" in names
     for n in names:
         assert hasattr(oqm.lib(), n), f"{n} declared in the header but not exported"
     assert set(oqm.EXPORTS) <= set(names)
