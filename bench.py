@@ -579,8 +579,169 @@ def run_stream(args, sh):
     }))
 
 
+CTR_SHAPE = {"T": 7200, "N": 196, "D": 1152, "G": 50, "tau_c": 0.9, "dtype": "bf16", "seed": 4242}
+CTR_CPU_FRAMES = 1200
+
+
+def bytes_ctr(T, N, D, G, elem=2):
+    """Algorithmic bytes of the CTR steps over T frames: every feature row once, saliency once, similarity written
+    and read once, the integer outputs written once."""
+    return T * N * D * elem + T * N * 4 + 2 * T * N * 4 + T * (N + G + 2) * 4
+
+
+def run_ctr(args):
+    """The CTR steps (paper Sec. 3.3: temporal similarity, static/dynamic split, budget, saliency top-k_d) over a
+    2-hour stream of synthetic encoder features.  `--impl reference` times the oracle on a sample of the frames."""
+    c = dict(CTR_SHAPE)
+    if args.frames:
+        c["T"] = args.frames
+    T, N, D, G = c["T"], c["N"], c["D"], c["G"]
+    name = "CTR-7B-2h" if not args.frames else f"CTR-7B-reduced-T{T}"
+    from paper_2510_18269_b200 import synth
+    if args.impl == "reference":
+        if int(os.environ.get("RANK", "0")) != 0:
+            return
+        from oracle import oqm_oracle as orc
+        frames = min(T, CTR_CPU_FRAMES)
+        F, alpha = synth.ctr_stream(frames, N, D, c["seed"], "cpu", c["dtype"])
+        Fn, an = synth.as_u16(F), alpha.numpy()
+        ts = []
+        for _ in range(args.steps):
+            t0 = time.perf_counter()
+            sim = orc.ctr_similarity(Fn, orc.BF16)
+            orc.ctr_select(sim, an, G, c["tau_c"])
+            ts.append(time.perf_counter() - t0)
+        v = bytes_ctr(frames, N, D, G) / statistics.mean(ts) / 1e9
+        sample = f"first {frames} frames (of {T})"
+        print(json.dumps({
+            "impl": "reference", "metric": "CTR reduce throughput", "value": v, "unit": "GB/s", "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": 0, "ms_per_step": 1e3 * statistics.mean(ts), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": name, "sample": sample},
+            "cpu_baseline": {"value": v, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": v, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}, "gpu_launches": 0}))
+        return
+    import torch
+    from paper_2510_18269_b200 import oqm, dist as sdist
+    rank, world, local = sdist.init_from_env(args.gpus)
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    oqm.lib()
+    peak, peak_src = measured_peak()
+    F, alpha = synth.ctr_stream(T, N, D, c["seed"] + 17 * rank, dev, c["dtype"])
+    sim = torch.empty(T, N, dtype=torch.float32, device=dev)
+    ks = torch.empty(T, dtype=torch.int32, device=dev)
+    kd = torch.empty_like(ks)
+    si = torch.empty(T, N, dtype=torch.int32, device=dev)
+    di = torch.empty(T, G, dtype=torch.int32, device=dev)
+    flush = torch.empty(512 << 20, dtype=torch.uint8, device=dev)
+
+    def ev():
+        return torch.cuda.Event(enable_timing=True)
+
+    def step(timers=None):
+        flush.fill_(1)
+        e = [ev() for _ in range(3)]
+        e[0].record()
+        oqm.stom_ctr_similarity(F, None, T, N, D, (N * D, D), sim)
+        e[1].record()
+        oqm.stom_ctr_select(sim, alpha, T, N, G, c["tau_c"], ks, kd, si, di)
+        e[2].record()
+        if timers is not None:
+            timers.append(e)
+
+    for _ in range(args.warmup):
+        step()
+    sampler = ClockSampler(nvml_index(local))
+    sampler.start()
+    sampler.ready.wait(10)
+    sdist.barrier()
+    torch.cuda.synchronize()
+    timers = []
+    for _ in range(args.steps):
+        step(timers)
+    torch.cuda.synchronize()
+    sdist.barrier()
+    clocks = sampler.result()
+    sim_ms = sdist.max_over_ranks(statistics.mean(t[0].elapsed_time(t[1]) for t in timers))
+    sel_ms = sdist.max_over_ranks(statistics.mean(t[1].elapsed_time(t[2]) for t in timers))
+    tot_ms = sdist.max_over_ranks(statistics.mean(t[0].elapsed_time(t[2]) for t in timers))
+    nbytes = bytes_ctr(T, N, D, G)
+    sbytes = T * N * D * 2 + T * N * 4
+    a = sbytes / (sim_ms * 1e-3) / 1e9
+    tpu = NCU_TRAFFIC_PER_UNIT.get("ctr_similarity_kernel")
+    out = {
+        "metric": "CTR reduce throughput", "value": world * nbytes / (tot_ms * 1e-3) / 1e9, "unit": "GB/s",
+        "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": tot_ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": name, **{k: c[k] for k in ("T", "N", "D", "G", "tau_c", "dtype")},
+                   "l2": "features 3.25 GB >> L2; 512 MB flush before every step",
+                   "multi_gpu": "independent stream per rank, no collective"},
+        "submetrics": {"frames_per_s": world * T / (tot_ms * 1e-3),
+                       "stage_us": {"similarity": sim_ms * 1e3, "select": sel_ms * 1e3},
+                       "mean_k_s": float(ks.float().mean().item())},
+        "roofline": {"kernel": "ctr_similarity_kernel", "bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s",
+                     "frac": a / peak, "traffic": None if tpu is None else tpu * T, "peak_source": peak_src,
+                     "algorithmic_bytes_per_launch": sbytes, "ms_per_launch": sim_ms},
+        "gpu_launches": 2, "clocks": clocks,
+    }
+    if not args.no_e2e:
+        # host buffers: features and saliency of a chunk of frames go up, the integer outputs come back; the frame
+        # before a chunk is the carried state (`prev`)
+        chunk = min(600, T)
+        Fh = torch.empty(chunk, N, D, dtype=F.dtype).pin_memory()
+        ah = torch.empty(chunk, N, dtype=torch.float32).pin_memory()
+        Fh.copy_(F[:chunk])
+        ah.copy_(alpha[:chunk])
+        outs_h = [torch.empty(chunk, dtype=torch.int32).pin_memory(), torch.empty(chunk, dtype=torch.int32).pin_memory(),
+                  torch.empty(chunk, G, dtype=torch.int32).pin_memory()]
+        Fd, ad = torch.empty_like(F[:chunk]), torch.empty_like(alpha[:chunk])
+        prev = torch.empty(N, D, dtype=F.dtype, device=dev)
+        n_chunks = (T + chunk - 1) // chunk
+        ts = []
+        for it in range(args.e2e_steps + 1):
+            torch.cuda.synchronize()
+            a0, a1 = ev(), ev()
+            a0.record()
+            for cidx in range(n_chunks):
+                Fd.copy_(Fh, non_blocking=True)
+                ad.copy_(ah, non_blocking=True)
+                oqm.stom_ctr_reduce(Fd, prev if cidx else None, chunk, N, D, (N * D, D), ad, G, c["tau_c"], sim[:chunk],
+                                    ks[:chunk], kd[:chunk], si[:chunk], di[:chunk])
+                prev.copy_(Fd[chunk - 1], non_blocking=True)
+                outs_h[0].copy_(ks[:chunk], non_blocking=True)
+                outs_h[1].copy_(kd[:chunk], non_blocking=True)
+                outs_h[2].copy_(di[:chunk], non_blocking=True)
+            a1.record()
+            torch.cuda.synchronize()
+            if it:
+                ts.append(a0.elapsed_time(a1))
+        e_ms = sdist.max_over_ranks(statistics.mean(ts))
+        frames = n_chunks * chunk
+        out["e2e"] = {"value": world * bytes_ctr(frames, N, D, G) / (e_ms * 1e-3) / 1e9, "unit": "GB/s",
+                      "h2d_bytes_per_step": n_chunks * (Fh.numel() * 2 + ah.numel() * 4),
+                      "d2h_bytes_per_step": n_chunks * sum(o.numel() * 4 for o in outs_h), "ms_per_step": e_ms,
+                      "note": f"{n_chunks} chunks of {chunk} frames from pinned host memory, one synthetic chunk cycled"}
+    if not args.no_cpu_baseline and rank == 0 and world == 1:
+        from oracle import oqm_oracle as orc
+        frames = min(T, CTR_CPU_FRAMES)
+        Fc, ac = F[:frames].cpu(), alpha[:frames].cpu()
+        t0 = time.perf_counter()
+        o_sim = orc.ctr_similarity(synth.as_u16(Fc), orc.BF16)
+        orc.ctr_select(o_sim, ac.numpy(), G, c["tau_c"])
+        dt = time.perf_counter() - t0
+        out["cpu_baseline"] = {"value": bytes_ctr(frames, N, D, G) / dt / 1e9, "unit": "GB/s", "cores": 1,
+                               "kind": "oracle", "sample": f"first {frames} frames (of {T})", "seconds": dt}
+    if rank == 0:
+        print(json.dumps(out))
+    sdist.finish()
+
+
 def main():
     args = parse()
+    if args.config == "CTR":
+        run_ctr(args)
+        return
     from paper_2510_18269_b200 import synth
     sh = synth.CONFIGS[args.config]
     if args.meta != "fp32":

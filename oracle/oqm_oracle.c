@@ -708,6 +708,7 @@ int32_t orc_ctr_select(const float *sim, const float *alpha, int32_t T, int32_t 
                 if (taken[i]) continue;
                 if (best < 0 || a[i] > a[best]) best = i; /* dyn is ascending: equal alpha keeps the earlier one */
             }
+            if (best < 0) break; /* cannot happen while r < nd; keeps the index provably in range */
             taken[best] = 1;
             ++got;
         }

@@ -32,12 +32,31 @@ struct SimParams {
     int32_t T, N, D, n_runs;
 };
 
+__device__ __forceinline__ uint64_t pair_f2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void split_f2(uint64_t v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+
 // T: element type; NP: 16-byte vectors of a row per lane
+// Blocks of wide rows are half as large: a thread then holds so many registers that whole blocks of 8 warps would
+// leave a third of the register file idle.
+template <int NP>
+__host__ __device__ constexpr int sim_warps() { return NP > 8 ? kSimWarps / 2 : kSimWarps; }
+
 template <typename T, int NP>
-__global__ void __launch_bounds__(kSimWarps * 32) ctr_similarity_kernel(const SimParams p) {
+__global__ void __launch_bounds__(sim_warps<NP>() * 32) ctr_similarity_kernel(const SimParams p) {
     constexpr int EPV = 16 / (int)sizeof(T);  // elements per vector
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t w = (int64_t)blockIdx.x * kSimWarps + warp;
+    const int64_t w = (int64_t)blockIdx.x * sim_warps<NP>() + warp;
     if (w >= (int64_t)p.n_runs * p.N) return;
     const int run = (int)(w / p.N), i = (int)(w - (int64_t)run * p.N);
     const int f0 = run * kSimRun, f1 = min(f0 + kSimRun, p.T);
@@ -50,25 +69,63 @@ __global__ void __launch_bounds__(kSimWarps * 32) ctr_similarity_kernel(const Si
             v[q] = e < p.D ? __ldg(reinterpret_cast<const uint4 *>(row + e)) : make_uint4(0u, 0u, 0u, 0u);
         }
     };
-    auto dot = [&](const uint4 (&a)[NP], const uint4 (&b)[NP]) {
-        float acc = 0.0f;
+    // sum over the lane's elements of a*b and of a*a.  Rows of up to 4 KB: two channels per instruction (f32x2),
+    // which also keeps the kernel at three blocks per SM; wider rows measured faster with scalar accumulation.
+    auto dots = [&](const uint4 (&a)[NP], const uint4 (&b)[NP], float &ab, float &aa) {
+        if constexpr (NP > 8) {
+            float s_ab = 0.0f, s_aa = 0.0f;
+#pragma unroll
+            for (int q = 0; q < NP; ++q) {
+                const uint32_t aw[4] = {a[q].x, a[q].y, a[q].z, a[q].w}, bw[4] = {b[q].x, b[q].y, b[q].z, b[q].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if constexpr (sizeof(T) == 4) {
+                        s_ab = fmaf(__uint_as_float(aw[j]), __uint_as_float(bw[j]), s_ab);
+                        s_aa = fmaf(__uint_as_float(aw[j]), __uint_as_float(aw[j]), s_aa);
+                    } else {
+                        float a0, a1, b0, b1;
+                        unpack2<T>(aw[j], a0, a1);
+                        unpack2<T>(bw[j], b0, b1);
+                        s_ab = fmaf(a0, b0, s_ab);
+                        s_ab = fmaf(a1, b1, s_ab);
+                        s_aa = fmaf(a0, a0, s_aa);
+                        s_aa = fmaf(a1, a1, s_aa);
+                    }
+                }
+            }
+            ab = s_ab;
+            aa = s_aa;
+            return;
+        }
+        uint64_t acc_ab = 0ull, acc_aa = 0ull;  // (+0, +0)
 #pragma unroll
         for (int q = 0; q < NP; ++q) {
             const uint32_t aw[4] = {a[q].x, a[q].y, a[q].z, a[q].w}, bw[4] = {b[q].x, b[q].y, b[q].z, b[q].w};
+            if constexpr (sizeof(T) == 4) {
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                if constexpr (sizeof(T) == 4) {
-                    acc = fmaf(__uint_as_float(aw[j]), __uint_as_float(bw[j]), acc);
-                } else {
+                for (int j = 0; j < 4; j += 2) {
+                    const uint64_t a2 = pair_f2(__uint_as_float(aw[j]), __uint_as_float(aw[j + 1]));
+                    const uint64_t b2 = pair_f2(__uint_as_float(bw[j]), __uint_as_float(bw[j + 1]));
+                    acc_ab = fma_f2(a2, b2, acc_ab);
+                    acc_aa = fma_f2(a2, a2, acc_aa);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
                     float a0, a1, b0, b1;
                     unpack2<T>(aw[j], a0, a1);
                     unpack2<T>(bw[j], b0, b1);
-                    acc = fmaf(a0, b0, acc);
-                    acc = fmaf(a1, b1, acc);
+                    const uint64_t a2 = pair_f2(a0, a1), b2 = pair_f2(b0, b1);
+                    acc_ab = fma_f2(a2, b2, acc_ab);
+                    acc_aa = fma_f2(a2, a2, acc_aa);
                 }
             }
         }
-        return acc;
+        float lo, hi;
+        split_f2(acc_ab, lo, hi);
+        ab = lo + hi;
+        split_f2(acc_aa, lo, hi);
+        aa = lo + hi;
     };
     auto warp_sum = [](float v) {
 #pragma unroll
@@ -88,11 +145,16 @@ __global__ void __launch_bounds__(kSimWarps * 32) ctr_similarity_kernel(const Si
         for (int q = 0; q < NP; ++q) prv[q] = make_uint4(0u, 0u, 0u, 0u);
     }
     load_row(base + (int64_t)f0 * p.sf, cur);
-    float n_prv = warp_sum(dot(prv, prv));
+    float n_prv, unused;
+    dots(prv, prv, unused, n_prv);
+    n_prv = warp_sum(n_prv);
     for (int f = f0; f < f1; ++f) {
         uint4 nxt[NP];
         if (f + 1 < f1) load_row(base + (int64_t)(f + 1) * p.sf, nxt);
-        const float d = warp_sum(dot(cur, prv)), n_cur = warp_sum(dot(cur, cur));
+        float d, n_cur;
+        dots(cur, prv, d, n_cur);
+        d = warp_sum(d);
+        n_cur = warp_sum(n_cur);
         if (lane == 0) {
             const float den = fmaxf(sqrtf(n_cur), 1e-12f) * fmaxf(sqrtf(n_prv), 1e-12f);
             p.sim[(int64_t)f * p.N + i] = have_prev ? d / den : -INFINITY;
@@ -189,21 +251,28 @@ __global__ void __launch_bounds__(kSelThreads) ctr_select_kernel(const SelParams
     for (int j = n_sel + tid; j < p.G; j += kSelThreads) d_out[j] = -1;
 }
 
+template <typename T, int NP>
+static void launch_similarity_np(const SimParams &p, cudaStream_t s) {
+    constexpr int W = sim_warps<NP>();
+    const int64_t warps = (int64_t)p.n_runs * p.N;
+    ctr_similarity_kernel<T, NP><<<(unsigned)((warps + W - 1) / W), W * 32, 0, s>>>(p);
+}
+
 template <typename T>
-static void launch_similarity(const SimParams &p, int np, unsigned blocks, cudaStream_t s) {
+static void launch_similarity(const SimParams &p, int np, cudaStream_t s) {
     switch (np) {
-    case 1: ctr_similarity_kernel<T, 1><<<blocks, kSimWarps * 32, 0, s>>>(p); break;
-    case 2: ctr_similarity_kernel<T, 2><<<blocks, kSimWarps * 32, 0, s>>>(p); break;
-    case 3: ctr_similarity_kernel<T, 3><<<blocks, kSimWarps * 32, 0, s>>>(p); break;
-    case 4: ctr_similarity_kernel<T, 4><<<blocks, kSimWarps * 32, 0, s>>>(p); break;
-    case 5: ctr_similarity_kernel<T, 5><<<blocks, kSimWarps * 32, 0, s>>>(p); break;
-    case 6: ctr_similarity_kernel<T, 6><<<blocks, kSimWarps * 32, 0, s>>>(p); break;
-    case 7: ctr_similarity_kernel<T, 7><<<blocks, kSimWarps * 32, 0, s>>>(p); break;
-    case 8: ctr_similarity_kernel<T, 8><<<blocks, kSimWarps * 32, 0, s>>>(p); break;
-    case 9: case 10: ctr_similarity_kernel<T, 10><<<blocks, kSimWarps * 32, 0, s>>>(p); break;
-    case 11: case 12: ctr_similarity_kernel<T, 12><<<blocks, kSimWarps * 32, 0, s>>>(p); break;
-    case 13: case 14: ctr_similarity_kernel<T, 14><<<blocks, kSimWarps * 32, 0, s>>>(p); break;
-    default: ctr_similarity_kernel<T, 16><<<blocks, kSimWarps * 32, 0, s>>>(p); break;  // rows of up to 8 KB
+    case 1: launch_similarity_np<T, 1>(p, s); break;
+    case 2: launch_similarity_np<T, 2>(p, s); break;
+    case 3: launch_similarity_np<T, 3>(p, s); break;
+    case 4: launch_similarity_np<T, 4>(p, s); break;
+    case 5: launch_similarity_np<T, 5>(p, s); break;
+    case 6: launch_similarity_np<T, 6>(p, s); break;
+    case 7: launch_similarity_np<T, 7>(p, s); break;
+    case 8: launch_similarity_np<T, 8>(p, s); break;
+    case 9: case 10: launch_similarity_np<T, 10>(p, s); break;
+    case 11: case 12: launch_similarity_np<T, 12>(p, s); break;
+    case 13: case 14: launch_similarity_np<T, 14>(p, s); break;
+    default: launch_similarity_np<T, 16>(p, s); break;  // rows of up to 8 KB
     }
 }
 
@@ -225,15 +294,13 @@ extern "C" int32_t stom_ctr_similarity(const void *F, const void *prev, int32_t 
     p.F = F; p.prev = prev; p.sf = stride_frame; p.st = stride_token; p.sim = sim;
     p.T = T; p.N = N; p.D = D;
     p.n_runs = (T + kSimRun - 1) / kSimRun;
-    const int64_t warps = (int64_t)p.n_runs * N;
-    const int64_t blocks = (warps + kSimWarps - 1) / kSimWarps;
-    if (blocks > 0x7fffffffLL) return STOM_ERR_SHAPE;
+    if ((int64_t)p.n_runs * N > 0x7fffffffLL) return STOM_ERR_SHAPE;
     const int np = (D * elem_bytes(dtype) + 511) / 512;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     switch (dtype) {
-    case STOM_BF16: launch_similarity<__nv_bfloat16>(p, np, (unsigned)blocks, s); break;
-    case STOM_FP16: launch_similarity<__half>(p, np, (unsigned)blocks, s); break;
-    default: launch_similarity<float>(p, np, (unsigned)blocks, s); break;
+    case STOM_BF16: launch_similarity<__nv_bfloat16>(p, np, s); break;
+    case STOM_FP16: launch_similarity<__half>(p, np, s); break;
+    default: launch_similarity<float>(p, np, s); break;
     }
     return finish_launch();
 }
