@@ -47,6 +47,8 @@ NCU_TRAFFIC_PER_UNIT = {
     "dequant_gather_kernel": 103985.0 / 4,
     "score_kernel": 2066.0 / 4,         # bytes per (layer, stored group): 59.25 MB over 28 x 1024 units
     "retrieve_kernel": 2178.0 / 4,      # bytes per (layer, stored group): 62.46 MB over 28 x 1024 units (Q re-read per block)
+    # bytes per frame of 196 tokens x 1152 bf16 channels (not per kv head): 561.8 MB over 1200 frames
+    "ctr_similarity_kernel": 468181.0,
 }
 
 
