@@ -305,9 +305,12 @@ int32_t stom_oqm_retrieve(const stom_oqm_config *cfg, const stom_oqm_store *stor
  * (H_q/H_k)):  out[l][h_q][:] = softmax_t(softmax_scale * <q[l][h_q], K_t>) V_t
  * over the tokens t of  [the sys_len system tokens of (l, h)] followed by [the
  * G tokens of every selected group idx[..][j] >= 0, j < k], where a group's K
- * and V rows are fmaf(code, s, m) of the bank (binary32, not rounded to a
- * 16-bit type on the way).  Accumulation is binary32; the output is rounded
- * once to cache_dtype.
+ * and V rows are code * s + m of the bank (not rounded to a 16-bit type on the
+ * way).  Accumulation is binary32; the output is rounded once to cache_dtype.
+ * With 4-bit codes both contractions run on the tensor cores with the raw
+ * codes as one operand (exact) and q*s, respectively the softmax weights, as
+ * the other, carried as a high and a low 16-bit part (16 significant bits);
+ * the affine terms are added in binary32.
  * idx: as for stom_oqm_dequant_gather (PER_LAYER [layer_count][k]; PER_HEAD
  *   [layer_count][H_k][k]); -1 entries are skipped, other out-of-range entries
  *   are skipped and flagged.  k may be 0 if sys_len > 0.

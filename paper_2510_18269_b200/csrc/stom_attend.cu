@@ -51,6 +51,60 @@ struct AttendParams {
     uint32_t *flags;
 };
 
+// Ticket and merge, the tail of both attention kernels: every block of a (layer, kv head) has written its partial
+// (max, sum, weighted sum) per query head to the workspace; the block that draws the last ticket combines them and
+// writes the output rows.  All threads of the block call it; nobody waits for another block.
+template <typename CT, int D>
+__device__ __forceinline__ void attend_merge(const AttendParams &p, int li, int h, int n_blocks, int *s_last_ptr) {
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, H = p.g.H;
+    int &s_last = *s_last_ptr;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) s_last = atomicAdd(&p.counters[li * H + h], 1u) == (unsigned)n_blocks - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (tid == 0) p.counters[li * H + h] = 0;  // as found
+    // one warp per query head: lanes first share out the blocks (max, then the sum of the weighted sums of
+    // weights), then the channels, with the loads of several blocks in flight
+    for (int hq = warp; hq < p.rep; hq += kAtWarps) {
+        const float *rec0 = p.part + (((int64_t)li * H + h) * n_blocks * p.rep + hq) * (D + 2);
+        const int64_t step = (int64_t)p.rep * (D + 2);
+        // lanes share out the blocks 32 at a time: their maxima and sums are loaded once, the weight of a block is
+        // then handed round by shuffle while every lane adds up its own channels, 8 blocks' loads in flight
+        float mx = -INFINITY;
+        for (int b = lane; b < n_blocks; b += 32) mx = fmaxf(mx, __ldcg(rec0 + b * step));
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+        float den = 0.0f;
+        float num[D / 32];
+#pragma unroll
+        for (int i = 0; i < D / 32; ++i) num[i] = 0.0f;
+        for (int b0 = 0; b0 < n_blocks; b0 += 32) {
+            float w_mine = 0.0f;
+            if (b0 + lane < n_blocks) {
+                const float mb = __ldcg(rec0 + (b0 + lane) * step);
+                if (mb != -INFINITY) {
+                    w_mine = exp2f(mb - mx);
+                    den = fmaf(__ldcg(rec0 + (b0 + lane) * step + 1), w_mine, den);
+                }
+            }
+            const int nb = min(32, n_blocks - b0);
+#pragma unroll 8
+            for (int j = 0; j < nb; ++j) {
+                const float w = __shfl_sync(0xffffffffu, w_mine, j);
+#pragma unroll
+                for (int i = 0; i < D / 32; ++i) num[i] = fmaf(__ldcg(rec0 + (b0 + j) * step + 2 + lane + 32 * i), w, num[i]);
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
+        CT *out = reinterpret_cast<CT *>(p.out) + (int64_t)li * p.o_sl + (int64_t)(h * p.rep + hq) * p.o_sh;
+#pragma unroll
+        for (int i = 0; i < D / 32; ++i) out[lane + 32 * i] = (CT)(den > 0.0f ? num[i] / den : 0.0f);
+    }
+}
+
 // QT: type of q_dec; CT: type of the system-token cache and of the output; LPR: lanes per token (d / 8);
 // BITS: width of a code
 template <typename QT, typename CT, int LPR, int BITS>
@@ -307,52 +361,379 @@ __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p
         __syncthreads();  // qf, buf and the statistics are rewritten by the next chunk of heads
     }
 
-    // ---- ticket: the block that completes (layer, kv head) merges the partial results
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) s_last = atomicAdd(&p.counters[li * H + h], 1u) == (unsigned)n_blocks - 1;
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    if (tid == 0) p.counters[li * H + h] = 0;  // as found
-    // one warp per query head: lanes first share out the blocks (max, then the sum of the weighted sums of
-    // weights), then the channels, with the loads of several blocks in flight
-    for (int hq = warp; hq < p.rep; hq += kAtWarps) {
-        const float *rec0 = p.part + (((int64_t)li * H + h) * n_blocks * p.rep + hq) * (D + 2);
-        const int64_t step = (int64_t)p.rep * (D + 2);
-        // lanes share out the blocks 32 at a time: their maxima and sums are loaded once, the weight of a block is
-        // then handed round by shuffle while every lane adds up its own channels, 8 blocks' loads in flight
-        float mx = -INFINITY;
-        for (int b = lane; b < n_blocks; b += 32) mx = fmaxf(mx, __ldcg(rec0 + b * step));
+    attend_merge<CT, D>(p, li, h, n_blocks, &s_last);
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// The same attention with the two contractions on the tensor cores (4-bit codes).
+//
+// Both products are small dense contractions -- scores: [tokens x d] . [d x 8 query heads]; values:
+// [d x tokens] . [tokens x 8 query heads] -- so they run as m16n8k16 warp-level matrix products (the query heads of a
+// GQA block are the 8 columns).  The affine map of the quantizer is moved out of the inner product: within a group
+// (s, m) depend on the channel only, so
+//     scores:  sum_c q_c (code_c s_c + m_c) = sum_c code_c (q_c s_c) + sum_c q_c m_c
+//     values:  sum_t w_t (code_tc s_c + m_c) = s_c sum_t w_t code_tc + m_c sum_t w_t
+// and the matrix operand is the raw code.  A code becomes a bfloat16 without arithmetic: 0x4300 | code is the number
+// 128 + code, exactly; the 128 is taken out again through the same sums.  The contraction index of a matrix product
+// may be permuted freely as long as both operands use the same permutation, and so may the output columns: a thread
+// therefore owns CONTIGUOUS code bytes (for the scores: d/4 adjacent channels of a token row; for the values: d/8
+// adjacent channels of four tokens), which it loads with one vector load and slices with byte permutes.
+// Segments, block layout, softmax statistics, partial results and the merge are those of the kernel above.
+// ---------------------------------------------------------------------------------------------------------------
+
+template <typename MT>
+__device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                          uint32_t b1);
+template <>
+__device__ __forceinline__ void mma_16816<__nv_bfloat16>(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                         uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+template <>
+__device__ __forceinline__ void mma_16816<__half>(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                                  uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// NW 32-bit words from p (p aligned to min(16, 4 * NW) bytes), or zeros
+template <int NW>
+__device__ __forceinline__ void load_words_or_zero(const void *p, bool valid, uint32_t (&w)[NW]) {
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        float den = 0.0f;
-        float num[D / 32];
+    for (int i = 0; i < NW; ++i) w[i] = 0u;
+    if (!valid) return;
+    if constexpr (NW == 1) {
+        w[0] = __ldg(static_cast<const uint32_t *>(p));
+    } else if constexpr (NW == 2) {
+        const uint2 v = __ldg(static_cast<const uint2 *>(p));
+        w[0] = v.x; w[1] = v.y;
+    } else {
 #pragma unroll
-        for (int i = 0; i < D / 32; ++i) num[i] = 0.0f;
-        for (int b0 = 0; b0 < n_blocks; b0 += 32) {
-            float w_mine = 0.0f;
-            if (b0 + lane < n_blocks) {
-                const float mb = __ldcg(rec0 + (b0 + lane) * step);
-                if (mb != -INFINITY) {
-                    w_mine = exp2f(mb - mx);
-                    den = fmaf(__ldcg(rec0 + (b0 + lane) * step + 1), w_mine, den);
+        for (int i = 0; i < NW / 4; ++i) {
+            const uint4 v = __ldg(static_cast<const uint4 *>(p) + i);
+            w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
+        }
+    }
+}
+
+// Byte `b` of x and byte `b` of y, each holding one 4-bit code (0x00..0x0F), as the bfloat16 pair
+// (128 + code of x, 128 + code of y): the permute puts the two bytes into the low byte of each half and fills the
+// other two with the sign of a source byte (selector values of 8 and above), which is zero.
+__device__ __forceinline__ uint32_t code_pair_bf16(uint32_t x, uint32_t y, int b) {
+    uint32_t v;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(v) : "r"(x), "r"(y), "r"(0x8480u + (uint32_t)b * 0x0101u));
+    return v | 0x43004300u;
+}
+
+// QT: type of q_dec; CT: type of the system-token cache and of the output; D: head dim
+// Two floats as a (high, low) pair of packed 16-bit pairs: hi = the values rounded to MT, lo = what the rounding
+// left over, rounded again.  A matrix product issued once with each part carries 16 significant bits of the operand.
+template <typename MT>
+__device__ __forceinline__ void split2(float a, float b, uint32_t &hi, uint32_t &lo, float &seen_a, float &seen_b) {
+    hi = pack2<MT>(a, b);
+    float ha, hb, la, lb;
+    unpack2<MT>(hi, ha, hb);
+    lo = pack2<MT>(a - ha, b - hb);
+    unpack2<MT>(lo, la, lb);
+    seen_a = ha + la;
+    seen_b = hb + lb;
+}
+
+template <typename QT, typename CT, int D>
+__global__ void __launch_bounds__(kAtThreads) attend_mma_kernel(const AttendParams p) {
+    constexpr int kSlots = kAtWarps * kAtSegTokens;
+    constexpr int kBuf = (32 * 1024) / (kAtHeads * D * 4) < kAtWarps ? (32 * 1024) / (kAtHeads * D * 4) : kAtWarps;
+    constexpr int KS = D / 16;  // k-steps of the score product (16 channels each)
+    constexpr int KC = D / 4;   // channels of a token row one thread owns in the score product
+    constexpr int MT = D / 16;  // m-tiles of the value product (16 channels each)
+    constexpr int VC = D / 8;   // channels one thread owns in the value product
+    using BF = __nv_bfloat16;
+    __shared__ __align__(16) float buf[8192];  // scores / weights [kAtHeads][kSlots]; then warp sums [kBuf][kAtHeads][D]
+    __shared__ __align__(16) float qf[kAtHeads][D];
+    __shared__ float blk_max[kAtHeads];
+    __shared__ float seg_sum[kAtWarps][kAtHeads];  // sum of a segment's weights per query head, as the tensor core sees them
+    __shared__ int s_last;
+    static_assert(kAtHeads * kSlots <= 8192 && kBuf * kAtHeads * D <= 8192, "shared buffer");
+    static_assert(kAtHeads == 8 && kAtSegTokens == 32, "fragment mapping");
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int g = lane >> 2, t = lane & 3;  // fragment coordinates of the thread
+    const int bx = blockIdx.x, h = blockIdx.y, li = blockIdx.z;
+    const int G = p.g.G, H = p.g.H;
+    const int seg = bx * kAtWarps + warp;
+    float(*sc)[kSlots] = reinterpret_cast<float(*)[kSlots]>(buf);
+
+    // ---- what the warp's segment is (as in the kernel above)
+    int n_tok = 0, tok0 = 0;
+    bool is_sys = false;
+    int64_t slot = 0;
+    if (seg < p.n_sys_seg) {
+        is_sys = true;
+        tok0 = seg * kAtSegTokens;
+        n_tok = min(kAtSegTokens, p.sys_len - tok0);
+    } else if (seg < p.n_seg) {
+        const int sg = seg - p.n_sys_seg;
+        const int j = sg / p.segs_per_group;
+        tok0 = (sg - j * p.segs_per_group) * kAtSegTokens;
+        const int tg = p.per_head ? p.idx[((int64_t)li * H + h) * p.k + j] : p.idx[(int64_t)li * p.k + j];
+        if (tg >= 0 && tg < p.n_groups) {
+            n_tok = min(kAtSegTokens, G - tok0);
+            slot = bank_slot(p.g, p.layer_begin + li, tg, h);
+        } else if (tg != -1 && p.flags && lane == 0 && tok0 == 0) {
+            atomicOr(p.flags, STOM_FLAG_BAD_INDEX);
+        }
+    }
+    n_tok = max(n_tok, 0);
+    const CT *ksys = reinterpret_cast<const CT *>(p.ksys) + (int64_t)li * p.s_sl + (int64_t)h * p.s_sh;
+    const CT *vsys = reinterpret_cast<const CT *>(p.vsys) + (int64_t)li * p.s_sl + (int64_t)h * p.s_sh;
+    const uint8_t *kcodes = p.codes_k + slot * (int64_t)G * p.g.row_bytes;
+    const uint8_t *vcodes = p.codes_v + slot * (int64_t)G * p.g.row_bytes;
+    const int md = p.g.meta_dtype;
+
+    const int n_blocks = gridDim.x;
+    for (int h0 = 0; h0 < p.rep; h0 += kAtHeads) {
+        const int nh = min(kAtHeads, p.rep - h0);
+        // ---- the query rows, scaled so that exp2 can be used
+        for (int e = tid; e < kAtHeads * D; e += kAtThreads) {
+            const int hh = e / D, c = e - hh * D;
+            float v = 0.0f;
+            if (hh < nh) {
+                const QT *q = reinterpret_cast<const QT *>(p.q) + (int64_t)li * p.q_sl + (int64_t)(h * p.rep + h0 + hh) * p.q_sh;
+                v = (float)q[c] * p.scale_log2e;
+            }
+            qf[hh][c] = v;
+        }
+        __syncthreads();
+
+        // ---- phase 1: scores.  Contraction slot (kk; 2t, 2t+1, 2t+8, 2t+9) of the matrix product stands for
+        //      channels KC*t + 4*kk + (0, 1, 2, 3); column g is query head g.
+        for (int e = lane; e < kAtHeads * kAtSegTokens; e += 32)
+            sc[e / kAtSegTokens][warp * kAtSegTokens + (e % kAtSegTokens)] = -INFINITY;  // slots without a token
+        __syncwarp();
+        if (n_tok > 0) {
+            uint32_t qb[KS][2], ql[KS][2];  // the thread's column of the right-hand operand, high and low parts
+            float bias = 0.0f;   // what the raw-code product leaves out, for query head g
+            if (!is_sys) {
+#pragma unroll
+                for (int c8 = 0; c8 < KC / 8; ++c8) {
+                    float s8[8], m8[8];
+                    load_scale_zero8(p.scale_k, p.zero_k, slot * D + KC * t + c8 * 8, md, s8, m8);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {  // 2 channels each
+                        const int c = KC * t + c8 * 8 + 2 * j;
+                        const float q0 = qf[g][c], q1 = qf[g][c + 1];
+                        uint32_t whi, wlo;
+                        float r0, r1;  // the two products as the tensor core sees them
+                        split2<BF>(q0 * s8[2 * j], q1 * s8[2 * j + 1], whi, wlo, r0, r1);
+                        bias = fmaf(q0, m8[2 * j], bias);
+                        bias = fmaf(q1, m8[2 * j + 1], bias);
+                        bias = fmaf(-128.0f, r0 + r1, bias);
+                        qb[(c8 * 8 + 2 * j) / 4][((c8 * 8 + 2 * j) / 2) & 1] = whi;
+                        ql[(c8 * 8 + 2 * j) / 4][((c8 * 8 + 2 * j) / 2) & 1] = wlo;
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < KC / 2; ++j) {
+                    const int c = KC * t + 2 * j;
+                    float r0, r1;
+                    split2<CT>(qf[g][c], qf[g][c + 1], qb[j / 2][j & 1], ql[j / 2][j & 1], r0, r1);
                 }
             }
-            const int nb = min(32, n_blocks - b0);
-#pragma unroll 8
-            for (int j = 0; j < nb; ++j) {
-                const float w = __shfl_sync(0xffffffffu, w_mine, j);
+            bias += __shfl_xor_sync(0xffffffffu, bias, 1);
+            bias += __shfl_xor_sync(0xffffffffu, bias, 2);
+            const float bias_a = __shfl_sync(0xffffffffu, bias, (2 * t) << 2);       // of query head 2t
+            const float bias_b = __shfl_sync(0xffffffffu, bias, (2 * t + 1) << 2);   // of query head 2t + 1
 #pragma unroll
-                for (int i = 0; i < D / 32; ++i) num[i] = fmaf(__ldcg(rec0 + (b0 + j) * step + 2 + lane + 32 * i), w, num[i]);
+            for (int mt = 0; mt < kAtSegTokens / 16; ++mt) {
+                const int r0 = mt * 16 + g, r1 = r0 + 8;
+                if (mt * 16 >= n_tok) break;  // warp-uniform
+                float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+                if (!is_sys) {
+                    uint32_t w0[D / 32], w1[D / 32];  // the thread's KC codes of the two token rows
+                    load_words_or_zero<D / 32>(kcodes + (int64_t)(tok0 + r0) * p.g.row_bytes + t * (KC / 2), r0 < n_tok, w0);
+                    load_words_or_zero<D / 32>(kcodes + (int64_t)(tok0 + r1) * p.g.row_bytes + t * (KC / 2), r1 < n_tok, w1);
+#pragma unroll
+                    for (int kk = 0; kk < KS; ++kk) {
+                        // codes 4kk .. 4kk+3 of the thread's run: bytes 2(kk&1) and 2(kk&1)+1 of the even-nibble and
+                        // odd-nibble views of word kk/2
+                        const uint32_t e0 = w0[kk / 2] & 0x0F0F0F0Fu, o0 = (w0[kk / 2] >> 4) & 0x0F0F0F0Fu;
+                        const uint32_t e1 = w1[kk / 2] & 0x0F0F0F0Fu, o1 = (w1[kk / 2] >> 4) & 0x0F0F0F0Fu;
+                        const int b = 2 * (kk & 1);
+                        const uint32_t a0 = code_pair_bf16(e0, o0, b), a1 = code_pair_bf16(e1, o1, b);
+                        const uint32_t a2 = code_pair_bf16(e0, o0, b + 1), a3 = code_pair_bf16(e1, o1, b + 1);
+                        mma_16816<BF>(c4, a0, a1, a2, a3, qb[kk][0], qb[kk][1]);
+                        mma_16816<BF>(c4, a0, a1, a2, a3, ql[kk][0], ql[kk][1]);
+                    }
+                } else {
+                    uint32_t w0[KC / 2], w1[KC / 2];  // the thread's KC channels of the two token rows, 16-bit pairs
+                    load_words_or_zero<KC / 2>(ksys + (int64_t)(tok0 + r0) * p.s_st + KC * t, r0 < n_tok, w0);
+                    load_words_or_zero<KC / 2>(ksys + (int64_t)(tok0 + r1) * p.s_st + KC * t, r1 < n_tok, w1);
+#pragma unroll
+                    for (int kk = 0; kk < KS; ++kk) {
+                        mma_16816<CT>(c4, w0[2 * kk], w1[2 * kk], w0[2 * kk + 1], w1[2 * kk + 1], qb[kk][0], qb[kk][1]);
+                        mma_16816<CT>(c4, w0[2 * kk], w1[2 * kk], w0[2 * kk + 1], w1[2 * kk + 1], ql[kk][0], ql[kk][1]);
+                    }
+                }
+                if (r0 < n_tok) {
+                    sc[2 * t][warp * kAtSegTokens + r0] = c4[0] + bias_a;
+                    sc[2 * t + 1][warp * kAtSegTokens + r0] = c4[1] + bias_b;
+                }
+                if (r1 < n_tok) {
+                    sc[2 * t][warp * kAtSegTokens + r1] = c4[2] + bias_a;
+                    sc[2 * t + 1][warp * kAtSegTokens + r1] = c4[3] + bias_b;
+                }
             }
         }
+        __syncthreads();
+
+        // ---- phase 2: the block's maximum per query head; scores become weights in place.  The sum of the weights is
+        //      taken in phase 3 from the ROUNDED weights the matrix product uses, so that numerator and denominator
+        //      of the softmax average see the same weights.
+        if (warp < kAtHeads) {
+            float mx = -INFINITY;
+            for (int i = lane; i < kSlots; i += 32) mx = fmaxf(mx, sc[warp][i]);
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
-        CT *out = reinterpret_cast<CT *>(p.out) + (int64_t)li * p.o_sl + (int64_t)(h * p.rep + hq) * p.o_sh;
+            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+            for (int i = lane; i < kSlots; i += 32) {
+                const float v = sc[warp][i];
+                sc[warp][i] = v == -INFINITY ? 0.0f : exp2f(v - mx);
+            }
+            if (lane == 0) blk_max[warp] = mx;
+        }
+        __syncthreads();
+
+        // ---- phase 3: weighted sum of the values.  Rows of the product are channels: rows g and g + 8 of m-tile mm
+        //      stand for channels VC*g + 2*mm and VC*g + 2*mm + 1; the contraction runs over the segment's tokens
+        //      (slot 2t, 2t+1, 2t+8, 2t+9 of k-step ks is token 16*ks + the same); columns are query heads.
+        float acc[MT][4];
 #pragma unroll
-        for (int i = 0; i < D / 32; ++i) out[lane + 32 * i] = (CT)(den > 0.0f ? num[i] / den : 0.0f);
+        for (int mm = 0; mm < MT; ++mm)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[mm][i] = 0.0f;
+        float wsum = 0.0f;  // sum of the weights of query head g as the tensor core sees them
+        if (n_tok > 0) {
+#pragma unroll
+            for (int ks = 0; ks < kAtSegTokens / 16; ++ks) {
+                if (ks * 16 >= n_tok) break;  // warp-uniform
+                const int ta = ks * 16 + 2 * t;  // tokens ta, ta + 1, ta + 8, ta + 9
+                const float2 wlo = *reinterpret_cast<const float2 *>(&sc[g][warp * kAtSegTokens + ta]);
+                const float2 whi = *reinterpret_cast<const float2 *>(&sc[g][warp * kAtSegTokens + ta + 8]);
+                uint32_t b0, b1, l0, l1;  // the weights, high and low parts
+                float r0, r1, r2, r3;
+                if (!is_sys) {
+                    split2<BF>(wlo.x, wlo.y, b0, l0, r0, r1);
+                    split2<BF>(whi.x, whi.y, b1, l1, r2, r3);
+                } else {
+                    split2<CT>(wlo.x, wlo.y, b0, l0, r0, r1);
+                    split2<CT>(whi.x, whi.y, b1, l1, r2, r3);
+                }
+                wsum += (r0 + r1) + (r2 + r3);
+                if (!is_sys) {
+                    uint32_t e[4][D / 64], o[4][D / 64];  // even / odd nibbles of the thread's VC codes of its 4 tokens
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int tok = ta + (i & 1) + 8 * (i >> 1);
+                        uint32_t w[D / 64];
+                        load_words_or_zero<D / 64>(vcodes + (int64_t)(tok0 + tok) * p.g.row_bytes + g * (VC / 2), tok < n_tok, w);
+#pragma unroll
+                        for (int j = 0; j < D / 64; ++j) {
+                            e[i][j] = w[j] & 0x0F0F0F0Fu;
+                            o[i][j] = (w[j] >> 4) & 0x0F0F0F0Fu;
+                        }
+                    }
+#pragma unroll
+                    for (int mm = 0; mm < MT; ++mm) {
+                        // byte mm % 4 of word mm / 4 of e: the code of channel VC*g + 2*mm; of o: of the next channel
+                        const int j = mm >> 2, b = mm & 3;
+                        const uint32_t a0 = code_pair_bf16(e[0][j], e[1][j], b), a1 = code_pair_bf16(o[0][j], o[1][j], b);
+                        const uint32_t a2 = code_pair_bf16(e[2][j], e[3][j], b), a3 = code_pair_bf16(o[2][j], o[3][j], b);
+                        mma_16816<BF>(acc[mm], a0, a1, a2, a3, b0, b1);
+                        mma_16816<BF>(acc[mm], a0, a1, a2, a3, l0, l1);
+                    }
+                } else {
+                    uint32_t w[4][VC / 2];  // the thread's VC channels of its 4 tokens, 16-bit pairs (channel 2mm, 2mm+1)
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const int tok = ta + (i & 1) + 8 * (i >> 1);
+                        load_words_or_zero<VC / 2>(vsys + (int64_t)(tok0 + tok) * p.s_st + VC * g, tok < n_tok, w[i]);
+                    }
+#pragma unroll
+                    for (int mm = 0; mm < MT; ++mm) {
+                        const uint32_t a0 = __byte_perm(w[0][mm], w[1][mm], 0x5410), a1 = __byte_perm(w[0][mm], w[1][mm], 0x7632);
+                        const uint32_t a2 = __byte_perm(w[2][mm], w[3][mm], 0x5410), a3 = __byte_perm(w[2][mm], w[3][mm], 0x7632);
+                        mma_16816<CT>(acc[mm], a0, a1, a2, a3, b0, b1);
+                        mma_16816<CT>(acc[mm], a0, a1, a2, a3, l0, l1);
+                    }
+                }
+            }
+        }
+        wsum += __shfl_xor_sync(0xffffffffu, wsum, 1);
+        wsum += __shfl_xor_sync(0xffffffffu, wsum, 2);
+        const float ws_a = __shfl_sync(0xffffffffu, wsum, (2 * t) << 2), ws_b = __shfl_sync(0xffffffffu, wsum, (2 * t + 1) << 2);
+        if (t == 0) seg_sum[warp][g] = wsum;
+        if (!is_sys && n_tok > 0) {
+            // acc holds sum_t w_t (128 + code): apply the group's scale and offset, channel by channel
+#pragma unroll
+            for (int c8 = 0; c8 < VC / 8; ++c8) {
+                float s8[8], m8[8];
+                load_scale_zero8(p.scale_v, p.zero_v, slot * D + VC * g + c8 * 8, md, s8, m8);
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int mm = c8 * 4 + j;
+                    acc[mm][0] = fmaf(s8[2 * j], fmaf(-128.0f, ws_a, acc[mm][0]), m8[2 * j] * ws_a);
+                    acc[mm][1] = fmaf(s8[2 * j], fmaf(-128.0f, ws_b, acc[mm][1]), m8[2 * j] * ws_b);
+                    acc[mm][2] = fmaf(s8[2 * j + 1], fmaf(-128.0f, ws_a, acc[mm][2]), m8[2 * j + 1] * ws_a);
+                    acc[mm][3] = fmaf(s8[2 * j + 1], fmaf(-128.0f, ws_b, acc[mm][3]), m8[2 * j + 1] * ws_b);
+                }
+            }
+        }
+        __syncthreads();  // every warp is done with the weights; the buffer now takes the warps' sums
+        float tot[kAtHeads * D / kAtThreads];
+#pragma unroll
+        for (int e = 0; e < kAtHeads * D / kAtThreads; ++e) tot[e] = 0.0f;
+        for (int r = 0; r < kAtWarps; r += kBuf) {
+            if (warp >= r && warp < r + kBuf) {
+                float *dst = buf + (size_t)(warp - r) * kAtHeads * D;
+#pragma unroll
+                for (int mm = 0; mm < MT; ++mm) {
+                    const int c = VC * g + 2 * mm;
+                    dst[(2 * t) * D + c] = acc[mm][0];
+                    dst[(2 * t + 1) * D + c] = acc[mm][1];
+                    dst[(2 * t) * D + c + 1] = acc[mm][2];
+                    dst[(2 * t + 1) * D + c + 1] = acc[mm][3];
+                }
+            }
+            __syncthreads();
+#pragma unroll
+            for (int e = 0; e < kAtHeads * D / kAtThreads; ++e) {
+                const int i = e * kAtThreads + tid;  // (head, channel) pair
+                for (int w = 0; w < kBuf && r + w < kAtWarps; ++w) tot[e] += buf[(size_t)w * kAtHeads * D + i];
+            }
+            __syncthreads();
+        }
+        // ---- partial result of this block: (max, sum, weighted sum) per query head
+#pragma unroll
+        for (int e = 0; e < kAtHeads * D / kAtThreads; ++e) {
+            const int i = e * kAtThreads + tid, hh = i / D, c = i - hh * D;
+            if (hh < nh) {
+                float *rec = p.part + ((((int64_t)li * H + h) * n_blocks + bx) * p.rep + h0 + hh) * (D + 2);
+                rec[2 + c] = tot[e];
+                if (c == 0) {
+                    float sum = 0.0f;
+#pragma unroll
+                    for (int w = 0; w < kAtWarps; ++w) sum += seg_sum[w][hh];
+                    rec[0] = blk_max[hh];
+                    rec[1] = sum;
+                }
+            }
+        }
+        __syncthreads();  // qf, buf and the statistics are rewritten by the next chunk of heads
     }
+    attend_merge<CT, D>(p, li, h, n_blocks, &s_last);
 }
 
 static int attend_segments(const stom_oqm_config *cfg, int32_t k, int32_t sys_len, int *n_sys_seg, int *segs_per_group) {
@@ -366,15 +747,15 @@ static int32_t launch_attend(const AttendParams &p, dim3 grid, cudaStream_t s) {
     const bool b4 = p.g.row_bytes * 2 == p.g.d;  // 4-bit codes: d/2 bytes per row
     switch (p.g.d) {
     case 64:
-        if (b4) attend_kernel<QT, CT, 8, 4><<<grid, kAtThreads, 0, s>>>(p);
+        if (b4) attend_mma_kernel<QT, CT, 64><<<grid, kAtThreads, 0, s>>>(p);
         else attend_kernel<QT, CT, 8, 2><<<grid, kAtThreads, 0, s>>>(p);
         break;
     case 128:
-        if (b4) attend_kernel<QT, CT, 16, 4><<<grid, kAtThreads, 0, s>>>(p);
+        if (b4) attend_mma_kernel<QT, CT, 128><<<grid, kAtThreads, 0, s>>>(p);
         else attend_kernel<QT, CT, 16, 2><<<grid, kAtThreads, 0, s>>>(p);
         break;
     case 256:
-        if (b4) attend_kernel<QT, CT, 32, 4><<<grid, kAtThreads, 0, s>>>(p);
+        if (b4) attend_mma_kernel<QT, CT, 256><<<grid, kAtThreads, 0, s>>>(p);
         else attend_kernel<QT, CT, 32, 2><<<grid, kAtThreads, 0, s>>>(p);
         break;
     default: return STOM_ERR_SHAPE;
