@@ -516,7 +516,7 @@ def run_stream(args, sh):
     idx = torch.empty(sh.L, sh.k, dtype=torch.int32, device=dev)
     out = torch.empty(sh.L, sh.H_q, sh.d, dtype=torch.bfloat16, device=dev)
     ws = torch.empty(oqm.stom_oqm_retrieve_workspace_bytes(cfg, sh.L, sh.T, sh.k), dtype=torch.uint8, device=dev)
-    aws = torch.empty(oqm.stom_oqm_attend_workspace_bytes(cfg, sh.L, sh.k, sys_len) + 256, dtype=torch.uint8, device=dev)
+    aws = torch.zeros(oqm.stom_oqm_attend_workspace_bytes(cfg, sh.L, sh.k, sys_len) + 256, dtype=torch.uint8, device=dev)
     aws = aws[(-aws.data_ptr()) % 256:]
     flags = torch.zeros(1, dtype=torch.int32, device=dev)
     scale = float(sh.d) ** -0.5

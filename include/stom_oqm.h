@@ -322,7 +322,14 @@ int32_t stom_oqm_retrieve(const stom_oqm_config *cfg, const stom_oqm_store *stor
  * out (cache_dtype): element (l, h_q, c) at (l-layer_begin)*out_stride_layer +
  *   h_q*out_stride_head + c.
  * workspace: DEVICE, 256-byte aligned, stom_oqm_attend_workspace_bytes() bytes;
- *   holds the partial results of the blocks that share a (layer, kv head).
+ *   holds the partial results of the blocks that share a (layer, kv head) and,
+ *   in its first 4 * n_layers * H_k bytes (rounded up to 256), their ticket
+ *   counters.  Those
+ *   bytes must be ZERO when a call starts: clear the workspace once after
+ *   allocating it (cudaMemsetAsync); every call that completes leaves them
+ *   zero again, so the same workspace serves call after call (one call at a
+ *   time) without further clearing.  Counters that are not zero make the call
+ *   write no output or an incomplete one; nothing waits on them.
  * Errors: INVALID_ARG, SHAPE, UNSUPPORTED, ALIGNMENT, CAPACITY, WORKSPACE, CUDA.
  */
 int64_t stom_oqm_attend_workspace_bytes(const stom_oqm_config *cfg, int32_t layer_count, int32_t k,

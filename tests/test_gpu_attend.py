@@ -85,7 +85,7 @@ def _check_attend(orc, L, H_q, H_k, d, G, T, k, n_sel, sys_len, mode, dtype, cac
     want = np.stack([orc.to_f32(orc.attend(H_q, H_k, d, qn[l], P.dt_code(dtype), oka[l], ova[l], ccode, S * d, d,
                                            n_tok, scale, out_dtype=ccode), ccode) for l in range(L)])
 
-    ws = torch.empty(oqm.stom_oqm_attend_workspace_bytes(gcfg, L, k, sys_len) + 256, dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(oqm.stom_oqm_attend_workspace_bytes(gcfg, L, k, sys_len) + 256, dtype=torch.uint8, device="cuda")
     ws = ws[(-ws.data_ptr()) % 256:]
     out_flat = torch.full((L * H_q * d + P.GUARD,), 3.0, dtype=cdt, device="cuda")
     out = out_flat[:L * H_q * d].view(L, H_q, d)
@@ -110,7 +110,7 @@ def test_attend_flags_bad_indices_and_skips_them(orc):
     sh = synth.Shape("attend-bad", L=1, H_q=4, H_k=2, d=128, G=8, T=12, T_q=1, k=4, seed=3)
     ocfg, gcfg, ost, gst, _ = P.random_bank(orc, oqm, sh, 0, seed=9)
     q = torch.randn(1, 4, 128).to(torch.bfloat16).cuda()
-    ws = torch.empty(oqm.stom_oqm_attend_workspace_bytes(gcfg, 1, 4, 0) + 256, dtype=torch.uint8, device="cuda")
+    ws = torch.zeros(oqm.stom_oqm_attend_workspace_bytes(gcfg, 1, 4, 0) + 256, dtype=torch.uint8, device="cuda")
     ws = ws[(-ws.data_ptr()) % 256:]
     outs = []
     for idx in ([1, 5, 99, -1], [1, 5, -1, -1]):   # 99 is out of range: skipped and flagged
@@ -122,3 +122,36 @@ def test_attend_flags_bad_indices_and_skips_them(orc):
         outs.append((out.clone(), int(flags.item())))
     assert outs[0][1] == oqm.FLAG_BAD_INDEX and outs[1][1] == 0
     assert torch.equal(outs[0][0], outs[1][0])
+
+
+def test_one_cleared_workspace_serves_calls_over_any_layer_range(orc):
+    """The workspace is cleared once; every call leaves its ticket counters at zero, so a call over all layers,
+    calls layer by layer and a call over a sub-range can follow each other and give the same rows."""
+    from paper_2510_18269_b200 import oqm
+    sh = synth.Shape("attend-ws", L=5, H_q=14, H_k=2, d=128, G=50, T=40, T_q=1, k=6, seed=3)
+    ocfg, gcfg, ost, gst, _ = P.random_bank(orc, oqm, sh, 0, seed=23)
+    L, Hq, d, k, sys_len = sh.L, sh.H_q, sh.d, sh.k, 9
+    rng = np.random.default_rng(2)
+    idx = torch.from_numpy(_selection(rng, L, sh.T, k, k)).cuda()
+    g = torch.Generator().manual_seed(8)
+    q = torch.randn(L, Hq, d, generator=g).to(torch.bfloat16).cuda()
+    S = sys_len + k * sh.G
+    ks = torch.randn(L, sh.H_k, S, d, generator=g).to(torch.bfloat16).cuda()
+    vs = torch.randn(L, sh.H_k, S, d, generator=g).to(torch.bfloat16).cuda()
+    ws = torch.zeros(oqm.stom_oqm_attend_workspace_bytes(gcfg, L, k, sys_len) + 256, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 256:]
+    act = P.active_strides(sh, S)
+
+    def run(l0, n):
+        out = torch.zeros(n, Hq, d, dtype=torch.bfloat16, device="cuda")
+        oqm.stom_oqm_attend(gcfg, gst, l0, n, idx[l0:], k, sh.T, q[l0:], (Hq * d, d), ks[l0:], vs[l0:], oqm.BF16, act, sys_len,
+                            d ** -0.5, out, (Hq * d, d), ws)
+        torch.cuda.synchronize()
+        return out
+
+    whole = run(0, L)
+    assert float(whole.float().abs().max()) > 0.05
+    for l in range(L):
+        assert torch.equal(run(l, 1)[0], whole[l])
+    assert torch.equal(run(1, 3), whole[1:4])
+    assert torch.equal(run(0, L), whole)

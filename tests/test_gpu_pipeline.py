@@ -35,7 +35,7 @@ def test_streaming_interleave_matches_oracle(orc):
     sys_k = torch.randn(sh.L, sh.H_k, sys_len, sh.d, generator=gen).to(torch.bfloat16)
     sys_v = torch.randn(sh.L, sh.H_k, sys_len, sh.d, generator=gen).to(torch.bfloat16)
     ws = torch.empty(oqm.stom_oqm_retrieve_workspace_bytes(gcfg, sh.L, sh.T, sh.k), dtype=torch.uint8, device="cuda")
-    aws = torch.empty(oqm.stom_oqm_attend_workspace_bytes(gcfg, sh.L, sh.k, sys_len) + 256, dtype=torch.uint8, device="cuda")
+    aws = torch.zeros(oqm.stom_oqm_attend_workspace_bytes(gcfg, sh.L, sh.k, sys_len) + 256, dtype=torch.uint8, device="cuda")
     aws = aws[(-aws.data_ptr()) % 256:]
     n_questions = 0
     for f in range(sh.T):
@@ -118,7 +118,7 @@ def test_question_sequence_replays_from_a_cuda_graph(orc):
     va = ka.clone()
     out = torch.zeros(sh.L, sh.H_q, sh.d, dtype=torch.bfloat16, device=dev)
     ws = torch.empty(oqm.stom_oqm_retrieve_workspace_bytes(gcfg, sh.L, sh.T, sh.k), dtype=torch.uint8, device=dev)
-    aws = torch.empty(oqm.stom_oqm_attend_workspace_bytes(gcfg, sh.L, sh.k, sys_len) + 256, dtype=torch.uint8, device=dev)
+    aws = torch.zeros(oqm.stom_oqm_attend_workspace_bytes(gcfg, sh.L, sh.k, sys_len) + 256, dtype=torch.uint8, device=dev)
     aws = aws[(-aws.data_ptr()) % 256:]
     flags = torch.zeros(1, dtype=torch.int32, device=dev)
 
