@@ -42,11 +42,11 @@ FALLBACK_HBM_GBS = 6650.0
 NCU_TRAFFIC_PER_UNIT = {
     # all figures are per kv head of the unit named (the captures ran the 4-head 7B geometry)
     "quantize_kernel": 137448.0 / 4,    # bytes per (layer, frame): 3.941 GB over 28 x 1024 units
-    # bytes per (layer, selected group): 186.3 MB over 28 x 64 units; of the 183.5 MB the kernel writes only
-    # 125.7 MB had left L2 when it ended (the rest is written back later), so this undercounts by design
-    "dequant_gather_kernel": 103985.0 / 4,
-    "score_kernel": 2066.0 / 4,         # bytes per (layer, stored group): 59.25 MB over 28 x 1024 units
-    "retrieve_kernel": 2178.0 / 4,      # bytes per (layer, stored group): 62.46 MB over 28 x 1024 units (Q re-read per block)
+    # bytes per (layer, selected group): 186.0 MB over 28 x 64 units; of the 183.5 MB the kernel writes only
+    # 125.4 MB had left L2 when it ended (the rest is written back later), so this undercounts by design
+    "dequant_gather_kernel": 103805.0 / 4,
+    "score_kernel": 2071.0 / 4,         # bytes per (layer, stored group): 59.39 MB over 28 x 1024 units
+    "retrieve_kernel": 2186.0 / 4,      # bytes per (layer, stored group): 62.68 MB over 28 x 1024 units (Q re-read per block)
     # bytes per frame of 196 tokens x 1152 bf16 channels (not per kv head): 561.8 MB over 1200 frames
     "ctr_similarity_kernel": 468181.0,
 }
