@@ -52,21 +52,19 @@ __device__ __forceinline__ uint64_t dq_sub2(uint64_t a, uint64_t b) {
     return d;
 }
 
-// LPR: lanes per token row (d / 8); BITS: width of a code
+// LPR: lanes per token row (d / 8); BITS: width of a code.
+// grid (ceil(4 H / kDqWarps), k, layer_count): a block serves one (layer, slot) and kDqWarps of its 4 H units
+// (kv head x keys|values x first|second half of the rows), so no unit index has to be divided out.
 template <typename OT, int LPR, int BITS>
 __global__ void __launch_bounds__(kDqWarps * 32) dequant_gather_kernel(const DequantParams p) {
     constexpr int RPP = 32 / LPR;          // rows one warp pass covers
     constexpr int kDqMaxRows = 32 / RPP;   // passes that cover half of the largest group (G <= 64)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t unit = (int64_t)blockIdx.x * kDqWarps + warp;
-    if (unit >= p.n_units) return;
     const int G = p.g.G, H = p.g.H, d = p.g.d;
-    const int half = (int)(unit & 1), which = (int)((unit >> 1) & 1);
-    int64_t rest = unit >> 2;
-    const int h = (int)(rest % H);
-    rest /= H;
-    const int j = (int)(rest % p.k);
-    const int li = (int)(rest / p.k);
+    const int u = blockIdx.x * kDqWarps + warp;
+    const int half = u & 1, which = (u >> 1) & 1, h = u >> 2;
+    if (h >= H) return;
+    const int j = blockIdx.y, li = blockIdx.z;
 
     grid_dependency_wait();  // idx may come from the kernel just ahead in the stream
     const int t = p.per_head ? p.idx[((int64_t)li * H + h) * p.k + j] : p.idx[(int64_t)li * p.k + j];
@@ -78,16 +76,15 @@ __global__ void __launch_bounds__(kDqWarps * 32) dequant_gather_kernel(const Deq
     const int sub = lane / LPR;       // which row of a warp pass this lane serves
     const int cl = lane - sub * LPR;  // channel block of this lane
     const int g_half = (G + 1) >> 1;
-    const int r_begin = half ? g_half : 0, r_end = half ? G : g_half;
+    const int r_first = (half ? g_half : 0) + sub, r_end = half ? G : g_half;
+    const int n_mine = r_first < r_end ? (r_end - r_first + RPP - 1) / RPP : 0;  // rows this lane serves
 
     // code words of all this lane's rows first, then the statistics
-    const uint8_t *codes = (which ? p.codes_v : p.codes_k) + slot * (int64_t)G * p.g.row_bytes;
+    const uint8_t *crow = (which ? p.codes_v : p.codes_k) + (slot * G + r_first) * (int64_t)p.g.row_bytes;
+    const int cstep = RPP * p.g.row_bytes;
     uint32_t w[kDqMaxRows];
 #pragma unroll
-    for (int b = 0; b < kDqMaxRows; ++b) {
-        const int r = r_begin + sub + b * RPP;
-        w[b] = r < r_end ? load_codes8<BITS>(codes + (int64_t)r * p.g.row_bytes, cl) : 0u;
-    }
+    for (int b = 0; b < kDqMaxRows; ++b) w[b] = b < n_mine ? load_codes8<BITS>(crow + b * cstep, cl) : 0u;
     uint64_t s2[4], m2[4];
     {
         float sf[8], mf[8];
@@ -100,23 +97,23 @@ __global__ void __launch_bounds__(kDqWarps * 32) dequant_gather_kernel(const Deq
         }
     }
     OT *out = reinterpret_cast<OT *>(which ? p.va : p.ka) + (int64_t)li * p.sl + (int64_t)h * p.sh +
-              ((int64_t)p.token_offset + (int64_t)j * G) * p.st + cl * 8;
+              ((int64_t)p.token_offset + (int64_t)j * G + r_first) * p.st + cl * 8;
+    const int64_t ostep = RPP * p.st;
     const uint64_t two23 = dq_pack(8388608.0f, 8388608.0f);
 #pragma unroll
     for (int b = 0; b < kDqMaxRows; ++b) {
-        const int r = r_begin + sub + b * RPP;
-        if (r < r_end) {
-            uint32_t f[8], o[4];
-            code_floats8<BITS>(w[b], f);
+        if (b >= n_mine) break;
+        uint32_t f[8], o[4];
+        code_floats8<BITS>(w[b], f);
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const uint64_t code = dq_sub2(dq_pack(__uint_as_float(f[2 * i]), __uint_as_float(f[2 * i + 1])), two23);
-                float v0, v1;
-                dq_unpack(dq_fma2(code, s2[i], m2[i]), v0, v1);
-                o[i] = pack2<OT>(v0, v1);
-            }
-            *reinterpret_cast<uint4 *>(out + (int64_t)r * p.st) = make_uint4(o[0], o[1], o[2], o[3]);
+        for (int i = 0; i < 4; ++i) {
+            const uint64_t code = dq_sub2(dq_pack(__uint_as_float(f[2 * i]), __uint_as_float(f[2 * i + 1])), two23);
+            float v0, v1;
+            dq_unpack(dq_fma2(code, s2[i], m2[i]), v0, v1);
+            o[i] = pack2<OT>(v0, v1);
         }
+        *reinterpret_cast<uint4 *>(out) = make_uint4(o[0], o[1], o[2], o[3]);
+        out += ostep;
     }
 }
 
@@ -163,15 +160,15 @@ int32_t stom::dequant_gather_launch(const stom_oqm_config *cfg, const stom_oqm_s
     p.per_head = cfg->score_mode == STOM_SCORE_PER_HEAD;
     p.flags = dev_flags;
     p.n_units = (int64_t)layer_count * k * cfg->n_kv_heads * 4;  // x (keys | values) x (first | second half of the rows)
-    const int64_t blocks = (p.n_units + kDqWarps - 1) / kDqWarps;
-    if (blocks > 0x7fffffffLL) return STOM_ERR_SHAPE;
+    if (k > 65535 || layer_count > 65535) return STOM_ERR_SHAPE;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const unsigned nb = (unsigned)blocks, nt = kDqWarps * 32;
+    const dim3 nb((unsigned)((cfg->n_kv_heads * 4 + kDqWarps - 1) / kDqWarps), (unsigned)k, (unsigned)layer_count);
+    const unsigned nt = kDqWarps * 32;
     const bool bf = out_dtype == STOM_BF16;
     cudaError_t le = cudaSuccess;
 #define STOM_DQ_KERNEL(OT_, LPR_, BITS_)                                                               \
     do {                                                                                               \
-        if (after_producer) le = launch_after_producer(dequant_gather_kernel<OT_, LPR_, BITS_>, dim3(nb), dim3(nt), 0, s, p); \
+        if (after_producer) le = launch_after_producer(dequant_gather_kernel<OT_, LPR_, BITS_>, nb, dim3(nt), 0, s, p); \
         else dequant_gather_kernel<OT_, LPR_, BITS_><<<nb, nt, 0, s>>>(p);                             \
     } while (0)
 #define STOM_DQ_LAUNCH(LPR_)                                                                           \
