@@ -65,15 +65,28 @@ __device__ __forceinline__ void attend_merge(const AttendParams &p, int li, int 
     if (!s_last) return;
     __threadfence();
     if (tid == 0) p.counters[li * H + h] = 0;  // as found
-    // one warp per query head: lanes first share out the blocks (max, then the sum of the weighted sums of
-    // weights), then the channels, with the loads of several blocks in flight
+    // One warp per query head.  Lanes share out the blocks 32 at a time: (max, sum) of a block come in one 8-byte
+    // load; the channel sums of the first kChunk blocks are requested in the same breath, before anything is
+    // reduced, and those of the next chunk while the current one is added up -- the merge is two memory round trips
+    // for up to kChunk blocks and one more per further chunk.
+    constexpr int kChunk = D >= 256 ? 4 : 8;
     for (int hq = warp; hq < p.rep; hq += kAtWarps) {
         const float *rec0 = p.part + (((int64_t)li * H + h) * n_blocks * p.rep + hq) * (D + 2);
         const int64_t step = (int64_t)p.rep * (D + 2);
-        // lanes share out the blocks 32 at a time: their maxima and sums are loaded once, the weight of a block is
-        // then handed round by shuffle while every lane adds up its own channels, 8 blocks' loads in flight
-        float mx = -INFINITY;
-        for (int b = lane; b < n_blocks; b += 32) mx = fmaxf(mx, __ldcg(rec0 + b * step));
+        auto load_chunk = [&](int b0, float (&v)[kChunk][D / 32]) {
+#pragma unroll
+            for (int j = 0; j < kChunk; ++j)
+#pragma unroll
+                for (int i = 0; i < D / 32; ++i)
+                    v[j][i] = b0 + j < n_blocks ? __ldcg(rec0 + (b0 + j) * step + 2 + lane + 32 * i) : 0.0f;
+        };
+        float cur[kChunk][D / 32];
+        load_chunk(0, cur);
+        // the global maximum over all blocks (several trips only beyond 32 blocks)
+        float2 ms = make_float2(-INFINITY, 0.0f);  // of block `lane` of the first trip
+        if (lane < n_blocks) ms = __ldcg(reinterpret_cast<const float2 *>(rec0 + lane * step));
+        float mx = ms.x;
+        for (int b = lane + 32; b < n_blocks; b += 32) mx = fmaxf(mx, __ldcg(rec0 + b * step));
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
         float den = 0.0f;
@@ -81,20 +94,29 @@ __device__ __forceinline__ void attend_merge(const AttendParams &p, int li, int 
 #pragma unroll
         for (int i = 0; i < D / 32; ++i) num[i] = 0.0f;
         for (int b0 = 0; b0 < n_blocks; b0 += 32) {
-            float w_mine = 0.0f;
-            if (b0 + lane < n_blocks) {
-                const float mb = __ldcg(rec0 + (b0 + lane) * step);
-                if (mb != -INFINITY) {
-                    w_mine = exp2f(mb - mx);
-                    den = fmaf(__ldcg(rec0 + (b0 + lane) * step + 1), w_mine, den);
-                }
+            if (b0 > 0) {
+                ms = make_float2(-INFINITY, 0.0f);
+                if (b0 + lane < n_blocks) ms = __ldcg(reinterpret_cast<const float2 *>(rec0 + (b0 + lane) * step));
             }
+            const float w_mine = ms.x == -INFINITY ? 0.0f : exp2f(ms.x - mx);
+            den = fmaf(ms.y, w_mine, den);
             const int nb = min(32, n_blocks - b0);
-#pragma unroll 8
-            for (int j = 0; j < nb; ++j) {
-                const float w = __shfl_sync(0xffffffffu, w_mine, j);
+            for (int c0 = 0; c0 < nb; c0 += kChunk) {
+                float nxt[kChunk][D / 32];
+                const bool more = b0 + c0 + kChunk < n_blocks;
+                if (more) load_chunk(b0 + c0 + kChunk, nxt);
 #pragma unroll
-                for (int i = 0; i < D / 32; ++i) num[i] = fmaf(__ldcg(rec0 + (b0 + j) * step + 2 + lane + 32 * i), w, num[i]);
+                for (int j = 0; j < kChunk; ++j) {
+                    const float w = __shfl_sync(0xffffffffu, w_mine, (c0 + j) & 31);
+#pragma unroll
+                    for (int i = 0; i < D / 32; ++i) num[i] = fmaf(cur[j][i], c0 + j < nb ? w : 0.0f, num[i]);
+                }
+                if (more) {
+#pragma unroll
+                    for (int j = 0; j < kChunk; ++j)
+#pragma unroll
+                        for (int i = 0; i < D / 32; ++i) cur[j][i] = nxt[j][i];
+                }
             }
         }
 #pragma unroll
@@ -428,7 +450,6 @@ __device__ __forceinline__ uint32_t code_pair_bf16(uint32_t x, uint32_t y, int b
     return v | 0x43004300u;
 }
 
-// QT: type of q_dec; CT: type of the system-token cache and of the output; D: head dim
 // Two floats as a (high, low) pair of packed 16-bit pairs: hi = the values rounded to MT, lo = what the rounding
 // left over, rounded again.  A matrix product issued once with each part carries 16 significant bits of the operand.
 template <typename MT>
@@ -442,6 +463,7 @@ __device__ __forceinline__ void split2(float a, float b, uint32_t &hi, uint32_t 
     seen_b = hb + lb;
 }
 
+// QT: type of q_dec; CT: type of the system-token cache and of the output; D: head dim
 template <typename QT, typename CT, int D>
 __global__ void __launch_bounds__(kAtThreads) attend_mma_kernel(const AttendParams p) {
     constexpr int kSlots = kAtWarps * kAtSegTokens;

@@ -241,7 +241,8 @@ def stom_oqm_attend_workspace_bytes(cfg: Config, layer_count: int, k: int, sys_l
 def stom_oqm_attend(cfg: Config, store: Store, layer_begin, layer_count, idx, k, n_groups, q_dec, q_strides,
                     k_sys, v_sys, cache_dtype, sys_strides, sys_len, softmax_scale, out, out_strides, workspace,
                     dev_flags=None, stream=None):
-    """q_strides = (layer, head); sys_strides = (layer, head, token); out_strides = (layer, head), all in elements."""
+    """q_strides = (layer, head); sys_strides = (layer, head, token); out_strides = (layer, head), all in elements.
+    `workspace` (256-byte aligned) must have been zero-filled once after it was allocated; calls leave it reusable."""
     rc = lib().stom_oqm_attend(
         C.byref(cfg), C.byref(store.desc), C.c_int32(layer_begin), C.c_int32(layer_count), _ptr(idx), C.c_int32(k),
         C.c_int32(n_groups), _ptr(q_dec), C.c_int64(q_strides[0]), C.c_int64(q_strides[1]), _ptr(k_sys), _ptr(v_sys),
