@@ -421,6 +421,8 @@ __device__ __forceinline__ void mma_16816<__half>(float (&c)[4], uint32_t a0, ui
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+__device__ __forceinline__ void prefetch_l1(const void *p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
+
 // NW 32-bit words from p (p aligned to min(16, 4 * NW) bytes), or zeros
 template <int NW>
 __device__ __forceinline__ void load_words_or_zero(const void *p, bool valid, uint32_t (&w)[NW]) {
@@ -514,6 +516,28 @@ __global__ void __launch_bounds__(kAtThreads) attend_mma_kernel(const AttendPara
     const uint8_t *kcodes = p.codes_k + slot * (int64_t)G * p.g.row_bytes;
     const uint8_t *vcodes = p.codes_v + slot * (int64_t)G * p.g.row_bytes;
     const int md = p.g.meta_dtype;
+
+    // A decode step is a chain of memory round trips.  Everything a group segment will read depends on the slot
+    // only, not on the query: ask for it now (no registers are tied up), so that it arrives while the query rows are
+    // staged and the loads below find it in L1.
+    if (!is_sys && n_tok > 0) {
+        const int esz = md == STOM_FP32 ? 4 : 2;
+        const int64_t kat = (slot * D + KC * t) * esz, vat = (slot * D + VC * g) * esz;
+        prefetch_l1(static_cast<const uint8_t *>(p.scale_k) + kat);
+        prefetch_l1(static_cast<const uint8_t *>(p.zero_k) + kat);
+        prefetch_l1(static_cast<const uint8_t *>(p.scale_v) + vat);
+        prefetch_l1(static_cast<const uint8_t *>(p.zero_v) + vat);
+#pragma unroll
+        for (int i = 0; i < kAtSegTokens / 8; ++i) {
+            const int row = g + 8 * i;  // the score product reads rows g, g+8, g+16, g+24
+            if (row < n_tok) prefetch_l1(kcodes + (int64_t)(tok0 + row) * p.g.row_bytes + t * (KC / 2));
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int tok = (i >> 2) * 16 + 2 * t + (i & 1) + 8 * ((i >> 1) & 1);  // the value product's tokens
+            if (tok < n_tok) prefetch_l1(vcodes + (int64_t)(tok0 + tok) * p.g.row_bytes + g * (VC / 2));
+        }
+    }
 
     const int n_blocks = gridDim.x;
     for (int h0 = 0; h0 < p.rep; h0 += kAtHeads) {
