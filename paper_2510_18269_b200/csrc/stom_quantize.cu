@@ -91,6 +91,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// the same question without waiting at all: has the phase with this parity completed?
+__device__ __forceinline__ bool mbar_test(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 __device__ __forceinline__ unsigned long long global_ns() {
     unsigned long long t;
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
@@ -366,7 +378,7 @@ __device__ __forceinline__ TileCoord tile_coord(uint32_t tau, const QuantParams 
 struct SlotInfo {
     int64_t bslot;  // index of (layer, group, head) in the bank
     int32_t kind;   // 0 keys, 1 values, 2 pre-rotary keys
-    int32_t pad;
+    int32_t round;  // fill number of the slot's latest fill, -1 before the first (read by the producer's final drain)
 };
 
 // shared memory: [full[2][kMaxSlots], empty[kMaxSlots]] [abort words] [SlotInfo[kMaxSlots]] [ring of input slots]
@@ -395,9 +407,9 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
     // Tile n of the block goes to ring slot n % N and to consumer warp n % n_warps.  A slot has TWO "full" barriers
     // used by alternate fills: a waiter only tells a barrier's phases apart by one parity bit, and with a single
     // barrier a warp that runs ahead could take fill k-1 of its slot, still on its way, for fill k.  With two, the
-    // fill it could be confused with is k-2, which lies at least N tiles behind the oldest unfinished tile of the
-    // block once n_warps <= N, so it has long completed.  The producer waits on "empty" phases strictly in order,
-    // so one barrier per slot is enough there.
+    // fill it could be confused with is k-2; the consumer rules that out by the fill number the producer publishes
+    // in the slot's info record before it starts a copy (see the consumers' wait).  The fills of ONE slot are issued
+    // in order and each waits for the release of the one before, so one "empty" barrier per slot is enough.
     const uint32_t WA = (uint32_t)p.n_warps;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -409,6 +421,7 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
             mbar_init(full0 + 8 * i, 1);
             mbar_init(full0 + 8 * (kMaxSlots + i), 1);
             mbar_init(empty0 + 8 * i, 1);
+            info[i].round = -1;
         }
         abort_flag[0] = 0;  // set by the first thread whose wait ran out
         abort_flag[1] = 0;  // never set: lets the final drain wait regardless of an abort
@@ -421,49 +434,107 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
 
     if (warp == kConsumerWarps) {
         // =============================================================== producer
-        // Tile coordinates cost a few integer divisions.  One warp doing them tile after tile would cap the block
-        // at about one tile per thousand cycles, so the 32 lanes work out 32 consecutive tiles at once and hand
-        // the results round by shuffle.
-        uint32_t issued = 0;
-        int slot = 0;
-        uint32_t round = 0;  // fill number of `slot`
         bool stop = false;
-        for (uint32_t n0 = 0; n0 < my_count && !stop; n0 += 32) {
-            const uint32_t mine = n0 + lane < my_count ? n0 + lane : my_count - 1;
-            const TileCoord tl = tile_coord(blockIdx.x + mine * gridDim.x, p);
-            const unsigned long long src_l = reinterpret_cast<unsigned long long>(
-                reinterpret_cast<const T *>(tl.kind == 0 ? p.K : (tl.kind == 1 ? p.V : p.Ksum)) +
-                (int64_t)tl.li * p.sl + (int64_t)tl.f * p.sg + (int64_t)tl.h * p.sh);
-            const long long bslot_l = bank_slot(p.g, p.layer_begin + tl.li, p.group_begin + tl.f, tl.h);
-            const int cnt = (int)(my_count - n0 < 32u ? my_count - n0 : 32u);
-            for (int i = 0; i < cnt; ++i) {
-                const uint32_t n = n0 + i;
-                bool ok = true;
-                if (round > 0) ok = mbar_wait(empty0 + 8 * slot, (round - 1) & 1u, abort_flag);
-                ok = __all_sync(0xffffffffu, ok && !*abort_flag);  // the whole warp stops together
-                if (!ok) {
-                    if (lane == 0) {
-                        if (!*abort_flag && p.flags) atomicOr(p.flags, STOM_FLAG_TIMEOUT);
-                        *abort_flag = 1;
+        if (p.contiguous) {
+            // One bulk copy per tile.  Issued tile by tile by one thread, a tile cost the warp about 500 cycles of
+            // dependent instructions (wait, publish, expect, copy) and the whole block no more than one tile per
+            // 0.3 us, whatever the consumers did.  So a group of up to N consecutive tiles -- N ring slots, each
+            // slot at most once -- is handled by N lanes at once: every lane polls (without blocking) whether its
+            // own slot has been released and fills it the moment it has, in whatever order the slots come free.
+            // Groups follow one another, so the fills of one slot are still issued in order; what is lost is the
+            // order BETWEEN slots, which the consumers make up for (see their wait).
+            int slot0 = 0;        // slot of the group's first tile
+            uint32_t round0 = 0;  // and its fill number
+            for (uint32_t n0 = 0; n0 < my_count && !stop; n0 += (uint32_t)N) {
+                const int cnt = (int)(my_count - n0 < (uint32_t)N ? my_count - n0 : (uint32_t)N);
+                bool pending = lane < cnt;
+                int my_slot = slot0 + lane;
+                uint32_t my_round = round0;
+                if (my_slot >= N) {
+                    my_slot -= N;
+                    ++my_round;
+                }
+                TileCoord tl = {0, 0, 0, 0};
+                const T *src = nullptr;
+                int64_t bslot = 0;
+                if (pending) {
+                    tl = tile_coord(blockIdx.x + (n0 + lane) * gridDim.x, p);
+                    src = reinterpret_cast<const T *>(tl.kind == 0 ? p.K : (tl.kind == 1 ? p.V : p.Ksum)) +
+                          (int64_t)tl.li * p.sl + (int64_t)tl.f * p.sg + (int64_t)tl.h * p.sh;
+                    bslot = bank_slot(p.g, p.layer_begin + tl.li, p.group_begin + tl.f, tl.h);
+                }
+                unsigned long long t0 = 0;
+                for (uint32_t spin = 0;; ++spin) {
+                    if (pending && (my_round == 0 || mbar_test(empty0 + 8 * my_slot, (my_round - 1) & 1u))) {
+                        info[my_slot].bslot = bslot;  // published by the release of the arrive below
+                        info[my_slot].kind = tl.kind;
+                        info[my_slot].round = (int32_t)my_round;
+                        const uint32_t bar = full_bar(my_slot, my_round);
+                        mbar_expect_tx(bar, tile_bytes);
+                        bulk_load(smem_u32(ring + (size_t)my_slot * p.slot_bytes), src, tile_bytes, bar);
+                        pending = false;
                     }
-                    stop = true;
-                    break;
+                    if (!__any_sync(0xffffffffu, pending)) break;
+#ifdef QSLEEP
+                    __nanosleep(QSLEEP);
+#endif
+                    if ((spin & 63u) == 63u) {  // bounded: a slot that never comes free ends the block
+                        if (t0 == 0) t0 = global_ns();
+                        if (__any_sync(0xffffffffu, *abort_flag || global_ns() - t0 > kWaitLimitNs)) {
+                            if (lane == 0) {
+                                if (!*abort_flag && p.flags) atomicOr(p.flags, STOM_FLAG_TIMEOUT);
+                                *abort_flag = 1;
+                            }
+                            stop = true;
+                            break;
+                        }
+                    }
                 }
-                const T *src = reinterpret_cast<const T *>(__shfl_sync(0xffffffffu, src_l, i));
-                const long long bslot = __shfl_sync(0xffffffffu, bslot_l, i);
-                const int kind = __shfl_sync(0xffffffffu, tl.kind, i);
-                const int f = __shfl_sync(0xffffffffu, tl.f, i);
-                const uint32_t bar = full_bar(slot, round);
-                const uint32_t dst = smem_u32(ring + (size_t)slot * p.slot_bytes);
-                if (lane == 0) {
-                    info[slot].bslot = bslot;  // published by the release of the arrive below
-                    info[slot].kind = kind;
-                    mbar_expect_tx(bar, tile_bytes);
+                slot0 += cnt;
+                if (slot0 >= N) {
+                    slot0 -= N;
+                    ++round0;
                 }
-                __syncwarp();
-                if (p.contiguous) {
-                    if (lane == 0) bulk_load(dst, src, tile_bytes, bar);
-                } else {
+            }
+        } else {
+            // Rows of a tile are strided or picked by token_idx: one bulk copy per row, the warp's lanes sharing out
+            // the rows of one tile at a time.  Tile coordinates cost a few integer divisions, so the 32 lanes work
+            // out 32 consecutive tiles at once and hand the results round by shuffle.
+            int slot = 0;
+            uint32_t round = 0;  // fill number of `slot`
+            for (uint32_t n0 = 0; n0 < my_count && !stop; n0 += 32) {
+                const uint32_t mine = n0 + lane < my_count ? n0 + lane : my_count - 1;
+                const TileCoord tl = tile_coord(blockIdx.x + mine * gridDim.x, p);
+                const unsigned long long src_l = reinterpret_cast<unsigned long long>(
+                    reinterpret_cast<const T *>(tl.kind == 0 ? p.K : (tl.kind == 1 ? p.V : p.Ksum)) +
+                    (int64_t)tl.li * p.sl + (int64_t)tl.f * p.sg + (int64_t)tl.h * p.sh);
+                const long long bslot_l = bank_slot(p.g, p.layer_begin + tl.li, p.group_begin + tl.f, tl.h);
+                const int cnt = (int)(my_count - n0 < 32u ? my_count - n0 : 32u);
+                for (int i = 0; i < cnt; ++i) {
+                    bool ok = true;
+                    if (round > 0) ok = mbar_wait(empty0 + 8 * slot, (round - 1) & 1u, abort_flag);
+                    ok = __all_sync(0xffffffffu, ok && !*abort_flag);  // the whole warp stops together
+                    if (!ok) {
+                        if (lane == 0) {
+                            if (!*abort_flag && p.flags) atomicOr(p.flags, STOM_FLAG_TIMEOUT);
+                            *abort_flag = 1;
+                        }
+                        stop = true;
+                        break;
+                    }
+                    const T *src = reinterpret_cast<const T *>(__shfl_sync(0xffffffffu, src_l, i));
+                    const long long bslot = __shfl_sync(0xffffffffu, bslot_l, i);
+                    const int kind = __shfl_sync(0xffffffffu, tl.kind, i);
+                    const int f = __shfl_sync(0xffffffffu, tl.f, i);
+                    const uint32_t bar = full_bar(slot, round);
+                    const uint32_t dst = smem_u32(ring + (size_t)slot * p.slot_bytes);
+                    if (lane == 0) {
+                        info[slot].bslot = bslot;  // published by the release of the arrive below
+                        info[slot].kind = kind;
+                        info[slot].round = (int32_t)round;
+                        mbar_expect_tx(bar, tile_bytes);
+                    }
+                    __syncwarp();
                     for (int r = lane; r < G; r += 32) {
                         int tok = r;
                         if (p.token_idx) {
@@ -473,20 +544,20 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
                         }
                         bulk_load(dst + (uint32_t)r * ROW_BYTES, src + (int64_t)tok * p.st, ROW_BYTES, bar);
                     }
-                }
-                issued = n + 1;
-                if (++slot == N) {
-                    slot = 0;
-                    ++round;
+                    if (++slot == N) {
+                        slot = 0;
+                        ++round;
+                    }
                 }
             }
         }
-        // nothing may still be landing in this block's shared memory when it exits: on the regular path every
-        // fill has been consumed already and these waits return at once
-        const uint32_t first = issued > (uint32_t)N ? issued - (uint32_t)N : 0u;
-        for (uint32_t n = first; n < issued; ++n) {
-            const uint32_t rnd = n / (uint32_t)N;
-            mbar_wait(full_bar((int)(n % (uint32_t)N), rnd), (rnd >> 1) & 1u, abort_flag + 1);
+        // nothing may still be landing in this block's shared memory when it exits: lane s looks after slot s and
+        // waits for its latest fill.  On the regular path every fill has been consumed already and these waits
+        // return at once.
+        __syncwarp();
+        if (lane < N) {
+            const int32_t r = info[lane].round;
+            if (r >= 0) mbar_wait(full_bar(lane, (uint32_t)r), ((uint32_t)r >> 1) & 1u, abort_flag + 1);
         }
         return;
     }
@@ -496,7 +567,26 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
     int slot = warp;       // n_warps <= N
     uint32_t round = 0;    // fill number of `slot` that holds tile n
     for (uint32_t n = warp; n < my_count; n += WA) {
-        bool ok = mbar_wait(full_bar(slot, round), (round >> 1) & 1u, abort_flag);
+        // A parity wait cannot tell the fill it is waiting for from the fill two rounds back on the same barrier,
+        // and the producer fills the slots of a group in whatever order they come free, so that older fill may
+        // still be on its way when this warp gets here.  The producer publishes the fill number of a slot before it
+        // starts the copy; a wait that returns while that number is not ours answered for the older fill: wait on.
+        bool ok;
+        {
+            unsigned long long t0 = 0;
+            for (uint32_t spin = 0;; ++spin) {
+                ok = mbar_wait(full_bar(slot, round), (round >> 1) & 1u, abort_flag);
+                if (!ok || *reinterpret_cast<volatile int32_t *>(&info[slot].round) == (int32_t)round) break;
+                __nanosleep(64);
+                if ((spin & 63u) == 63u) {
+                    if (t0 == 0) t0 = global_ns();
+                    if (*abort_flag || global_ns() - t0 > kWaitLimitNs) {
+                        ok = false;
+                        break;
+                    }
+                }
+            }
+        }
         ok = __all_sync(0xffffffffu, ok && !*abort_flag);  // the whole warp stops together
         if (!ok) {
             if (lane == 0) {
