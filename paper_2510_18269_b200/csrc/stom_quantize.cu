@@ -5,14 +5,17 @@
 // of V (12.8 KB at G = 50, d = 128, bf16).  The kernel is persistent: one
 // block per SM, up to kConsumerWarps consumer warps and one producer warp.
 //
-//   producer  walks the block's tiles in order and, for each, issues bulk
-//             asynchronous copies (cp.async.bulk, completion counted on an
-//             mbarrier) from global memory into the next free slot of a ring
-//             of shared-memory slots that fills the SM's shared memory (18
-//             slots at 12.8 KB); a tile whose rows are contiguous is one
-//             copy, a strided or index-gathered tile is one copy per row.
-//             Whatever is not being read by a consumer is in flight, which
-//             is what hides HBM latency; no register is tied up by a load.
+//   producer  walks the block's tiles and, for each, issues bulk asynchronous
+//             copies (cp.async.bulk, completion counted on an mbarrier) from
+//             global memory into a ring of shared-memory slots that fills
+//             the SM's shared memory (18 slots at 12.8 KB): tile n goes to
+//             slot n % N.  A tile whose rows are contiguous is one copy, and
+//             the lanes of the warp each look after one slot of a group of N
+//             consecutive tiles, filling it the moment its consumer lets go;
+//             a strided or index-gathered tile is one copy per row, issued
+//             by the whole warp tile after tile.  Whatever is not being read
+//             by a consumer is in flight, which is what hides HBM latency;
+//             no register is tied up by a load.
 //   consumer  warp w takes every n_warps-th tile of the block outright.
 //             A lane owns d/32 adjacent channels of ALL G rows, so the
 //             per-channel statistics need no cross-lane traffic at all:
