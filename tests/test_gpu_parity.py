@@ -342,3 +342,22 @@ def test_retrieve_convenience_call_matches_the_three_calls(orc, oqm):
     P.compare_topk(idx_b, idx_a.view(sh.L, sh.k).cpu().numpy(), sc_a.view(sh.L, sh.T).cpu().numpy(), sh.k)
     if torch.equal(idx_a, idx_b):
         assert torch.equal(ka_a, ka_b) and torch.equal(va_a, va_b)
+
+
+@pytest.mark.parametrize("G,d,H_k,T,dtype", [(8, 64, 2, 3000, "bf16"), (25, 128, 4, 900, "bf16"), (3, 128, 1, 5000, "fp16")])
+def test_many_small_tiles_wrap_the_ring_many_times(orc, oqm, G, d, H_k, T, dtype):
+    """Small groups make the consumers fast and the producer the slow side, and every block's ring of shared-memory
+    slots is refilled dozens of times: the bank must equal the oracle's for the whole stream, must not depend on how
+    the stream is cut into calls (another tile -> slot mapping), and must come out the same twice."""
+    sh = synth.Shape("ring", L=2, H_q=2 * H_k, H_k=H_k, d=d, G=G, T=T, T_q=1, k=4, dtype=dtype, seed=900 + G)
+    K, V = synth.kv_stream(sh)
+    gst, ost, gcfg, ocfg = _quantize_both(orc, oqm, sh, K, V)
+    P.compare_store(gst, ost, _keys_f32(orc, sh, K))
+    again, _, _, _ = _quantize_both(orc, oqm, sh, K, V, frames_per_call=997)
+    for name in ("codes_k", "codes_v", "scale_k", "zero_k", "scale_v", "zero_v", "rep_key", "rep_norm2"):
+        assert torch.equal(getattr(gst, name), getattr(again, name)), f"{name} depends on how the stream was cut"
+    twice = oqm.Store(gcfg)
+    Kd, Vd = K.cuda(), V.cuda()
+    oqm.stom_oqm_quantize_frame(gcfg, twice, 0, sh.L, 0, sh.T, Kd, Vd, P.contiguous_strides(sh, sh.G))
+    torch.cuda.synchronize()
+    assert torch.equal(twice.codes_k, gst.codes_k) and torch.equal(twice.codes_v, gst.codes_v)
