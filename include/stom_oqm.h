@@ -63,6 +63,8 @@ extern "C" {
 /* bits of dev_flags set by kernels */
 #define STOM_FLAG_BAD_INDEX 1u /* an entry of idx was < -1 or >= n_groups and was skipped */
 #define STOM_FLAG_TIMEOUT 2u   /* a bounded wait inside a kernel ran out; the call's outputs are incomplete */
+#define STOM_FLAG_DIRTY_WORKSPACE 4u /* stom_oqm_attend found a ticket counter that cannot follow from a cleared
+                                        workspace: the workspace was not zero-filled; outputs are missing */
 
 /* Geometry of one memory bank (paper notation: L, H_q, H_k, d, G). */
 typedef struct stom_oqm_config {
@@ -329,7 +331,8 @@ int32_t stom_oqm_retrieve(const stom_oqm_config *cfg, const stom_oqm_store *stor
  *   allocating it (cudaMemsetAsync); every call that completes leaves them
  *   zero again, so the same workspace serves call after call (one call at a
  *   time) without further clearing.  Counters that are not zero make the call
- *   write no output or an incomplete one; nothing waits on them.
+ *   write no output or an incomplete one; nothing waits on them, and a counter
+ *   beyond the number of blocks sets STOM_FLAG_DIRTY_WORKSPACE in dev_flags.
  * Errors: INVALID_ARG, SHAPE, UNSUPPORTED, ALIGNMENT, CAPACITY, WORKSPACE, CUDA.
  */
 int64_t stom_oqm_attend_workspace_bytes(const stom_oqm_config *cfg, int32_t layer_count, int32_t k,

@@ -60,7 +60,12 @@ __device__ __forceinline__ void attend_merge(const AttendParams &p, int li, int 
     int &s_last = *s_last_ptr;
     __threadfence();
     __syncthreads();
-    if (tid == 0) s_last = atomicAdd(&p.counters[li * H + h], 1u) == (unsigned)n_blocks - 1;
+    if (tid == 0) {
+        const unsigned ticket = atomicAdd(&p.counters[li * H + h], 1u);
+        // tickets of a cleared workspace run from 0 to n_blocks - 1; anything else was there before the call
+        if (ticket >= (unsigned)n_blocks && p.flags) atomicOr(p.flags, STOM_FLAG_DIRTY_WORKSPACE);
+        s_last = ticket == (unsigned)n_blocks - 1;
+    }
     __syncthreads();
     if (!s_last) return;
     __threadfence();

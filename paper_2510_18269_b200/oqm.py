@@ -17,6 +17,8 @@ LIB_PATH = _PKG / "libstom_oqm.so"
 BF16, FP16, FP32 = 0, 1, 2
 PER_LAYER, PER_HEAD = 0, 1
 FLAG_BAD_INDEX = 1
+FLAG_TIMEOUT = 2
+FLAG_DIRTY_WORKSPACE = 4
 
 _TORCH_DTYPE = {BF16: torch.bfloat16, FP16: torch.float16, FP32: torch.float32}
 _DTYPE_CODE = {v: k for k, v in _TORCH_DTYPE.items()}

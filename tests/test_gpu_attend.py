@@ -155,3 +155,31 @@ def test_one_cleared_workspace_serves_calls_over_any_layer_range(orc):
         assert torch.equal(run(l, 1)[0], whole[l])
     assert torch.equal(run(1, 3), whole[1:4])
     assert torch.equal(run(0, L), whole)
+
+
+def test_workspace_that_was_never_cleared_is_flagged(orc):
+    """The ticket counters must be zero on entry.  A workspace full of other bytes cannot give a valid ticket: the
+    call says so in dev_flags instead of returning rows that look plausible; after clearing, the same workspace works."""
+    from paper_2510_18269_b200 import oqm
+    sh = synth.Shape("attend-dirty", L=2, H_q=8, H_k=2, d=128, G=16, T=20, T_q=1, k=5, seed=3)
+    ocfg, gcfg, ost, gst, _ = P.random_bank(orc, oqm, sh, 0, seed=31)
+    idx = torch.from_numpy(_selection(np.random.default_rng(4), sh.L, sh.T, sh.k, sh.k)).cuda()
+    q = torch.randn(sh.L, sh.H_q, sh.d).to(torch.bfloat16).cuda()
+    ws = torch.full((oqm.stom_oqm_attend_workspace_bytes(gcfg, sh.L, sh.k, 0) + 256,), 0xAB, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 256:]
+
+    def run():
+        out = torch.zeros(sh.L, sh.H_q, sh.d, dtype=torch.bfloat16, device="cuda")
+        flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+        oqm.stom_oqm_attend(gcfg, gst, 0, sh.L, idx, sh.k, sh.T, q, (sh.H_q * sh.d, sh.d), None, None, oqm.BF16,
+                            (0, 0, sh.d), 0, 0.09, out, (sh.H_q * sh.d, sh.d), ws, dev_flags=flags)
+        torch.cuda.synchronize()
+        return out, int(flags.item())
+
+    _, flags = run()
+    assert flags & oqm.FLAG_DIRTY_WORKSPACE
+    ws.zero_()
+    out, flags = run()
+    assert flags == 0 and float(out.float().abs().max()) > 0.01
+    again, flags = run()
+    assert flags == 0 and torch.equal(out, again)
