@@ -30,7 +30,7 @@ struct TopkParams {
 // Scratch of one block-wide selection.
 struct TopkSmem {
     uint32_t hist[256];
-    uint32_t s_prefix, s_need;
+    uint32_t s_prefix, s_need, s_done;
     uint32_t warp_gt[32], warp_eq[32];
 };
 
@@ -42,7 +42,7 @@ template <int NT, int MODE>
 __device__ __forceinline__ void block_topk(const float *sc, int n, int k, int32_t *idx_out, float *score_out,
                                            int32_t *n_sel_out, uint32_t *skeys, TopkSmem &sm) {
     uint32_t(&hist)[256] = sm.hist;
-    uint32_t &s_prefix = sm.s_prefix, &s_need = sm.s_need;
+    uint32_t &s_prefix = sm.s_prefix, &s_need = sm.s_need, &s_done = sm.s_done;
     uint32_t(&warp_gt)[32] = sm.warp_gt, (&warp_eq)[32] = sm.warp_eq;
     constexpr int kTopkThreads = NT;
     const int tid = threadIdx.x;
@@ -90,8 +90,10 @@ __device__ __forceinline__ void block_topk(const float *sc, int n, int k, int32_
         }
     };
 
-    // ---- radix select of the ksel-th largest key: 4 passes of 8 bits.  The bin in which the running count from the
-    //      top reaches `need` is found by one warp: a lane owns 8 bins, suffix sums go round by shuffle.
+    // ---- radix select of the ksel-th largest key: up to 4 passes of 8 bits.  The bin in which the running count from
+    //      the top reaches `need` is found by one warp: a lane owns 8 bins, suffix sums go round by shuffle.  The
+    //      passes stop as soon as that bin has exactly as many keys as are still needed: all of them are taken, so
+    //      their lower bits no longer matter (with well-spread scores that is after two passes).
     uint32_t prefix = 0, mask = 0, need = (uint32_t)ksel;
     for (int shift = 24; shift >= 0; shift -= 8) {
         if (tid < 256) hist[tid] = 0;
@@ -123,20 +125,23 @@ __device__ __forceinline__ void block_topk(const float *sc, int n, int k, int32_
                 }
                 s_prefix = prefix | ((uint32_t)(tid * 8 + j) << shift);
                 s_need = left;
+                s_done = c[j] == left;
             }
         }
         __syncthreads();
         prefix = s_prefix;
         need = s_need;
         mask |= 255u << shift;
+        if (s_done) break;  // block-uniform
     }
-    const uint32_t kth = prefix;  // exact key of the ksel-th largest; `need` of the elements equal to it are taken
+    // keys whose bits under `mask` exceed `prefix` are taken; of those that equal it, the first `need` in index order
+    // (after all four passes `prefix` is the exact key of the ksel-th largest)
 
     // ---- ordered compaction over the threads' contiguous ranges
     uint32_t gt = 0, eq = 0;
     for_my_keys([&](int, uint32_t key) {
-        gt += key > kth;
-        eq += key == kth;
+        gt += (key & mask) > prefix;
+        eq += (key & mask) == prefix;
     });
     // exclusive prefix sums of (gt, eq) over threads: warp scan, then scan of warp totals
     const int lane = tid & 31, warp = tid >> 5;
@@ -174,14 +179,14 @@ __device__ __forceinline__ void block_topk(const float *sc, int n, int k, int32_
     uint32_t gt_before = warp_gt[warp] + igt - gt;
     uint32_t eq_before = warp_eq[warp] + ieq - eq;
     for_my_keys([&](int i, uint32_t key) {
-        const bool take = key > kth || (key == kth && eq_before < need);
+        const bool take = (key & mask) > prefix || ((key & mask) == prefix && eq_before < need);
         if (take) {
             const uint32_t pos = gt_before + min(eq_before, need);
             idx_out[pos] = i;
             if (score_out) score_out[pos] = __ldcg(sc + i);
         }
-        gt_before += key > kth;
-        eq_before += key == kth;
+        gt_before += (key & mask) > prefix;
+        eq_before += (key & mask) == prefix;
     });
 }
 
