@@ -107,29 +107,47 @@ __device__ __forceinline__ void embed_layer(const ScoreParams &p, int li, float 
 #pragma unroll
             for (int c = 0; c < 8; ++c) acc[c] = 0.0f;
         };
+        // The walk i = 0 .. n_i-1 visits (head hh of the group, k-th row of this slot in that head); the row is
+        // r = rs + k * RG = query head hr of the GQA block, token j.  All four are stepped, never divided out: an
+        // integer division per load was a third of this prologue's instructions.
+        const int hr0 = rs / p.T_q, j0 = rs - hr0 * p.T_q;
+        int l_hh = 0, l_k = 0, l_hr = hr0, l_j = j0;  // state of the loading walk
+        int a_hh = 0, a_k = 0;                        // state of the adding walk
         for (int i0 = 0; i0 < n_i; i0 += kInFlight) {
             QRow<T> x[kInFlight];
 #pragma unroll
             for (int b = 0; b < kInFlight; ++b) {
-                const int i = i0 + b;
-                const int hh = i / per_head, r = rs + (i - hh * per_head) * RG;
 #pragma unroll
                 for (int j = 0; j < QRow<T>::W; ++j) x[b].w[j] = 0u;  // +0.0 in every format
-                if (i < n_i && r < rows) {
-                    const int hr = r / p.T_q, j = r - hr * p.T_q;
-                    x[b].load(qbase + (int64_t)((h0 + hh) * p.rep + hr) * p.qh + (int64_t)j * p.qt);
+                if (i0 + b < n_i) {
+                    if (rs + l_k * RG < rows)
+                        x[b].load(qbase + (int64_t)((h0 + l_hh) * p.rep + l_hr) * p.qh + (int64_t)l_j * p.qt);
+                    if (++l_k == per_head) {  // next head of the group: back to the slot's first row
+                        l_k = 0;
+                        ++l_hh;
+                        l_hr = hr0;
+                        l_j = j0;
+                    } else {
+                        l_j += RG;
+                        while (l_j >= p.T_q) {
+                            l_j -= p.T_q;
+                            ++l_hr;
+                        }
+                    }
                 }
             }
 #pragma unroll
             for (int b = 0; b < kInFlight; ++b) {
-                const int i = i0 + b;
-                if (i < n_i) {
-                    const int hh = i / per_head;
-                    if (hh != cur) {
+                if (i0 + b < n_i) {
+                    if (a_hh != cur) {
                         flush(cur);
-                        cur = hh;
+                        cur = a_hh;
                     }
                     x[b].add_to(acc);
+                    if (++a_k == per_head) {
+                        a_k = 0;
+                        ++a_hh;
+                    }
                 }
             }
         }
