@@ -35,13 +35,16 @@
 // Bit-exactness of the codes: the contract is code = rne(fl((x - m) / s)) in
 // binary32 with a true division.  A hardware-exact division per element would
 // make the kernel instruction-bound, so the quotient is formed with the
-// correctly rounded reciprocal y = rn(1/s) and two residual corrections
-//     q0 = rn(diff*y); e = rn(diff - q0*s); q1 = rn(q0 + e*y);
-//     e = rn(diff - q1*s); q2 = rn(q1 + e*y)
-// (q1 is a faithful quotient, and a faithful quotient corrected once more with
-// an exact FMA residual and a correctly rounded reciprocal is the correctly
-// rounded quotient -- Markstein's division theorem), followed by the
-// add-magic-constant trick for round-half-even.  Tiles with a channel whose
+// correctly rounded reciprocal y = rn(1/s), its remainder y_lo = rn(1/s - y)
+// (both per channel, once per tile) and one residual correction
+//     q0 = rn(diff*y + rn(diff*y_lo)); e = rn(diff - q0*s); q1 = rn(q0 + e*y)
+// (y + y_lo carries 1/s to about 47 bits, so q0 is within half an ulp of the
+// quotient up to 2^-22 ulp: a faithful quotient; and a faithful quotient
+// corrected once with an exact FMA residual and a correctly rounded reciprocal
+// is the correctly rounded quotient -- Markstein's division theorem), followed
+// by the add-magic-constant trick for round-half-even.  That is six packed
+// operations per pair of channels; starting from rn(diff*y) alone, which is
+// not always faithful, took two corrections and seven.  Tiles with a channel whose
 // scale is zero or outside (2^-60, 2^60) take a slow path with the IEEE division.
 #include "stom_internal.cuh"
 
@@ -202,14 +205,15 @@ __device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
     return d;
 }
 
-// Two adjacent channels at once: x - m, the doubly corrected quotient, the rounding add.  Returns the two
-// floats 1.5*2^23 + code as a pair.
-__device__ __forceinline__ uint64_t code_pair(uint64_t x, uint64_t m, uint64_t neg_s, uint64_t y, uint64_t magic) {
+// Two adjacent channels at once: x - m, the correctly rounded quotient, the rounding add.  Returns the two floats
+// 1.5*2^23 + code as a pair.  y = rn(1/s) and y_lo = rn(1/s - y) together carry 1/s to about 47 bits, so
+// q0 = rn(diff*y + rn(diff*y_lo)) is within 0.5 ulp (plus 2^-22 ulp) of diff/s: a faithful quotient, which one
+// correction with the exact FMA residual turns into the correctly rounded one.
+__device__ __forceinline__ uint64_t code_pair(uint64_t x, uint64_t m, uint64_t neg_s, uint64_t y, uint64_t y_lo,
+                                              uint64_t magic) {
     const uint64_t diff = sub2(x, m);
-    uint64_t q = mul2(diff, y);
-    uint64_t e = fma2(q, neg_s, diff);
-    q = fma2(e, y, q);
-    e = fma2(q, neg_s, diff);
+    uint64_t q = fma2(diff, y, mul2(diff, y_lo));
+    const uint64_t e = fma2(q, neg_s, diff);
     q = fma2(e, y, q);
     return add2(q, magic);
 }
@@ -316,7 +320,8 @@ __device__ __forceinline__ void store_codes(unsigned char *dst, uint32_t cw, int
 template <typename T, int C, int BITS, bool SUM>
 __device__ __forceinline__ void code_rows(const unsigned char *tile, unsigned char *out_lane, int G, int lane,
                                           const uint64_t (&m2)[C / 2], const uint64_t (&ns2)[C / 2],
-                                          const uint64_t (&y2)[C / 2], uint64_t (&sum2)[C / 2]) {
+                                          const uint64_t (&y2)[C / 2], const uint64_t (&yl2)[C / 2],
+                                          uint64_t (&sum2)[C / 2]) {
     constexpr int ROW_BYTES = 32 * C * (int)sizeof(T), CODE_ROW = 4 * C * BITS;
     const uint64_t magic = pack_f2(12582912.0f, 12582912.0f);  // 1.5 * 2^23: rounds to integer, ties to even
     // every float 1.5*2^23 + code has the bit pattern 0x4B400000 + code; summing pattern << (BITS * channel) over
@@ -331,7 +336,7 @@ __device__ __forceinline__ void code_rows(const unsigned char *tile, unsigned ch
             row.pair(j, x0, x1);
             const uint64_t x = pack_f2(x0, x1);
             if constexpr (SUM) sum2[j] = add2(sum2[j], x);
-            const uint64_t u = code_pair(x, m2[j], ns2[j], y2[j], magic);
+            const uint64_t u = code_pair(x, m2[j], ns2[j], y2[j], yl2[j], magic);
             float u0, u1;
             unpack_f2(u, u0, u1);
             cw += __float_as_uint(u0) << (2 * BITS * j);
@@ -665,15 +670,18 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
 
             // ---- pass 2: codes (and, for keys, the channel sums of the rows as a by-product)
             if (safe) {
-                uint64_t m2[C / 2], ns2[C / 2], y2[C / 2];
+                uint64_t m2[C / 2], ns2[C / 2], y2[C / 2], yl2[C / 2];
 #pragma unroll
                 for (int j = 0; j < C / 2; ++j) {
                     m2[j] = pack_f2(m[2 * j], m[2 * j + 1]);
                     ns2[j] = pack_f2(-s[2 * j], -s[2 * j + 1]);
                     y2[j] = pack_f2(y[2 * j], y[2 * j + 1]);
+                    // what rn(1/s) leaves out: (1 - s*y) / s, the residual being exact in one FMA
+                    yl2[j] = pack_f2(__fmul_rn(__fmaf_rn(-s[2 * j], y[2 * j], 1.0f), y[2 * j]),
+                                     __fmul_rn(__fmaf_rn(-s[2 * j + 1], y[2 * j + 1], 1.0f), y[2 * j + 1]));
                 }
-                if (want_sum) code_rows<T, C, BITS, true>(tile, out_lane, G, lane, m2, ns2, y2, sum2);
-                else code_rows<T, C, BITS, false>(tile, out_lane, G, lane, m2, ns2, y2, sum2);
+                if (want_sum) code_rows<T, C, BITS, true>(tile, out_lane, G, lane, m2, ns2, y2, yl2, sum2);
+                else code_rows<T, C, BITS, false>(tile, out_lane, G, lane, m2, ns2, y2, yl2, sum2);
             } else {
 #pragma unroll 2
                 for (int r = 0; r < G; ++r) {
