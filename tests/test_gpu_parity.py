@@ -252,6 +252,41 @@ def test_bf16_structured_data_has_no_code_mismatch(orc, oqm):
     P.compare_store(gst, ost, K.float().numpy())
 
 
+@pytest.mark.parametrize("bits", [4, 2])
+def test_quotients_one_float_away_from_a_rounding_boundary(orc, oqm, bits):
+    """binary32 inputs placed 0, 1, 2 and 3 floats to either side of m + (k + 1/2) s for every level k and many
+    random (m, s): the codes flip exactly where the true division says, so a quotient that is only nearly correctly
+    rounded (one correction too few, a reciprocal that is off by an ulp) shows up here as a mismatch."""
+    levels = (1 << bits) - 1
+    sh = synth.Shape("boundary", L=1, H_q=2, H_k=2, d=128, G=64, T=40, T_q=1, k=2, dtype="fp32", seed=5,
+                     extra={"bits": bits})
+    rng = np.random.default_rng(17 + bits)
+    shape = (1, sh.T, sh.H_k, sh.d)
+    lo = rng.uniform(-4, 4, shape).astype(np.float32)
+    span = (rng.uniform(0.05, 8.0, shape) * 2.0 ** rng.integers(-6, 7, shape)).astype(np.float32)
+    hi = (lo + span).astype(np.float32)
+    s = ((hi - lo).astype(np.float32) / np.float32(levels)).astype(np.float32)      # what both sides will compute
+    X = np.empty((1, sh.T, sh.H_k, sh.G, sh.d), np.float32)
+    X[:, :, :, 0] = lo
+    X[:, :, :, 1] = hi
+    for g in range(2, sh.G):
+        k = (g - 2) % levels
+        off = ((g - 2) // levels) % 7 - 3                                              # -3 .. 3 floats
+        mid = (lo.astype(np.float64) + (k + 0.5) * s.astype(np.float64)).astype(np.float32)
+        x = mid.copy()
+        for _ in range(abs(off)):
+            x = np.nextafter(x, np.float32(np.inf if off > 0 else -np.inf), dtype=np.float32)
+        X[:, :, :, g] = np.clip(x, lo, hi)                                             # the range stays (lo, hi)
+    K = torch.from_numpy(X)
+    V = torch.from_numpy(X[:, ::-1].copy())
+    gst, ost, gcfg, ocfg = _quantize_both(orc, oqm, sh, K, V)
+    P.compare_store(gst, ost, X)
+    # the construction does what it says: a good share of the elements sits within 2^-20 of a boundary
+    q = (X - lo[:, :, :, None]) / s[:, :, :, None]
+    near = np.abs(q - np.floor(q) - 0.5) < 2.0 ** -20
+    assert near.mean() > 0.3
+
+
 # ------------------------------------------------------------------ keep-mask, summary keys, strided inputs
 
 def test_keep_mask_summary_keys_and_token_major_layout(orc, oqm):
