@@ -11,15 +11,12 @@
 // group of 50 tokens is two segments) or of the system tokens.  A block of 8
 // warps takes 8 consecutive segments of one (layer, kv head) and all the query
 // heads of that kv head's GQA block (in chunks of 8); warp w owns segment w:
-//   phase 1  scores: a lane owns 8 adjacent channels, d/8 lanes share a token;
-//            the code words of the whole segment are requested at once, K is
-//            rebuilt as fmaf(code, s, m) in registers, dotted with the query
-//            heads, and the 8 partial dot products of a lane are summed across
-//            the token's lanes by a reduce-scatter (8 shuffles, not 32)
+//   phase 1  scores of the segment's tokens against the query heads, a
+//            tensor-core product whose matrix operand is the raw codes
 //   phase 2  block-local softmax statistics per query head (max, sum) in the
 //            base-2 domain (the scores carry softmax_scale * log2(e))
-//   phase 3  weighted sum of V, rebuilt the same way, per warp; the warps'
-//            sums are combined through shared memory
+//   phase 3  weighted sum of V, again a tensor-core product over raw codes,
+//            per warp; the warps' sums are combined through shared memory
 // and writes (max, sum, weighted sum) per query head to the workspace.  The
 // block that draws the last ticket of its (layer, kv head) merges the partial
 // results of all its blocks and writes the output row.  Nobody waits.
@@ -51,7 +48,7 @@ struct AttendParams {
     uint32_t *flags;
 };
 
-// Ticket and merge, the tail of both attention kernels: every block of a (layer, kv head) has written its partial
+// Ticket and merge, the tail of the attention kernel: every block of a (layer, kv head) has written its partial
 // (max, sum, weighted sum) per query head to the workspace; the block that draws the last ticket combines them and
 // writes the output rows.  All threads of the block call it; nobody waits for another block.
 template <typename CT, int D>
@@ -132,267 +129,8 @@ __device__ __forceinline__ void attend_merge(const AttendParams &p, int li, int 
     }
 }
 
-// QT: type of q_dec; CT: type of the system-token cache and of the output; LPR: lanes per token (d / 8);
-// BITS: width of a code
-template <typename QT, typename CT, int LPR, int BITS>
-__global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p) {
-    constexpr int D = LPR * 8;
-    constexpr int TPW = 32 / LPR;  // tokens one warp pass covers
-    constexpr int kSlots = kAtWarps * kAtSegTokens;
-    constexpr int kBuf = (32 * 1024) / (kAtHeads * D * 4) < kAtWarps ? (32 * 1024) / (kAtHeads * D * 4) : kAtWarps;
-    __shared__ __align__(16) float buf[8192];  // phases 1-3: scores [kAtHeads][kSlots]; then warp sums [kBuf][kAtHeads][D]
-    __shared__ __align__(16) float qf[kAtHeads][D];
-    __shared__ float blk_max[kAtHeads], blk_sum[kAtHeads];
-    __shared__ int s_last;
-    static_assert(kAtHeads * kSlots <= 8192 && kBuf * kAtHeads * D <= 8192, "shared buffer");
-
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int sub = lane / LPR, cl = lane - sub * LPR;
-    const int bx = blockIdx.x, h = blockIdx.y, li = blockIdx.z;
-    const int G = p.g.G, H = p.g.H;
-    const int seg = bx * kAtWarps + warp;  // this warp's segment of (li, h)
-    float(*sc)[kSlots] = reinterpret_cast<float(*)[kSlots]>(buf);
-
-    // ---- what the warp's segment is
-    int n_tok = 0;          // tokens in the segment
-    int tok0 = 0;           // first token of the segment inside its group / inside the system tokens
-    bool is_sys = false;
-    int64_t slot = 0;       // bank slot of a group segment
-    if (seg < p.n_sys_seg) {
-        is_sys = true;
-        tok0 = seg * kAtSegTokens;
-        n_tok = min(kAtSegTokens, p.sys_len - tok0);
-    } else if (seg < p.n_seg) {
-        const int sg = seg - p.n_sys_seg;
-        const int j = sg / p.segs_per_group;
-        tok0 = (sg - j * p.segs_per_group) * kAtSegTokens;
-        const int t = p.per_head ? p.idx[((int64_t)li * H + h) * p.k + j] : p.idx[(int64_t)li * p.k + j];
-        if (t >= 0 && t < p.n_groups) {
-            n_tok = min(kAtSegTokens, G - tok0);
-            slot = bank_slot(p.g, p.layer_begin + li, t, h);
-        } else if (t != -1 && p.flags && lane == 0 && tok0 == 0) {
-            atomicOr(p.flags, STOM_FLAG_BAD_INDEX);
-        }
-    }
-    const CT *ksys = reinterpret_cast<const CT *>(p.ksys) + (int64_t)li * p.s_sl + (int64_t)h * p.s_sh + cl * 8;
-    const CT *vsys = reinterpret_cast<const CT *>(p.vsys) + (int64_t)li * p.s_sl + (int64_t)h * p.s_sh + cl * 8;
-
-    // All loads of a segment (16 passes of group tokens: one code word per lane and pass) or of a quarter of it (4
-    // passes of system tokens: 16 bytes per lane and pass) are issued at once -- a decode step is pure latency -- and
-    // parked in a per-warp staging area; the passes then run in a ROLLED loop.  Unrolling them instead made the
-    // kernel several thousand instructions long, executed once per warp, and instruction fetch became the bottleneck.
-    constexpr int kStageWords = 16;
-    uint32_t *stage = reinterpret_cast<uint32_t *>(buf) + kAtHeads * kSlots + warp * kStageWords * 32 + lane;
-    static_assert(kAtHeads * kSlots + kAtWarps * kStageWords * 32 <= 8192, "shared buffer");
-    const int n_pass = (n_tok + TPW - 1) / TPW;
-    const int batch_passes = is_sys ? kStageWords / 4 : kStageWords;
-    auto load_batch = [&](bool keys, int p0) {
-        if (is_sys) {
-            const CT *base = keys ? ksys : vsys;
-#pragma unroll
-            for (int b = 0; b < kStageWords / 4; ++b) {
-                const int g = (p0 + b) * TPW + sub;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (g < n_tok) v = __ldg(reinterpret_cast<const uint4 *>(base + (int64_t)(tok0 + g) * p.s_st));
-                stage[(4 * b) * 32] = v.x; stage[(4 * b + 1) * 32] = v.y;
-                stage[(4 * b + 2) * 32] = v.z; stage[(4 * b + 3) * 32] = v.w;
-            }
-        } else {
-            const uint8_t *codes = (keys ? p.codes_k : p.codes_v) + slot * (int64_t)G * p.g.row_bytes;
-#pragma unroll
-            for (int b = 0; b < kStageWords; ++b) {
-                const int g = (p0 + b) * TPW + sub;
-                stage[b * 32] = g < n_tok ? load_codes8<BITS>(codes + (int64_t)(tok0 + g) * p.g.row_bytes, cl) : 0u;
-            }
-        }
-    };
-    // runs f(g, x) for every token of the warp's segment (x: 8 channels as floats), keys or values
-    auto for_tokens = [&](bool keys, const float (&s)[8], const float (&m)[8], auto &&f) {
-        for (int p0 = 0; p0 < n_pass; p0 += batch_passes) {
-            load_batch(keys, p0);
-            __syncwarp();
-            const int nb = min(batch_passes, n_pass - p0);
-#pragma unroll 1
-            for (int b = 0; b < nb; ++b) {
-                float x[8];
-                if (is_sys) {
-                    unpack2<CT>(stage[(4 * b) * 32], x[0], x[1]);
-                    unpack2<CT>(stage[(4 * b + 1) * 32], x[2], x[3]);
-                    unpack2<CT>(stage[(4 * b + 2) * 32], x[4], x[5]);
-                    unpack2<CT>(stage[(4 * b + 3) * 32], x[6], x[7]);
-                } else {
-                    uint32_t fbits[8];
-                    code_floats8<BITS>(stage[b * 32], fbits);
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) x[c] = __fmaf_rn(__uint_as_float(fbits[c]) - 8388608.0f, s[c], m[c]);
-                }
-                f((p0 + b) * TPW + sub, x);
-            }
-            __syncwarp();
-        }
-    };
-    auto load_stats = [&](bool keys, float (&s)[8], float (&m)[8]) {
-        if (is_sys || n_tok == 0) return;
-        load_scale_zero8(keys ? p.scale_k : p.scale_v, keys ? p.zero_k : p.zero_v, slot * D + cl * 8, p.g.meta_dtype, s, m);
-    };
-
-    const int n_blocks = gridDim.x;
-    for (int h0 = 0; h0 < p.rep; h0 += kAtHeads) {  // query heads of this kv head, kAtHeads at a time
-        const int nh = min(kAtHeads, p.rep - h0);
-        // ---- the query rows, scaled so that exp2 can be used
-        for (int e = tid; e < kAtHeads * D; e += kAtThreads) {
-            const int hh = e / D, c = e - hh * D;
-            float v = 0.0f;
-            if (hh < nh) {
-                const QT *q = reinterpret_cast<const QT *>(p.q) + (int64_t)li * p.q_sl + (int64_t)(h * p.rep + h0 + hh) * p.q_sh;
-                v = (float)q[c] * p.scale_log2e;
-            }
-            qf[hh][c] = v;
-        }
-        __syncthreads();
-
-        // ---- phase 1: scores of the warp's segment
-        {
-            float s[8], m[8];
-            load_stats(true, s, m);
-            float q8[kAtHeads][8];
-#pragma unroll
-            for (int hh = 0; hh < kAtHeads; ++hh) {
-                const float4 a = *reinterpret_cast<const float4 *>(&qf[hh][cl * 8]);
-                const float4 b = *reinterpret_cast<const float4 *>(&qf[hh][cl * 8 + 4]);
-                q8[hh][0] = a.x; q8[hh][1] = a.y; q8[hh][2] = a.z; q8[hh][3] = a.w;
-                q8[hh][4] = b.x; q8[hh][5] = b.y; q8[hh][6] = b.z; q8[hh][7] = b.w;
-            }
-            // slots without a token score -inf
-            for (int e = lane; e < kAtHeads * kAtSegTokens; e += 32)
-                sc[e / kAtSegTokens][warp * kAtSegTokens + (e % kAtSegTokens)] = -INFINITY;
-            __syncwarp();
-            for_tokens(true, s, m, [&](int g, const float (&x)[8]) {
-                float dot[kAtHeads];
-#pragma unroll
-                for (int hh = 0; hh < kAtHeads; ++hh) {
-                    dot[hh] = 0.0f;
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) dot[hh] = fmaf(x[c], q8[hh][c], dot[hh]);
-                }
-                // reduce-scatter over the token's lanes: each step halves the heads a lane still carries, so that lane
-                // cl ends with the full sum of query head cl & 7 (8 channel blocks cover 3 steps; wider rows add plain steps)
-                float v4[4], v2[2], mine;
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float keep = (cl & 4) ? dot[4 + i] : dot[i], give = (cl & 4) ? dot[i] : dot[4 + i];
-                    v4[i] = keep + __shfl_xor_sync(0xffffffffu, give, 4);
-                }
-#pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const float keep = (cl & 2) ? v4[2 + i] : v4[i], give = (cl & 2) ? v4[i] : v4[2 + i];
-                    v2[i] = keep + __shfl_xor_sync(0xffffffffu, give, 2);
-                }
-                {
-                    const float keep = (cl & 1) ? v2[1] : v2[0], give = (cl & 1) ? v2[0] : v2[1];
-                    mine = keep + __shfl_xor_sync(0xffffffffu, give, 1);
-                }
-#pragma unroll
-                for (int o = 8; o < LPR; o <<= 1) mine += __shfl_xor_sync(0xffffffffu, mine, o);
-                if (cl < kAtHeads && g < n_tok) {
-                    sc[cl][warp * kAtSegTokens + g] = mine;
-                }
-            });
-        }
-        __syncthreads();
-
-        // ---- phase 2: the block's softmax statistics; scores become weights in place
-        if (warp < kAtHeads) {
-            float mx = -INFINITY;
-            for (int i = lane; i < kSlots; i += 32) mx = fmaxf(mx, sc[warp][i]);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            float sum = 0.0f;
-            for (int i = lane; i < kSlots; i += 32) {
-                const float v = sc[warp][i];
-                const float w = v == -INFINITY ? 0.0f : exp2f(v - mx);
-                sc[warp][i] = w;
-                sum += w;
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-            if (lane == 0) {
-                blk_max[warp] = mx;
-                blk_sum[warp] = sum;
-            }
-        }
-        __syncthreads();
-
-        // ---- phase 3: weighted sum of the values of the warp's segment
-        float acc[kAtHeads][8];
-#pragma unroll
-        for (int hh = 0; hh < kAtHeads; ++hh)
-#pragma unroll
-            for (int c = 0; c < 8; ++c) acc[hh][c] = 0.0f;
-        {
-            float s[8], m[8];
-            load_stats(false, s, m);
-            for_tokens(false, s, m, [&](int g, const float (&x)[8]) {
-                if (g < n_tok) {
-#pragma unroll
-                    for (int hh = 0; hh < kAtHeads; ++hh) {
-                        const float w = sc[hh][warp * kAtSegTokens + g];
-#pragma unroll
-                        for (int c = 0; c < 8; ++c) acc[hh][c] = fmaf(w, x[c], acc[hh][c]);
-                    }
-                }
-            });
-            // the token slots of a warp pass hold different tokens of the same channels
-#pragma unroll
-            for (int o = LPR; o < 32; o <<= 1) {
-#pragma unroll
-                for (int hh = 0; hh < kAtHeads; ++hh)
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) acc[hh][c] += __shfl_xor_sync(0xffffffffu, acc[hh][c], o);
-            }
-        }
-        __syncthreads();  // every warp is done with the weights; the buffer now takes the warps' sums
-        float tot[kAtHeads * D / kAtThreads];
-#pragma unroll
-        for (int e = 0; e < kAtHeads * D / kAtThreads; ++e) tot[e] = 0.0f;
-        for (int r = 0; r < kAtWarps; r += kBuf) {
-            if (warp >= r && warp < r + kBuf && sub == 0) {
-                float *dst = buf + (size_t)(warp - r) * kAtHeads * D + cl * 8;
-#pragma unroll
-                for (int hh = 0; hh < kAtHeads; ++hh) {
-                    *reinterpret_cast<float4 *>(dst + hh * D) = make_float4(acc[hh][0], acc[hh][1], acc[hh][2], acc[hh][3]);
-                    *reinterpret_cast<float4 *>(dst + hh * D + 4) = make_float4(acc[hh][4], acc[hh][5], acc[hh][6], acc[hh][7]);
-                }
-            }
-            __syncthreads();
-#pragma unroll
-            for (int e = 0; e < kAtHeads * D / kAtThreads; ++e) {
-                const int i = e * kAtThreads + tid;  // (head, channel) pair
-                for (int w = 0; w < kBuf && r + w < kAtWarps; ++w) tot[e] += buf[(size_t)w * kAtHeads * D + i];
-            }
-            __syncthreads();
-        }
-        // ---- partial result of this block: (max, sum, weighted sum) per query head
-#pragma unroll
-        for (int e = 0; e < kAtHeads * D / kAtThreads; ++e) {
-            const int i = e * kAtThreads + tid, hh = i / D, c = i - hh * D;
-            if (hh < nh) {
-                float *rec = p.part + ((((int64_t)li * H + h) * n_blocks + bx) * p.rep + h0 + hh) * (D + 2);
-                rec[2 + c] = tot[e];
-                if (c == 0) {
-                    rec[0] = blk_max[hh];
-                    rec[1] = blk_sum[hh];
-                }
-            }
-        }
-        __syncthreads();  // qf, buf and the statistics are rewritten by the next chunk of heads
-    }
-
-    attend_merge<CT, D>(p, li, h, n_blocks, &s_last);
-}
-
 // ---------------------------------------------------------------------------------------------------------------
-// The same attention with the two contractions on the tensor cores (4-bit codes).
+// The two contractions on the tensor cores (4-bit and 2-bit codes).
 //
 // Both products are small dense contractions -- scores: [tokens x d] . [d x 8 query heads]; values:
 // [d x tokens] . [tokens x 8 query heads] -- so they run as m16n8k16 warp-level matrix products (the query heads of a
@@ -405,7 +143,6 @@ __global__ void __launch_bounds__(kAtThreads) attend_kernel(const AttendParams p
 // may be permuted freely as long as both operands use the same permutation, and so may the output columns: a thread
 // therefore owns CONTIGUOUS code bytes (for the scores: d/4 adjacent channels of a token row; for the values: d/8
 // adjacent channels of four tokens), which it loads with one vector load and slices with byte permutes.
-// Segments, block layout, softmax statistics, partial results and the merge are those of the kernel above.
 // ---------------------------------------------------------------------------------------------------------------
 
 template <typename MT>
@@ -448,7 +185,28 @@ __device__ __forceinline__ void load_words_or_zero(const void *p, bool valid, ui
     }
 }
 
-// Byte `b` of x and byte `b` of y, each holding one 4-bit code (0x00..0x0F), as the bfloat16 pair
+// Field f of every byte of a word of packed codes (a byte holds 8/BITS codes, lowest channel in the lowest bits):
+// byte b of the result is the code of channel (8/BITS) * b + f of the word, alone in its byte.
+template <int BITS>
+__device__ __forceinline__ uint32_t code_view(uint32_t w, int f) {
+    return (w >> (BITS * f)) & (BITS == 4 ? 0x0F0F0F0Fu : 0x03030303u);
+}
+// Where code i of a run of packed codes sits: word, byte of the word, field of the byte.
+template <int BITS> __device__ __forceinline__ constexpr int code_word_of(int i) { return i / (32 / BITS); }
+template <int BITS> __device__ __forceinline__ constexpr int code_byte_of(int i) { return (i % (32 / BITS)) / (8 / BITS); }
+template <int BITS> __device__ __forceinline__ constexpr int code_field_of(int i) { return i % (8 / BITS); }
+
+// NB bytes of packed codes from p (aligned to min(16, NB) bytes) as 32-bit words, or zeros
+template <int NB>
+__device__ __forceinline__ void load_code_bytes(const uint8_t *p, bool valid, uint32_t (&w)[(NB + 3) / 4]) {
+    if constexpr (NB == 2) {
+        w[0] = valid ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(p)) : 0u;
+    } else {
+        load_words_or_zero<NB / 4>(p, valid, w);
+    }
+}
+
+// Byte `b` of x and byte `b` of y, each holding one code (0x00..0x0F), as the bfloat16 pair
 // (128 + code of x, 128 + code of y): the permute puts the two bytes into the low byte of each half and fills the
 // other two with the sign of a source byte (selector values of 8 and above), which is zero.
 __device__ __forceinline__ uint32_t code_pair_bf16(uint32_t x, uint32_t y, int b) {
@@ -470,8 +228,8 @@ __device__ __forceinline__ void split2(float a, float b, uint32_t &hi, uint32_t 
     seen_b = hb + lb;
 }
 
-// QT: type of q_dec; CT: type of the system-token cache and of the output; D: head dim
-template <typename QT, typename CT, int D>
+// QT: type of q_dec; CT: type of the system-token cache and of the output; D: head dim; BITS: width of a code
+template <typename QT, typename CT, int D, int BITS>
 __global__ void __launch_bounds__(kAtThreads) attend_mma_kernel(const AttendParams p) {
     constexpr int kSlots = kAtWarps * kAtSegTokens;
     constexpr int kBuf = (32 * 1024) / (kAtHeads * D * 4) < kAtWarps ? (32 * 1024) / (kAtHeads * D * 4) : kAtWarps;
@@ -479,6 +237,7 @@ __global__ void __launch_bounds__(kAtThreads) attend_mma_kernel(const AttendPara
     constexpr int KC = D / 4;   // channels of a token row one thread owns in the score product
     constexpr int MT = D / 16;  // m-tiles of the value product (16 channels each)
     constexpr int VC = D / 8;   // channels one thread owns in the value product
+    constexpr int KB = KC * BITS / 8, VB = VC * BITS / 8;  // bytes of packed codes behind them
     using BF = __nv_bfloat16;
     __shared__ __align__(16) float buf[8192];  // scores / weights [kAtHeads][kSlots]; then warp sums [kBuf][kAtHeads][D]
     __shared__ __align__(16) float qf[kAtHeads][D];
@@ -495,7 +254,7 @@ __global__ void __launch_bounds__(kAtThreads) attend_mma_kernel(const AttendPara
     const int seg = bx * kAtWarps + warp;
     float(*sc)[kSlots] = reinterpret_cast<float(*)[kSlots]>(buf);
 
-    // ---- what the warp's segment is (as in the kernel above)
+    // ---- what the warp's segment is
     int n_tok = 0, tok0 = 0;
     bool is_sys = false;
     int64_t slot = 0;
@@ -535,12 +294,12 @@ __global__ void __launch_bounds__(kAtThreads) attend_mma_kernel(const AttendPara
 #pragma unroll
         for (int i = 0; i < kAtSegTokens / 8; ++i) {
             const int row = g + 8 * i;  // the score product reads rows g, g+8, g+16, g+24
-            if (row < n_tok) prefetch_l1(kcodes + (int64_t)(tok0 + row) * p.g.row_bytes + t * (KC / 2));
+            if (row < n_tok) prefetch_l1(kcodes + (int64_t)(tok0 + row) * p.g.row_bytes + t * KB);
         }
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const int tok = (i >> 2) * 16 + 2 * t + (i & 1) + 8 * ((i >> 1) & 1);  // the value product's tokens
-            if (tok < n_tok) prefetch_l1(vcodes + (int64_t)(tok0 + tok) * p.g.row_bytes + g * (VC / 2));
+            if (tok < n_tok) prefetch_l1(vcodes + (int64_t)(tok0 + tok) * p.g.row_bytes + g * VB);
         }
     }
 
@@ -604,18 +363,19 @@ __global__ void __launch_bounds__(kAtThreads) attend_mma_kernel(const AttendPara
                 if (mt * 16 >= n_tok) break;  // warp-uniform
                 float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
                 if (!is_sys) {
-                    uint32_t w0[D / 32], w1[D / 32];  // the thread's KC codes of the two token rows
-                    load_words_or_zero<D / 32>(kcodes + (int64_t)(tok0 + r0) * p.g.row_bytes + t * (KC / 2), r0 < n_tok, w0);
-                    load_words_or_zero<D / 32>(kcodes + (int64_t)(tok0 + r1) * p.g.row_bytes + t * (KC / 2), r1 < n_tok, w1);
+                    uint32_t w0[(KB + 3) / 4], w1[(KB + 3) / 4];  // the thread's KC codes of the two token rows
+                    load_code_bytes<KB>(kcodes + (int64_t)(tok0 + r0) * p.g.row_bytes + t * KB, r0 < n_tok, w0);
+                    load_code_bytes<KB>(kcodes + (int64_t)(tok0 + r1) * p.g.row_bytes + t * KB, r1 < n_tok, w1);
 #pragma unroll
                     for (int kk = 0; kk < KS; ++kk) {
-                        // codes 4kk .. 4kk+3 of the thread's run: bytes 2(kk&1) and 2(kk&1)+1 of the even-nibble and
-                        // odd-nibble views of word kk/2
-                        const uint32_t e0 = w0[kk / 2] & 0x0F0F0F0Fu, o0 = (w0[kk / 2] >> 4) & 0x0F0F0F0Fu;
-                        const uint32_t e1 = w1[kk / 2] & 0x0F0F0F0Fu, o1 = (w1[kk / 2] >> 4) & 0x0F0F0F0Fu;
-                        const int b = 2 * (kk & 1);
-                        const uint32_t a0 = code_pair_bf16(e0, o0, b), a1 = code_pair_bf16(e1, o1, b);
-                        const uint32_t a2 = code_pair_bf16(e0, o0, b + 1), a3 = code_pair_bf16(e1, o1, b + 1);
+                        // codes 4kk, 4kk+1 of the thread's run share a byte, and so do 4kk+2, 4kk+3
+                        const int ca = 4 * kk, cb = 4 * kk + 2;
+                        const int wa = code_word_of<BITS>(ca), ba = code_byte_of<BITS>(ca), fa = code_field_of<BITS>(ca);
+                        const int wb = code_word_of<BITS>(cb), bb = code_byte_of<BITS>(cb), fb = code_field_of<BITS>(cb);
+                        const uint32_t a0 = code_pair_bf16(code_view<BITS>(w0[wa], fa), code_view<BITS>(w0[wa], fa + 1), ba);
+                        const uint32_t a1 = code_pair_bf16(code_view<BITS>(w1[wa], fa), code_view<BITS>(w1[wa], fa + 1), ba);
+                        const uint32_t a2 = code_pair_bf16(code_view<BITS>(w0[wb], fb), code_view<BITS>(w0[wb], fb + 1), bb);
+                        const uint32_t a3 = code_pair_bf16(code_view<BITS>(w1[wb], fb), code_view<BITS>(w1[wb], fb + 1), bb);
                         mma_16816<BF>(c4, a0, a1, a2, a3, qb[kk][0], qb[kk][1]);
                         mma_16816<BF>(c4, a0, a1, a2, a3, ql[kk][0], ql[kk][1]);
                     }
@@ -684,24 +444,21 @@ __global__ void __launch_bounds__(kAtThreads) attend_mma_kernel(const AttendPara
                 }
                 wsum += (r0 + r1) + (r2 + r3);
                 if (!is_sys) {
-                    uint32_t e[4][D / 64], o[4][D / 64];  // even / odd nibbles of the thread's VC codes of its 4 tokens
+                    uint32_t w[4][(VB + 3) / 4];  // the thread's VC codes of its 4 tokens
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         const int tok = ta + (i & 1) + 8 * (i >> 1);
-                        uint32_t w[D / 64];
-                        load_words_or_zero<D / 64>(vcodes + (int64_t)(tok0 + tok) * p.g.row_bytes + g * (VC / 2), tok < n_tok, w);
-#pragma unroll
-                        for (int j = 0; j < D / 64; ++j) {
-                            e[i][j] = w[j] & 0x0F0F0F0Fu;
-                            o[i][j] = (w[j] >> 4) & 0x0F0F0F0Fu;
-                        }
+                        load_code_bytes<VB>(vcodes + (int64_t)(tok0 + tok) * p.g.row_bytes + g * VB, tok < n_tok, w[i]);
                     }
 #pragma unroll
                     for (int mm = 0; mm < MT; ++mm) {
-                        // byte mm % 4 of word mm / 4 of e: the code of channel VC*g + 2*mm; of o: of the next channel
-                        const int j = mm >> 2, b = mm & 3;
-                        const uint32_t a0 = code_pair_bf16(e[0][j], e[1][j], b), a1 = code_pair_bf16(o[0][j], o[1][j], b);
-                        const uint32_t a2 = code_pair_bf16(e[2][j], e[3][j], b), a3 = code_pair_bf16(o[2][j], o[3][j], b);
+                        // channels VC*g + 2*mm and the next one share a byte; rows g and g + 8 of the m-tile
+                        const int c = 2 * mm;
+                        const int j = code_word_of<BITS>(c), b = code_byte_of<BITS>(c), f = code_field_of<BITS>(c);
+                        const uint32_t a0 = code_pair_bf16(code_view<BITS>(w[0][j], f), code_view<BITS>(w[1][j], f), b);
+                        const uint32_t a1 = code_pair_bf16(code_view<BITS>(w[0][j], f + 1), code_view<BITS>(w[1][j], f + 1), b);
+                        const uint32_t a2 = code_pair_bf16(code_view<BITS>(w[2][j], f), code_view<BITS>(w[3][j], f), b);
+                        const uint32_t a3 = code_pair_bf16(code_view<BITS>(w[2][j], f + 1), code_view<BITS>(w[3][j], f + 1), b);
                         mma_16816<BF>(acc[mm], a0, a1, a2, a3, b0, b1);
                         mma_16816<BF>(acc[mm], a0, a1, a2, a3, l0, l1);
                     }
@@ -804,16 +561,16 @@ static int32_t launch_attend(const AttendParams &p, dim3 grid, cudaStream_t s) {
     const bool b4 = p.g.row_bytes * 2 == p.g.d;  // 4-bit codes: d/2 bytes per row
     switch (p.g.d) {
     case 64:
-        if (b4) attend_mma_kernel<QT, CT, 64><<<grid, kAtThreads, 0, s>>>(p);
-        else attend_kernel<QT, CT, 8, 2><<<grid, kAtThreads, 0, s>>>(p);
+        if (b4) attend_mma_kernel<QT, CT, 64, 4><<<grid, kAtThreads, 0, s>>>(p);
+        else attend_mma_kernel<QT, CT, 64, 2><<<grid, kAtThreads, 0, s>>>(p);
         break;
     case 128:
-        if (b4) attend_mma_kernel<QT, CT, 128><<<grid, kAtThreads, 0, s>>>(p);
-        else attend_kernel<QT, CT, 16, 2><<<grid, kAtThreads, 0, s>>>(p);
+        if (b4) attend_mma_kernel<QT, CT, 128, 4><<<grid, kAtThreads, 0, s>>>(p);
+        else attend_mma_kernel<QT, CT, 128, 2><<<grid, kAtThreads, 0, s>>>(p);
         break;
     case 256:
-        if (b4) attend_mma_kernel<QT, CT, 256><<<grid, kAtThreads, 0, s>>>(p);
-        else attend_kernel<QT, CT, 32, 2><<<grid, kAtThreads, 0, s>>>(p);
+        if (b4) attend_mma_kernel<QT, CT, 256, 4><<<grid, kAtThreads, 0, s>>>(p);
+        else attend_mma_kernel<QT, CT, 256, 2><<<grid, kAtThreads, 0, s>>>(p);
         break;
     default: return STOM_ERR_SHAPE;
     }
