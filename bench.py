@@ -549,7 +549,7 @@ def run_stream(args, sh):
     question(8)
     decode(8)
     torch.cuda.synchronize()
-    ing, qry, dec = [], [], []
+    ing, qry, dec, rep, graphs = [], [], [], [], []
     every = args.query_every
     t0 = time.perf_counter()
     for f in range(sh.T):
@@ -560,8 +560,17 @@ def run_stream(args, sh):
             a, b, c = ev(), ev(), ev()
             a.record(); question(f + 1); b.record(); decode(f + 1); c.record()
             qry.append((a, b)); dec.append((b, c))
+            # the same question (retrieval, then one decode step) captured as a CUDA graph and replayed once
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                question(f + 1)
+                decode(f + 1)
+            a, b = ev(), ev()
+            a.record(); g.replay(); b.record()
+            rep.append((a, b)); graphs.append(g)   # a graph lives until its replay has run
         if f % 256 == 255:
             torch.cuda.synchronize()             # bounds the number of events in flight
+            graphs.clear()
     torch.cuda.synchronize()
     wall = time.perf_counter() - t0
     assert int(flags.item()) == 0
@@ -571,7 +580,7 @@ def run_stream(args, sh):
         return {"p50_us": v[len(v) // 2], "p99_us": v[min(len(v) - 1, int(0.99 * len(v)))], "mean_us": statistics.mean(v),
                 "max_us": v[-1], "n": len(v)}
 
-    i_st, q_st, d_st = stats(ing), stats(qry), stats(dec)
+    i_st, q_st, d_st, r_st = stats(ing), stats(qry), stats(dec), stats(rep)
     frame_bytes = sh.L * (2 * sh.H_k * sh.G * sh.d * 2 + 2 * sh.H_k * sh.G * sh.d // 2 + 5 * sh.H_k * sh.d * 4 + sh.H_k * 4)
     print(json.dumps({
         "metric": "per-query OQM latency (score + top-k + dequant-gather + decode attention), streaming interleave",
@@ -582,6 +591,7 @@ def run_stream(args, sh):
                    "system_tokens": sys_len, "frame_pool": pool},
         "per_frame_ingest": dict(i_st, algorithmic_bytes=frame_bytes),
         "per_query_retrieve": q_st, "per_decode_step_attend_all_layers": d_st,
+        "per_query_retrieve_plus_decode_step_graph_replay": r_st,
         "wall_s_including_python": wall,
         "note": "CUDA-event times of single calls issued from Python one after the other; latencies, not bandwidths",
     }))
