@@ -10,7 +10,13 @@
 //             tokens) in shared memory -- Q of one layer is small and comes
 //             from L2 for all but the first block that touches it; the rows
 //             of several heads are in flight together, because this step is
-//             all memory latency;
+//             memory latency -- and L2 bandwidth: every block of a layer wants
+//             the same rows.  So the blocks of a layer are launched as
+//             thread-block clusters: each block of a cluster embeds only its
+//             share of the kv heads and the cluster exchanges the results
+//             through distributed shared memory (one hardware cluster
+//             barrier on each side of the exchange; no block returns before
+//             them);
 //   stream    cosine scores of the block's groups (the software-pipelined
 //             loop of the stand-alone scoring kernel), written to `scores`;
 //   select    every block takes a ticket on its layer's counter when its
@@ -82,9 +88,10 @@ struct QRow {
 // channels; the rows of a head (rep * T_q of them) are dealt to RG = kFusedThreads / (d/8) row slots.  The heads go
 // through in groups of kEmbedHeadGroup: a thread walks its rows of the whole group with kInFlight loads outstanding,
 // whatever head they belong to, so the wait for memory is paid once or twice per group instead of once per head;
-// part[head of the group][RG][d+4] combines the slots.
+// part[head of the group][RG][d+4] combines the slots.  The call embeds heads h_first, h_first + h_step, ... only.
 template <typename T>
-__device__ __forceinline__ void embed_layer(const ScoreParams &p, int li, float *sq, float *qn, float *part) {
+__device__ __forceinline__ void embed_layer(const ScoreParams &p, int li, float *sq, float *qn, float *part,
+                                            int h_first, int h_step) {
     constexpr int kInFlight = sizeof(T) == 4 ? 8 : 16;
     const int d = p.g.d, H = p.g.H, tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int lanes_per_row = d >> 3;
@@ -93,8 +100,10 @@ __device__ __forceinline__ void embed_layer(const ScoreParams &p, int li, float 
     const int rows = p.rep * p.T_q, pitch = d + 4;
     const int per_head = (rows + RG - 1) / RG;  // rows of one head that a row slot walks
     const T *qbase = reinterpret_cast<const T *>(p.Q) + (int64_t)li * p.ql + cq * 8;
-    for (int h0 = 0; h0 < H; h0 += kEmbedHeadGroup) {
-        const int hg = min(kEmbedHeadGroup, H - h0);
+    const int n_mine = h_first < H ? (H - h_first + h_step - 1) / h_step : 0;  // heads this call embeds
+    auto head_of = [&](int j) { return h_first + j * h_step; };                  // its j-th head
+    for (int h0 = 0; h0 < n_mine; h0 += kEmbedHeadGroup) {
+        const int hg = min(kEmbedHeadGroup, n_mine - h0);
         const int n_i = hg * per_head;
         float acc[8];
 #pragma unroll
@@ -121,7 +130,7 @@ __device__ __forceinline__ void embed_layer(const ScoreParams &p, int li, float 
                 for (int j = 0; j < QRow<T>::W; ++j) x[b].w[j] = 0u;  // +0.0 in every format
                 if (i0 + b < n_i) {
                     if (rs + l_k * RG < rows)
-                        x[b].load(qbase + (int64_t)((h0 + l_hh) * p.rep + l_hr) * p.qh + (int64_t)l_j * p.qt);
+                        x[b].load(qbase + (int64_t)(head_of(h0 + l_hh) * p.rep + l_hr) * p.qh + (int64_t)l_j * p.qt);
                     if (++l_k == per_head) {  // next head of the group: back to the slot's first row
                         l_k = 0;
                         ++l_hh;
@@ -157,26 +166,62 @@ __device__ __forceinline__ void embed_layer(const ScoreParams &p, int li, float 
             const int hh = e / d, c = e - hh * d;
             float a = 0.0f;
             for (int g = 0; g < RG; ++g) a += part[(hh * RG + g) * pitch + c];
-            sq[(h0 + hh) * d + c] = a / (float)rows;
+            sq[head_of(h0 + hh) * d + c] = a / (float)rows;
         }
         __syncthreads();
         for (int hh = warp; hh < hg; hh += kFusedThreads / 32) {  // |q_h|^2: one warp per head
             float n2 = 0.0f;
             for (int c = lane; c < d; c += 32) {
-                const float v = sq[(h0 + hh) * d + c];
+                const float v = sq[head_of(h0 + hh) * d + c];
                 n2 = fmaf(v, v, n2);
             }
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) n2 += __shfl_xor_sync(0xffffffffu, n2, o);
-            if (lane == 0) qn[h0 + hh] = n2;
+            if (lane == 0) qn[head_of(h0 + hh)] = n2;
         }
         // part is rewritten by the next group only after that group's loads; the barrier below orders it for all
         __syncthreads();
     }
 }
 
-// grid (chunks, layer_count), kFusedThreads threads.  Dynamic shared memory: q (H*d floats), norms (H rounded up
-// to 4 floats), then a region used first as the embedding scratch and, in a selecting block, as the key array.
+// Thread-block cluster primitives (sm_90+).  A kernel launched without a cluster dimension is a cluster of one.
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_size() {
+    uint32_t n;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(n));
+    return n;
+}
+// Hardware barrier over all threads of the cluster; every thread of every block must call it (no spinning involved)
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// The word(s) at the same shared-memory offset as `mine` in block `rank` of the cluster
+__device__ __forceinline__ uint32_t cluster_addr(const void *mine, uint32_t rank) {
+    uint32_t a = (uint32_t)__cvta_generic_to_shared(mine), ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(rank));
+    return ra;
+}
+__device__ __forceinline__ float4 ld_cluster_f4(const float4 *mine, uint32_t rank) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"(cluster_addr(mine, rank))
+                 : "memory");
+    return v;
+}
+__device__ __forceinline__ float ld_cluster_f(const float *mine, uint32_t rank) {
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr(mine, rank)) : "memory");
+    return v;
+}
+
+// grid (chunks, layer_count), kFusedThreads threads, optionally in clusters of consecutive chunks of a layer.
+// Dynamic shared memory: q (H*d floats), norms (H rounded up to 4 floats), then a region used first as the embedding
+// scratch and, in a selecting block, as the key array.
 template <typename T, int V4, typename KT>
 __global__ void __launch_bounds__(kFusedThreads) retrieve_kernel(const RetrieveParams rp) {
     extern __shared__ __align__(16) float dyn[];
@@ -187,7 +232,20 @@ __global__ void __launch_bounds__(kFusedThreads) retrieve_kernel(const RetrieveP
     float *sq = dyn, *qn = dyn + HD, *region = qn + ((H + 3) & ~3);
 
     grid_launch_dependents();  // the gather that follows may be scheduled as this grid drains; it waits before it reads idx
-    embed_layer<T>(p, li, sq, qn, region);
+    // The blocks of a cluster (consecutive chunks of one layer) share the embedding: block r of C embeds heads
+    // r, r + C, ... and fetches the others from their owners' shared memory.  Launched without clusters, C = 1.
+    const uint32_t C = cluster_size(), r = cluster_rank();
+    embed_layer<T>(p, li, sq, qn, region, (int)r, (int)C);
+    if (C > 1) {
+        cluster_sync();  // every block's heads are in its shared memory
+        const int d4 = p.g.d >> 2;
+        for (int e = tid; e < HD / 4; e += kFusedThreads) {
+            const uint32_t owner = (uint32_t)(e / d4) % C;
+            if (owner != r) reinterpret_cast<float4 *>(sq)[e] = ld_cluster_f4(reinterpret_cast<float4 *>(sq) + e, owner);
+        }
+        if (tid < H && (uint32_t)tid % C != r) qn[tid] = ld_cluster_f(qn + tid, (uint32_t)tid % C);
+        cluster_sync();  // nobody leaves, or goes on to reuse its scratch, while a neighbour still reads from it
+    }
 
     const int t_begin = blockIdx.x * p.groups_per_block;
     const int t_end = min(t_begin + p.groups_per_block, p.n_groups);
@@ -246,27 +304,57 @@ __global__ void __launch_bounds__(kFusedThreads) retrieve_kernel(const RetrieveP
     }
 }
 
+// Launch with thread-block clusters along x when `clusters` is set: the largest divisor of grid.x, up to the portable
+// limit of 8, with which the whole grid is still resident at once (as it is without clusters); else single blocks.
+template <typename KernelT>
+static void launch_fused(KernelT kernel, const RetrieveParams &rp, dim3 grid, size_t smem, int clusters, cudaStream_t s) {
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = grid;
+    lc.blockDim = dim3(kFusedThreads);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 1;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    lc.attrs = at;
+    lc.numAttrs = 1;
+    for (int c = 8; clusters && c > 1; --c) {
+        if (grid.x % c) continue;
+        int resident = 0;
+        at[0].val.clusterDim.x = (unsigned)c;
+        if (cudaOccupancyMaxActiveClusters(&resident, kernel, &lc) == cudaSuccess &&
+            (int64_t)resident * c >= (int64_t)grid.x * grid.y)
+            break;
+        (void)cudaGetLastError();
+        at[0].val.clusterDim.x = 1;
+    }
+    (void)cudaLaunchKernelEx(&lc, kernel, rp);  // a failure is picked up by the caller's finish_launch()
+}
+
 template <typename T, typename KT>
-static void launch_retrieve_kt(const RetrieveParams &rp, dim3 grid, size_t smem, int v4, cudaStream_t s) {
+static void launch_retrieve_kt(const RetrieveParams &rp, dim3 grid, size_t smem, int v4, int cluster, cudaStream_t s) {
     switch (v4) {
-    case 4: retrieve_kernel<T, 4, KT><<<grid, kFusedThreads, smem, s>>>(rp); break;  // 4 kv heads x 128
-    case 8: retrieve_kernel<T, 8, KT><<<grid, kFusedThreads, smem, s>>>(rp); break;  // 8 kv heads x 128
-    case 2: retrieve_kernel<T, 2, KT><<<grid, kFusedThreads, smem, s>>>(rp); break;
+    case 4: launch_fused(retrieve_kernel<T, 4, KT>, rp, grid, smem, cluster, s); break;  // 4 kv heads x 128
+    case 8: launch_fused(retrieve_kernel<T, 8, KT>, rp, grid, smem, cluster, s); break;  // 8 kv heads x 128
+    case 2: launch_fused(retrieve_kernel<T, 2, KT>, rp, grid, smem, cluster, s); break;
     case 1:
         if constexpr (sizeof(KT) == 4) {
-            retrieve_kernel<T, 1, KT><<<grid, kFusedThreads, smem, s>>>(rp);
+            launch_fused(retrieve_kernel<T, 1, KT>, rp, grid, smem, cluster, s);
             break;
         }
-    default: retrieve_kernel<T, 0, KT><<<grid, kFusedThreads, smem, s>>>(rp); break;
+    default: launch_fused(retrieve_kernel<T, 0, KT>, rp, grid, smem, cluster, s); break;
     }
 }
 
 template <typename T>
-static void launch_retrieve(const RetrieveParams &rp, dim3 grid, size_t smem, int HD, bool fast, cudaStream_t s) {
+static void launch_retrieve(const RetrieveParams &rp, dim3 grid, size_t smem, int HD, bool fast, int cluster,
+                            cudaStream_t s) {
     const int md = rp.sp.g.meta_dtype, v4 = score_fast_v4(HD, fast, md);
-    if (md == STOM_BF16) launch_retrieve_kt<T, __nv_bfloat16>(rp, grid, smem, v4, s);
-    else if (md == STOM_FP16) launch_retrieve_kt<T, __half>(rp, grid, smem, v4, s);
-    else launch_retrieve_kt<T, float>(rp, grid, smem, v4, s);
+    if (md == STOM_BF16) launch_retrieve_kt<T, __nv_bfloat16>(rp, grid, smem, v4, cluster, s);
+    else if (md == STOM_FP16) launch_retrieve_kt<T, __half>(rp, grid, smem, v4, cluster, s);
+    else launch_retrieve_kt<T, float>(rp, grid, smem, v4, cluster, s);
 }
 
 }  // namespace stom
@@ -364,10 +452,11 @@ extern "C" int32_t stom_oqm_retrieve(const stom_oqm_config *cfg, const stom_oqm_
         if (smem > 48 * 1024) return STOM_ERR_SHAPE;
         const dim3 grid((n_groups + p.groups_per_block - 1) / p.groups_per_block, layer_count);
         const bool fast = !p.per_head && H <= 32;
+        const int cluster = grid.x > 1;  // several blocks per layer: let them share the embedding
         switch (dt) {
-        case STOM_BF16: launch_retrieve<__nv_bfloat16>(rp, grid, smem, HD, fast, s); break;
-        case STOM_FP16: launch_retrieve<__half>(rp, grid, smem, HD, fast, s); break;
-        default: launch_retrieve<float>(rp, grid, smem, HD, fast, s); break;
+        case STOM_BF16: launch_retrieve<__nv_bfloat16>(rp, grid, smem, HD, fast, cluster, s); break;
+        case STOM_FP16: launch_retrieve<__half>(rp, grid, smem, HD, fast, cluster, s); break;
+        default: launch_retrieve<float>(rp, grid, smem, HD, fast, cluster, s); break;
         }
         if ((rc = finish_launch())) return rc;
     } else if (layer_count > 0) {

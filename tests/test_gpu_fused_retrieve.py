@@ -107,3 +107,50 @@ def test_fused_retrieve_on_an_empty_bank_marks_every_slot_unused(orc):
                           P.active_strides(sh, S), 0, ws)
     torch.cuda.synchronize()
     assert torch.all(idx == -1) and torch.all(ka == 3.0) and torch.all(va == 3.0)
+
+
+@pytest.mark.parametrize("copies", [3, 40, 200, "all"])
+def test_fused_retrieve_equal_scores_go_to_the_lower_index(orc, copies):
+    """Stored groups with identical representative keys score identically; which of them make the top-K is then
+    decided by index alone (the lower one wins), although the candidates reach the completing block from several
+    blocks' pre-selections.  Cases: a few copies of the group ranked around K, many, and a bank of identical groups.
+    Expected: the stable ordering (score descending, index ascending) of the scores the call itself wrote, cut at
+    K, ascending; the scores are checked against the oracle as everywhere else."""
+    from paper_2510_18269_b200 import oqm
+    oqm.lib()
+    L, H_q, H_k, d, G, T, T_q, k = 2, 28, 4, 128, 4, 2400, 4, 64
+    sh = synth.Shape("ties", L=L, H_q=H_q, H_k=H_k, d=d, G=G, T=T, T_q=T_q, k=k, dtype="bf16", seed=5, extra={})
+    ocfg, gcfg, ost, gst, u = P.random_bank(orc, oqm, sh, 0, seed=77)
+    g = torch.Generator().manual_seed(3)
+    base = torch.from_numpy(u[:, 0]).repeat_interleave(H_q // H_k, dim=1)[:, :, None, :]
+    Q = (base + 0.5 * torch.randn(L, H_q, T_q, d, generator=g)).to(torch.bfloat16).contiguous()
+    # the group the oracle ranks K-th in layer 0 is copied over other slots, spread over the bank
+    o_scores = orc.score_groups(ocfg, ost, 0, L, T, P.as_np16(Q), T_q, P.q_strides(sh))
+    kth = int(np.argsort(-o_scores[0], kind="stable")[k - 1])
+    rng = np.random.default_rng(11)
+    where = np.arange(T) if copies == "all" else rng.choice(T, size=copies, replace=False)
+    for l in range(L):
+        ost.rep_key[l, where] = ost.rep_key[l, kth]
+        ost.rep_norm2[l, where] = ost.rep_norm2[l, kth]
+    gst.rep_key.copy_(torch.from_numpy(ost.rep_key))
+    gst.rep_norm2.copy_(torch.from_numpy(ost.rep_norm2))
+    o_scores = orc.score_groups(ocfg, ost, 0, L, T, P.as_np16(Q), T_q, P.q_strides(sh))
+
+    S = k * G
+    _, ka = P.out_buffers(sh, L, S, torch.bfloat16, "cuda", 3.0)
+    _, va = P.out_buffers(sh, L, S, torch.bfloat16, "cuda", 3.0)
+    scores = torch.empty(L * T, dtype=torch.float32, device="cuda")
+    idx = torch.full((L * k,), -9, dtype=torch.int32, device="cuda")
+    ws = torch.full((oqm.stom_oqm_retrieve_workspace_bytes(gcfg, L, T, k) + 256,), 0xAB, dtype=torch.uint8, device="cuda")
+    ws = ws[(-ws.data_ptr()) % 256:]
+    oqm.stom_oqm_retrieve(gcfg, gst, 0, L, T, Q.cuda(), T_q, P.q_strides(sh), k, scores, idx, ka, va, oqm.BF16,
+                          P.active_strides(sh, S), 0, ws)
+    torch.cuda.synchronize()
+    P.compare_scores(scores, o_scores)
+    got_scores = scores.view(L, T).cpu().numpy()
+    got = idx.view(L, k).cpu().numpy()
+    for l in range(L):
+        same = got_scores[l, where]
+        assert np.all(same == same[0]), "identical groups must score identically"
+        order = np.lexsort((np.arange(T), -got_scores[l].astype(np.float64)))  # score descending, then index ascending
+        assert np.array_equal(got[l], np.sort(order[:k])), f"layer {l}"
