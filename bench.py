@@ -46,7 +46,7 @@ NCU_TRAFFIC_PER_UNIT = {
     # 125.4 MB had left L2 when it ended (the rest is written back later), so this undercounts by design
     "dequant_gather_kernel": 103805.0 / 4,
     "score_kernel": 2071.0 / 4,         # bytes per (layer, stored group): 59.39 MB over 28 x 1024 units
-    "retrieve_kernel": 2186.0 / 4,      # bytes per (layer, stored group): 62.68 MB over 28 x 1024 units (Q re-read per block)
+    "retrieve_kernel": 2188.0 / 4,      # bytes per (layer, stored group): 62.75 MB over 28 x 1024 units (Q read per cluster)
     # bytes per frame of 196 tokens x 1152 bf16 channels (not per kv head): 561.8 MB over 1200 frames
     "ctr_similarity_kernel": 468181.0,
 }
