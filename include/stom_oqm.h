@@ -71,7 +71,7 @@ typedef struct stom_oqm_config {
     int32_t n_layers;        /* L                                               */
     int32_t n_q_heads;       /* H_q, a multiple of n_kv_heads                   */
     int32_t n_kv_heads;      /* H_k                                             */
-    int32_t head_dim;        /* d: 32, 64, 128 or 256                           */
+    int32_t head_dim;        /* d: 64, 128 or 256                               */
     int32_t group_tokens;    /* G, tokens per group (frame); 1..64              */
     int32_t capacity_groups; /* groups the bank can hold per layer              */
     int32_t bits;            /* 4 (the paper's setting) or 2 (its ablation)     */
@@ -378,6 +378,8 @@ int64_t stom_oqm_retrieve_host_scratch_bytes(const stom_oqm_config *cfg, int32_t
  * stom_oqm_topk).  k_active_host, v_active_host: HOST compact
  * [layer_count][H_k][k*G][d] of out_dtype, both given or both NULL (NULL: the
  * reconstructed cache stays in scratch on the device and is not copied back).
+ * When fewer than k groups are stored, the token slots behind the last
+ * selected group (those of idx == -1) come back as zeros.
  * scratch: DEVICE, 256-byte aligned.
  * Errors: as the three device calls, plus WORKSPACE. */
 int32_t stom_oqm_retrieve_host(const stom_oqm_config *cfg, const stom_oqm_store *store,

@@ -100,6 +100,14 @@ extern "C" int32_t stom_oqm_retrieve_host(const stom_oqm_config *cfg, const stom
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const int64_t d = cfg->head_dim, S = (int64_t)k * cfg->group_tokens;
     if ((rc = copy_async(b + r.off_q, Q_host, r.bytes_q, cudaMemcpyHostToDevice, s))) return rc;
+    if (n_groups < k && k_active_host) {
+        // slots behind the last stored group are not written by the gather: hand back zeros, not stale scratch
+        cudaError_t e = cudaMemsetAsync(b + r.off_ka, 0, (size_t)(r.off_va + up256(r.bytes_act) - r.off_ka), s);
+        if (e != cudaSuccess) {
+            set_last_cuda_error(e);
+            return STOM_ERR_CUDA;
+        }
+    }
     rc = stom_oqm_retrieve(cfg, store, layer_begin, layer_count, n_groups, b + r.off_q, T_q,
                            (int64_t)cfg->n_q_heads * T_q * d, (int64_t)T_q * d, d, k,
                            reinterpret_cast<float *>(b + r.off_scores), reinterpret_cast<int32_t *>(b + r.off_idx),

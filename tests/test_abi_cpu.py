@@ -123,6 +123,37 @@ def test_entry_points_reject_bad_arguments_before_any_launch(oqm):
     assert gather(st=(i64(4 * 300 * 128), i64(300 * 128), i64(64))) == -1       # token stride shorter than a row
 
 
+def test_host_buffer_entry_points_reject_bad_arguments_before_any_cuda_call(oqm):
+    L = oqm.lib()
+    cfg = oqm.make_config(2, 8, 4, 128, 50, 10)
+    desc = oqm.StoreDesc(*[0x7f0000000000 + 4096 * i for i in range(8)])
+    p = C.c_void_p(0x7f1000000000)          # never dereferenced: every call below is refused on the host
+    i64, i32 = C.c_int64, C.c_int32
+    need_q = oqm.stom_oqm_quantize_host_scratch_bytes(cfg, 2, 10)
+    assert need_q >= 2 * 2 * 10 * 4 * 50 * 128 * 2 and need_q % 256 == 0
+
+    def quant(K=p, V=p, scr=p, nbytes=need_q, lc=2, gc=10):
+        return L.stom_oqm_quantize_frame_host(C.byref(cfg), C.byref(desc), 0, i32(lc), 0, i32(gc), K, V, scr,
+                                              i64(nbytes), None, None)
+    assert quant(K=None) == -1 and quant(V=None) == -1 and quant(gc=-1) == -1
+    assert quant(scr=None) == -8 and quant(nbytes=need_q - 1) == -8
+    assert quant(scr=C.c_void_p(0x7f1000000004)) == -8        # scratch must be 16-byte aligned
+
+    need_r = oqm.stom_oqm_retrieve_host_scratch_bytes(cfg, 2, 10, 4, 4, oqm.BF16)
+    assert need_r > 2 * 2 * 4 * 4 * 50 * 128 * 2              # holds the reconstructed K and V of the call
+    assert oqm.stom_oqm_retrieve_host_scratch_bytes(cfg, 2, 10, 0, 4, oqm.BF16) == -1
+    assert oqm.stom_oqm_retrieve_host_scratch_bytes(cfg, 2, 10, 4, 4, oqm.FP32) == -6
+
+    def retr(Q=p, idx=p, ka=p, va=p, scr=p, nbytes=need_r, od=0, k=4, Tq=4):
+        return L.stom_oqm_retrieve_host(C.byref(cfg), C.byref(desc), 0, 2, 10, Q, i32(Tq), i32(k), idx, ka, va,
+                                        i32(od), scr, i64(nbytes), None, None)
+    assert retr(Q=None) == -1 and retr(idx=None) == -1 and retr(k=0) == -1 and retr(Tq=0) == -1
+    assert retr(ka=None) == -1 and retr(va=None) == -1        # both cache pointers or neither
+    assert retr(od=2) == -6
+    assert retr(scr=None) == -8 and retr(nbytes=need_r - 1) == -8
+    assert retr(scr=C.c_void_p(0x7f1000000010)) == -8         # scratch must be 256-byte aligned
+
+
 def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
     from paper_2510_18269_b200 import oqm as m
     monkeypatch.setattr(m, "_lib", None)
