@@ -483,9 +483,6 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
                         pending = false;
                     }
                     if (!__any_sync(0xffffffffu, pending)) break;
-#ifdef QSLEEP
-                    __nanosleep(QSLEEP);
-#endif
                     if ((spin & 63u) == 63u) {  // bounded: a slot that never comes free ends the block
                         if (t0 == 0) t0 = global_ns();
                         if (__any_sync(0xffffffffu, *abort_flag || global_ns() - t0 > kWaitLimitNs)) {
@@ -578,14 +575,14 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
         // A parity wait cannot tell the fill it is waiting for from the fill two rounds back on the same barrier,
         // and the producer fills the slots of a group in whatever order they come free, so that older fill may
         // still be on its way when this warp gets here.  The producer publishes the fill number of a slot before it
-        // starts the copy; a wait that returns while that number is not ours answered for the older fill: wait on.
-        bool ok;
+        // starts the copy, and it starts that copy only after every earlier fill of the slot has been consumed.  So
+        // the warp first waits (bounded) until the published number is its own: from then on the barrier has
+        // completed exactly the earlier fills, and the parity wait that follows can only be answered by this one.
+        bool ok = true;
         {
             unsigned long long t0 = 0;
-            for (uint32_t spin = 0;; ++spin) {
-                ok = mbar_wait(full_bar(slot, round), (round >> 1) & 1u, abort_flag);
-                if (!ok || *reinterpret_cast<volatile int32_t *>(&info[slot].round) == (int32_t)round) break;
-                __nanosleep(64);
+            for (uint32_t spin = 0; *reinterpret_cast<volatile int32_t *>(&info[slot].round) != (int32_t)round; ++spin) {
+                __nanosleep(32);
                 if ((spin & 63u) == 63u) {
                     if (t0 == 0) t0 = global_ns();
                     if (*abort_flag || global_ns() - t0 > kWaitLimitNs) {
@@ -594,6 +591,7 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
                     }
                 }
             }
+            if (ok) ok = mbar_wait(full_bar(slot, round), (round >> 1) & 1u, abort_flag);
         }
         ok = __all_sync(0xffffffffu, ok && !*abort_flag);  // the whole warp stops together
         if (!ok) {

@@ -1,6 +1,7 @@
-"""Parity at the size and in the launch configuration the benchmark times: the 7B-shaped 2-hour stream (28 layers,
-7 200 frames of 50 tokens, 4 kv heads, d = 128; 20.6 GB of bf16 K/V), quantized in ONE call over all layers, then one
-question through the fused retrieval call.
+"""Parity at the sizes and in the launch configuration the benchmark times: the 7B-shaped 2-hour stream (28 layers,
+7 200 frames of 50 tokens, 4 kv heads, d = 128; 20.6 GB of bf16 K/V) and the 72B-shaped stream (80 layers, 3 600
+frames, 8 kv heads, 64 query heads, 32 question tokens; 59 GB of bf16 K/V), each quantized in ONE call over all
+layers, then one question through the fused retrieval call.
 
 The oracle cannot redo 20 GB in a test, so it redoes one whole layer (every frame of it: codes, scales, offsets,
 representative keys, then that layer's 7 200 scores, its selection and its reconstructed cache) and a sample of
@@ -20,12 +21,20 @@ pytestmark = pytest.mark.gpu
 
 
 def test_c3_full_stream_one_layer_in_full_and_samples_elsewhere(orc):
+    _full_stream(orc, synth.C3, lf=13, need_gib=40)
+
+
+def test_c5_full_stream_one_layer_in_full_and_samples_elsewhere(orc):
+    _full_stream(orc, synth.C5, lf=47, need_gib=100)
+
+
+def _full_stream(orc, sh, lf, need_gib):
     from paper_2510_18269_b200 import oqm
     oqm.lib()
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
-    if free < 40 * 2 ** 30:
-        pytest.skip("needs 40 GB of free device memory")
-    sh = synth.C3
+    if free < need_gib * 2 ** 30:
+        pytest.skip(f"needs {need_gib} GB of free device memory")
     dev = torch.device("cuda")
     gcfg = P.gpu_cfg(oqm, sh)
     gst = oqm.Store(gcfg, device=dev, zero=False)
@@ -57,7 +66,6 @@ def test_c3_full_stream_one_layer_in_full_and_samples_elsewhere(orc):
         assert sc_all[l, sel].min() >= sc_all[l, rest].max(), f"layer {l}: a left-out group outscores a selected one"
 
     # ---- one layer in full
-    lf = 13
     one = dataclasses.replace(sh, L=1)
     ocfg = P.oracle_cfg(orc, one)
     ost = orc.Store(ocfg)
