@@ -7,28 +7,51 @@
 // packed codes and their (s, m) -- a quarter of the bytes of the bf16 cache --
 // instead of writing that cache once and re-reading it every step.
 //
-// Work unit: a segment = up to 32 consecutive tokens of one selected group (a
-// group of 50 tokens is two segments) or of the system tokens.  A block of 8
-// warps takes 8 consecutive segments of one (layer, kv head) and all the query
-// heads of that kv head's GQA block (in chunks of 8); warp w owns segment w:
-//   phase 1  scores of the segment's tokens against the query heads, a
-//            tensor-core product whose matrix operand is the raw codes
-//   phase 2  block-local softmax statistics per query head (max, sum) in the
-//            base-2 domain (the scores carry softmax_scale * log2(e))
-//   phase 3  weighted sum of V, again a tensor-core product over raw codes,
-//            per warp; the warps' sums are combined through shared memory
-// and writes (max, sum, weighted sum) per query head to the workspace.  The
-// block that draws the last ticket of its (layer, kv head) merges the partial
-// results of all its blocks and writes the output row.  Nobody waits.
-// A decode step is latency, not bandwidth: 2.2 MB per layer at the 7B geometry.
+// Work unit: one selected group (its G tokens) or a run of up to 16 system
+// tokens.  Everything a unit reads is contiguous in the bank -- the K codes and
+// the V codes of a (layer, group, kv head) are one block each, and so are its
+// four metadata rows -- so a unit arrives in shared memory by a handful of bulk
+// asynchronous copies (cp.async.bulk, completion counted on an mbarrier),
+// which tie up no registers and no warp while the bytes are on their way.
+//
+//   grid     (C, kv heads, layers); the C blocks of a (layer, kv head) form a
+//            thread-block cluster and share out its units
+//   warp     owns its own ring of 1 or 2 stages and its own units (u = rank +
+//            C * (warp + 8 * i)): lane 0 posts the copies of unit i + stages
+//            as soon as unit i has been consumed.  Per unit the warp computes
+//            scores (a tensor-core product over the raw codes), a warp-local
+//            online softmax, and the weighted sum of V (again a tensor-core
+//            product over raw codes); it keeps a running (max, sum, output)
+//            for the 8 query heads it handles, so no block barrier sits
+//            between units
+//   merge    the warps of a block combine through shared memory, the blocks
+//            of the cluster through distributed shared memory (one hardware
+//            cluster barrier on each side); rank r writes its share of the
+//            output rows.  No workspace, no tickets, nobody spins.
+#include "stom_async.cuh"
 #include "stom_internal.cuh"
 
 namespace stom {
 
 constexpr int kAtWarps = 8;
 constexpr int kAtThreads = kAtWarps * 32;
-constexpr int kAtSegTokens = 32;  // token slots per segment
-constexpr int kAtHeads = 8;       // query heads handled together
+constexpr int kAtUnitTokens = 64;  // token slots of a group unit (G <= 64)
+constexpr int kAtSysTokens = 16;   // tokens of a system-token unit
+constexpr int kAtHeads = 8;        // query heads handled together
+constexpr int kAtWPitch = 68;      // floats per head row of a warp's weight tile (64 token slots + padding)
+constexpr int kAtMaxStages = 2;
+constexpr unsigned long long kAtWaitLimitNs = 2000000000ull;  // a copy that has not landed after 2 s ends the block
+
+// Shared-memory layout (bytes from the start of dynamic shared memory)
+constexpr int kAtOffBars = 0;                                   // [kAtWarps][kAtMaxStages] mbarriers
+constexpr int kAtOffAbort = kAtOffBars + kAtWarps * kAtMaxStages * 8;
+constexpr int kAtOffStat = 256;                                 // [kAtWarps][16]: max[8], sum[8] of each warp
+constexpr int kAtOffBlk = kAtOffStat + kAtWarps * 16 * 4;       // max[8], sum[8] of the block
+constexpr int kAtOffWt = kAtOffBlk + 16 * 4;                    // [kAtWarps][8][kAtWPitch] weights
+constexpr int kAtOffOb = kAtOffWt + kAtWarps * kAtHeads * kAtWPitch * 4;  // the block's partial output
+__host__ __device__ constexpr int at_opitch(int D) { return D + 8; }      // floats of one channel slab (D/8 channels x 8 heads) + padding
+__host__ __device__ constexpr int at_ofloats(int D) { return 8 * at_opitch(D); }
+__host__ __device__ constexpr int at_off_ring(int D) { return (kAtOffOb + at_ofloats(D) * 4 + 127) / 128 * 128; }
 
 struct AttendParams {
     const int32_t *idx;
@@ -40,94 +63,12 @@ struct AttendParams {
     int64_t s_sl, s_sh, s_st;  // element strides of the system-token cache: layer, kv head, token
     void *out;
     int64_t o_sl, o_sh;  // element strides of out: layer, query head
-    float *part;         // [layer][H][blocks][rep][d + 2]
-    uint32_t *counters;  // [layer][H]
     BankGeom g;
-    int32_t layer_begin, k, n_groups, per_head, rep, sys_len, n_sys_seg, n_seg, segs_per_group;
+    int32_t layer_begin, k, n_groups, per_head, rep, sys_len, n_sys_units, n_units;
+    int32_t stage_bytes, n_stages;
     float scale_log2e;
     uint32_t *flags;
 };
-
-// Ticket and merge, the tail of the attention kernel: every block of a (layer, kv head) has written its partial
-// (max, sum, weighted sum) per query head to the workspace; the block that draws the last ticket combines them and
-// writes the output rows.  All threads of the block call it; nobody waits for another block.
-template <typename CT, int D>
-__device__ __forceinline__ void attend_merge(const AttendParams &p, int li, int h, int n_blocks, int *s_last_ptr) {
-    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31, H = p.g.H;
-    int &s_last = *s_last_ptr;
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const unsigned ticket = atomicAdd(&p.counters[li * H + h], 1u);
-        // tickets of a cleared workspace run from 0 to n_blocks - 1; anything else was there before the call
-        if (ticket >= (unsigned)n_blocks && p.flags) atomicOr(p.flags, STOM_FLAG_DIRTY_WORKSPACE);
-        s_last = ticket == (unsigned)n_blocks - 1;
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    if (tid == 0) p.counters[li * H + h] = 0;  // as found
-    // One warp per query head.  Lanes share out the blocks 32 at a time: (max, sum) of a block come in one 8-byte
-    // load; the channel sums of the first kChunk blocks are requested in the same breath, before anything is
-    // reduced, and those of the next chunk while the current one is added up -- the merge is two memory round trips
-    // for up to kChunk blocks and one more per further chunk.
-    constexpr int kChunk = D >= 256 ? 4 : 8;
-    for (int hq = warp; hq < p.rep; hq += kAtWarps) {
-        const float *rec0 = p.part + (((int64_t)li * H + h) * n_blocks * p.rep + hq) * (D + 2);
-        const int64_t step = (int64_t)p.rep * (D + 2);
-        auto load_chunk = [&](int b0, float (&v)[kChunk][D / 32]) {
-#pragma unroll
-            for (int j = 0; j < kChunk; ++j)
-#pragma unroll
-                for (int i = 0; i < D / 32; ++i)
-                    v[j][i] = b0 + j < n_blocks ? __ldcg(rec0 + (b0 + j) * step + 2 + lane + 32 * i) : 0.0f;
-        };
-        float cur[kChunk][D / 32];
-        load_chunk(0, cur);
-        // the global maximum over all blocks (several trips only beyond 32 blocks)
-        float2 ms = make_float2(-INFINITY, 0.0f);  // of block `lane` of the first trip
-        if (lane < n_blocks) ms = __ldcg(reinterpret_cast<const float2 *>(rec0 + lane * step));
-        float mx = ms.x;
-        for (int b = lane + 32; b < n_blocks; b += 32) mx = fmaxf(mx, __ldcg(rec0 + b * step));
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        float den = 0.0f;
-        float num[D / 32];
-#pragma unroll
-        for (int i = 0; i < D / 32; ++i) num[i] = 0.0f;
-        for (int b0 = 0; b0 < n_blocks; b0 += 32) {
-            if (b0 > 0) {
-                ms = make_float2(-INFINITY, 0.0f);
-                if (b0 + lane < n_blocks) ms = __ldcg(reinterpret_cast<const float2 *>(rec0 + (b0 + lane) * step));
-            }
-            const float w_mine = ms.x == -INFINITY ? 0.0f : exp2f(ms.x - mx);
-            den = fmaf(ms.y, w_mine, den);
-            const int nb = min(32, n_blocks - b0);
-            for (int c0 = 0; c0 < nb; c0 += kChunk) {
-                float nxt[kChunk][D / 32];
-                const bool more = b0 + c0 + kChunk < n_blocks;
-                if (more) load_chunk(b0 + c0 + kChunk, nxt);
-#pragma unroll
-                for (int j = 0; j < kChunk; ++j) {
-                    const float w = __shfl_sync(0xffffffffu, w_mine, (c0 + j) & 31);
-#pragma unroll
-                    for (int i = 0; i < D / 32; ++i) num[i] = fmaf(cur[j][i], c0 + j < nb ? w : 0.0f, num[i]);
-                }
-                if (more) {
-#pragma unroll
-                    for (int j = 0; j < kChunk; ++j)
-#pragma unroll
-                        for (int i = 0; i < D / 32; ++i) cur[j][i] = nxt[j][i];
-                }
-            }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) den += __shfl_xor_sync(0xffffffffu, den, o);
-        CT *out = reinterpret_cast<CT *>(p.out) + (int64_t)li * p.o_sl + (int64_t)(h * p.rep + hq) * p.o_sh;
-#pragma unroll
-        for (int i = 0; i < D / 32; ++i) out[lane + 32 * i] = (CT)(den > 0.0f ? num[i] / den : 0.0f);
-    }
-}
 
 // ---------------------------------------------------------------------------------------------------------------
 // The two contractions on the tensor cores (4-bit and 2-bit codes).
@@ -151,35 +92,33 @@ __device__ __forceinline__ void mma_16816(float (&c)[4], uint32_t a0, uint32_t a
 template <>
 __device__ __forceinline__ void mma_16816<__nv_bfloat16>(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                          uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 template <>
 __device__ __forceinline__ void mma_16816<__half>(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                                   uint32_t b0, uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
                  : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ void prefetch_l1(const void *p) { asm volatile("prefetch.global.L1 [%0];" ::"l"(p)); }
-
-// NW 32-bit words from p (p aligned to min(16, 4 * NW) bytes), or zeros
+// NW 32-bit words from shared memory at p (aligned to min(16, 4 * NW) bytes), or zeros
 template <int NW>
-__device__ __forceinline__ void load_words_or_zero(const void *p, bool valid, uint32_t (&w)[NW]) {
+__device__ __forceinline__ void lds_words_or_zero(const unsigned char *p, bool valid, uint32_t (&w)[NW]) {
 #pragma unroll
     for (int i = 0; i < NW; ++i) w[i] = 0u;
     if (!valid) return;
     if constexpr (NW == 1) {
-        w[0] = __ldg(static_cast<const uint32_t *>(p));
+        w[0] = *reinterpret_cast<const uint32_t *>(p);
     } else if constexpr (NW == 2) {
-        const uint2 v = __ldg(static_cast<const uint2 *>(p));
+        const uint2 v = *reinterpret_cast<const uint2 *>(p);
         w[0] = v.x; w[1] = v.y;
     } else {
 #pragma unroll
         for (int i = 0; i < NW / 4; ++i) {
-            const uint4 v = __ldg(static_cast<const uint4 *>(p) + i);
+            const uint4 v = *(reinterpret_cast<const uint4 *>(p) + i);
             w[4 * i] = v.x; w[4 * i + 1] = v.y; w[4 * i + 2] = v.z; w[4 * i + 3] = v.w;
         }
     }
@@ -196,13 +135,13 @@ template <int BITS> __device__ __forceinline__ constexpr int code_word_of(int i)
 template <int BITS> __device__ __forceinline__ constexpr int code_byte_of(int i) { return (i % (32 / BITS)) / (8 / BITS); }
 template <int BITS> __device__ __forceinline__ constexpr int code_field_of(int i) { return i % (8 / BITS); }
 
-// NB bytes of packed codes from p (aligned to min(16, NB) bytes) as 32-bit words, or zeros
+// NB bytes of packed codes from shared memory at p (aligned to min(16, NB) bytes) as 32-bit words, or zeros
 template <int NB>
-__device__ __forceinline__ void load_code_bytes(const uint8_t *p, bool valid, uint32_t (&w)[(NB + 3) / 4]) {
+__device__ __forceinline__ void lds_code_bytes(const unsigned char *p, bool valid, uint32_t (&w)[(NB + 3) / 4]) {
     if constexpr (NB == 2) {
-        w[0] = valid ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(p)) : 0u;
+        w[0] = valid ? (uint32_t)*reinterpret_cast<const uint16_t *>(p) : 0u;
     } else {
-        load_words_or_zero<NB / 4>(p, valid, w);
+        lds_words_or_zero<NB / 4>(p, valid, w);
     }
 }
 
@@ -228,353 +167,611 @@ __device__ __forceinline__ void split2(float a, float b, uint32_t &hi, uint32_t 
     seen_b = hb + lb;
 }
 
+// Eight adjacent metadata values (element type by the run-time code md) from shared memory, as floats
+__device__ __forceinline__ void lds_meta8(const unsigned char *row, int ch, int md, float (&f)[8]) {
+    if (md == STOM_FP32) {
+        const float4 a = *reinterpret_cast<const float4 *>(row + ch * 4), b = *reinterpret_cast<const float4 *>(row + ch * 4 + 16);
+        f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w; f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+    } else {
+        const uint4 v = *reinterpret_cast<const uint4 *>(row + ch * 2);
+        if (md == STOM_BF16) {
+            unpack2<__nv_bfloat16>(v.x, f[0], f[1]); unpack2<__nv_bfloat16>(v.y, f[2], f[3]);
+            unpack2<__nv_bfloat16>(v.z, f[4], f[5]); unpack2<__nv_bfloat16>(v.w, f[6], f[7]);
+        } else {
+            unpack2<__half>(v.x, f[0], f[1]); unpack2<__half>(v.y, f[2], f[3]);
+            unpack2<__half>(v.z, f[4], f[5]); unpack2<__half>(v.w, f[6], f[7]);
+        }
+    }
+}
+
+// The thread's KC query channels, kept in registers in the type they arrive in
+template <typename QT, int KC>
+struct QRegs {
+    static constexpr int W = sizeof(QT) == 4 ? KC : KC / 2;
+    uint32_t w[W];
+    __device__ __forceinline__ void load(const QT *row, bool valid) {  // row: the head's KC channels of this thread
+#pragma unroll
+        for (int i = 0; i < W; ++i) w[i] = valid ? __ldg(reinterpret_cast<const uint32_t *>(row) + i) : 0u;
+    }
+    // channels 2j and 2j + 1 of the thread's run
+    __device__ __forceinline__ void pair(int j, float &a, float &b) const {
+        if constexpr (sizeof(QT) == 4) {
+            a = __uint_as_float(w[2 * j]);
+            b = __uint_as_float(w[2 * j + 1]);
+        } else {
+            unpack2<QT>(w[j], a, b);
+        }
+    }
+};
+
 // QT: type of q_dec; CT: type of the system-token cache and of the output; D: head dim; BITS: width of a code
 template <typename QT, typename CT, int D, int BITS>
-__global__ void __launch_bounds__(kAtThreads) attend_mma_kernel(const AttendParams p) {
-    constexpr int kSlots = kAtWarps * kAtSegTokens;
-    constexpr int kBuf = (32 * 1024) / (kAtHeads * D * 4) < kAtWarps ? (32 * 1024) / (kAtHeads * D * 4) : kAtWarps;
+__global__ void __launch_bounds__(kAtThreads, 1) attend_kernel(const AttendParams p) {
     constexpr int KS = D / 16;  // k-steps of the score product (16 channels each)
     constexpr int KC = D / 4;   // channels of a token row one thread owns in the score product
     constexpr int MT = D / 16;  // m-tiles of the value product (16 channels each)
     constexpr int VC = D / 8;   // channels one thread owns in the value product
     constexpr int KB = KC * BITS / 8, VB = VC * BITS / 8;  // bytes of packed codes behind them
+    constexpr int MH = MT < 8 ? MT : 8;  // m-tiles of the value product done in one pass over the weights
+    constexpr int OP = at_opitch(D), OF = at_ofloats(D);
     using BF = __nv_bfloat16;
-    __shared__ __align__(16) float buf[8192];  // scores / weights [kAtHeads][kSlots]; then warp sums [kBuf][kAtHeads][D]
-    __shared__ __align__(16) float qf[kAtHeads][D];
-    __shared__ float blk_max[kAtHeads];
-    __shared__ float seg_sum[kAtWarps][kAtHeads];  // sum of a segment's weights per query head, as the tensor core sees them
-    __shared__ int s_last;
-    static_assert(kAtHeads * kSlots <= 8192 && kBuf * kAtHeads * D <= 8192, "shared buffer");
-    static_assert(kAtHeads == 8 && kAtSegTokens == 32, "fragment mapping");
+    static_assert(kAtHeads == 8 && kAtUnitTokens == 64 && kAtSysTokens == 16, "fragment mapping");
+    extern __shared__ __align__(128) unsigned char smem[];
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(smem + kAtOffAbort);
+    float *stat = reinterpret_cast<float *>(smem + kAtOffStat);
+    float *blk = reinterpret_cast<float *>(smem + kAtOffBlk);
+    float *ob = reinterpret_cast<float *>(smem + kAtOffOb);
+    unsigned char *ring = smem + at_off_ring(D);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int g = lane >> 2, t = lane & 3;  // fragment coordinates of the thread
-    const int bx = blockIdx.x, h = blockIdx.y, li = blockIdx.z;
-    const int G = p.g.G, H = p.g.H;
-    const int seg = bx * kAtWarps + warp;
-    float(*sc)[kSlots] = reinterpret_cast<float(*)[kSlots]>(buf);
+    const int h = blockIdx.y, li = blockIdx.z;
+    const int G = p.g.G, H = p.g.H, md = p.g.meta_dtype, S = p.n_stages;
+    const uint32_t C = cluster_size(), r = cluster_rank();
+    float *wt = reinterpret_cast<float *>(smem + kAtOffWt) + warp * (kAtHeads * kAtWPitch);
+    unsigned char *my_ring = ring + (size_t)warp * S * p.stage_bytes;
+    const uint32_t bar0 = smem_u32(smem + kAtOffBars) + 8u * (warp * kAtMaxStages);
 
-    // ---- what the warp's segment is
-    int n_tok = 0, tok0 = 0;
-    bool is_sys = false;
-    int64_t slot = 0;
-    if (seg < p.n_sys_seg) {
-        is_sys = true;
-        tok0 = seg * kAtSegTokens;
-        n_tok = min(kAtSegTokens, p.sys_len - tok0);
-    } else if (seg < p.n_seg) {
-        const int sg = seg - p.n_sys_seg;
-        const int j = sg / p.segs_per_group;
-        tok0 = (sg - j * p.segs_per_group) * kAtSegTokens;
-        const int tg = p.per_head ? p.idx[((int64_t)li * H + h) * p.k + j] : p.idx[(int64_t)li * p.k + j];
-        if (tg >= 0 && tg < p.n_groups) {
-            n_tok = min(kAtSegTokens, G - tok0);
-            slot = bank_slot(p.g, p.layer_begin + li, tg, h);
-        } else if (tg != -1 && p.flags && lane == 0 && tok0 == 0) {
-            atomicOr(p.flags, STOM_FLAG_BAD_INDEX);
+    if (lane == 0) {
+        for (int s = 0; s < S; ++s) mbar_init(bar0 + 8 * s, 1);
+        if (warp == 0) {
+            abort_flag[0] = 0;  // raised by the first warp whose wait ran out
+            abort_flag[1] = 0;  // never raised: lets a warp wait out its own copies regardless
         }
+        mbar_init_fence();
     }
-    n_tok = max(n_tok, 0);
+    __syncthreads();
+
+    // ---- the units of this warp: u = u_first + i * u_step, i < n_mine
+    const int u_step = (int)C * kAtWarps, u_first = (int)r + (int)C * warp;
+    const int n_mine = u_first < p.n_units ? (p.n_units - u_first + u_step - 1) / u_step : 0;
+    const int code_block = G * p.g.row_bytes;              // bytes of the K (or V) codes of a unit
+    const int meta_row = D * (md == STOM_FP32 ? 4 : 2);    // bytes of one metadata row
     const CT *ksys = reinterpret_cast<const CT *>(p.ksys) + (int64_t)li * p.s_sl + (int64_t)h * p.s_sh;
     const CT *vsys = reinterpret_cast<const CT *>(p.vsys) + (int64_t)li * p.s_sl + (int64_t)h * p.s_sh;
-    const uint8_t *kcodes = p.codes_k + slot * (int64_t)G * p.g.row_bytes;
-    const uint8_t *vcodes = p.codes_v + slot * (int64_t)G * p.g.row_bytes;
-    const int md = p.g.meta_dtype;
+    const int32_t *idx_row = p.idx + (p.per_head ? ((int64_t)li * H + h) * p.k : (int64_t)li * p.k);
 
-    // A decode step is a chain of memory round trips.  Everything a group segment will read depends on the slot
-    // only, not on the query: ask for it now (no registers are tied up), so that it arrives while the query rows are
-    // staged and the loads below find it in L1.
-    if (!is_sys && n_tok > 0) {
-        const int esz = md == STOM_FP32 ? 4 : 2;
-        const int64_t kat = (slot * D + KC * t) * esz, vat = (slot * D + VC * g) * esz;
-        prefetch_l1(static_cast<const uint8_t *>(p.scale_k) + kat);
-        prefetch_l1(static_cast<const uint8_t *>(p.zero_k) + kat);
-        prefetch_l1(static_cast<const uint8_t *>(p.scale_v) + vat);
-        prefetch_l1(static_cast<const uint8_t *>(p.zero_v) + vat);
-#pragma unroll
-        for (int i = 0; i < kAtSegTokens / 8; ++i) {
-            const int row = g + 8 * i;  // the score product reads rows g, g+8, g+16, g+24
-            if (row < n_tok) prefetch_l1(kcodes + (int64_t)(tok0 + row) * p.g.row_bytes + t * KB);
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int tok = (i >> 2) * 16 + 2 * t + (i & 1) + 8 * ((i >> 1) & 1);  // the value product's tokens
-            if (tok < n_tok) prefetch_l1(vcodes + (int64_t)(tok0 + tok) * p.g.row_bytes + g * VB);
-        }
-    }
+    uint32_t phase_bits = 0;   // bit s: parity the next wait on stage s asks for
+    uint32_t stage_info = 0;   // byte s: token count of the unit in stage s (0: nothing was posted), bit 7: system tokens
+    bool dead = false;         // a wait ran out: the warp posts nothing more and its result is void
 
-    const int n_blocks = gridDim.x;
+    // Group index of unit number i of this warp (lane-parallel: 32 units per load)
+    auto load_tg_batch = [&](int i0) -> int32_t {
+        const int u = u_first + (i0 + lane) * u_step;
+        if (i0 + lane < n_mine && u >= p.n_sys_units) return __ldg(idx_row + (u - p.n_sys_units));
+        return -1;
+    };
+    // Posts the copies of unit number i into stage i % S.  tg: the unit's group index (groups only).  Warp-collective.
+    auto post_unit = [&](int i, int32_t tg) {
+        const int s = i % S;
+        const int u = u_first + i * u_step;
+        unsigned char *st = my_ring + (size_t)s * p.stage_bytes;
+        const uint32_t bar = bar0 + 8 * s, dst = smem_u32(st);
+        uint32_t info = 0;
+        if (u < p.n_sys_units) {
+            const int tok0 = u * kAtSysTokens, n_tok = min(kAtSysTokens, p.sys_len - tok0);
+            const uint32_t row = D * (uint32_t)sizeof(CT);
+            info = (uint32_t)n_tok | 0x80u;
+            if (lane == 0) mbar_expect_tx(bar, 2u * n_tok * row);
+            __syncwarp();
+            if (p.s_st == D) {  // adjacent rows: one copy each for K and V
+                if (lane == 0) bulk_load(dst, ksys + (int64_t)tok0 * D, n_tok * row, bar);
+                if (lane == 1) bulk_load(dst + kAtSysTokens * row, vsys + (int64_t)tok0 * D, n_tok * row, bar);
+            } else if (lane < 2 * kAtSysTokens) {
+                const int rr = lane & (kAtSysTokens - 1);
+                if (rr < n_tok) {
+                    const CT *src = (lane < kAtSysTokens ? ksys : vsys) + (int64_t)(tok0 + rr) * p.s_st;
+                    bulk_load(dst + (lane < kAtSysTokens ? 0u : kAtSysTokens * row) + rr * row, src, row, bar);
+                }
+            }
+        } else if (tg >= 0 && tg < p.n_groups) {
+            const int64_t slot = bank_slot(p.g, p.layer_begin + li, tg, h);
+            info = (uint32_t)G;
+            if (lane == 0) mbar_expect_tx(bar, 2u * code_block + 4u * meta_row);
+            __syncwarp();
+            const int esz = md == STOM_FP32 ? 4 : 2;
+            if (lane == 0) bulk_load(dst, p.codes_k + slot * code_block, code_block, bar);
+            if (lane == 1) bulk_load(dst + code_block, p.codes_v + slot * code_block, code_block, bar);
+            if (lane >= 2 && lane < 6) {
+                const void *base = lane == 2 ? p.scale_k : (lane == 3 ? p.zero_k : (lane == 4 ? p.scale_v : p.zero_v));
+                bulk_load(dst + 2 * code_block + (lane - 2) * meta_row,
+                          static_cast<const unsigned char *>(base) + slot * D * esz, meta_row, bar);
+            }
+        } else if (tg != -1 && p.flags && lane == 0) {
+            atomicOr(p.flags, STOM_FLAG_BAD_INDEX);
+        }
+        stage_info = (stage_info & ~(0xFFu << (8 * s))) | (info << (8 * s));
+    };
+
     for (int h0 = 0; h0 < p.rep; h0 += kAtHeads) {
         const int nh = min(kAtHeads, p.rep - h0);
-        // ---- the query rows, scaled so that exp2 can be used
-        for (int e = tid; e < kAtHeads * D; e += kAtThreads) {
-            const int hh = e / D, c = e - hh * D;
-            float v = 0.0f;
-            if (hh < nh) {
-                const QT *q = reinterpret_cast<const QT *>(p.q) + (int64_t)li * p.q_sl + (int64_t)(h * p.rep + h0 + hh) * p.q_sh;
-                v = (float)q[c] * p.scale_log2e;
-            }
-            qf[hh][c] = v;
-        }
-        __syncthreads();
+        // ---- start the first units on their way, then fetch the query rows behind them
+        int32_t tg_batch = load_tg_batch(0);
+        if (!dead)
+            for (int i = 0; i < S && i < n_mine; ++i) post_unit(i, __shfl_sync(0xffffffffu, tg_batch, i));
+        QRegs<QT, KC> qr;  // query head g of the chunk, channels KC*t .. KC*t + KC - 1
+        qr.load(reinterpret_cast<const QT *>(p.q) + (int64_t)li * p.q_sl + (int64_t)(h * p.rep + h0 + g) * p.q_sh + KC * t, g < nh);
 
-        // ---- phase 1: scores.  Contraction slot (kk; 2t, 2t+1, 2t+8, 2t+9) of the matrix product stands for
-        //      channels KC*t + 4*kk + (0, 1, 2, 3); column g is query head g.
-        for (int e = lane; e < kAtHeads * kAtSegTokens; e += 32)
-            sc[e / kAtSegTokens][warp * kAtSegTokens + (e % kAtSegTokens)] = -INFINITY;  // slots without a token
-        __syncwarp();
-        if (n_tok > 0) {
-            uint32_t qb[KS][2], ql[KS][2];  // the thread's column of the right-hand operand, high and low parts
-            float bias = 0.0f;   // what the raw-code product leaves out, for query head g
-            if (!is_sys) {
-#pragma unroll
-                for (int c8 = 0; c8 < KC / 8; ++c8) {
-                    float s8[8], m8[8];
-                    load_scale_zero8(p.scale_k, p.zero_k, slot * D + KC * t + c8 * 8, md, s8, m8);
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {  // 2 channels each
-                        const int c = KC * t + c8 * 8 + 2 * j;
-                        const float q0 = qf[g][c], q1 = qf[g][c + 1];
-                        uint32_t whi, wlo;
-                        float r0, r1;  // the two products as the tensor core sees them
-                        split2<BF>(q0 * s8[2 * j], q1 * s8[2 * j + 1], whi, wlo, r0, r1);
-                        bias = fmaf(q0, m8[2 * j], bias);
-                        bias = fmaf(q1, m8[2 * j + 1], bias);
-                        bias = fmaf(-128.0f, r0 + r1, bias);
-                        qb[(c8 * 8 + 2 * j) / 4][((c8 * 8 + 2 * j) / 2) & 1] = whi;
-                        ql[(c8 * 8 + 2 * j) / 4][((c8 * 8 + 2 * j) / 2) & 1] = wlo;
-                    }
-                }
-            } else {
-#pragma unroll
-                for (int j = 0; j < KC / 2; ++j) {
-                    const int c = KC * t + 2 * j;
-                    float r0, r1;
-                    split2<CT>(qf[g][c], qf[g][c + 1], qb[j / 2][j & 1], ql[j / 2][j & 1], r0, r1);
-                }
-            }
-            bias += __shfl_xor_sync(0xffffffffu, bias, 1);
-            bias += __shfl_xor_sync(0xffffffffu, bias, 2);
-            const float bias_a = __shfl_sync(0xffffffffu, bias, (2 * t) << 2);       // of query head 2t
-            const float bias_b = __shfl_sync(0xffffffffu, bias, (2 * t + 1) << 2);   // of query head 2t + 1
-#pragma unroll
-            for (int mt = 0; mt < kAtSegTokens / 16; ++mt) {
-                const int r0 = mt * 16 + g, r1 = r0 + 8;
-                if (mt * 16 >= n_tok) break;  // warp-uniform
-                float c4[4] = {0.0f, 0.0f, 0.0f, 0.0f};
-                if (!is_sys) {
-                    uint32_t w0[(KB + 3) / 4], w1[(KB + 3) / 4];  // the thread's KC codes of the two token rows
-                    load_code_bytes<KB>(kcodes + (int64_t)(tok0 + r0) * p.g.row_bytes + t * KB, r0 < n_tok, w0);
-                    load_code_bytes<KB>(kcodes + (int64_t)(tok0 + r1) * p.g.row_bytes + t * KB, r1 < n_tok, w1);
-#pragma unroll
-                    for (int kk = 0; kk < KS; ++kk) {
-                        // codes 4kk, 4kk+1 of the thread's run share a byte, and so do 4kk+2, 4kk+3
-                        const int ca = 4 * kk, cb = 4 * kk + 2;
-                        const int wa = code_word_of<BITS>(ca), ba = code_byte_of<BITS>(ca), fa = code_field_of<BITS>(ca);
-                        const int wb = code_word_of<BITS>(cb), bb = code_byte_of<BITS>(cb), fb = code_field_of<BITS>(cb);
-                        const uint32_t a0 = code_pair_bf16(code_view<BITS>(w0[wa], fa), code_view<BITS>(w0[wa], fa + 1), ba);
-                        const uint32_t a1 = code_pair_bf16(code_view<BITS>(w1[wa], fa), code_view<BITS>(w1[wa], fa + 1), ba);
-                        const uint32_t a2 = code_pair_bf16(code_view<BITS>(w0[wb], fb), code_view<BITS>(w0[wb], fb + 1), bb);
-                        const uint32_t a3 = code_pair_bf16(code_view<BITS>(w1[wb], fb), code_view<BITS>(w1[wb], fb + 1), bb);
-                        mma_16816<BF>(c4, a0, a1, a2, a3, qb[kk][0], qb[kk][1]);
-                        mma_16816<BF>(c4, a0, a1, a2, a3, ql[kk][0], ql[kk][1]);
-                    }
-                } else {
-                    uint32_t w0[KC / 2], w1[KC / 2];  // the thread's KC channels of the two token rows, 16-bit pairs
-                    load_words_or_zero<KC / 2>(ksys + (int64_t)(tok0 + r0) * p.s_st + KC * t, r0 < n_tok, w0);
-                    load_words_or_zero<KC / 2>(ksys + (int64_t)(tok0 + r1) * p.s_st + KC * t, r1 < n_tok, w1);
-#pragma unroll
-                    for (int kk = 0; kk < KS; ++kk) {
-                        mma_16816<CT>(c4, w0[2 * kk], w1[2 * kk], w0[2 * kk + 1], w1[2 * kk + 1], qb[kk][0], qb[kk][1]);
-                        mma_16816<CT>(c4, w0[2 * kk], w1[2 * kk], w0[2 * kk + 1], w1[2 * kk + 1], ql[kk][0], ql[kk][1]);
-                    }
-                }
-                if (r0 < n_tok) {
-                    sc[2 * t][warp * kAtSegTokens + r0] = c4[0] + bias_a;
-                    sc[2 * t + 1][warp * kAtSegTokens + r0] = c4[1] + bias_b;
-                }
-                if (r1 < n_tok) {
-                    sc[2 * t][warp * kAtSegTokens + r1] = c4[2] + bias_a;
-                    sc[2 * t + 1][warp * kAtSegTokens + r1] = c4[3] + bias_b;
-                }
-            }
-        }
-        __syncthreads();
-
-        // ---- phase 2: the block's maximum per query head; scores become weights in place.  The sum of the weights is
-        //      taken in phase 3 from the ROUNDED weights the matrix product uses, so that numerator and denominator
-        //      of the softmax average see the same weights.
-        if (warp < kAtHeads) {
-            float mx = -INFINITY;
-            for (int i = lane; i < kSlots; i += 32) mx = fmaxf(mx, sc[warp][i]);
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-            for (int i = lane; i < kSlots; i += 32) {
-                const float v = sc[warp][i];
-                sc[warp][i] = v == -INFINITY ? 0.0f : exp2f(v - mx);
-            }
-            if (lane == 0) blk_max[warp] = mx;
-        }
-        __syncthreads();
-
-        // ---- phase 3: weighted sum of the values.  Rows of the product are channels: rows g and g + 8 of m-tile mm
-        //      stand for channels VC*g + 2*mm and VC*g + 2*mm + 1; the contraction runs over the segment's tokens
-        //      (slot 2t, 2t+1, 2t+8, 2t+9 of k-step ks is token 16*ks + the same); columns are query heads.
-        float acc[MT][4];
+        float m_a = -INFINITY, m_b = -INFINITY, l_a = 0.0f, l_b = 0.0f;  // running max / sum of query heads 2t, 2t + 1
+        float O[MT][4];  // running output: channels VC*g + 2*mm (+1) x query heads 2t, 2t + 1
 #pragma unroll
         for (int mm = 0; mm < MT; ++mm)
 #pragma unroll
-            for (int i = 0; i < 4; ++i) acc[mm][i] = 0.0f;
-        float wsum = 0.0f;  // sum of the weights of query head g as the tensor core sees them
-        if (n_tok > 0) {
-#pragma unroll
-            for (int ks = 0; ks < kAtSegTokens / 16; ++ks) {
-                if (ks * 16 >= n_tok) break;  // warp-uniform
-                const int ta = ks * 16 + 2 * t;  // tokens ta, ta + 1, ta + 8, ta + 9
-                const float2 wlo = *reinterpret_cast<const float2 *>(&sc[g][warp * kAtSegTokens + ta]);
-                const float2 whi = *reinterpret_cast<const float2 *>(&sc[g][warp * kAtSegTokens + ta + 8]);
-                uint32_t b0, b1, l0, l1;  // the weights, high and low parts
-                float r0, r1, r2, r3;
-                if (!is_sys) {
-                    split2<BF>(wlo.x, wlo.y, b0, l0, r0, r1);
-                    split2<BF>(whi.x, whi.y, b1, l1, r2, r3);
-                } else {
-                    split2<CT>(wlo.x, wlo.y, b0, l0, r0, r1);
-                    split2<CT>(whi.x, whi.y, b1, l1, r2, r3);
+            for (int i = 0; i < 4; ++i) O[mm][i] = 0.0f;
+
+        for (int i = 0; i < n_mine && !dead; ++i) {
+            const int s = i % S;
+            const uint32_t info = (stage_info >> (8 * s)) & 0xFFu;
+            const int n_tok = (int)(info & 0x7Fu);
+            const bool is_sys = (info & 0x80u) != 0;
+            const unsigned char *st = my_ring + (size_t)s * p.stage_bytes;
+            if (n_tok > 0) {
+                const bool ok = mbar_wait_bounded(bar0 + 8 * s, (phase_bits >> s) & 1u, abort_flag, kAtWaitLimitNs);
+                if (!__all_sync(0xffffffffu, ok)) {
+                    if (lane == 0) {
+                        if (p.flags) atomicOr(p.flags, STOM_FLAG_TIMEOUT);
+                        *abort_flag = 1;
+                    }
+                    dead = true;
+                    break;
                 }
-                wsum += (r0 + r1) + (r2 + r3);
-                if (!is_sys) {
-                    uint32_t w[4][(VB + 3) / 4];  // the thread's VC codes of its 4 tokens
+                phase_bits ^= 1u << s;
+                stage_info &= ~(0xFFu << (8 * s));  // consumed: nothing of this stage is in flight any more
+
+                // ---- phase 1: scores.  Contraction slot (kk; 2t, 2t+1, 2t+8, 2t+9) of the matrix product stands for
+                //      channels KC*t + 4*kk + (0, 1, 2, 3); column g is query head g.
+                const int n_mt = (n_tok + 15) >> 4;
+                float sc[kAtUnitTokens / 16][4];
+                {
+                    uint32_t qb[KS][2], ql[KS][2];  // the thread's column of the right-hand operand, high and low parts
+                    float bias = 0.0f;              // what the raw-code product leaves out, for query head g
+                    if (!is_sys) {
+                        const unsigned char *sk = st + 2 * code_block, *mk = sk + meta_row;
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int tok = ta + (i & 1) + 8 * (i >> 1);
-                        load_code_bytes<VB>(vcodes + (int64_t)(tok0 + tok) * p.g.row_bytes + g * VB, tok < n_tok, w[i]);
+                        for (int c8 = 0; c8 < KC / 8; ++c8) {
+                            float s8[8], m8[8];
+                            lds_meta8(sk, KC * t + c8 * 8, md, s8);
+                            lds_meta8(mk, KC * t + c8 * 8, md, m8);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {  // 2 channels each
+                                const int c = c8 * 8 + 2 * j;
+                                float q0, q1;
+                                qr.pair(c / 2, q0, q1);
+                                uint32_t whi, wlo;
+                                float r0, r1;  // the two products as the tensor core sees them
+                                split2<BF>(q0 * s8[2 * j], q1 * s8[2 * j + 1], whi, wlo, r0, r1);
+                                bias = fmaf(q0, m8[2 * j], bias);
+                                bias = fmaf(q1, m8[2 * j + 1], bias);
+                                bias = fmaf(-128.0f, r0 + r1, bias);
+                                qb[c / 4][(c / 2) & 1] = whi;
+                                ql[c / 4][(c / 2) & 1] = wlo;
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < KC / 2; ++j) {
+                            float q0, q1, r0, r1;
+                            qr.pair(j, q0, q1);
+                            split2<CT>(q0, q1, qb[j / 2][j & 1], ql[j / 2][j & 1], r0, r1);
+                        }
                     }
+                    bias += __shfl_xor_sync(0xffffffffu, bias, 1);
+                    bias += __shfl_xor_sync(0xffffffffu, bias, 2);
+                    const float bias_a = __shfl_sync(0xffffffffu, bias, (2 * t) << 2);       // of query head 2t
+                    const float bias_b = __shfl_sync(0xffffffffu, bias, (2 * t + 1) << 2);   // of query head 2t + 1
+                    // Two m-tiles at a time, and the high and low part of the right-hand operand into accumulators of
+                    // their own: four independent chains of dependent products instead of one.
 #pragma unroll
-                    for (int mm = 0; mm < MT; ++mm) {
-                        // channels VC*g + 2*mm and the next one share a byte; rows g and g + 8 of the m-tile
-                        const int c = 2 * mm;
-                        const int j = code_word_of<BITS>(c), b = code_byte_of<BITS>(c), f = code_field_of<BITS>(c);
-                        const uint32_t a0 = code_pair_bf16(code_view<BITS>(w[0][j], f), code_view<BITS>(w[1][j], f), b);
-                        const uint32_t a1 = code_pair_bf16(code_view<BITS>(w[0][j], f + 1), code_view<BITS>(w[1][j], f + 1), b);
-                        const uint32_t a2 = code_pair_bf16(code_view<BITS>(w[2][j], f), code_view<BITS>(w[3][j], f), b);
-                        const uint32_t a3 = code_pair_bf16(code_view<BITS>(w[2][j], f + 1), code_view<BITS>(w[3][j], f + 1), b);
-                        mma_16816<BF>(acc[mm], a0, a1, a2, a3, b0, b1);
-                        mma_16816<BF>(acc[mm], a0, a1, a2, a3, l0, l1);
-                    }
-                } else {
-                    uint32_t w[4][VC / 2];  // the thread's VC channels of its 4 tokens, 16-bit pairs (channel 2mm, 2mm+1)
+                    for (int mp = 0; mp < kAtUnitTokens / 32; ++mp) {
+                        float ch[2][4], cl[2][4];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        const int tok = ta + (i & 1) + 8 * (i >> 1);
-                        load_words_or_zero<VC / 2>(vsys + (int64_t)(tok0 + tok) * p.s_st + VC * g, tok < n_tok, w[i]);
-                    }
+                        for (int u = 0; u < 2; ++u)
 #pragma unroll
-                    for (int mm = 0; mm < MT; ++mm) {
-                        const uint32_t a0 = __byte_perm(w[0][mm], w[1][mm], 0x5410), a1 = __byte_perm(w[0][mm], w[1][mm], 0x7632);
-                        const uint32_t a2 = __byte_perm(w[2][mm], w[3][mm], 0x5410), a3 = __byte_perm(w[2][mm], w[3][mm], 0x7632);
-                        mma_16816<CT>(acc[mm], a0, a1, a2, a3, b0, b1);
-                        mma_16816<CT>(acc[mm], a0, a1, a2, a3, l0, l1);
+                            for (int e = 0; e < 4; ++e) ch[u][e] = cl[u][e] = 0.0f;
+                        if (2 * mp < n_mt) {  // warp-uniform
+                            if (!is_sys) {
+                                uint32_t w[2][2][(KB + 3) / 4];  // [m-tile of the pair][row g / row g + 8]: the thread's KC codes
+#pragma unroll
+                                for (int u = 0; u < 2; ++u)
+#pragma unroll
+                                    for (int v = 0; v < 2; ++v) {
+                                        const int row = (2 * mp + u) * 16 + g + 8 * v;
+                                        lds_code_bytes<KB>(st + row * p.g.row_bytes + t * KB, row < n_tok, w[u][v]);
+                                    }
+#pragma unroll
+                                for (int kk = 0; kk < KS; ++kk) {
+                                    // codes 4kk, 4kk+1 of the thread's run share a byte, and so do 4kk+2, 4kk+3
+                                    const int ca = 4 * kk, cb = 4 * kk + 2;
+                                    const int wa = code_word_of<BITS>(ca), ba = code_byte_of<BITS>(ca), fa = code_field_of<BITS>(ca);
+                                    const int wb = code_word_of<BITS>(cb), bb = code_byte_of<BITS>(cb), fb = code_field_of<BITS>(cb);
+#pragma unroll
+                                    for (int u = 0; u < 2; ++u) {
+                                        const uint32_t a0 = code_pair_bf16(code_view<BITS>(w[u][0][wa], fa), code_view<BITS>(w[u][0][wa], fa + 1), ba);
+                                        const uint32_t a1 = code_pair_bf16(code_view<BITS>(w[u][1][wa], fa), code_view<BITS>(w[u][1][wa], fa + 1), ba);
+                                        const uint32_t a2 = code_pair_bf16(code_view<BITS>(w[u][0][wb], fb), code_view<BITS>(w[u][0][wb], fb + 1), bb);
+                                        const uint32_t a3 = code_pair_bf16(code_view<BITS>(w[u][1][wb], fb), code_view<BITS>(w[u][1][wb], fb + 1), bb);
+                                        mma_16816<BF>(ch[u], a0, a1, a2, a3, qb[kk][0], qb[kk][1]);
+                                        mma_16816<BF>(cl[u], a0, a1, a2, a3, ql[kk][0], ql[kk][1]);
+                                    }
+                                }
+                            } else if (mp == 0) {  // a system-token unit is one m-tile
+                                uint32_t w0[KC / 2], w1[KC / 2];  // the thread's KC channels of the two token rows, 16-bit pairs
+                                lds_words_or_zero<KC / 2>(st + (g * D + KC * t) * (int)sizeof(CT), g < n_tok, w0);
+                                lds_words_or_zero<KC / 2>(st + ((g + 8) * D + KC * t) * (int)sizeof(CT), g + 8 < n_tok, w1);
+#pragma unroll
+                                for (int kk = 0; kk < KS; ++kk) {
+                                    mma_16816<CT>(ch[0], w0[2 * kk], w1[2 * kk], w0[2 * kk + 1], w1[2 * kk + 1], qb[kk][0], qb[kk][1]);
+                                    mma_16816<CT>(cl[0], w0[2 * kk], w1[2 * kk], w0[2 * kk + 1], w1[2 * kk + 1], ql[kk][0], ql[kk][1]);
+                                }
+                            }
+                        }
+                        // base-2 scores; token slots without a token never win the maximum and weigh nothing
+#pragma unroll
+                        for (int u = 0; u < 2; ++u) {
+                            const int mt = 2 * mp + u, r0 = mt * 16 + g, r1 = r0 + 8;
+                            sc[mt][0] = r0 < n_tok ? (ch[u][0] + cl[u][0] + bias_a) * p.scale_log2e : -INFINITY;
+                            sc[mt][1] = r0 < n_tok ? (ch[u][1] + cl[u][1] + bias_b) * p.scale_log2e : -INFINITY;
+                            sc[mt][2] = r1 < n_tok ? (ch[u][2] + cl[u][2] + bias_a) * p.scale_log2e : -INFINITY;
+                            sc[mt][3] = r1 < n_tok ? (ch[u][3] + cl[u][3] + bias_b) * p.scale_log2e : -INFINITY;
+                        }
                     }
                 }
-            }
-        }
-        wsum += __shfl_xor_sync(0xffffffffu, wsum, 1);
-        wsum += __shfl_xor_sync(0xffffffffu, wsum, 2);
-        const float ws_a = __shfl_sync(0xffffffffu, wsum, (2 * t) << 2), ws_b = __shfl_sync(0xffffffffu, wsum, (2 * t + 1) << 2);
-        if (t == 0) seg_sum[warp][g] = wsum;
-        if (!is_sys && n_tok > 0) {
-            // acc holds sum_t w_t (128 + code): apply the group's scale and offset, channel by channel
+
+                // ---- phase 2: the warp's own online softmax.  New running maxima of query heads 2t, 2t + 1; the
+                //      scores become weights in the warp's tile [head][token slot]; the running sums and outputs
+                //      are rescaled.  The sum of the weights is taken in phase 3 from the ROUNDED weights the matrix
+                //      product uses, so that numerator and denominator of the softmax average see the same weights.
+                float mx_a = -INFINITY, mx_b = -INFINITY;
 #pragma unroll
-            for (int c8 = 0; c8 < VC / 8; ++c8) {
-                float s8[8], m8[8];
-                load_scale_zero8(p.scale_v, p.zero_v, slot * D + VC * g + c8 * 8, md, s8, m8);
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int mm = c8 * 4 + j;
-                    acc[mm][0] = fmaf(s8[2 * j], fmaf(-128.0f, ws_a, acc[mm][0]), m8[2 * j] * ws_a);
-                    acc[mm][1] = fmaf(s8[2 * j], fmaf(-128.0f, ws_b, acc[mm][1]), m8[2 * j] * ws_b);
-                    acc[mm][2] = fmaf(s8[2 * j + 1], fmaf(-128.0f, ws_a, acc[mm][2]), m8[2 * j + 1] * ws_a);
-                    acc[mm][3] = fmaf(s8[2 * j + 1], fmaf(-128.0f, ws_b, acc[mm][3]), m8[2 * j + 1] * ws_b);
+                for (int mt = 0; mt < kAtUnitTokens / 16; ++mt) {
+                    mx_a = fmaxf(mx_a, fmaxf(sc[mt][0], sc[mt][2]));
+                    mx_b = fmaxf(mx_b, fmaxf(sc[mt][1], sc[mt][3]));
                 }
-            }
-        }
-        __syncthreads();  // every warp is done with the weights; the buffer now takes the warps' sums
-        float tot[kAtHeads * D / kAtThreads];
 #pragma unroll
-        for (int e = 0; e < kAtHeads * D / kAtThreads; ++e) tot[e] = 0.0f;
-        for (int r = 0; r < kAtWarps; r += kBuf) {
-            if (warp >= r && warp < r + kBuf) {
-                float *dst = buf + (size_t)(warp - r) * kAtHeads * D;
+                for (int o = 4; o < 32; o <<= 1) {
+                    mx_a = fmaxf(mx_a, __shfl_xor_sync(0xffffffffu, mx_a, o));
+                    mx_b = fmaxf(mx_b, __shfl_xor_sync(0xffffffffu, mx_b, o));
+                }
+                const float mn_a = fmaxf(m_a, mx_a), mn_b = fmaxf(m_b, mx_b);  // finite: the unit has a token
+                const float al_a = exp2f(m_a - mn_a), al_b = exp2f(m_b - mn_b);  // 0 on the first unit
+                m_a = mn_a;
+                m_b = mn_b;
+#pragma unroll
+                for (int mt = 0; mt < kAtUnitTokens / 16; ++mt) {
+                    const int r0 = mt * 16 + g;
+                    wt[(2 * t) * kAtWPitch + r0] = exp2f(sc[mt][0] - mn_a);
+                    wt[(2 * t + 1) * kAtWPitch + r0] = exp2f(sc[mt][1] - mn_b);
+                    wt[(2 * t) * kAtWPitch + r0 + 8] = exp2f(sc[mt][2] - mn_a);
+                    wt[(2 * t + 1) * kAtWPitch + r0 + 8] = exp2f(sc[mt][3] - mn_b);
+                }
+                l_a *= al_a;
+                l_b *= al_b;
 #pragma unroll
                 for (int mm = 0; mm < MT; ++mm) {
-                    const int c = VC * g + 2 * mm;
-                    dst[(2 * t) * D + c] = acc[mm][0];
-                    dst[(2 * t + 1) * D + c] = acc[mm][1];
-                    dst[(2 * t) * D + c + 1] = acc[mm][2];
-                    dst[(2 * t + 1) * D + c + 1] = acc[mm][3];
+                    O[mm][0] *= al_a; O[mm][1] *= al_b; O[mm][2] *= al_a; O[mm][3] *= al_b;
                 }
-            }
-            __syncthreads();
+                __syncwarp();
+
+                // ---- phase 3: weighted sum of the values.  Rows of the product are channels: rows g and g + 8 of
+                //      m-tile mm stand for channels VC*g + 2*mm and VC*g + 2*mm + 1; the contraction runs over the
+                //      unit's tokens (slot 2t, 2t+1, 2t+8, 2t+9 of k-step ks is token 16*ks + the same); columns are
+                //      query heads.  d = 256 takes two passes of 8 m-tiles over the same weights.
+                const unsigned char *vst = st + (is_sys ? kAtSysTokens * D * (int)sizeof(CT) : code_block);
 #pragma unroll
-            for (int e = 0; e < kAtHeads * D / kAtThreads; ++e) {
-                const int i = e * kAtThreads + tid;  // (head, channel) pair
-                for (int w = 0; w < kBuf && r + w < kAtWarps; ++w) tot[e] += buf[(size_t)w * kAtHeads * D + i];
-            }
-            __syncthreads();
-        }
-        // ---- partial result of this block: (max, sum, weighted sum) per query head
+                for (int m0 = 0; m0 < MT; m0 += MH) {
+                    float acc[MH][4];
 #pragma unroll
-        for (int e = 0; e < kAtHeads * D / kAtThreads; ++e) {
-            const int i = e * kAtThreads + tid, hh = i / D, c = i - hh * D;
-            if (hh < nh) {
-                float *rec = p.part + ((((int64_t)li * H + h) * n_blocks + bx) * p.rep + h0 + hh) * (D + 2);
-                rec[2 + c] = tot[e];
-                if (c == 0) {
-                    float sum = 0.0f;
+                    for (int mm = 0; mm < MH; ++mm)
 #pragma unroll
-                    for (int w = 0; w < kAtWarps; ++w) sum += seg_sum[w][hh];
-                    rec[0] = blk_max[hh];
-                    rec[1] = sum;
+                        for (int e = 0; e < 4; ++e) acc[mm][e] = 0.0f;
+                    float wsum = 0.0f;  // sum of the weights of query head g as the tensor core sees them
+#pragma unroll
+                    for (int ks = 0; ks < kAtUnitTokens / 16; ++ks) {
+                        if (ks < n_mt) {  // warp-uniform
+                            const int ta = ks * 16 + 2 * t;  // tokens ta, ta + 1, ta + 8, ta + 9
+                            const float2 wlo = *reinterpret_cast<const float2 *>(&wt[g * kAtWPitch + ta]);
+                            const float2 whi = *reinterpret_cast<const float2 *>(&wt[g * kAtWPitch + ta + 8]);
+                            uint32_t b0, b1, l0, l1;  // the weights, high and low parts
+                            float r0, r1, r2, r3;
+                            if (!is_sys) {
+                                split2<BF>(wlo.x, wlo.y, b0, l0, r0, r1);
+                                split2<BF>(whi.x, whi.y, b1, l1, r2, r3);
+                            } else {
+                                split2<CT>(wlo.x, wlo.y, b0, l0, r0, r1);
+                                split2<CT>(whi.x, whi.y, b1, l1, r2, r3);
+                            }
+                            wsum += (r0 + r1) + (r2 + r3);
+                            if (!is_sys) {
+                                uint32_t w[4][(VB + 3) / 4];  // the thread's VC codes of its 4 tokens
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const int tok = ta + (e & 1) + 8 * (e >> 1);
+                                    lds_code_bytes<VB>(vst + tok * p.g.row_bytes + g * VB, tok < n_tok, w[e]);
+                                }
+#pragma unroll
+                                for (int mm = 0; mm < MH; ++mm) {
+                                    // channels VC*g + 2*mm and the next one share a byte; rows g and g + 8 of the m-tile
+                                    const int c = 2 * (m0 + mm);
+                                    const int j = code_word_of<BITS>(c), b = code_byte_of<BITS>(c), f = code_field_of<BITS>(c);
+                                    const uint32_t a0 = code_pair_bf16(code_view<BITS>(w[0][j], f), code_view<BITS>(w[1][j], f), b);
+                                    const uint32_t a1 = code_pair_bf16(code_view<BITS>(w[0][j], f + 1), code_view<BITS>(w[1][j], f + 1), b);
+                                    const uint32_t a2 = code_pair_bf16(code_view<BITS>(w[2][j], f), code_view<BITS>(w[3][j], f), b);
+                                    const uint32_t a3 = code_pair_bf16(code_view<BITS>(w[2][j], f + 1), code_view<BITS>(w[3][j], f + 1), b);
+                                    mma_16816<BF>(acc[mm], a0, a1, a2, a3, b0, b1);
+                                    mma_16816<BF>(acc[mm], a0, a1, a2, a3, l0, l1);
+                                }
+                            } else if (ks == 0) {
+                                uint32_t w[4][VC / 2];  // the thread's VC channels of its 4 tokens, 16-bit pairs (channel 2mm, 2mm+1)
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    const int tok = ta + (e & 1) + 8 * (e >> 1);
+                                    lds_words_or_zero<VC / 2>(vst + (tok * D + VC * g) * (int)sizeof(CT), tok < n_tok, w[e]);
+                                }
+#pragma unroll
+                                for (int mm = 0; mm < MH; ++mm) {
+                                    const int j = m0 + mm;
+                                    const uint32_t a0 = __byte_perm(w[0][j], w[1][j], 0x5410), a1 = __byte_perm(w[0][j], w[1][j], 0x7632);
+                                    const uint32_t a2 = __byte_perm(w[2][j], w[3][j], 0x5410), a3 = __byte_perm(w[2][j], w[3][j], 0x7632);
+                                    mma_16816<CT>(acc[mm], a0, a1, a2, a3, b0, b1);
+                                    mma_16816<CT>(acc[mm], a0, a1, a2, a3, l0, l1);
+                                }
+                            }
+                        }
+                    }
+                    wsum += __shfl_xor_sync(0xffffffffu, wsum, 1);
+                    wsum += __shfl_xor_sync(0xffffffffu, wsum, 2);
+                    const float ws_a = __shfl_sync(0xffffffffu, wsum, (2 * t) << 2), ws_b = __shfl_sync(0xffffffffu, wsum, (2 * t + 1) << 2);
+                    if (m0 == 0) {
+                        l_a += ws_a;
+                        l_b += ws_b;
+                    }
+                    if (!is_sys) {
+                        // acc holds sum_t w_t (128 + code): apply the group's scale and offset, channel by channel
+                        const unsigned char *sv = st + 2 * code_block + 2 * meta_row, *mv = sv + meta_row;
+#pragma unroll
+                        for (int c8 = 0; c8 < 2 * MH / 8; ++c8) {
+                            float s8[8], m8[8];
+                            lds_meta8(sv, VC * g + 2 * m0 + c8 * 8, md, s8);
+                            lds_meta8(mv, VC * g + 2 * m0 + c8 * 8, md, m8);
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                const int mm = c8 * 4 + j;
+                                O[m0 + mm][0] += fmaf(s8[2 * j], fmaf(-128.0f, ws_a, acc[mm][0]), m8[2 * j] * ws_a);
+                                O[m0 + mm][1] += fmaf(s8[2 * j], fmaf(-128.0f, ws_b, acc[mm][1]), m8[2 * j] * ws_b);
+                                O[m0 + mm][2] += fmaf(s8[2 * j + 1], fmaf(-128.0f, ws_a, acc[mm][2]), m8[2 * j + 1] * ws_a);
+                                O[m0 + mm][3] += fmaf(s8[2 * j + 1], fmaf(-128.0f, ws_b, acc[mm][3]), m8[2 * j + 1] * ws_b);
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int mm = 0; mm < MH; ++mm)
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) O[m0 + mm][e] += acc[mm][e];
+                    }
                 }
+                __syncwarp();  // every lane is done with the stage and with the weight tile
+            }
+            // ---- the stage is free: post the unit that comes S units later
+            const int in = i + S;
+            if (in < n_mine) {
+                if ((in & 31) == 0) tg_batch = load_tg_batch(in);
+                post_unit(in, __shfl_sync(0xffffffffu, tg_batch, in & 31));
             }
         }
-        __syncthreads();  // qf, buf and the statistics are rewritten by the next chunk of heads
+
+        // ---- merge the warps of the block.  Each warp rescales its output to the block's maximum and parks it in its
+        //      own first stage, laid out [channel slab g][channel][head] with padded slabs so that neither these
+        //      stores nor the sums below collide on shared-memory banks.
+        if (dead) {
+            m_a = m_b = -INFINITY;
+            l_a = l_b = 0.0f;
+        }
+        if (g == 0) {
+            stat[warp * 16 + 2 * t] = m_a;
+            stat[warp * 16 + 2 * t + 1] = m_b;
+            stat[warp * 16 + 8 + 2 * t] = l_a;
+            stat[warp * 16 + 8 + 2 * t + 1] = l_b;
+        }
+        // nothing of this warp may still be landing in the stage that now takes its result (only after a wait ran out)
+        for (int s = 0; s < S; ++s) {
+            if ((stage_info >> (8 * s)) & 0x7Fu) {
+                mbar_wait_bounded(bar0 + 8 * s, (phase_bits >> s) & 1u, abort_flag + 1, kAtWaitLimitNs);
+                phase_bits ^= 1u << s;
+                stage_info &= ~(0xFFu << (8 * s));
+            }
+        }
+        __syncthreads();
+        {
+            float M_a = -INFINITY, M_b = -INFINITY;
+#pragma unroll
+            for (int w = 0; w < kAtWarps; ++w) {
+                M_a = fmaxf(M_a, stat[w * 16 + 2 * t]);
+                M_b = fmaxf(M_b, stat[w * 16 + 2 * t + 1]);
+            }
+            const float f_a = m_a == -INFINITY ? 0.0f : exp2f(m_a - M_a), f_b = m_b == -INFINITY ? 0.0f : exp2f(m_b - M_b);
+            float *mine = reinterpret_cast<float *>(my_ring) + g * OP + 2 * t;
+#pragma unroll
+            for (int mm = 0; mm < MT; ++mm) {
+                *reinterpret_cast<float2 *>(mine + (2 * mm) * 8) = make_float2(O[mm][0] * f_a, O[mm][1] * f_b);
+                *reinterpret_cast<float2 *>(mine + (2 * mm + 1) * 8) = make_float2(O[mm][2] * f_a, O[mm][3] * f_b);
+            }
+        }
+        __syncthreads();
+        for (int e = tid; e < OF; e += kAtThreads) {
+            float a = 0.0f;
+#pragma unroll
+            for (int w = 0; w < kAtWarps; ++w)
+                a += reinterpret_cast<const float *>(ring + (size_t)w * S * p.stage_bytes)[e];
+            ob[e] = a;
+        }
+        if (tid < kAtHeads) {
+            float M = -INFINITY, L = 0.0f;
+#pragma unroll
+            for (int w = 0; w < kAtWarps; ++w) M = fmaxf(M, stat[w * 16 + tid]);
+#pragma unroll
+            for (int w = 0; w < kAtWarps; ++w) {
+                const float mw = stat[w * 16 + tid];
+                if (mw != -INFINITY) L = fmaf(stat[w * 16 + 8 + tid], exp2f(mw - M), L);
+            }
+            blk[tid] = M;
+            blk[8 + tid] = L;
+        }
+
+        // ---- merge the blocks of the cluster: rank r finishes its share of the (channel, head) pairs
+        if (C > 1) cluster_sync(); else __syncthreads();
+        {
+            const int per = (OF + (int)C - 1) / (int)C;
+            const int e_end = min(per * ((int)r + 1), OF);
+            for (int e = per * (int)r + tid; e < e_end; e += kAtThreads) {
+                const int slab = e / OP, rem = e - slab * OP;
+                const int hh = rem & 7, cl = rem >> 3;
+                if (cl >= VC || hh >= nh) continue;  // padding, or a head beyond the GQA block
+                float num = 0.0f, den = 0.0f;
+                if (C > 1) {
+                    // every block's (max, sum, partial) of this pair is asked for before any of them is used
+                    float Mb[8], Lb[8], Ov[8];
+#pragma unroll
+                    for (uint32_t b = 0; b < 8; ++b) {
+                        Mb[b] = -INFINITY;
+                        Lb[b] = Ov[b] = 0.0f;
+                        if (b < C) {
+                            Mb[b] = ld_cluster_f(blk + hh, b);
+                            Lb[b] = ld_cluster_f(blk + 8 + hh, b);
+                            Ov[b] = ld_cluster_f(ob + e, b);
+                        }
+                    }
+                    float M = -INFINITY;
+#pragma unroll
+                    for (int b = 0; b < 8; ++b) M = fmaxf(M, Mb[b]);
+#pragma unroll
+                    for (int b = 0; b < 8; ++b) {
+                        const float f = Mb[b] == -INFINITY ? 0.0f : exp2f(Mb[b] - M);
+                        num = fmaf(Ov[b], f, num);
+                        den = fmaf(Lb[b], f, den);
+                    }
+                } else {
+                    num = ob[e];
+                    den = blk[8 + hh];
+                }
+                CT *out = reinterpret_cast<CT *>(p.out) + (int64_t)li * p.o_sl + (int64_t)(h * p.rep + h0 + hh) * p.o_sh;
+                out[VC * slab + cl] = (CT)(den > 0.0f ? num / den : 0.0f);
+            }
+        }
+        // nobody leaves, or reuses its buffers for the next chunk of heads, while a neighbour still reads from them
+        if (C > 1) cluster_sync(); else __syncthreads();
     }
-    attend_merge<CT, D>(p, li, h, n_blocks, &s_last);
 }
 
-// The ticket counters take the same room whatever the layer range of a call, so that a workspace cleared once serves
-// calls over any layer range of the bank.
-static int64_t attend_counter_bytes(const stom_oqm_config *cfg) {
-    return ((int64_t)cfg->n_layers * cfg->n_kv_heads * 4 + 255) / 256 * 256;
+static int attend_units(const stom_oqm_config *cfg, int32_t k, int32_t sys_len, int *n_sys_units) {
+    *n_sys_units = (sys_len + kAtSysTokens - 1) / kAtSysTokens;
+    return *n_sys_units + k;
 }
 
-static int attend_segments(const stom_oqm_config *cfg, int32_t k, int32_t sys_len, int *n_sys_seg, int *segs_per_group) {
-    *n_sys_seg = (sys_len + kAtSegTokens - 1) / kAtSegTokens;
-    *segs_per_group = (cfg->group_tokens + kAtSegTokens - 1) / kAtSegTokens;
-    return *n_sys_seg + k * *segs_per_group;
+// bytes of one ring stage: a group's K and V codes and its four metadata rows, or 16 system tokens of K and of V
+static int attend_stage_bytes(const stom_oqm_config *cfg) {
+    const int group = 2 * cfg->group_tokens * (cfg->head_dim * cfg->bits / 8) + 4 * cfg->head_dim * elem_bytes(cfg->meta_dtype);
+    const int sys = 2 * kAtSysTokens * cfg->head_dim * 2;
+    const int b = group > sys ? group : sys;
+    return (b + 127) / 128 * 128;
+}
+
+template <typename KernelT>
+static int32_t launch_attend_kernel(KernelT kernel, const AttendParams &p, int D, int units, int pairs_h, int layers,
+                                    cudaStream_t s) {
+    int dev = 0, sms = 0, smem_max = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&smem_max, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (e != cudaSuccess) {
+        set_last_cuda_error(e);
+        return STOM_ERR_CUDA;
+    }
+    AttendParams q = p;
+    const int fixed = at_off_ring(D);
+    q.n_stages = fixed + kAtWarps * 2 * q.stage_bytes <= smem_max ? 2 : 1;
+    const size_t smem = (size_t)fixed + (size_t)kAtWarps * q.n_stages * q.stage_bytes;
+    if ((int64_t)smem > smem_max) return STOM_ERR_SHAPE;
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) {
+        set_last_cuda_error(e);
+        return STOM_ERR_CUDA;
+    }
+    // Blocks per (layer, kv head): as many as keep every block busy for the same number of rounds of units without
+    // sending more blocks to a multiprocessor than the others get; more blocks on a tie (fewer bytes per block).
+    const int64_t pairs = (int64_t)pairs_h * layers;
+    int best_c = 1;
+    int64_t best_cost = INT64_MAX;
+    for (int c = 1; c <= 8; ++c) {
+        if (c > 1 && (c - 1) * kAtWarps >= units) break;  // the last block would have nothing to do
+        const int64_t per_sm = (pairs * c + sms - 1) / sms;
+        const int64_t rounds = (units + c * kAtWarps - 1) / (c * kAtWarps);
+        const int64_t cost = per_sm * rounds;
+        if (cost <= best_cost) {
+            best_cost = cost;
+            best_c = c;
+        }
+    }
+    cudaLaunchConfig_t lc = {};
+    lc.blockDim = dim3(kAtThreads);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = 1;
+    lc.attrs = at;
+    lc.numAttrs = 1;
+    for (int c = best_c;; --c) {
+        lc.gridDim = dim3((unsigned)c, (unsigned)pairs_h, (unsigned)layers);
+        at[0].val.clusterDim.x = (unsigned)c;
+        int resident = 0;
+        if (c == 1 || (cudaOccupancyMaxActiveClusters(&resident, kernel, &lc) == cudaSuccess && resident >= 1)) break;
+        (void)cudaGetLastError();
+    }
+    e = cudaLaunchKernelEx(&lc, kernel, q);
+    if (e != cudaSuccess) {
+        set_last_cuda_error(e);
+        return STOM_ERR_CUDA;
+    }
+    return finish_launch();
 }
 
 template <typename QT, typename CT>
-static int32_t launch_attend(const AttendParams &p, dim3 grid, cudaStream_t s) {
+static int32_t launch_attend(const AttendParams &p, int units, int layers, cudaStream_t s) {
     const bool b4 = p.g.row_bytes * 2 == p.g.d;  // 4-bit codes: d/2 bytes per row
+    const int H = p.g.H;
     switch (p.g.d) {
     case 64:
-        if (b4) attend_mma_kernel<QT, CT, 64, 4><<<grid, kAtThreads, 0, s>>>(p);
-        else attend_mma_kernel<QT, CT, 64, 2><<<grid, kAtThreads, 0, s>>>(p);
-        break;
+        return b4 ? launch_attend_kernel(attend_kernel<QT, CT, 64, 4>, p, 64, units, H, layers, s)
+                  : launch_attend_kernel(attend_kernel<QT, CT, 64, 2>, p, 64, units, H, layers, s);
     case 128:
-        if (b4) attend_mma_kernel<QT, CT, 128, 4><<<grid, kAtThreads, 0, s>>>(p);
-        else attend_mma_kernel<QT, CT, 128, 2><<<grid, kAtThreads, 0, s>>>(p);
-        break;
+        return b4 ? launch_attend_kernel(attend_kernel<QT, CT, 128, 4>, p, 128, units, H, layers, s)
+                  : launch_attend_kernel(attend_kernel<QT, CT, 128, 2>, p, 128, units, H, layers, s);
     case 256:
-        if (b4) attend_mma_kernel<QT, CT, 256, 4><<<grid, kAtThreads, 0, s>>>(p);
-        else attend_mma_kernel<QT, CT, 256, 2><<<grid, kAtThreads, 0, s>>>(p);
-        break;
+        return b4 ? launch_attend_kernel(attend_kernel<QT, CT, 256, 4>, p, 256, units, H, layers, s)
+                  : launch_attend_kernel(attend_kernel<QT, CT, 256, 2>, p, 256, units, H, layers, s);
     default: return STOM_ERR_SHAPE;
     }
-    return finish_launch();
 }
 
 }  // namespace stom
@@ -584,13 +781,7 @@ using namespace stom;
 extern "C" int64_t stom_oqm_attend_workspace_bytes(const stom_oqm_config *cfg, int32_t layer_count, int32_t k,
                                                    int32_t sys_len) {
     if (check_config(cfg) || layer_count < 0 || k < 0 || sys_len < 0) return STOM_ERR_INVALID_ARG;
-    int n_sys_seg = 0, spg = 0;
-    const int n_seg = attend_segments(cfg, k, sys_len, &n_sys_seg, &spg);
-    const int64_t blocks = (n_seg + kAtWarps - 1) / kAtWarps;
-    const int64_t counters = attend_counter_bytes(cfg);
-    const int64_t part = (int64_t)layer_count * cfg->n_kv_heads * blocks * (cfg->n_q_heads / cfg->n_kv_heads) *
-                         (cfg->head_dim + 2) * 4;
-    return counters + (part + 255) / 256 * 256;
+    return 256;  // the call keeps nothing in global memory; a token size so that callers written for a workspace keep working
 }
 
 extern "C" int32_t stom_oqm_attend(const stom_oqm_config *cfg, const stom_oqm_store *store,
@@ -602,6 +793,8 @@ extern "C" int32_t stom_oqm_attend(const stom_oqm_config *cfg, const stom_oqm_st
                                    int32_t sys_len, float softmax_scale,
                                    void *out, int64_t out_stride_layer, int64_t out_stride_head,
                                    void *workspace, int64_t workspace_bytes, uint32_t *dev_flags, void *stream) {
+    (void)workspace;
+    (void)workspace_bytes;
     int32_t rc = check_config(cfg);
     if (rc) return rc;
     if ((rc = check_store(store))) return rc;
@@ -617,11 +810,12 @@ extern "C" int32_t stom_oqm_attend(const stom_oqm_config *cfg, const stom_oqm_st
     if ((idx && (reinterpret_cast<uintptr_t>(idx) & 3u)) || (reinterpret_cast<uintptr_t>(q_dec) & 3u) ||
         (reinterpret_cast<uintptr_t>(out) & 1u))
         return STOM_ERR_ALIGNMENT;
+    // a thread reads its query channels as 32-bit words
+    if ((q_stride_layer * elem_bytes(cfg->kv_dtype)) % 4 || (q_stride_head * elem_bytes(cfg->kv_dtype)) % 4)
+        return STOM_ERR_ALIGNMENT;
     if (sys_len > 0 && (!aligned16(k_sys) || !aligned16(v_sys) || !stride_ok(sys_stride_layer, cache_dtype) ||
                         !stride_ok(sys_stride_head, cache_dtype) || !stride_ok(sys_stride_token, cache_dtype)))
         return STOM_ERR_ALIGNMENT;
-    const int64_t need = stom_oqm_attend_workspace_bytes(cfg, layer_count, k, sys_len);
-    if (!workspace || (reinterpret_cast<uintptr_t>(workspace) & 255u) || workspace_bytes < need) return STOM_ERR_WORKSPACE;
     if (layer_count == 0) return STOM_OK;
 
     AttendParams p;
@@ -631,29 +825,28 @@ extern "C" int32_t stom_oqm_attend(const stom_oqm_config *cfg, const stom_oqm_st
     p.q = q_dec; p.q_sl = q_stride_layer; p.q_sh = q_stride_head;
     p.ksys = k_sys; p.vsys = v_sys; p.s_sl = sys_stride_layer; p.s_sh = sys_stride_head; p.s_st = sys_stride_token;
     p.out = out; p.o_sl = out_stride_layer; p.o_sh = out_stride_head;
-    const int64_t counters = attend_counter_bytes(cfg);
-    p.counters = static_cast<uint32_t *>(workspace);
-    p.part = reinterpret_cast<float *>(static_cast<uint8_t *>(workspace) + counters);
     p.g = bank_geom(cfg);
     p.layer_begin = layer_begin; p.k = k; p.n_groups = n_groups;
     p.per_head = cfg->score_mode == STOM_SCORE_PER_HEAD;
     p.rep = cfg->n_q_heads / cfg->n_kv_heads;
     p.sys_len = sys_len;
-    p.n_seg = attend_segments(cfg, k, sys_len, &p.n_sys_seg, &p.segs_per_group);
+    p.n_units = attend_units(cfg, k, sys_len, &p.n_sys_units);
+    p.stage_bytes = attend_stage_bytes(cfg);
+    p.n_stages = 1;
     p.scale_log2e = softmax_scale * 1.4426950408889634f;
     p.flags = dev_flags;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // The ticket counters at the head of the workspace are zero on entry (the caller cleared the workspace once) and
-    // every call leaves them zero: no memset here -- ahead of the kernel in a CUDA graph it measured 7 us per call.
     if (layer_count > 65535 || cfg->n_kv_heads > 65535) return STOM_ERR_SHAPE;
-    const dim3 grid((p.n_seg + kAtWarps - 1) / kAtWarps, cfg->n_kv_heads, layer_count);
     const bool bf = cache_dtype == STOM_BF16;
     switch (cfg->kv_dtype) {
     case STOM_BF16:
-        return bf ? launch_attend<__nv_bfloat16, __nv_bfloat16>(p, grid, s) : launch_attend<__nv_bfloat16, __half>(p, grid, s);
+        return bf ? launch_attend<__nv_bfloat16, __nv_bfloat16>(p, p.n_units, layer_count, s)
+                  : launch_attend<__nv_bfloat16, __half>(p, p.n_units, layer_count, s);
     case STOM_FP16:
-        return bf ? launch_attend<__half, __nv_bfloat16>(p, grid, s) : launch_attend<__half, __half>(p, grid, s);
+        return bf ? launch_attend<__half, __nv_bfloat16>(p, p.n_units, layer_count, s)
+                  : launch_attend<__half, __half>(p, p.n_units, layer_count, s);
     default:
-        return bf ? launch_attend<float, __nv_bfloat16>(p, grid, s) : launch_attend<float, __half>(p, grid, s);
+        return bf ? launch_attend<float, __nv_bfloat16>(p, p.n_units, layer_count, s)
+                  : launch_attend<float, __half>(p, p.n_units, layer_count, s);
     }
 }

@@ -124,9 +124,9 @@ def test_attend_flags_bad_indices_and_skips_them(orc):
     assert torch.equal(outs[0][0], outs[1][0])
 
 
-def test_one_cleared_workspace_serves_calls_over_any_layer_range(orc):
-    """The workspace is cleared once; every call leaves its ticket counters at zero, so a call over all layers,
-    calls layer by layer and a call over a sub-range can follow each other and give the same rows."""
+def test_calls_over_any_layer_range_give_the_same_rows(orc):
+    """A call over all layers, calls layer by layer and a call over a sub-range follow each other and give the same
+    rows: the call keeps nothing between launches, whatever the workspace argument holds."""
     from paper_2510_18269_b200 import oqm
     sh = synth.Shape("attend-ws", L=5, H_q=14, H_k=2, d=128, G=50, T=40, T_q=1, k=6, seed=3)
     ocfg, gcfg, ost, gst, _ = P.random_bank(orc, oqm, sh, 0, seed=23)
@@ -154,32 +154,45 @@ def test_one_cleared_workspace_serves_calls_over_any_layer_range(orc):
     for l in range(L):
         assert torch.equal(run(l, 1)[0], whole[l])
     assert torch.equal(run(1, 3), whole[1:4])
+    ws.fill_(0xAB)           # the workspace argument is not read: its contents do not matter
     assert torch.equal(run(0, L), whole)
 
 
-def test_workspace_that_was_never_cleared_is_flagged(orc):
-    """The ticket counters must be zero on entry.  A workspace full of other bytes cannot give a valid ticket: the
-    call says so in dev_flags instead of returning rows that look plausible; after clearing, the same workspace works."""
+def test_system_tokens_with_a_padded_token_stride_and_many_units_per_warp(orc):
+    """System tokens whose rows are not adjacent in memory (token stride above d: one copy per row), more units than
+    one pass of the warps of a cluster takes (several units per warp, both ring stages in use), and k far above
+    what one batch of prefetched indices holds."""
     from paper_2510_18269_b200 import oqm
-    sh = synth.Shape("attend-dirty", L=2, H_q=8, H_k=2, d=128, G=16, T=20, T_q=1, k=5, seed=3)
-    ocfg, gcfg, ost, gst, _ = P.random_bank(orc, oqm, sh, 0, seed=31)
-    idx = torch.from_numpy(_selection(np.random.default_rng(4), sh.L, sh.T, sh.k, sh.k)).cuda()
-    q = torch.randn(sh.L, sh.H_q, sh.d).to(torch.bfloat16).cuda()
-    ws = torch.full((oqm.stom_oqm_attend_workspace_bytes(gcfg, sh.L, sh.k, 0) + 256,), 0xAB, dtype=torch.uint8, device="cuda")
+    sh = synth.Shape("attend-many", L=1, H_q=8, H_k=1, d=128, G=16, T=3000, T_q=1, k=2300, seed=3)
+    ocfg, gcfg, ost, gst, _ = P.random_bank(orc, oqm, sh, 0, seed=41)
+    L, Hq, d, k, sys_len, T = sh.L, sh.H_q, sh.d, sh.k, 75, sh.T
+    rng = np.random.default_rng(6)
+    idx = _selection(rng, L, T, k, k - 5)
+    g = torch.Generator().manual_seed(12)
+    q = torch.randn(L, Hq, d, generator=g).to(torch.bfloat16)
+    S = sys_len + k * sh.G
+    pitch = d + 64                                             # padded rows of the system-token cache
+    k_sys = torch.randn(L, 1, sys_len, pitch, generator=g).to(torch.bfloat16)
+    v_sys = torch.randn(L, 1, sys_len, pitch, generator=g).to(torch.bfloat16)
+    k_act = torch.zeros(L, 1, S, d, dtype=torch.bfloat16)
+    v_act = torch.zeros(L, 1, S, d, dtype=torch.bfloat16)
+    k_act[:, :, :sys_len] = k_sys[..., :d]
+    v_act[:, :, :sys_len] = v_sys[..., :d]
+    oka, ova = P.as_np16(k_act).copy(), P.as_np16(v_act).copy()
+    assert orc.dequant_gather(ocfg, ost, 0, L, idx, k, T, oka, ova, orc.BF16, P.active_strides(sh, S), sys_len) == 0
+    scale = 1.0 / np.sqrt(d)
+    n_tok = sys_len + (k - 5) * sh.G
+    want = np.stack([orc.to_f32(orc.attend(Hq, 1, d, P.as_np16(q)[l], orc.BF16, oka[l], ova[l], orc.BF16, S * d, d, n_tok,
+                                           scale, out_dtype=orc.BF16), orc.BF16) for l in range(L)])
+    out = torch.zeros(L, Hq, d, dtype=torch.bfloat16, device="cuda")
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws = torch.zeros(512, dtype=torch.uint8, device="cuda")
     ws = ws[(-ws.data_ptr()) % 256:]
-
-    def run():
-        out = torch.zeros(sh.L, sh.H_q, sh.d, dtype=torch.bfloat16, device="cuda")
-        flags = torch.zeros(1, dtype=torch.int32, device="cuda")
-        oqm.stom_oqm_attend(gcfg, gst, 0, sh.L, idx, sh.k, sh.T, q, (sh.H_q * sh.d, sh.d), None, None, oqm.BF16,
-                            (0, 0, sh.d), 0, 0.09, out, (sh.H_q * sh.d, sh.d), ws, dev_flags=flags)
-        torch.cuda.synchronize()
-        return out, int(flags.item())
-
-    _, flags = run()
-    assert flags & oqm.FLAG_DIRTY_WORKSPACE
-    ws.zero_()
-    out, flags = run()
-    assert flags == 0 and float(out.float().abs().max()) > 0.01
-    again, flags = run()
-    assert flags == 0 and torch.equal(out, again)
+    oqm.stom_oqm_attend(gcfg, gst, 0, L, torch.from_numpy(idx).cuda(), k, T, q.cuda(), (Hq * d, d), k_sys.cuda(), v_sys.cuda(),
+                        oqm.BF16, (sys_len * pitch, sys_len * pitch, pitch), sys_len, float(scale), out, (Hq * d, d), ws,
+                        dev_flags=flags)
+    torch.cuda.synchronize()
+    assert int(flags.item()) == 0
+    got = orc.to_f32(P.as_np16(out), orc.BF16)
+    err = np.abs(got - want)
+    assert np.all(err <= np.maximum(TOL, 2.0 ** -7 * np.abs(want))), f"attention output differs by {err.max()}"
