@@ -750,6 +750,20 @@ def run_stream(args, sh, dev=None):
         torch.cuda.synchronize()
         if i >= 2:
             lay.append(a.elapsed_time(b) * 1e3 / sh.L)
+    # the same step as ONE call over all layers, captured and replayed: the device's share of that call
+    g_all = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_all):
+        decode(n)
+    allr = []
+    for i in range(12):
+        a, b = ev(), ev()
+        a.record()
+        for _ in range(10):
+            g_all.replay()
+        b.record()
+        torch.cuda.synchronize()
+        if i >= 2:
+            allr.append(a.elapsed_time(b) * 1e3 / 10)
     clocks = sampler.result()
     assert int(flags.item()) == 0
 
@@ -770,6 +784,7 @@ def run_stream(args, sh, dev=None):
         "per_frame_ingest": dict(i_st, algorithmic_bytes=frame_bytes),
         "per_query_retrieve": q_st, "per_decode_step_attend_all_layers": d_st,
         "per_decode_step_attend_one_layer_per_call_graph_replay_us": statistics.median(lay),
+        "per_decode_step_attend_all_layers_graph_replay_us": statistics.median(allr),
         "per_query_retrieve_plus_decode_step_graph_replay": r_st,
         "wall_s_including_python": wall, "clocks": clocks,
         "note": "CUDA-event times of single calls issued from Python one after the other; latencies, not bandwidths",

@@ -63,8 +63,8 @@ extern "C" {
 /* bits of dev_flags set by kernels */
 #define STOM_FLAG_BAD_INDEX 1u /* an entry of idx was < -1 or >= n_groups and was skipped */
 #define STOM_FLAG_TIMEOUT 2u   /* a bounded wait inside a kernel ran out; the call's outputs are incomplete */
-#define STOM_FLAG_DIRTY_WORKSPACE 4u /* stom_oqm_attend found a ticket counter that cannot follow from a cleared
-                                        workspace: the workspace was not zero-filled; outputs are missing */
+#define STOM_FLAG_DIRTY_WORKSPACE 4u /* reserved: raised by an earlier form of stom_oqm_attend that kept counters in a
+                                        caller-cleared workspace; the call no longer uses one */
 
 /* Geometry of one memory bank (paper notation: L, H_q, H_k, d, G). */
 typedef struct stom_oqm_config {
@@ -309,31 +309,31 @@ int32_t stom_oqm_retrieve(const stom_oqm_config *cfg, const stom_oqm_store *stor
  * G tokens of every selected group idx[..][j] >= 0, j < k], where a group's K
  * and V rows are code * s + m of the bank (not rounded to a 16-bit type on the
  * way).  Accumulation is binary32; the output is rounded once to cache_dtype.
- * With 4-bit codes both contractions run on the tensor cores with the raw
- * codes as one operand (exact) and q*s, respectively the softmax weights, as
- * the other, carried as a high and a low 16-bit part (16 significant bits);
- * the affine terms are added in binary32.
+ * Both contractions run on the tensor cores with the raw codes as one operand
+ * (exact) and q*s, respectively the softmax weights, as the other, carried as
+ * a high and a low 16-bit part (16 significant bits); the affine terms are
+ * added in binary32.
  * idx: as for stom_oqm_dequant_gather (PER_LAYER [layer_count][k]; PER_HEAD
  *   [layer_count][H_k][k]); -1 entries are skipped, other out-of-range entries
  *   are skipped and flagged.  k may be 0 if sys_len > 0.
  * q_dec (cfg->kv_dtype): element (l, h_q, c) at (l-layer_begin)*q_stride_layer
- *   + h_q*q_stride_head + c.
+ *   + h_q*q_stride_head + c; 4-byte aligned, both strides a multiple of 4 bytes.
  * k_sys, v_sys (cache_dtype = STOM_BF16 | STOM_FP16; may be NULL if sys_len == 0):
  *   element (l, h, tok, c) at (l-layer_begin)*sys_stride_layer + h*sys_stride_head
  *   + tok*sys_stride_token + c -- the first sys_len tokens of the active cache.
  * out (cache_dtype): element (l, h_q, c) at (l-layer_begin)*out_stride_layer +
  *   h_q*out_stride_head + c.
- * workspace: DEVICE, 256-byte aligned, stom_oqm_attend_workspace_bytes() bytes;
- *   holds the partial results of the blocks that share a (layer, kv head) and,
- *   in its first 4 * n_layers * H_k bytes (rounded up to 256), their ticket
- *   counters.  Those
- *   bytes must be ZERO when a call starts: clear the workspace once after
- *   allocating it (cudaMemsetAsync); every call that completes leaves them
- *   zero again, so the same workspace serves call after call (one call at a
- *   time) without further clearing.  Counters that are not zero make the call
- *   write no output or an incomplete one; nothing waits on them, and a counter
- *   beyond the number of blocks sets STOM_FLAG_DIRTY_WORKSPACE in dev_flags.
- * Errors: INVALID_ARG, SHAPE, UNSUPPORTED, ALIGNMENT, CAPACITY, WORKSPACE, CUDA.
+ * workspace, workspace_bytes: not used.  The blocks that share a (layer, kv
+ *   head) combine their partial results through the shared memory of a
+ *   thread-block cluster, so the call keeps nothing in global memory between
+ *   or during launches; the two arguments remain so that callers written for
+ *   the earlier form of the call (which took a cleared scratch buffer) keep
+ *   working, and may be NULL / 0.  stom_oqm_attend_workspace_bytes() returns a
+ *   small constant.  STOM_FLAG_DIRTY_WORKSPACE is no longer raised.
+ * A bulk copy into shared memory that has not landed after 2 s ends the block
+ * that waits for it: STOM_FLAG_TIMEOUT is set in dev_flags and the output rows
+ * of that (layer, kv head) are void.
+ * Errors: INVALID_ARG, SHAPE, UNSUPPORTED, ALIGNMENT, CAPACITY, CUDA.
  */
 int64_t stom_oqm_attend_workspace_bytes(const stom_oqm_config *cfg, int32_t layer_count, int32_t k,
                                         int32_t sys_len);

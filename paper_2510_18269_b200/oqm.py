@@ -244,13 +244,14 @@ def stom_oqm_attend(cfg: Config, store: Store, layer_begin, layer_count, idx, k,
                     k_sys, v_sys, cache_dtype, sys_strides, sys_len, softmax_scale, out, out_strides, workspace,
                     dev_flags=None, stream=None):
     """q_strides = (layer, head); sys_strides = (layer, head, token); out_strides = (layer, head), all in elements.
-    `workspace` (256-byte aligned) must have been zero-filled once after it was allocated; calls leave it reusable."""
+    `workspace` is not used by the call (it may be None); the argument remains for callers of the earlier form."""
     rc = lib().stom_oqm_attend(
         C.byref(cfg), C.byref(store.desc), C.c_int32(layer_begin), C.c_int32(layer_count), _ptr(idx), C.c_int32(k),
         C.c_int32(n_groups), _ptr(q_dec), C.c_int64(q_strides[0]), C.c_int64(q_strides[1]), _ptr(k_sys), _ptr(v_sys),
         C.c_int32(cache_dtype), C.c_int64(sys_strides[0]), C.c_int64(sys_strides[1]), C.c_int64(sys_strides[2]),
         C.c_int32(sys_len), C.c_float(softmax_scale), _ptr(out), C.c_int64(out_strides[0]), C.c_int64(out_strides[1]),
-        _ptr(workspace), C.c_int64(workspace.numel() * workspace.element_size()), _ptr(dev_flags), _stream(stream))
+        _ptr(workspace), C.c_int64(0 if workspace is None else workspace.numel() * workspace.element_size()),
+        _ptr(dev_flags), _stream(stream))
     _check(rc, "stom_oqm_attend")
 
 
