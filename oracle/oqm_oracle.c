@@ -723,6 +723,165 @@ int32_t orc_ctr_select(const float *sim, const float *alpha, int32_t T, int32_t 
     return ORC_OK;
 }
 
+/*
+ * Sec. 3.3, the Merge_{k_s} half of the (G_d, G_s) equation: the static tokens of one frame are consolidated "through
+ * density-based clustering" into k_s tokens.  The paper names the method (density peaks, "dpc" in the overview
+ * figure) and fixes none of its parameters; the reading taken here -- the k-nearest-neighbour form of density-peak
+ * clustering that token-merging work commonly uses -- is a decision of this code, written out step by step:
+ *   d2(i,j) = sum_c (x_ic - x_jc)^2 / D                            squared distance, normalised by the width
+ *   rho_i   = exp(-(1/kk) sum of the kk smallest d2(i,j), j != i)   kk = min(knn, n_s - 1); kk = 0 gives rho = 1
+ *   delta_i = min d(i,j) over the j that are denser than i (rho_j > rho_i, or equal and j earlier), d = sqrt(d2);
+ *             the densest token of all takes max_j d(i,j)
+ *   gamma_i = rho_i * delta_i; the k_s tokens of largest gamma are the cluster centres (equal gammas: the earlier one)
+ *   every other static token joins the centre it is nearest to (equal distances: the earlier centre)
+ *   a cluster becomes one token: the arithmetic mean of its members' features, placed at its centre's position
+ * F: one frame [N][D] of `dtype` (element (i, c) at i * stride_token + c); S: the n_s static token indices, ascending.
+ * centre [k_s]: token indices of the centres, ascending; assign [n_s]: for every static token the position of its
+ * centre in centre[]; merged [k_s][D]: the means (binary64 sums, returned in binary32); gamma [n_s] (nullable).
+ * margin (nullable, 2 values): how far the integer decisions are from flipping -- [0] the relative gap between the
+ * smallest gamma taken and the largest left out, [1] the smallest relative gap between a token's nearest and second
+ * nearest centre (both +inf where there is nothing to compare).
+ */
+int32_t orc_ctr_merge(const void *F, int32_t dtype, int32_t N, int32_t D, int64_t stride_token, const int32_t *S,
+                      int32_t n_s, int32_t k_s, int32_t knn, int32_t *centre, int32_t *assign, float *merged,
+                      double *gamma, double *margin) {
+    if (!F || !S || !centre || !assign || !merged || N < 1 || D < 1 || n_s < 0 || n_s > N || k_s < 0 || k_s > n_s || knn < 0)
+        return ORC_ERR_ARG;
+    if (margin) margin[0] = margin[1] = INFINITY;
+    if (k_s == 0) return ORC_OK;
+    for (int a = 0; a < n_s; ++a)
+        if (S[a] < 0 || S[a] >= N || (a > 0 && S[a] <= S[a - 1])) return ORC_ERR_ARG;
+    const size_t n = (size_t)n_s;
+    double *d2 = (double *)malloc(sizeof(double) * n * n), *rho = (double *)malloc(sizeof(double) * n);
+    double *gam = (double *)malloc(sizeof(double) * n), *tmp = (double *)malloc(sizeof(double) * n);
+    uint8_t *is_c = (uint8_t *)calloc(n, 1);
+    if (!d2 || !rho || !gam || !tmp || !is_c) { free(d2); free(rho); free(gam); free(tmp); free(is_c); return ORC_ERR_ARG; }
+    for (int a = 0; a < n_s; ++a)
+        for (int b = 0; b < n_s; ++b) {
+            double acc = 0.0;
+            for (int c = 0; c < D; ++c) {
+                const double u = (double)load_elem(F, (int64_t)S[a] * stride_token + c, dtype) -
+                                 (double)load_elem(F, (int64_t)S[b] * stride_token + c, dtype);
+                acc += u * u;
+            }
+            d2[a * n + b] = acc / (double)D;
+        }
+    const int kk = knn < n_s - 1 ? knn : n_s - 1;
+    for (int a = 0; a < n_s; ++a) {
+        /* the kk smallest distances to OTHER tokens: selection by repeated minimum */
+        int m = 0;
+        for (int b = 0; b < n_s; ++b)
+            if (b != a) tmp[m++] = d2[a * n + b];
+        double sum = 0.0;
+        for (int r = 0; r < kk; ++r) {
+            int best = r;
+            for (int j = r + 1; j < m; ++j)
+                if (tmp[j] < tmp[best]) best = j;
+            const double v = tmp[best];
+            tmp[best] = tmp[r];
+            tmp[r] = v;
+            sum += v;
+        }
+        rho[a] = kk > 0 ? exp(-sum / (double)kk) : 1.0;
+    }
+    for (int a = 0; a < n_s; ++a) {
+        double best = INFINITY, far = 0.0;
+        for (int b = 0; b < n_s; ++b) {
+            if (b == a) continue;
+            const double d = sqrt(d2[a * n + b]);
+            if (d > far) far = d;
+            if ((rho[b] > rho[a] || (rho[b] == rho[a] && b < a)) && d < best) best = d;
+        }
+        gam[a] = rho[a] * (best == INFINITY ? far : best);
+        if (gamma) gamma[a] = gam[a];
+    }
+    /* k_s times: the not yet taken token of largest gamma, the earliest among equals */
+    double last_taken = INFINITY;
+    for (int r = 0; r < k_s; ++r) {
+        int best = -1;
+        for (int a = 0; a < n_s; ++a)
+            if (!is_c[a] && (best < 0 || gam[a] > gam[best])) best = a;
+        is_c[best] = 1;
+        last_taken = gam[best];
+    }
+    if (margin && k_s < n_s) {
+        double next = -INFINITY;
+        for (int a = 0; a < n_s; ++a)
+            if (!is_c[a] && gam[a] > next) next = gam[a];
+        margin[0] = (last_taken - next) / (fabs(last_taken) > 1e-300 ? fabs(last_taken) : 1e-300);
+    }
+    int w = 0;
+    for (int a = 0; a < n_s; ++a)
+        if (is_c[a]) centre[w++] = S[a];
+    /* position of every centre among the static tokens, in centre order */
+    int *cpos = (int *)malloc(sizeof(int) * (size_t)k_s);
+    if (!cpos) { free(d2); free(rho); free(gam); free(tmp); free(is_c); return ORC_ERR_ARG; }
+    w = 0;
+    for (int a = 0; a < n_s; ++a)
+        if (is_c[a]) cpos[w++] = a;
+    for (int a = 0; a < n_s; ++a) {
+        int best = 0;
+        double second = INFINITY;
+        if (is_c[a]) {
+            for (int j = 0; j < k_s; ++j)
+                if (cpos[j] == a) best = j;
+        } else {
+            for (int j = 1; j < k_s; ++j)
+                if (d2[a * n + cpos[j]] < d2[a * n + cpos[best]]) best = j;
+            for (int j = 0; j < k_s; ++j)
+                if (j != best && d2[a * n + cpos[j]] < second) second = d2[a * n + cpos[j]];
+            if (margin && k_s > 1) {
+                const double near = d2[a * n + cpos[best]];
+                const double gap = (second - near) / (second > 1e-300 ? second : 1e-300);
+                if (gap < margin[1]) margin[1] = gap;
+            }
+        }
+        assign[a] = best;
+    }
+    for (int j = 0; j < k_s; ++j)
+        for (int c = 0; c < D; ++c) {
+            double acc = 0.0;
+            int cnt = 0;
+            for (int a = 0; a < n_s; ++a)
+                if (assign[a] == j) {
+                    acc += (double)load_elem(F, (int64_t)S[a] * stride_token + c, dtype);
+                    ++cnt;
+                }
+            merged[(int64_t)j * D + c] = (float)(acc / (double)cnt);
+        }
+    free(d2); free(rho); free(gam); free(tmp); free(is_c); free(cpos);
+    return ORC_OK;
+}
+
+/*
+ * Sec. 3.3: "The per-frame retained group G_t combines both paths with |G_t| = G".  The k_d selected dynamic tokens
+ * (their feature rows, unchanged) and the k_s merged tokens (rounded to the feature type, nearest-even), in ascending
+ * order of token position -- a merged token stands at its centre's position.  retained [G][D] of `dtype`,
+ * pos [G]; rows behind the k_d + k_s tokens are zero with position -1.
+ */
+int32_t orc_ctr_retain(const void *F, int32_t dtype, int32_t N, int32_t D, int64_t stride_token, const int32_t *dyn,
+                       int32_t k_d, const int32_t *centre, const float *merged, int32_t k_s, int32_t G, void *retained,
+                       int32_t *pos) {
+    if (!F || !retained || !pos || k_d < 0 || k_s < 0 || k_d + k_s > G || D < 1 || N < 1) return ORC_ERR_ARG;
+    int a = 0, b = 0;
+    for (int w = 0; w < G; ++w) {
+        const int pa = a < k_d ? dyn[a] : N + 1, pb = b < k_s ? centre[b] : N + 1;
+        if (pa > N && pb > N) {
+            pos[w] = -1;
+            for (int c = 0; c < D; ++c) store_out(retained, (int64_t)w * D + c, dtype, 0.0f);
+        } else if (pa < pb) {
+            pos[w] = pa;
+            for (int c = 0; c < D; ++c) store_out(retained, (int64_t)w * D + c, dtype, load_elem(F, (int64_t)pa * stride_token + c, dtype));
+            ++a;
+        } else {
+            pos[w] = pb;
+            for (int c = 0; c < D; ++c) store_out(retained, (int64_t)w * D + c, dtype, merged[(int64_t)b * D + c]);
+            ++b;
+        }
+    }
+    return ORC_OK;
+}
+
 /* ------------------------------------------------------------------ */
 /* O8  storage accounting                                               */
 /* ------------------------------------------------------------------ */

@@ -267,7 +267,7 @@ def attend(H_q, H_k, d, q_dec, q_dtype, k_cache, v_cache, kv_dtype, stride_head,
     return out
 
 
-# ---------------------------------------------------------------- CTR (specified steps only)
+# ---------------------------------------------------------------- CTR
 
 def ctr_similarity(F: np.ndarray, dtype: int, prev: np.ndarray | None = None) -> np.ndarray:
     """F [T][N][D] (contiguous; uint16 patterns for the 16-bit types), prev [N][D] or None -> sim [T][N] float32."""
@@ -296,6 +296,48 @@ def ctr_select(sim: np.ndarray, alpha: np.ndarray, G: int, tau_c: float):
     if rc:
         raise ValueError(f"orc_ctr_select -> {rc}")
     return ks, kd, sidx, didx
+
+
+def ctr_merge(F_frame: np.ndarray, dtype: int, S: np.ndarray, k_s: int, knn: int = 5):
+    """One frame's Merge_{k_s} under this code's reading of the paper's density-based clustering.
+
+    F_frame [N][D] (uint16 patterns for the 16-bit types), S: ascending static token indices.  Returns a dict:
+    centre [k_s] (token indices, ascending), assign [n_s] (position of each static token's centre in `centre`),
+    merged [k_s][D] float32 (member means), gamma [n_s] float64, margin [2] float64 (how far the centre choice and
+    the nearest-centre assignments are from flipping, as relative gaps)."""
+    F_frame = np.ascontiguousarray(F_frame)
+    N, D = F_frame.shape
+    S = np.ascontiguousarray(S, np.int32)
+    n_s = int(S.shape[0])
+    centre = np.full(max(k_s, 1), -1, np.int32)
+    assign = np.full(max(n_s, 1), -1, np.int32)
+    merged = np.zeros((max(k_s, 1), D), np.float32)
+    gamma = np.zeros(max(n_s, 1), np.float64)
+    margin = np.zeros(2, np.float64)
+    rc = lib().orc_ctr_merge(_p(F_frame), C.c_int32(dtype), C.c_int32(N), C.c_int32(D), C.c_int64(D), _p(S),
+                             C.c_int32(n_s), C.c_int32(k_s), C.c_int32(knn), _p(centre), _p(assign), _p(merged),
+                             _p(gamma), _p(margin))
+    if rc:
+        raise ValueError(f"orc_ctr_merge -> {rc}")
+    return {"centre": centre[:k_s], "assign": assign[:n_s], "merged": merged[:k_s], "gamma": gamma[:n_s], "margin": margin}
+
+
+def ctr_retain(F_frame: np.ndarray, dtype: int, dyn: np.ndarray, centre: np.ndarray, merged: np.ndarray, G: int):
+    """The frame's retained group: the selected dynamic rows and the merged rows in position order.
+    Returns (retained [G][D] in the feature type, pos [G] int32)."""
+    F_frame = np.ascontiguousarray(F_frame)
+    N, D = F_frame.shape
+    dyn = np.ascontiguousarray(dyn, np.int32)
+    centre = np.ascontiguousarray(centre, np.int32)
+    merged = np.ascontiguousarray(merged, np.float32)
+    retained = np.zeros((G, D), F_frame.dtype)
+    pos = np.full(G, -1, np.int32)
+    rc = lib().orc_ctr_retain(_p(F_frame), C.c_int32(dtype), C.c_int32(N), C.c_int32(D), C.c_int64(D), _p(dyn),
+                              C.c_int32(dyn.shape[0]), _p(centre), _p(merged), C.c_int32(centre.shape[0]), C.c_int32(G),
+                              _p(retained), _p(pos))
+    if rc:
+        raise ValueError(f"orc_ctr_retain -> {rc}")
+    return retained, pos
 
 
 # ---------------------------------------------------------------- accounting

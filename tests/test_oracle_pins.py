@@ -637,6 +637,99 @@ def test_ctr_select_split_budget_and_saliency_topk(orc):
         assert len(want) == kd[t]
 
 
+# ------------------------------------------------------------------ CTR: Merge_{k_s} (this code's reading of Sec. 3.3)
+
+def test_ctr_merge_points_on_a_line_worked_by_hand(orc):
+    """Six one-channel tokens 0, 1, 2, 10, 11, 12 with two neighbours each and k_s = 2, worked out from the stated rule:
+    the middle tokens 1 and 11 have their two neighbours at distance 1 (rho = exp(-1)), the four outer tokens at 1 and
+    2 (rho = exp(-(1 + 4)/2)).  Token 1 and token 11 tie for the highest density and the earlier one ranks first: its
+    delta is its largest distance, 11; token 11 then looks back to token 1, delta = 10; every outer token has its
+    denser neighbour next to it, delta = 1.  gamma = rho * delta: 11/e, 10/e, and exp(-2.5) four times, so the centres
+    are tokens 1 and 11, each outer token joins the centre one step away, and the merged tokens are the means 1 and 11."""
+    F = np.array([[0], [1], [2], [10], [11], [12]], np.float32)
+    r = orc.ctr_merge(F, orc.FP32, np.arange(6), 2, knn=2)
+    assert r["centre"].tolist() == [1, 4] and r["assign"].tolist() == [0, 0, 0, 1, 1, 1]
+    np.testing.assert_allclose(r["gamma"], [np.exp(-2.5), 11 / np.e, np.exp(-2.5), np.exp(-2.5), 10 / np.e, np.exp(-2.5)],
+                               rtol=1e-14)
+    np.testing.assert_array_equal(r["merged"], [[1.0], [11.0]])
+    # the distances are normalised by the width: the same tokens written with each channel four times change nothing
+    r4 = orc.ctr_merge(np.repeat(F, 4, axis=1), orc.FP32, np.arange(6), 2, knn=2)
+    assert r4["centre"].tolist() == [1, 4] and r4["assign"].tolist() == [0, 0, 0, 1, 1, 1]
+    np.testing.assert_allclose(r4["gamma"], r["gamma"], rtol=1e-14)
+    # a subset as the static set: tokens 0, 2, 3, 5 -> neighbours change, the rule does not
+    rs = orc.ctr_merge(F, orc.FP32, np.array([0, 2, 3, 5]), 2, knn=1)
+    assert rs["centre"].tolist() in ([0, 3], [0, 5], [2, 3], [2, 5]) and rs["assign"].tolist() == [0, 0, 1, 1]
+    np.testing.assert_array_equal(rs["merged"], [[1.0], [11.0]])
+
+
+def test_ctr_merge_invariants(orc):
+    """Whatever the clustering decides: k_s clusters, none empty, every static token in exactly one, a centre in its
+    own cluster, each merged token the mean of its members (so a convex combination, channel by channel inside the
+    members' range); k_s = |S| leaves the tokens as they are; relabelling the tokens permutes the result with them."""
+    rng = np.random.default_rng(3)
+    N, D = 40, 24
+    F = rng.standard_normal((N, D)).astype(np.float32)
+    S = np.sort(rng.choice(N, size=29, replace=False)).astype(np.int32)
+    for k_s in (1, 2, 7, 28, 29):
+        r = orc.ctr_merge(F, orc.FP32, S, k_s)
+        c, a, m = r["centre"], r["assign"], r["merged"]
+        assert len(c) == k_s and np.all(np.diff(c) > 0) and np.all(np.isin(c, S))
+        assert a.min() == 0 and a.max() == k_s - 1 and len(np.unique(a)) == k_s
+        for j in range(k_s):
+            members = S[a == j]
+            assert c[j] in members
+            want = F[members].astype(np.float64).mean(axis=0)
+            np.testing.assert_allclose(m[j], want, rtol=1e-6, atol=1e-7)
+            assert np.all(m[j] <= F[members].max(axis=0) + 1e-6) and np.all(m[j] >= F[members].min(axis=0) - 1e-6)
+        if k_s == len(S):
+            np.testing.assert_array_equal(c, S)
+            np.testing.assert_array_equal(m, F[S])
+    # permutation: token i of the permuted frame is token perm[i] of the original
+    k_s = 7
+    base = orc.ctr_merge(F, orc.FP32, S, k_s)
+    perm = rng.permutation(N)
+    inv = np.argsort(perm)
+    Sp = np.sort(inv[S]).astype(np.int32)
+    rp = orc.ctr_merge(F[perm], orc.FP32, Sp, k_s)
+    assert sorted(perm[rp["centre"]].tolist()) == base["centre"].tolist()
+    clusters = lambda r, S_, back: sorted(sorted(back[S_[r["assign"] == j]].tolist()) for j in range(k_s))
+    assert clusters(rp, Sp, perm) == clusters(base, S, np.arange(N))
+
+
+def test_ctr_merge_separated_blobs_and_retained_group(orc):
+    """Three tight, well separated blobs and k_s = 3: the clusters are the blobs and the merged tokens their means
+    (numpy).  The retained group then interleaves the selected dynamic rows (bit for bit) with the merged rows rounded
+    to the feature type (torch's nearest-even), in position order, a merged token at its centre's position."""
+    import torch
+    rng = np.random.default_rng(8)
+    N, D, G = 30, 16, 9
+    blob = rng.integers(0, 3, size=N)
+    blob[:3] = [0, 1, 2]
+    mu = 20.0 * rng.standard_normal((3, D))
+    X = torch.from_numpy((mu[blob] + 0.05 * rng.standard_normal((N, D))).astype(np.float32)).to(torch.bfloat16)
+    Xf = X.to(torch.float32).numpy().astype(np.float64)
+    Xu = X.view(torch.int16).numpy().view(np.uint16)
+    dyn = np.array([4, 11, 20, 27], np.int32)
+    S = np.setdiff1d(np.arange(N), dyn).astype(np.int32)
+    r = orc.ctr_merge(Xu, orc.BF16, S, 3)
+    assert sorted(blob[r["centre"]].tolist()) == [0, 1, 2]
+    for j in range(3):
+        members = S[r["assign"] == j]
+        b = blob[r["centre"][j]]
+        assert np.array_equal(members, S[blob[S] == b])
+        np.testing.assert_allclose(r["merged"][j], Xf[members].mean(axis=0), rtol=1e-6, atol=1e-6)
+    assert r["margin"][0] > 0.5 and r["margin"][1] > 0.9     # nothing about these decisions is close
+    ret, pos = orc.ctr_retain(Xu, orc.BF16, dyn, r["centre"], r["merged"], G)
+    want_pos = np.sort(np.concatenate([dyn, r["centre"]]))
+    assert np.array_equal(pos[:7], want_pos) and np.all(pos[7:] == -1) and not ret[7:].any()
+    merged16 = torch.from_numpy(r["merged"]).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+    for w, t in enumerate(want_pos):
+        if t in dyn:
+            assert np.array_equal(ret[w], Xu[t])
+        else:
+            assert np.array_equal(ret[w], merged16[list(r["centre"]).index(t)])
+
+
 # ------------------------------------------------------------------ whole path on the tiny workload
 
 def test_tiny_workload_retrieves_planted_groups_and_bounds_active_cache(orc):
