@@ -852,15 +852,20 @@ def run_ctr(args):
     def ev():
         return torch.cuda.Event(enable_timing=True)
 
+    ret = torch.empty(T, G, D, dtype=F.dtype, device=dev)
+    rpos = torch.empty(T, G, dtype=torch.int32, device=dev)
+
     def step(timers=None):
         flush.fill_(1)       # evict everything ...
         flush_rd.sum()       # ... and leave no dirty lines whose write-back would run during the timed kernels
-        e = [ev() for _ in range(3)]
+        e = [ev() for _ in range(4)]
         e[0].record()
         oqm.stom_ctr_similarity(F, None, T, N, D, (N * D, D), sim)
         e[1].record()
         oqm.stom_ctr_select(sim, alpha, T, N, G, c["tau_c"], ks, kd, si, di)
         e[2].record()
+        oqm.stom_ctr_merge(F, T, N, D, (N * D, D), ks, kd, si, di, G, 5, ret, rpos)
+        e[3].record()
         if timers is not None:
             timers.append(e)
 
@@ -880,6 +885,12 @@ def run_ctr(args):
     sim_ms = sdist.max_over_ranks(statistics.mean(t[0].elapsed_time(t[1]) for t in timers))
     sel_ms = sdist.max_over_ranks(statistics.mean(t[1].elapsed_time(t[2]) for t in timers))
     tot_ms = sdist.max_over_ranks(statistics.mean(t[0].elapsed_time(t[2]) for t in timers))
+    mg_ms = sdist.max_over_ranks(statistics.median(t[2].elapsed_time(t[3]) for t in timers))
+    # Merge: the Gram matrix of a frame's N tokens is a [N x D] . [D x N] contraction; only the 16 x 16 blocks on and
+    # below the diagonal are computed.  Its bytes: the frame's features once, the retained group written once.
+    tiles = (N + 15) // 16
+    mg_flops = T * (tiles * (tiles + 1) // 2) * 2 * 16 * 16 * D
+    mg_bytes = T * (N * D * 2 + G * D * 2 + (N + 3 * G + 2) * 4)
     nbytes = bytes_ctr(T, N, D, G)
     sbytes = T * N * D * 2 + T * N * 4
     a = sbytes / (sim_ms * 1e-3) / 1e9
@@ -892,12 +903,19 @@ def run_ctr(args):
                    "l2": "features 3.25 GB >> L2; a 512 MB write then a 512 MB read before every step",
                    "multi_gpu": "independent stream per rank, no collective"},
         "submetrics": {"frames_per_s": world * T / (tot_ms * 1e-3),
-                       "stage_us": {"similarity": sim_ms * 1e3, "select": sel_ms * 1e3},
-                       "mean_k_s": float(ks.float().mean().item())},
+                       "stage_us": {"similarity": sim_ms * 1e3, "select": sel_ms * 1e3, "merge": mg_ms * 1e3},
+                       "mean_k_s": float(ks.float().mean().item()),
+                       "merge": {"ms": mg_ms, "frames_per_s": world * T / (mg_ms * 1e-3),
+                                 "gram_TFLOPs": mg_flops / (mg_ms * 1e-3) / 1e12,
+                                 "GBps": mg_bytes / (mg_ms * 1e-3) / 1e9,
+                                 "frac_of_measured_hbm": mg_bytes / (mg_ms * 1e-3) / 1e9 / peak,
+                                 "note": "Merge_{k_s} + retained group; the Gram matrix runs on the tensor cores (warp-level "
+                                         "matrix products); not part of `value`, which covers similarity + select"},
+                       "whole_ctr_frames_per_s": world * T / ((tot_ms + mg_ms) * 1e-3)},
         "roofline": {"kernel": "ctr_similarity_kernel", "bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s",
                      "frac": a / peak, "traffic": None if tpu is None else tpu * T, "peak_source": peak_src,
                      "algorithmic_bytes_per_launch": sbytes, "ms_per_launch": sim_ms},
-        "gpu_launches": 2, "clocks": clocks,
+        "gpu_launches": 3, "clocks": clocks,
     }
     if not args.no_e2e:
         # host buffers: features and saliency of a chunk of frames go up, the integer outputs come back; the frame

@@ -738,16 +738,17 @@ int32_t orc_ctr_select(const float *sim, const float *alpha, int32_t T, int32_t 
  * F: one frame [N][D] of `dtype` (element (i, c) at i * stride_token + c); S: the n_s static token indices, ascending.
  * centre [k_s]: token indices of the centres, ascending; assign [n_s]: for every static token the position of its
  * centre in centre[]; merged [k_s][D]: the means (binary64 sums, returned in binary32); gamma [n_s] (nullable).
- * margin (nullable, 2 values): how far the integer decisions are from flipping -- [0] the relative gap between the
- * smallest gamma taken and the largest left out, [1] the smallest relative gap between a token's nearest and second
- * nearest centre (both +inf where there is nothing to compare).
+ * margin (nullable, 1 + n_s values): how far the integer decisions are from flipping -- [0] the relative gap between
+ * the smallest gamma taken and the largest left out, [1 + a] the relative gap between static token a's nearest and
+ * second nearest centre (+inf where there is nothing to compare: a centre, or a single cluster).
  */
 int32_t orc_ctr_merge(const void *F, int32_t dtype, int32_t N, int32_t D, int64_t stride_token, const int32_t *S,
                       int32_t n_s, int32_t k_s, int32_t knn, int32_t *centre, int32_t *assign, float *merged,
                       double *gamma, double *margin) {
     if (!F || !S || !centre || !assign || !merged || N < 1 || D < 1 || n_s < 0 || n_s > N || k_s < 0 || k_s > n_s || knn < 0)
         return ORC_ERR_ARG;
-    if (margin) margin[0] = margin[1] = INFINITY;
+    if (margin)
+        for (int a = 0; a <= n_s; ++a) margin[a] = INFINITY;
     if (k_s == 0) return ORC_OK;
     for (int a = 0; a < n_s; ++a)
         if (S[a] < 0 || S[a] >= N || (a > 0 && S[a] <= S[a - 1])) return ORC_ERR_ARG;
@@ -832,8 +833,7 @@ int32_t orc_ctr_merge(const void *F, int32_t dtype, int32_t N, int32_t D, int64_
                 if (j != best && d2[a * n + cpos[j]] < second) second = d2[a * n + cpos[j]];
             if (margin && k_s > 1) {
                 const double near = d2[a * n + cpos[best]];
-                const double gap = (second - near) / (second > 1e-300 ? second : 1e-300);
-                if (gap < margin[1]) margin[1] = gap;
+                margin[1 + a] = (second - near) / (second > 1e-300 ? second : 1e-300);
             }
         }
         assign[a] = best;

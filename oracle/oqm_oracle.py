@@ -303,8 +303,9 @@ def ctr_merge(F_frame: np.ndarray, dtype: int, S: np.ndarray, k_s: int, knn: int
 
     F_frame [N][D] (uint16 patterns for the 16-bit types), S: ascending static token indices.  Returns a dict:
     centre [k_s] (token indices, ascending), assign [n_s] (position of each static token's centre in `centre`),
-    merged [k_s][D] float32 (member means), gamma [n_s] float64, margin [2] float64 (how far the centre choice and
-    the nearest-centre assignments are from flipping, as relative gaps)."""
+    merged [k_s][D] float32 (member means), gamma [n_s] float64, margin_centres (relative gap between the last gamma
+    taken and the first left out) and margin_assign [n_s] (relative gap between each token's nearest and second
+    nearest centre): how far the integer decisions are from flipping."""
     F_frame = np.ascontiguousarray(F_frame)
     N, D = F_frame.shape
     S = np.ascontiguousarray(S, np.int32)
@@ -313,13 +314,14 @@ def ctr_merge(F_frame: np.ndarray, dtype: int, S: np.ndarray, k_s: int, knn: int
     assign = np.full(max(n_s, 1), -1, np.int32)
     merged = np.zeros((max(k_s, 1), D), np.float32)
     gamma = np.zeros(max(n_s, 1), np.float64)
-    margin = np.zeros(2, np.float64)
+    margin = np.zeros(1 + max(n_s, 1), np.float64)
     rc = lib().orc_ctr_merge(_p(F_frame), C.c_int32(dtype), C.c_int32(N), C.c_int32(D), C.c_int64(D), _p(S),
                              C.c_int32(n_s), C.c_int32(k_s), C.c_int32(knn), _p(centre), _p(assign), _p(merged),
                              _p(gamma), _p(margin))
     if rc:
         raise ValueError(f"orc_ctr_merge -> {rc}")
-    return {"centre": centre[:k_s], "assign": assign[:n_s], "merged": merged[:k_s], "gamma": gamma[:n_s], "margin": margin}
+    return {"centre": centre[:k_s], "assign": assign[:n_s], "merged": merged[:k_s], "gamma": gamma[:n_s],
+            "margin_centres": float(margin[0]), "margin_assign": margin[1:1 + n_s]}
 
 
 def ctr_retain(F_frame: np.ndarray, dtype: int, dyn: np.ndarray, centre: np.ndarray, merged: np.ndarray, G: int):

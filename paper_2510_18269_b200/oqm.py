@@ -31,7 +31,7 @@ EXPORTS = (
     "stom_oqm_retrieve_host_scratch_bytes", "stom_oqm_retrieve_host",
     "stom_oqm_score_groups_noalloc", "stom_oqm_attend_workspace_bytes", "stom_oqm_attend",
     "stom_oqm_retrieve_workspace_bytes",
-    "stom_ctr_similarity", "stom_ctr_select", "stom_ctr_reduce",
+    "stom_ctr_similarity", "stom_ctr_select", "stom_ctr_reduce", "stom_ctr_merge", "stom_ctr_reduce_tokens",
 )
 
 
@@ -315,3 +315,23 @@ def stom_ctr_reduce(F, prev, T, N, D, strides, alpha, G, tau_c, sim, k_s, k_d, s
                                  C.c_int32(D), C.c_int64(sf), C.c_int64(st), _ptr(alpha), C.c_int32(G),
                                  C.c_float(tau_c), _ptr(sim), _ptr(k_s), _ptr(k_d), _ptr(static_idx), _ptr(dyn_idx),
                                  _stream(stream)), "stom_ctr_reduce")
+
+
+def stom_ctr_merge(F, T, N, D, strides, k_s, k_d, static_idx, dyn_idx, G, knn, retained, retained_pos, centre=None,
+                   assign=None, stream=None):
+    """Merge_{k_s} of the static tokens and the retained group [T][G][D] (see include/stom_ctr.h for the rule)."""
+    sf, st = strides
+    _check(lib().stom_ctr_merge(_ptr(F), C.c_int32(dtype_code(F.dtype)), C.c_int32(T), C.c_int32(N), C.c_int32(D),
+                                C.c_int64(sf), C.c_int64(st), _ptr(k_s), _ptr(k_d), _ptr(static_idx), _ptr(dyn_idx),
+                                C.c_int32(G), C.c_int32(knn), _ptr(retained), _ptr(retained_pos), _ptr(centre),
+                                _ptr(assign), _stream(stream)), "stom_ctr_merge")
+
+
+def stom_ctr_reduce_tokens(F, prev, T, N, D, strides, alpha, G, tau_c, knn, sim, k_s, k_d, static_idx, dyn_idx, retained,
+                           retained_pos, stream=None):
+    sf, st = strides
+    _check(lib().stom_ctr_reduce_tokens(_ptr(F), _ptr(prev), C.c_int32(dtype_code(F.dtype)), C.c_int32(T), C.c_int32(N),
+                                        C.c_int32(D), C.c_int64(sf), C.c_int64(st), _ptr(alpha), C.c_int32(G),
+                                        C.c_float(tau_c), C.c_int32(knn), _ptr(sim), _ptr(k_s), _ptr(k_d),
+                                        _ptr(static_idx), _ptr(dyn_idx), _ptr(retained), _ptr(retained_pos),
+                                        _stream(stream)), "stom_ctr_reduce_tokens")
