@@ -138,13 +138,15 @@ __global__ void __launch_bounds__(kMgThreads, 1) ctr_merge_kernel(const MergePar
 
     if (k_s > 0) {
         // ================================================================= Gram matrix on the tensor cores
-        // 16 x 16 blocks (i, j), j <= i, numbered row by row; warp w owns blocks w, w + 8, ...
-        const int n_blk = NT * (NT + 1) / 2;
+        // 16 x 16 blocks (i, j), j <= i, numbered row by row; warp w owns a run of consecutive blocks, most of them in
+        // one row, so that the row's operand fragment is loaded once per run of equal rows
+        const int n_blk = NT * (NT + 1) / 2, per_warp = (n_blk + kMgWarps - 1) / kMgWarps;
+        const int blk0 = warp * per_warp, n_mine_blk = max(0, min(per_warp, n_blk - blk0));
         int bi_[kMgMaxBlocks], bj_[kMgMaxBlocks];
         float acc[kMgMaxBlocks][2][4];
 #pragma unroll
         for (int b = 0; b < kMgMaxBlocks; ++b) {
-            const int n = warp + b * kMgWarps;
+            const int n = blk0 + b;
             int i = 0;
             while ((i + 1) * (i + 2) / 2 <= n) ++i;  // row of block n
             bi_[b] = i;
@@ -193,11 +195,13 @@ __global__ void __launch_bounds__(kMgThreads, 1) ctr_merge_kernel(const MergePar
 #pragma unroll
             for (int ks = 0; ks < kMgSlabCh / 16; ++ks) {
                 const uint32_t pa = base + offA[ks], pb = base + offB[ks];
+                uint32_t a0 = 0, a1 = 0, a2 = 0, a3 = 0;
 #pragma unroll
                 for (int b = 0; b < kMgMaxBlocks; ++b) {
-                    if (warp + b * kMgWarps < n_blk) {  // warp-uniform
-                        uint32_t a0, a1, a2, a3, b0, b1, b2, b3;
-                        ldmatrix_x4(pa + (bi_[b] << 11), a0, a1, a2, a3);  // a tile of 16 rows is 2048 bytes of a slab
+                    if (b < n_mine_blk) {  // warp-uniform
+                        uint32_t b0, b1, b2, b3;
+                        if (b == 0 || bi_[b] != bi_[b - 1])  // (warp-uniform) a tile of 16 rows is 2048 bytes of a slab
+                            ldmatrix_x4(pa + (bi_[b] << 11), a0, a1, a2, a3);
                         ldmatrix_x4(pb + (bj_[b] << 11), b0, b1, b2, b3);
                         mg_mma<T>(acc[b][0], a0, a1, a2, a3, b0, b1);
                         mg_mma<T>(acc[b][1], a0, a1, a2, a3, b2, b3);
@@ -211,7 +215,7 @@ __global__ void __launch_bounds__(kMgThreads, 1) ctr_merge_kernel(const MergePar
         const int g = lane >> 2, tq = lane & 3;
 #pragma unroll
         for (int b = 0; b < kMgMaxBlocks; ++b) {
-            if (warp + b * kMgWarps < n_blk && bi_[b] == bj_[b]) {
+            if (b < n_mine_blk && bi_[b] == bj_[b]) {
 #pragma unroll
                 for (int u = 0; u < 2; ++u)
 #pragma unroll
@@ -225,7 +229,7 @@ __global__ void __launch_bounds__(kMgThreads, 1) ctr_merge_kernel(const MergePar
         const float inv_d = 1.0f / (float)D;
 #pragma unroll
         for (int b = 0; b < kMgMaxBlocks; ++b) {
-            if (warp + b * kMgWarps < n_blk) {
+            if (b < n_mine_blk) {
 #pragma unroll
                 for (int u = 0; u < 2; ++u)
 #pragma unroll
@@ -246,10 +250,13 @@ __global__ void __launch_bounds__(kMgThreads, 1) ctr_merge_kernel(const MergePar
             float best[kMgMaxKnn];  // the smallest squared distances, ascending
 #pragma unroll
             for (int q = 0; q < kMgMaxKnn; ++q) best[q] = INFINITY;
+            const int row = ia * (ia + 1) / 2;
+#pragma unroll 4
             for (int b = 0; b < n_s; ++b) {
-                if (b == a) continue;
-                float v = d2[tri(ia, slist[b])];
-                far2 = fmaxf(far2, v);
+                const int ib = slist[b];
+                float v = d2[ib <= ia ? row + ib : ib * (ib + 1) / 2 + ia];
+                far2 = fmaxf(far2, v);          // (the token itself adds 0)
+                v = b == a ? INFINITY : v;      // ... and is no neighbour of itself
 #pragma unroll
                 for (int q = 0; q < kMgMaxKnn; ++q) {  // insertion: v sinks to its place, the largest falls out
                     const float lo = fminf(best[q], v);
@@ -268,10 +275,12 @@ __global__ void __launch_bounds__(kMgThreads, 1) ctr_merge_kernel(const MergePar
             const int ia = slist[a];
             const float ra = rho[a];
             float near2 = INFINITY;
-            for (int b = 0; b < n_s; ++b) {
-                if (b == a) continue;
-                const float rb = rho[b];
-                if (rb > ra || (rb == ra && b < a)) near2 = fminf(near2, d2[tri(ia, slist[b])]);
+            const int row = ia * (ia + 1) / 2;
+#pragma unroll 4
+            for (int b = 0; b < n_s; ++b) {  // (b == a is never denser than a)
+                const int ib = slist[b];
+                const float rb = rho[b], v = d2[ib <= ia ? row + ib : ib * (ib + 1) / 2 + ia];
+                near2 = (rb > ra || (rb == ra && b < a)) ? fminf(near2, v) : near2;
             }
             gam[a] = ra * sqrtf(near2 == INFINITY ? far2 : near2);
         }
@@ -365,15 +374,23 @@ __global__ void __launch_bounds__(kMgThreads, 1) ctr_merge_kernel(const MergePar
 #pragma unroll
         for (int q = 0; q < 8; ++q) s8[q] = 0.0f;
         const int m0 = coff[j], m1 = coff[j + 1];
-        for (int m = m0; m < m1; ++m) {
-            const uint4 v = __ldg(reinterpret_cast<const uint4 *>(Ft + (int64_t)member[m] * p.st) + c);
-            const uint32_t w4[4] = {v.x, v.y, v.z, v.w};
+        for (int m = m0; m < m1; m += 4) {  // the loads of four members are in flight together; added in member order
+            uint4 v[4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                float lo, hi;
-                unpack2<T>(w4[q], lo, hi);
-                s8[2 * q] += lo;
-                s8[2 * q + 1] += hi;
+            for (int u = 0; u < 4; ++u)
+                v[u] = m + u < m1 ? __ldg(reinterpret_cast<const uint4 *>(Ft + (int64_t)member[m + u] * p.st) + c) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (m + u < m1) {
+                    const uint32_t w4[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        float lo, hi;
+                        unpack2<T>(w4[q], lo, hi);
+                        s8[2 * q] += lo;
+                        s8[2 * q + 1] += hi;
+                    }
+                }
             }
         }
         // true division: the binary32 sum of a few 16-bit values is exact, so the quotient is the correctly rounded mean
