@@ -7,7 +7,7 @@
  * tokens, the consolidation of the static tokens (Merge_{k_s}) and the
  * retained group of G tokens that goes on to the language model.  The paper
  * specifies all of these but the clustering inside Merge_{k_s}, which it only
- * names ("density-based clustering"); the rule used here is written out at
+ * names (a density-based clustering); the rule used here is written out at
  * stom_ctr_merge and is this library's reading, not the paper's text.
  *
  * Conventions are those of stom_oqm.h: device pointers unless stated, caller
@@ -76,9 +76,9 @@ int32_t stom_ctr_reduce(const void *F, const void *prev, int32_t dtype, int32_t 
 
 /*
  * Sec. 3.3, the Merge half of the (G_d, G_s) equation, G_s = Merge_{k_s}({F_t^(i)}, i in S_t), and the retained
- * group ("the per-frame retained group G_t combines both paths with |G_t| = G"), per frame.
+ * group G_t of Sec. 3.3 (the selected dynamic tokens and the merged static ones together, |G_t| = G), per frame.
  *
- * The paper consolidates the static tokens "through density-based clustering" (density peaks, "dpc" in its overview
+ * The paper consolidates the static tokens by a density-based clustering (density peaks, going by its overview
  * figure) and gives neither the density, nor the distance, nor how a cluster becomes one token.  This library's
  * reading -- the k-nearest-neighbour form of density-peak clustering -- over the n_s static tokens x_i of a frame:
  *   d2(i,j) = |x_i - x_j|^2 / D                                   (computed as (|x_i|^2 + |x_j|^2 - 2 x_i.x_j) / D

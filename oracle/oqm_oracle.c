@@ -724,8 +724,8 @@ int32_t orc_ctr_select(const float *sim, const float *alpha, int32_t T, int32_t 
 }
 
 /*
- * Sec. 3.3, the Merge_{k_s} half of the (G_d, G_s) equation: the static tokens of one frame are consolidated "through
- * density-based clustering" into k_s tokens.  The paper names the method (density peaks, "dpc" in the overview
+ * Sec. 3.3, the Merge_{k_s} half of the (G_d, G_s) equation: the static tokens of one frame are consolidated into
+ * k_s tokens by a density-based clustering.  The paper names the method (density peaks, going by its overview
  * figure) and fixes none of its parameters; the reading taken here -- the k-nearest-neighbour form of density-peak
  * clustering that token-merging work commonly uses -- is a decision of this code, written out step by step:
  *   d2(i,j) = sum_c (x_ic - x_jc)^2 / D                            squared distance, normalised by the width
@@ -854,7 +854,7 @@ int32_t orc_ctr_merge(const void *F, int32_t dtype, int32_t N, int32_t D, int64_
 }
 
 /*
- * Sec. 3.3: "The per-frame retained group G_t combines both paths with |G_t| = G".  The k_d selected dynamic tokens
+ * Sec. 3.3, the retained group G_t of a frame (both paths together, |G_t| = G).  The k_d selected dynamic tokens
  * (their feature rows, unchanged) and the k_s merged tokens (rounded to the feature type, nearest-even), in ascending
  * order of token position -- a merged token stands at its centre's position.  retained [G][D] of `dtype`,
  * pos [G]; rows behind the k_d + k_s tokens are zero with position -1.

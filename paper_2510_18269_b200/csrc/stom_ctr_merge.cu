@@ -1,6 +1,6 @@
 // Merge_{k_s} of Causal Temporal Reduction and the retained group (paper Sec. 3.3, the static half of the (G_d, G_s)
-// equation and "the per-frame retained group combines both paths with |G_t| = G").  The paper consolidates the static
-// tokens "through density-based clustering" and fixes none of that method's parameters; the reading implemented here
+// equation, and the retained group G_t that holds both paths, |G_t| = G).  The paper consolidates the static tokens
+// by a density-based clustering and fixes none of that method's parameters; the reading implemented here
 // is the k-nearest-neighbour form of density-peak clustering (see include/stom_ctr.h for the rule, step by step).
 //
 // One block per frame.
