@@ -19,10 +19,13 @@
 //   team     the warps that work on one unit together.  The kernel comes in
 //            two shapes.  Four warps per team, warp j on tokens 16j .. 16j+15
 //            of the group: the shortest path through one unit, for calls that
-//            are latency (a decoder calling layer by layer).  One warp per
-//            team, walking the four 16-token tiles itself: the fewest
-//            instructions per unit, for calls with many units per
-//            multiprocessor (all layers at once).  The right-hand operand of
+//            are latency (a decoder calling layer by layer).  Two warps per
+//            team, each walking two 16-token tiles: fewer instructions per
+//            unit (the team's shared preparation is paid once per two tiles)
+//            and eight teams with a ring of two stages each in one block, for
+//            calls with many units per multiprocessor (all layers at once):
+//            the next unit is on its way while a team works on this one.
+//            The right-hand operand of
 //            the score product (q * s of the group, as a high and a low
 //            16-bit part) is the same for all tokens: the team prepares it
 //            once per unit, each warp a share, and passes it through shared
@@ -46,7 +49,6 @@ namespace stom {
 
 constexpr int kAtMaxWarps = 16;
 constexpr int kAtMaxThreads = kAtMaxWarps * 32;
-constexpr int kAtMaxWarpsOne = 14;  // warps of a block whose teams are single warps (more registers each)
 constexpr int kAtSysTokens = 16;   // tokens of a system-token unit (one 16-token tile)
 constexpr int kAtHeads = 8;        // query heads handled together
 constexpr int kAtMaxStages = 3;
@@ -268,9 +270,9 @@ template <int VC>
 __device__ __forceinline__ int at_oidx(int slab, int c, int head) { return slab * (VC * 8) + ((c + slab) % VC) * 8 + head; }
 
 // QT: type of q_dec; CT: type of the system-token cache and of the output; D: head dim; BITS: width of a code;
-// MPW: 16-token tiles of a unit that one warp takes (1: four warps per team; 4: one warp per team)
+// MPW: 16-token tiles of a unit that one warp takes (1: four warps per team; 2: two; 4: one warp per team)
 template <typename QT, typename CT, int D, int BITS, int MPW>
-__global__ void __launch_bounds__(MPW == 4 ? kAtMaxWarpsOne * 32 : kAtMaxThreads, 1) attend_kernel(const AttendParams p) {
+__global__ void __launch_bounds__(kAtMaxThreads, 1) attend_kernel(const AttendParams p) {
     constexpr int TW = 4 / MPW;  // warps per team
     constexpr int KS = D / 16;   // k-steps of the score product (16 channels each)
     constexpr int KC = D / 4;    // channels of a token row one thread owns in the score product
@@ -857,15 +859,13 @@ static cudaError_t attend_probe(KernelT kernel, AttendResidency &res, int dev, i
     if (e != cudaSuccess) return e;
     const int TW = 4 / MPW;
     res.n_shapes = 0;
-    // four warps per team: 4 teams (16 warps), as deep a ring as fits.  One warp per team: as many warps as fit with
-    // one stage each (half as many in two blocks per multiprocessor measured slower).
-    int cand[3], n_cand = 0;
-    if (MPW == 4) {
-        int most = kAtMaxWarpsOne;
-        while (most > 1 && at_layout(D, MPW, most, 1, stage_bytes).total > smem_max) --most;
+    // as many teams as a block of 16 warps has, fewer if their rings (two stages at least where a team has several
+    // warps) do not fit beside each other; then as deep a ring as fits
+    int cand[1], n_cand = 0;
+    {
+        int most = kAtMaxWarps / TW;
+        while (most > 1 && at_layout(D, MPW, most, TW > 1 ? 2 : 1, stage_bytes).total > smem_max) --most;
         cand[n_cand++] = most;
-    } else {
-        cand[n_cand++] = kAtMaxWarps / TW;
     }
     for (int ci = 0; ci < n_cand; ++ci) {
         AttendShape &sh = res.shapes[res.n_shapes];
@@ -900,10 +900,10 @@ static cudaError_t attend_probe(KernelT kernel, AttendResidency &res, int dev, i
     return cudaSuccess;
 }
 
-// Estimated run time (arbitrary units) of `pairs` (layer, kv head) pairs of `units` units each (n_sys of them short
-// ones) on clusters of c blocks of `teams` teams: waves of resident clusters x (fixed cost of a block + the longest
-// walk of a team x the time a team takes over a unit).
-static double attend_cost(const AttendShape &sh, int c, int64_t pairs, int units, int n_sys, double unit_time) {
+// Estimated run time (microseconds, roughly) of `pairs` (layer, kv head) pairs of `units` units each (n_sys of them
+// short ones) on clusters of c blocks of `teams` teams: waves of resident clusters x (fixed cost of a block + the
+// longest walk of a team x the time a team takes over a unit).
+static double attend_cost(const AttendShape &sh, int c, int64_t pairs, int units, int n_sys, double fixed, double unit_time) {
     if (sh.clusters[c] < 1) return 1e30;
     const int teams = c * sh.teams;
     if (c > 1 && (c - 1) * sh.teams >= units) return 1e30;  // the last block would have nothing to do
@@ -916,18 +916,18 @@ static double attend_cost(const AttendShape &sh, int c, int64_t pairs, int units
         if (load > worst) worst = load;
     }
     const double waves = (double)((pairs + sh.clusters[c] - 1) / sh.clusters[c]);
-    return waves * (6.0 + worst * unit_time) + 0.02 * c;
+    return waves * (fixed + worst * unit_time) + 0.02 * c;
 }
 
 struct AttendPlan {
     double cost = 1e30;
     int shape = -1, c = 0;
 };
-static AttendPlan attend_plan(const AttendResidency &res, int64_t pairs, int units, int n_sys, double unit_time) {
+static AttendPlan attend_plan(const AttendResidency &res, int64_t pairs, int units, int n_sys, double fixed, double unit_time) {
     AttendPlan best;
     for (int si = 0; si < res.n_shapes; ++si)
         for (int c = 1; c <= kAtMaxCluster; ++c) {
-            const double cost = attend_cost(res.shapes[si], c, pairs, units, n_sys, unit_time);
+            const double cost = attend_cost(res.shapes[si], c, pairs, units, n_sys, fixed, unit_time);
             if (cost < best.cost) {
                 best.cost = cost;
                 best.shape = si;
@@ -964,19 +964,20 @@ static int32_t attend_launch(KernelT kernel, const AttendResidency &res, const A
     return finish_launch();
 }
 
-// Both shapes of the kernel for one combination of types: the plan with the shorter estimate runs.  A team of four
-// warps takes about 3 us over a group, a team of one warp about 9 us when the multiprocessor is full of them, and a
-// block costs about 6 us before and after its units (measured on B200).
+// Both shapes of the kernel for one combination of types: the plan with the shorter estimate runs.  Measured on
+// B200: a block of four-warp teams costs about 6 us before and after its units and a team takes about 3.2 us over a
+// group; a block of two-warp teams costs about 7 us and a team takes about 4.3 us over a group with the multiprocessor
+// full of them (8 teams against 4).
 template <typename QT, typename CT, int D, int BITS>
 static int32_t launch_attend_inst(const AttendParams &p, int layers, cudaStream_t s) {
-    static AttendResidency res1, res4;
+    static AttendResidency res1, res2;
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) {
         std::lock_guard<std::mutex> lock(res1.mu);
         if (res1.dev != dev || res1.stage_bytes != p.stage_bytes) {
             e = attend_probe(attend_kernel<QT, CT, D, BITS, 1>, res1, dev, D, 1, p.stage_bytes);
-            if (e == cudaSuccess) e = attend_probe(attend_kernel<QT, CT, D, BITS, 4>, res4, dev, D, 4, p.stage_bytes);
+            if (e == cudaSuccess) e = attend_probe(attend_kernel<QT, CT, D, BITS, 2>, res2, dev, D, 2, p.stage_bytes);
         }
     }
     if (e != cudaSuccess) {
@@ -984,11 +985,11 @@ static int32_t launch_attend_inst(const AttendParams &p, int layers, cudaStream_
         return STOM_ERR_CUDA;
     }
     const int64_t pairs = (int64_t)p.g.H * layers;
-    const AttendPlan p1 = attend_plan(res1, pairs, p.n_units, p.n_sys_units, 3.2);
-    const AttendPlan p4 = attend_plan(res4, pairs, p.n_units, p.n_sys_units, 9.0);
-    if (p1.shape < 0 && p4.shape < 0) return STOM_ERR_SHAPE;
-    if (p1.cost <= p4.cost) return attend_launch(attend_kernel<QT, CT, D, BITS, 1>, res1, p1, p, 1, layers, s);
-    return attend_launch(attend_kernel<QT, CT, D, BITS, 4>, res4, p4, p, 4, layers, s);
+    const AttendPlan p1 = attend_plan(res1, pairs, p.n_units, p.n_sys_units, 6.0, 3.2);
+    const AttendPlan p2 = attend_plan(res2, pairs, p.n_units, p.n_sys_units, 7.2, 4.3);
+    if (p1.shape < 0 && p2.shape < 0) return STOM_ERR_SHAPE;
+    if (p1.cost <= p2.cost) return attend_launch(attend_kernel<QT, CT, D, BITS, 1>, res1, p1, p, 1, layers, s);
+    return attend_launch(attend_kernel<QT, CT, D, BITS, 2>, res2, p2, p, 2, layers, s);
 }
 
 template <typename QT, typename CT>
