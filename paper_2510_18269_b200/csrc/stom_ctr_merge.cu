@@ -22,7 +22,7 @@
 
 namespace stom {
 
-constexpr int kMgThreads = 256;
+constexpr int kMgThreads = 512;
 constexpr int kMgWarps = kMgThreads / 32;
 constexpr int kMgMaxTokens = 224;              // 14 row tiles of 16
 constexpr int kMgMaxTiles = kMgMaxTokens / 16;
@@ -241,24 +241,44 @@ __global__ void __launch_bounds__(kMgThreads, 1) ctr_merge_kernel(const MergePar
         }
         __syncthreads();
 
-        // ================================================================= density peaks: a thread per static token
-        // (n_s <= N <= kMgMaxTokens < kMgThreads: every loop below gives a thread at most one token)
+        // ================================================================= density peaks: two threads per static token
+        // (n_s <= N <= kMgMaxTokens, 2 * kMgMaxTokens <= kMgThreads: thread 2a + h takes the candidates b = h, h + 2, ...
+        // of token a; the two are neighbours in a warp and combine by shuffle)
+        static_assert(2 * kMgMaxTokens <= kMgThreads, "two threads per token");
         const int kk = min(p.knn, n_s - 1);
-        float far2 = 0.0f;  // the thread's largest squared distance to another static token
-        for (int a = tid; a < n_s; a += kMgThreads) {
-            const int ia = slist[a];
-            float best[kMgMaxKnn];  // the smallest squared distances, ascending
+        const int a = tid >> 1, hf = tid & 1;
+        const bool mine = a < n_s;
+        const int ia = mine ? slist[a] : 0, row = ia * (ia + 1) / 2;
+        float far2 = 0.0f;  // the token's largest squared distance to another static token
+        {
+            float best[kMgMaxKnn];  // the smallest squared distances among this thread's candidates, ascending
 #pragma unroll
             for (int q = 0; q < kMgMaxKnn; ++q) best[q] = INFINITY;
-            const int row = ia * (ia + 1) / 2;
+            if (mine) {
 #pragma unroll 4
-            for (int b = 0; b < n_s; ++b) {
-                const int ib = slist[b];
-                float v = d2[ib <= ia ? row + ib : ib * (ib + 1) / 2 + ia];
-                far2 = fmaxf(far2, v);          // (the token itself adds 0)
-                v = b == a ? INFINITY : v;      // ... and is no neighbour of itself
+                for (int b = hf; b < n_s; b += 2) {
+                    const int ib = slist[b];
+                    float v = d2[ib <= ia ? row + ib : ib * (ib + 1) / 2 + ia];
+                    far2 = fmaxf(far2, v);          // (the token itself adds 0)
+                    v = b == a ? INFINITY : v;      // ... and is no neighbour of itself
 #pragma unroll
-                for (int q = 0; q < kMgMaxKnn; ++q) {  // insertion: v sinks to its place, the largest falls out
+                    for (int q = 0; q < kMgMaxKnn; ++q) {  // insertion: v sinks to its place, the largest falls out
+                        const float lo = fminf(best[q], v);
+                        v = fmaxf(best[q], v);
+                        best[q] = lo;
+                    }
+                }
+            }
+            // the partner's list sinks into this one: both threads end with the smallest of all candidates
+            float theirs[kMgMaxKnn];
+#pragma unroll
+            for (int q = 0; q < kMgMaxKnn; ++q) theirs[q] = __shfl_xor_sync(0xffffffffu, best[q], 1);
+            far2 = fmaxf(far2, __shfl_xor_sync(0xffffffffu, far2, 1));
+#pragma unroll
+            for (int e = 0; e < kMgMaxKnn; ++e) {
+                float v = theirs[e];
+#pragma unroll
+                for (int q = 0; q < kMgMaxKnn; ++q) {
                     const float lo = fminf(best[q], v);
                     v = fmaxf(best[q], v);
                     best[q] = lo;
@@ -268,29 +288,32 @@ __global__ void __launch_bounds__(kMgThreads, 1) ctr_merge_kernel(const MergePar
 #pragma unroll
             for (int q = 0; q < kMgMaxKnn; ++q)
                 if (q < kk) sum += best[q];
-            rho[a] = kk > 0 ? expf(-sum / (float)kk) : 1.0f;
+            if (mine && hf == 0) rho[a] = kk > 0 ? expf(-sum / (float)kk) : 1.0f;
         }
         __syncthreads();
-        for (int a = tid; a < n_s; a += kMgThreads) {
-            const int ia = slist[a];
-            const float ra = rho[a];
+        {
+            const float ra = mine ? rho[a] : 0.0f;
             float near2 = INFINITY;
-            const int row = ia * (ia + 1) / 2;
+            if (mine) {
 #pragma unroll 4
-            for (int b = 0; b < n_s; ++b) {  // (b == a is never denser than a)
-                const int ib = slist[b];
-                const float rb = rho[b], v = d2[ib <= ia ? row + ib : ib * (ib + 1) / 2 + ia];
-                near2 = (rb > ra || (rb == ra && b < a)) ? fminf(near2, v) : near2;
+                for (int b = hf; b < n_s; b += 2) {  // (b == a is never denser than a)
+                    const int ib = slist[b];
+                    const float rb = rho[b], v = d2[ib <= ia ? row + ib : ib * (ib + 1) / 2 + ia];
+                    near2 = (rb > ra || (rb == ra && b < a)) ? fminf(near2, v) : near2;
+                }
             }
-            gam[a] = ra * sqrtf(near2 == INFINITY ? far2 : near2);
+            near2 = fminf(near2, __shfl_xor_sync(0xffffffffu, near2, 1));
+            if (mine && hf == 0) gam[a] = ra * sqrtf(near2 == INFINITY ? far2 : near2);
         }
         __syncthreads();
         // the k_s tokens of largest gamma (rank count; the earlier token among equals), in ascending token order
-        for (int a = tid; a < n_s; a += kMgThreads) {
-            const float ga = gam[a];
+        {
+            const float ga = mine ? gam[a] : 0.0f;
             int rank = 0;
-            for (int b = 0; b < n_s; ++b) rank += gam[b] > ga || (gam[b] == ga && b < a);
-            if (rank < k_s) flag[slist[a]] = 3;
+            if (mine)
+                for (int b = hf; b < n_s; b += 2) rank += gam[b] > ga || (gam[b] == ga && b < a);
+            rank += __shfl_xor_sync(0xffffffffu, rank, 1);
+            if (mine && hf == 0 && rank < k_s) flag[ia] = 3;
         }
         __syncthreads();
         for (int a = tid; a < n_s; a += kMgThreads) {
