@@ -98,12 +98,14 @@ int32_t stom_ctr_reduce(const void *F, const void *prev, int32_t dtype, int32_t 
  *   retained_pos out, [T][G] int32: token position of every retained row, -1 behind them
  *   centre       out, nullable, [T][G] int32: the centres in ascending order, -1 padded
  *   assign       out, nullable, [T][N] int32: for the a-th static token the index of its cluster in `centre`, -1 padded
+ *   dev_flags    nullable device word: STOM_FLAG_TIMEOUT is OR-ed in when a tensor-core product of a frame had not
+ *                completed after 0.1 s (that frame's outputs are then undefined; nothing traps, the call ends)
  * 1 <= G <= N <= 224, D a multiple of 64, at most 8192.  Errors: INVALID_ARG, SHAPE, UNSUPPORTED, ALIGNMENT, CUDA.
  */
 int32_t stom_ctr_merge(const void *F, int32_t dtype, int32_t T, int32_t N, int32_t D, int64_t stride_frame,
                        int64_t stride_token, const int32_t *k_s, const int32_t *k_d, const int32_t *static_idx,
                        const int32_t *dyn_idx, int32_t G, int32_t knn, void *retained, int32_t *retained_pos,
-                       int32_t *centre, int32_t *assign, void *stream);
+                       int32_t *centre, int32_t *assign, uint32_t *dev_flags, void *stream);
 
 /*
  * The whole of CTR for the T frames of one call, back to back on `stream`: stom_ctr_reduce (similarity, split,
@@ -114,7 +116,8 @@ int32_t stom_ctr_merge(const void *F, int32_t dtype, int32_t T, int32_t N, int32
 int32_t stom_ctr_reduce_tokens(const void *F, const void *prev, int32_t dtype, int32_t T, int32_t N, int32_t D,
                                int64_t stride_frame, int64_t stride_token, const float *alpha, int32_t G, float tau_c,
                                int32_t knn, float *sim, int32_t *k_s, int32_t *k_d, int32_t *static_idx,
-                               int32_t *dyn_idx, void *retained, int32_t *retained_pos, void *stream);
+                               int32_t *dyn_idx, void *retained, int32_t *retained_pos, uint32_t *dev_flags,
+                               void *stream);
 
 #ifdef __cplusplus
 }

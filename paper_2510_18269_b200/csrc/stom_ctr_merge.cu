@@ -5,17 +5,24 @@
 //
 // One block per frame.
 //   Gram     all pairwise inner products of the frame's N feature rows: a [N x D] . [D x N] contraction, the one dense
-//            product of CTR, on the tensor cores (mma.sync m16n8k16 on the 16-bit features, binary32 accumulation).
-//            The rows arrive in shared memory in slabs of 64 channels (cp.async, a ring of four slabs, three on their
-//            way while one is consumed; 16-byte columns swizzled by the row so that ldmatrix reads without bank
-//            conflicts); only the 16 x 16 blocks on and below the diagonal are computed and a warp keeps the
-//            accumulators of its blocks in registers over the whole contraction.  Squared distances d2(i,j) =
-//            (|x_i|^2 + |x_j|^2 - 2 x_i.x_j) / D go to a packed triangle that takes the slabs' place.
+//            product of CTR, on the fifth-generation tensor cores (tcgen05.mma, kind::f16, binary32 accumulators in
+//            tensor memory).  The rows arrive in shared memory in slabs of 64 channels (cp.async, a ring of slabs) in
+//            the canonical K-major layout with 128-byte swizzle -- a row is 128 bytes, its 16-byte columns XOR-ed
+//            with the row number modulo 8 -- so the same slab is both operands: the left one is a tile of 128 rows
+//            (rows 0..127, and a second tile that ends at the last row), the right one all rows.  One thread issues
+//            the products of a slab (4 steps of 16 channels x 2 tiles) and commits them to the slab's mbarrier, on
+//            which the loaders wait before they refill the slab.  When the last slab's products have completed, the
+//            16 warps read the accumulators from tensor memory (a warp reaches the 32 lanes of its quarter), and the
+//            squared distances d2(i,j) = (|x_i|^2 + |x_j|^2 - 2 x_i.x_j) / D, j <= i, go to a packed triangle that
+//            takes the slabs' place.
 //   cluster  a thread per token: density from the k nearest static neighbours, distance to the nearest denser token,
 //            rank count of gamma = rho * delta for the centres, nearest centre for the rest -- a few passes over rows
 //            of the triangle, N is a few hundred at most.
 //   merge    a cluster's mean, 8 channels per thread, members in ascending token order, written straight into the
 //            cluster's slot of the retained group; the selected dynamic rows are copied beside them.
+#include <type_traits>
+
+#include "stom_async.cuh"
 #include "stom_internal.cuh"
 
 #include "stom_ctr.h"
@@ -25,8 +32,8 @@ namespace stom {
 constexpr int kMgThreads = 512;
 constexpr int kMgWarps = kMgThreads / 32;
 constexpr int kMgMaxTokens = 224;              // 14 row tiles of 16
-constexpr int kMgMaxTiles = kMgMaxTokens / 16;
-constexpr int kMgMaxBlocks = (kMgMaxTiles * (kMgMaxTiles + 1) / 2 + kMgWarps - 1) / kMgWarps;  // 16 x 16 blocks per warp
+constexpr int kMgTmemCols = 512;               // tile 0: 128 columns, tile 1: up to 224; a power of two
+constexpr unsigned long long kMgWaitLimitNs = 100000000ull;  // a product that has not completed after 0.1 s ends the block
 constexpr int kMgSlabCh = 64;                  // channels per slab: 128 bytes of a row
 constexpr int kMgSlabs = 4;                    // slabs in the ring: three on their way while one is consumed
 constexpr int kMgMaxKnn = 8;
@@ -38,6 +45,7 @@ struct MergeParams {
     void *retained;
     int32_t *retained_pos, *centre, *assign;
     int32_t N, D, G, knn;
+    uint32_t *flags;
 };
 
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
@@ -46,26 +54,57 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
-                 : "r"(addr));
+
+// ---- tcgen05: tensor memory and the matrix product that reads both operands from shared memory
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t cols) {  // one whole warp; writes the base address
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
 }
-template <typename T>
-__device__ __forceinline__ void mg_mma(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1);
-template <>
-__device__ __forceinline__ void mg_mma<__nv_bfloat16>(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                                      uint32_t b0, uint32_t b1) {
-    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {  // the same warp
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
 }
-template <>
-__device__ __forceinline__ void mg_mma<__half>(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                               uint32_t b1) {
-    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+__device__ __forceinline__ void tc_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// writes of the generic proxy (cp.async, plain stores) become visible to the asynchronous proxy (the tensor cores)
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// Shared-memory matrix descriptor of a K-major operand in the 128-byte-swizzle layout: rows of 128 bytes, groups of 8
+// rows 1024 bytes apart; `addr` is where the tile starts (a multiple of 1024) plus 32 bytes per step of 16 channels.
+__device__ __forceinline__ uint64_t umma_desc_k128(uint32_t addr) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | (1ull << 16) | ((uint64_t)(1024 >> 4) << 32) | (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor of kind::f16: binary32 accumulator, both operands of type `fmt` (0 fp16, 1 bf16) and K-major,
+// a tile of 128 rows by n columns
+__device__ __forceinline__ uint32_t umma_idesc(uint32_t fmt, uint32_t n) {
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | ((n >> 3) << 17) | ((128u >> 4) << 24);
+}
+// D[tmem] (+)= A[smem] . B[smem]^T, issued by one thread
+__device__ __forceinline__ void umma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// all products issued so far by this thread arrive (once) on the mbarrier when they have completed
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 32 consecutive accumulator columns of this thread's lane (row) of tensor memory
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32]) {
+    uint32_t r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, "
+        "%18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+          "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+          "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+          "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
 
 // position of d2(a, b) in the packed lower triangle
@@ -74,12 +113,13 @@ __device__ __forceinline__ int tri(int a, int b) { return a >= b ? a * (a + 1) /
 // Shared-memory layout (bytes): the slab ring (later the triangle), then the per-token arrays
 struct MergeLayout {
     int rows, slab_bytes, off_tri, off_nrm, off_rho, off_gam, off_slist, off_cid, off_clist, off_member, off_coff, off_slot,
-        off_flag, total;
+        off_flag, off_bar, total;
 };
 __host__ __device__ inline MergeLayout merge_layout(int N) {
     MergeLayout l;
     l.rows = (N + 15) / 16 * 16;
-    l.slab_bytes = l.rows * kMgSlabCh * 2;
+    // a slab holds at least the 128 rows a tile of the left operand spans (rows past the frame's are never used)
+    l.slab_bytes = (l.rows > 128 ? l.rows : 128) * kMgSlabCh * 2;
     // the triangle is written when the last slab has been consumed: it lies over the slabs
     const int slabs = kMgSlabs * l.slab_bytes, tri_bytes = l.rows * (l.rows + 1) / 2 * 4;
     l.off_tri = 0;
@@ -94,13 +134,15 @@ __host__ __device__ inline MergeLayout merge_layout(int N) {
     l.off_coff = off; off += (l.rows + 1) * 4;  // where each cluster's members start in `member`
     l.off_slot = off; off += l.rows * 4;     // retained slot of every cluster
     l.off_flag = off; off += l.rows;         // per token: 1 static, 3 centre
+    off = (off + 15) / 16 * 16;
+    l.off_bar = off; off += kMgSlabs * 8 + 16;  // one mbarrier per slab, the tensor-memory base address, the abort word
     l.total = (off + 15) / 16 * 16;
     return l;
 }
 
 template <typename T>
 __global__ void __launch_bounds__(kMgThreads, 1) ctr_merge_kernel(const MergeParams p) {
-    extern __shared__ __align__(128) unsigned char smem[];
+    extern __shared__ __align__(1024) unsigned char smem[];
     const int N = p.N, D = p.D, G = p.G, t = blockIdx.x;
     const MergeLayout L = merge_layout(N);
     const int NT = L.rows / 16;
@@ -138,46 +180,39 @@ __global__ void __launch_bounds__(kMgThreads, 1) ctr_merge_kernel(const MergePar
 
     if (k_s > 0) {
         // ================================================================= Gram matrix on the tensor cores
-        // 16 x 16 blocks (i, j), j <= i, numbered row by row; warp w owns a run of consecutive blocks, most of them in
-        // one row, so that the row's operand fragment is loaded once per run of equal rows
-        const int n_blk = NT * (NT + 1) / 2, per_warp = (n_blk + kMgWarps - 1) / kMgWarps;
-        const int blk0 = warp * per_warp, n_mine_blk = max(0, min(per_warp, n_blk - blk0));
-        int bi_[kMgMaxBlocks], bj_[kMgMaxBlocks];
-        float acc[kMgMaxBlocks][2][4];
-#pragma unroll
-        for (int b = 0; b < kMgMaxBlocks; ++b) {
-            const int n = blk0 + b;
-            int i = 0;
-            while ((i + 1) * (i + 2) / 2 <= n) ++i;  // row of block n
-            bi_[b] = i;
-            bj_[b] = n - i * (i + 1) / 2;
-#pragma unroll
-            for (int u = 0; u < 2; ++u)
-#pragma unroll
-                for (int e = 0; e < 4; ++e) acc[b][u][e] = 0.0f;
+        // Tile 0 of the left operand is rows 0..127, tile 1 the 128 rows that end at the last one (they overlap where
+        // the frame has fewer than 256 rows; a frame of up to 128 rows has tile 0 only).  The right operand is all rows.
+        const uint32_t slab0 = smem_u32(smem), bar0 = smem_u32(smem + L.off_bar);
+        volatile uint32_t *tmem_word = reinterpret_cast<volatile uint32_t *>(smem + L.off_bar + kMgSlabs * 8);
+        volatile uint32_t *abort_flag = tmem_word + 1;
+        const bool two_tiles = L.rows > 128;
+        const int R1 = L.rows - 128;  // first row of tile 1 (a multiple of 16)
+        const bool aligned = (slab0 & 1023u) == 0;  // the swizzle is a function of the address: slabs start on 1024 bytes
+        if (tid == 0) {
+            for (int sl = 0; sl < kMgSlabs; ++sl) mbar_init(bar0 + 8 * sl, 1);
+            // (a frame is not started on the tensor cores once another frame of the call has given up)
+            const bool gave_up = p.flags && (*reinterpret_cast<volatile uint32_t *>(p.flags) & STOM_FLAG_TIMEOUT);
+            *abort_flag = aligned && !gave_up ? 0u : 1u;
+            mbar_init_fence();
         }
-        const uint32_t slab0 = (uint32_t)__cvta_generic_to_shared(smem);
-        // rows beyond N stay zero in every slab
-        for (int e = tid; e < (L.rows - N) * 8 * kMgSlabs; e += kMgThreads) {
-            const int sl = e / ((L.rows - N) * 8), r = N + (e % ((L.rows - N) * 8)) / 8, c = e % 8;
+        if (warp == 0) tmem_alloc(smem_u32(const_cast<uint32_t *>(tmem_word)), kMgTmemCols);
+        // rows beyond N stay zero in every slab (their products are never read, but they must be numbers)
+        for (int e = tid; e < (L.slab_bytes / 128 - N) * 8 * kMgSlabs; e += kMgThreads) {
+            const int per = (L.slab_bytes / 128 - N) * 8;
+            const int sl = e / per, r = N + (e % per) / 8, c = e % 8;
             *reinterpret_cast<uint4 *>(smem + sl * L.slab_bytes + r * 128 + c * 16) = make_uint4(0, 0, 0, 0);
         }
-        // Where a lane's ldmatrix row sits inside a tile, per k-step of a slab: the left operand's lane l supplies row
-        // l % 16 and the 16-byte column 2 ks + l / 16; the right operand's, row l % 8 + 8 (l / 16) and column 2 ks +
-        // (l / 8) % 2.  A tile starts at a multiple of 16 rows, so the swizzle (column ^ row % 8) depends on the lane only.
-        uint32_t offA[kMgSlabCh / 16], offB[kMgSlabCh / 16];
-#pragma unroll
-        for (int ks = 0; ks < kMgSlabCh / 16; ++ks) {
-            const int ra = lane & 15, ca = 2 * ks + (lane >> 4);
-            const int rb = (lane & 7) + ((lane >> 4) << 3), cb = 2 * ks + ((lane >> 3) & 1);
-            offA[ks] = (uint32_t)(ra * 128 + ((ca ^ (ra & 7)) << 4));
-            offB[ks] = (uint32_t)(rb * 128 + ((cb ^ (rb & 7)) << 4));
-        }
+        tc_fence_before_sync();
+        __syncthreads();
+        tc_fence_after_sync();
+        const uint32_t tmem = *tmem_word;
+        bool dead = *abort_flag != 0;
+        if (dead && tid == 0 && p.flags) atomicOr(p.flags, STOM_FLAG_TIMEOUT);
         const int n_chunks = D / kMgSlabCh;
         // channels [64 chunk, 64 chunk + 64) of rows 0 .. N-1 into slab chunk % kMgSlabs; always one group per call, an
         // empty one past the last chunk, so that the number of groups in flight tells which chunk has landed
         auto load_slab = [&](int chunk) {
-            if (chunk < n_chunks) {
+            if (chunk < n_chunks && !dead) {
                 const uint32_t to = slab0 + (chunk % kMgSlabs) * L.slab_bytes;
                 for (int e = tid; e < N * 8; e += kMgThreads) {
                     const int r = e >> 3, c = e & 7;
@@ -186,60 +221,109 @@ __global__ void __launch_bounds__(kMgThreads, 1) ctr_merge_kernel(const MergePar
             }
             cp_async_commit();
         };
+        const uint32_t fmt = sizeof(T) == 2 && std::is_same<T, __nv_bfloat16>::value ? 1u : 0u;
+        const uint32_t idesc0 = umma_idesc(fmt, 128u < (uint32_t)L.rows ? 128u : (uint32_t)L.rows);
+        const uint32_t idesc1 = umma_idesc(fmt, (uint32_t)L.rows);
         for (int ch = 0; ch < kMgSlabs - 1; ++ch) load_slab(ch);
         for (int ch = 0; ch < n_chunks; ++ch) {
             cp_async_wait<kMgSlabs - 2>();  // chunk ch has landed (this thread's part of it)
-            __syncthreads();                // ... everybody's; and everybody is done with chunk ch - 1
-            load_slab(ch + kMgSlabs - 1);   // into the slab chunk ch - 1 has just left
-            const uint32_t base = slab0 + (ch % kMgSlabs) * L.slab_bytes;
+            fence_proxy_async();            // ... and the tensor cores may read it
+            __syncthreads();                // ... everybody's
+            if (tid == 0 && !dead) {
+                tc_fence_after_sync();
+                const uint32_t base = slab0 + (ch % kMgSlabs) * L.slab_bytes;
 #pragma unroll
-            for (int ks = 0; ks < kMgSlabCh / 16; ++ks) {
-                const uint32_t pa = base + offA[ks], pb = base + offB[ks];
-                uint32_t a0 = 0, a1 = 0, a2 = 0, a3 = 0;
+                for (int ks = 0; ks < kMgSlabCh / 16; ++ks) {
+                    const uint64_t b = umma_desc_k128(base + ks * 32);
+                    const uint32_t acc = (ch | ks) != 0;
+                    umma_ss(tmem, b, b, idesc0, acc);  // rows 0..127 against columns 0..127 (only j <= i is read)
+                    if (two_tiles) umma_ss(tmem + 128, umma_desc_k128(base + R1 * 128 + ks * 32), b, idesc1, acc);
+                }
+                umma_commit(bar0 + 8 * (ch % kMgSlabs));  // arrives when these products no longer need the slab
+            }
+            // the slab of chunk ch - 1 takes chunk ch + kMgSlabs - 1 once that chunk's products have completed
+            if (ch > 0 && ch + kMgSlabs - 1 < n_chunks && !dead) {
+                const int pc = ch - 1;
+                if (!mbar_wait_bounded(bar0 + 8 * (pc % kMgSlabs), (pc / kMgSlabs) & 1, abort_flag, kMgWaitLimitNs)) {
+                    dead = true;
+                    *abort_flag = 1;  // everybody else's waits end at once
+                }
+            }
+            load_slab(ch + kMgSlabs - 1);
+        }
+        cp_async_wait<0>();
+        // every product has completed when the last chunk's have (a commit covers all products issued before it)
+        if (!dead) {
+            const int lc = n_chunks - 1;
+            if (!mbar_wait_bounded(bar0 + 8 * (lc % kMgSlabs), (lc / kMgSlabs) & 1, abort_flag, kMgWaitLimitNs)) {
+                dead = true;
+                *abort_flag = 1;
+            }
+        }
+        if (dead) {
+            *abort_flag = 1;
+            if (p.flags && (tid & 31) == 0) atomicOr(p.flags, STOM_FLAG_TIMEOUT);
+        }
+        tc_fence_after_sync();
+        __syncthreads();  // the slabs are dead: the triangle takes their place
+        dead = *abort_flag != 0;
+
+        // ---- a warp reaches lanes 32 q .. 32 q + 31 of tensor memory, q = warp % 4: lane l of the warp is row 32 q + l of
+        //      tile 0 and row R1 + 32 q + l of tile 1; the four warps of a quarter share out the blocks of 32 columns
+        const int q = warp & 3, jw = warp >> 2;
+        const uint32_t lane_base = tmem + ((uint32_t)(32 * q) << 16);
+        const int r0 = 32 * q + lane, r1 = R1 + 32 * q + lane;  // this thread's row in tile 0 and in tile 1
+        float v[32];
+        if (!dead) {
+            // squared norms from the diagonal: row r of tile 0 for r < 128, of tile 1 above
+            if (jw == 0 && 32 * q < L.rows) {
+                tmem_ld32(lane_base + 32 * q, v);
+                float dg = 0.0f;
 #pragma unroll
-                for (int b = 0; b < kMgMaxBlocks; ++b) {
-                    if (b < n_mine_blk) {  // warp-uniform
-                        uint32_t b0, b1, b2, b3;
-                        if (b == 0 || bi_[b] != bi_[b - 1])  // (warp-uniform) a tile of 16 rows is 2048 bytes of a slab
-                            ldmatrix_x4(pa + (bi_[b] << 11), a0, a1, a2, a3);
-                        ldmatrix_x4(pb + (bj_[b] << 11), b0, b1, b2, b3);
-                        mg_mma<T>(acc[b][0], a0, a1, a2, a3, b0, b1);
-                        mg_mma<T>(acc[b][1], a0, a1, a2, a3, b2, b3);
+                for (int i = 0; i < 32; ++i) dg = i == lane ? v[i] : dg;
+                if (r0 < N) nrm[r0] = dg;
+            }
+            if (jw == 1 && two_tiles) {
+                tmem_ld32(lane_base + 128 + R1 + 32 * q, v);
+                float dg = 0.0f;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) dg = i == lane ? v[i] : dg;
+                if (r1 >= 128 && r1 < N) nrm[r1] = dg;
+            }
+        }
+        __syncthreads();
+        if (!dead) {
+            const float inv_d = 1.0f / (float)D;
+            // tile 0: rows 32 q .. 32 q + 31 need column blocks 0 .. q
+            for (int cb = jw; cb <= q && 32 * q < L.rows; cb += 4) {
+                tmem_ld32(lane_base + 32 * cb, v);
+                if (r0 < N) {
+                    const float nr = nrm[r0];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int c = 32 * cb + i;
+                        if (c <= r0) d2[r0 * (r0 + 1) / 2 + c] = fmaxf(0.0f, (nr + nrm[c]) - 2.0f * v[i]) * inv_d;
+                    }
+                }
+            }
+            // tile 1: rows R1 + 32 q .. need column blocks 0 .. (R1 + 32 q + 31) / 32; only rows from 128 on are new
+            if (two_tiles && R1 + 32 * q + 31 >= 128) {
+                for (int cb = jw; cb <= (R1 + 32 * q + 31) >> 5; cb += 4) {
+                    tmem_ld32(lane_base + 128 + 32 * cb, v);
+                    if (r1 >= 128 && r1 < N) {
+                        const float nr = nrm[r1];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const int c = 32 * cb + i;
+                            if (c <= r1) d2[r1 * (r1 + 1) / 2 + c] = fmaxf(0.0f, (nr + nrm[c]) - 2.0f * v[i]) * inv_d;
+                        }
                     }
                 }
             }
         }
-        cp_async_wait<0>();
-        __syncthreads();  // the slabs are dead: the triangle takes their place
-        // ---- squared norms from the diagonal blocks, then the distances
-        const int g = lane >> 2, tq = lane & 3;
-#pragma unroll
-        for (int b = 0; b < kMgMaxBlocks; ++b) {
-            if (b < n_mine_blk && bi_[b] == bj_[b]) {
-#pragma unroll
-                for (int u = 0; u < 2; ++u)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int r = g + 8 * (e >> 1), c = 8 * u + 2 * tq + (e & 1);
-                        if (r == c) nrm[16 * bi_[b] + r] = acc[b][u][e];
-                    }
-            }
-        }
+        tc_fence_before_sync();
         __syncthreads();
-        const float inv_d = 1.0f / (float)D;
-#pragma unroll
-        for (int b = 0; b < kMgMaxBlocks; ++b) {
-            if (b < n_mine_blk) {
-#pragma unroll
-                for (int u = 0; u < 2; ++u)
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int r = 16 * bi_[b] + g + 8 * (e >> 1), c = 16 * bj_[b] + 8 * u + 2 * tq + (e & 1);
-                        if (c <= r) d2[r * (r + 1) / 2 + c] = fmaxf(0.0f, (nrm[r] + nrm[c]) - 2.0f * acc[b][u][e]) * inv_d;
-                    }
-            }
-        }
-        __syncthreads();
+        if (warp == 0) tmem_dealloc(tmem, kMgTmemCols);  // the tensor memory goes back before the clustering starts
 
         // ================================================================= density peaks: two threads per static token
         // (n_s <= N <= kMgMaxTokens, 2 * kMgMaxTokens <= kMgThreads: thread 2a + h takes the candidates b = h, h + 2, ...
@@ -434,7 +518,7 @@ using namespace stom;
 extern "C" int32_t stom_ctr_merge(const void *F, int32_t dtype, int32_t T, int32_t N, int32_t D, int64_t stride_frame,
                                   int64_t stride_token, const int32_t *k_s, const int32_t *k_d, const int32_t *static_idx,
                                   const int32_t *dyn_idx, int32_t G, int32_t knn, void *retained, int32_t *retained_pos,
-                                  int32_t *centre, int32_t *assign, void *stream) {
+                                  int32_t *centre, int32_t *assign, uint32_t *dev_flags, void *stream) {
     if (!F || !k_s || !k_d || !static_idx || !dyn_idx || !retained || !retained_pos || T < 0 || N < 1 || D < 1 || G < 1 || knn < 0)
         return STOM_ERR_INVALID_ARG;
     if (dtype != STOM_BF16 && dtype != STOM_FP16) return STOM_ERR_UNSUPPORTED;
@@ -442,11 +526,11 @@ extern "C" int32_t stom_ctr_merge(const void *F, int32_t dtype, int32_t T, int32
     if (stride_token < D || stride_frame < 0) return STOM_ERR_INVALID_ARG;
     if (!aligned16(F) || !aligned16(retained) || !stride_ok(stride_frame, dtype) || !stride_ok(stride_token, dtype))
         return STOM_ERR_ALIGNMENT;
-    const void *ptrs[7] = {k_s, k_d, static_idx, dyn_idx, retained_pos, centre, assign};
+    const void *ptrs[8] = {k_s, k_d, static_idx, dyn_idx, retained_pos, centre, assign, dev_flags};
     for (const void *q : ptrs)
         if (reinterpret_cast<uintptr_t>(q) & 3u) return STOM_ERR_ALIGNMENT;
     if (T == 0) return STOM_OK;
-    MergeParams p{F, stride_frame, stride_token, k_s, k_d, static_idx, dyn_idx, retained, retained_pos, centre, assign, N, D, G, knn};
+    MergeParams p{F, stride_frame, stride_token, k_s, k_d, static_idx, dyn_idx, retained, retained_pos, centre, assign, N, D, G, knn, dev_flags};
     const size_t smem = (size_t)merge_layout(N).total;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     cudaError_t e;
@@ -468,15 +552,16 @@ extern "C" int32_t stom_ctr_reduce_tokens(const void *F, const void *prev, int32
                                           int64_t stride_frame, int64_t stride_token, const float *alpha, int32_t G,
                                           float tau_c, int32_t knn, float *sim, int32_t *k_s, int32_t *k_d,
                                           int32_t *static_idx, int32_t *dyn_idx, void *retained, int32_t *retained_pos,
-                                          void *stream) {
+                                          uint32_t *dev_flags, void *stream) {
     // every argument list is checked before the first launch
     if (!retained || !retained_pos || knn < 0) return STOM_ERR_INVALID_ARG;
     if (dtype != STOM_BF16 && dtype != STOM_FP16) return STOM_ERR_UNSUPPORTED;
     if (N < 1 || G < 1 || G > N || N > kMgMaxTokens || D < 1 || D % kMgSlabCh || D > 8192 || knn > kMgMaxKnn) return STOM_ERR_SHAPE;
-    if (!aligned16(retained) || (reinterpret_cast<uintptr_t>(retained_pos) & 3u)) return STOM_ERR_ALIGNMENT;
+    if (!aligned16(retained) || (reinterpret_cast<uintptr_t>(retained_pos) & 3u) || (reinterpret_cast<uintptr_t>(dev_flags) & 3u))
+        return STOM_ERR_ALIGNMENT;
     int32_t rc = stom_ctr_reduce(F, prev, dtype, T, N, D, stride_frame, stride_token, alpha, G, tau_c, sim, k_s, k_d,
                                  static_idx, dyn_idx, stream);
     if (rc) return rc;
     return stom_ctr_merge(F, dtype, T, N, D, stride_frame, stride_token, k_s, k_d, static_idx, dyn_idx, G, knn, retained,
-                          retained_pos, nullptr, nullptr, stream);
+                          retained_pos, nullptr, nullptr, dev_flags, stream);
 }

@@ -318,20 +318,20 @@ def stom_ctr_reduce(F, prev, T, N, D, strides, alpha, G, tau_c, sim, k_s, k_d, s
 
 
 def stom_ctr_merge(F, T, N, D, strides, k_s, k_d, static_idx, dyn_idx, G, knn, retained, retained_pos, centre=None,
-                   assign=None, stream=None):
+                   assign=None, dev_flags=None, stream=None):
     """Merge_{k_s} of the static tokens and the retained group [T][G][D] (see include/stom_ctr.h for the rule)."""
     sf, st = strides
     _check(lib().stom_ctr_merge(_ptr(F), C.c_int32(dtype_code(F.dtype)), C.c_int32(T), C.c_int32(N), C.c_int32(D),
                                 C.c_int64(sf), C.c_int64(st), _ptr(k_s), _ptr(k_d), _ptr(static_idx), _ptr(dyn_idx),
                                 C.c_int32(G), C.c_int32(knn), _ptr(retained), _ptr(retained_pos), _ptr(centre),
-                                _ptr(assign), _stream(stream)), "stom_ctr_merge")
+                                _ptr(assign), _ptr(dev_flags), _stream(stream)), "stom_ctr_merge")
 
 
 def stom_ctr_reduce_tokens(F, prev, T, N, D, strides, alpha, G, tau_c, knn, sim, k_s, k_d, static_idx, dyn_idx, retained,
-                           retained_pos, stream=None):
+                           retained_pos, dev_flags=None, stream=None):
     sf, st = strides
     _check(lib().stom_ctr_reduce_tokens(_ptr(F), _ptr(prev), C.c_int32(dtype_code(F.dtype)), C.c_int32(T), C.c_int32(N),
                                         C.c_int32(D), C.c_int64(sf), C.c_int64(st), _ptr(alpha), C.c_int32(G),
                                         C.c_float(tau_c), C.c_int32(knn), _ptr(sim), _ptr(k_s), _ptr(k_d),
                                         _ptr(static_idx), _ptr(dyn_idx), _ptr(retained), _ptr(retained_pos),
-                                        _stream(stream)), "stom_ctr_reduce_tokens")
+                                        _ptr(dev_flags), _stream(stream)), "stom_ctr_reduce_tokens")

@@ -152,7 +152,11 @@ def _check_merge(orc, oqm, F, alpha, G, knn, dtype, o_sim=None, min_clear=0.3):
     cen = torch.full((T * G + P.GUARD,), -9, dtype=torch.int32, device="cuda")
     asg = torch.full((T * N + P.GUARD,), -9, dtype=torch.int32, device="cuda")
     up = lambda a: torch.from_numpy(a).cuda()
-    oqm.stom_ctr_merge(F.cuda(), T, N, D, (N * D, D), up(ks), up(kd), up(sidx), up(didx), G, knn, ret_flat, pos, cen, asg)
+    flags = torch.zeros(1, dtype=torch.int32, device="cuda")
+    oqm.stom_ctr_merge(F.cuda(), T, N, D, (N * D, D), up(ks), up(kd), up(sidx), up(didx), G, knn, ret_flat, pos, cen, asg,
+                       dev_flags=flags)
+    torch.cuda.synchronize()
+    assert int(flags.item()) == 0
     torch.cuda.synchronize()
     assert torch.all(ret_flat[T * G * D:] == 3.0) and torch.all(pos[T * G:] == -9), "guard band overwritten"
     assert torch.all(cen[T * G:] == -9) and torch.all(asg[T * N:] == -9), "guard band overwritten"
