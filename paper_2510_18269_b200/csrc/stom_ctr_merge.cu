@@ -35,7 +35,7 @@ constexpr int kMgMaxTokens = 224;              // 14 row tiles of 16
 constexpr int kMgTmemCols = 512;               // tile 0: 128 columns, tile 1: up to 224; a power of two
 constexpr unsigned long long kMgWaitLimitNs = 100000000ull;  // a product that has not completed after 0.1 s ends the block
 constexpr int kMgSlabCh = 64;                  // channels per slab: 128 bytes of a row
-constexpr int kMgSlabs = 4;                    // slabs in the ring: three on their way while one is consumed
+constexpr int kMgSlabs = 3;                    // slabs in the ring: two on their way while one is consumed
 constexpr int kMgMaxKnn = 8;
 
 struct MergeParams {
@@ -141,7 +141,7 @@ __host__ __device__ inline MergeLayout merge_layout(int N) {
 }
 
 template <typename T>
-__global__ void __launch_bounds__(kMgThreads, 1) ctr_merge_kernel(const MergeParams p) {
+__global__ void __launch_bounds__(kMgThreads, 2) ctr_merge_kernel(const MergeParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     const int N = p.N, D = p.D, G = p.G, t = blockIdx.x;
     const MergeLayout L = merge_layout(N);
