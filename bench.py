@@ -886,8 +886,9 @@ def run_ctr(args):
     sel_ms = sdist.max_over_ranks(statistics.mean(t[1].elapsed_time(t[2]) for t in timers))
     tot_ms = sdist.max_over_ranks(statistics.mean(t[0].elapsed_time(t[2]) for t in timers))
     mg_ms = sdist.max_over_ranks(statistics.median(t[2].elapsed_time(t[3]) for t in timers))
-    # Merge: the Gram matrix of a frame's N tokens is a [N x D] . [D x N] contraction; only the 16 x 16 blocks on and
-    # below the diagonal are computed.  Its bytes: the frame's features once, the retained group written once.
+    # Merge: the Gram matrix of a frame's N tokens is a [N x D] . [D x N] contraction of which only the part on and
+    # below the diagonal is needed (counted here in 16 x 16 blocks; the kernel's two 128-row tiles compute more).  Its
+    # bytes: the frame's features once, the retained group written once.
     tiles = (N + 15) // 16
     mg_flops = T * (tiles * (tiles + 1) // 2) * 2 * 16 * 16 * D
     mg_bytes = T * (N * D * 2 + G * D * 2 + (N + 3 * G + 2) * 4)
@@ -909,8 +910,9 @@ def run_ctr(args):
                                  "gram_TFLOPs": mg_flops / (mg_ms * 1e-3) / 1e12,
                                  "GBps": mg_bytes / (mg_ms * 1e-3) / 1e9,
                                  "frac_of_measured_hbm": mg_bytes / (mg_ms * 1e-3) / 1e9 / peak,
-                                 "note": "Merge_{k_s} + retained group; the Gram matrix runs on the tensor cores (warp-level "
-                                         "matrix products); not part of `value`, which covers similarity + select"},
+                                 "note": "Merge_{k_s} + retained group; the Gram matrix runs on the tensor cores (tcgen05, "
+                                         "accumulators in tensor memory); flops and bytes are the algorithmic ones; not part "
+                                         "of `value`, which covers similarity + select"},
                        "whole_ctr_frames_per_s": world * T / ((tot_ms + mg_ms) * 1e-3)},
         "roofline": {"kernel": "ctr_similarity_kernel", "bound": "hbm", "achieved": a, "peak": peak, "unit": "GB/s",
                      "frac": a / peak, "traffic": None if tpu is None else tpu * T, "peak_source": peak_src,
