@@ -1,4 +1,5 @@
-"""The streaming interleave end to end, CUDA library against the oracle driven by the same call sequence: frames of
+"""The streaming interleave end to end (at a small geometry, and at the 7B stack's own: 28 layers, 240 frames), CUDA
+library against the oracle driven by the same call sequence: frames of
 196 tokens arrive one at a time, 50 of them are kept by a seeded mask, quantized and appended; every few frames a
 question is scored against what has been stored so far, the top groups are selected and reconstructed behind the
 system tokens, and one decode step attends over the result.  Checked at every question: scores, selection, the
@@ -17,11 +18,18 @@ from paper_2510_18269_b200 import synth
 pytestmark = pytest.mark.gpu
 
 
-def test_streaming_interleave_matches_oracle(orc):
+@pytest.mark.parametrize("name,geom,every,sys_len", [
+    ("C4-small", dict(L=2, H_q=8, H_k=4, T=40, T_q=5, k=8), 6, 11),
+    # the 7B stack as it streams: all 28 layers, 240 frames, a question every 60 frames, 64 groups + 32 system tokens
+    ("C4-7B-240-frames", dict(L=28, H_q=28, H_k=4, T=240, T_q=16, k=64), 60, 32),
+])
+def test_streaming_interleave_matches_oracle(orc, name, geom, every, sys_len):
     from paper_2510_18269_b200 import oqm
     oqm.lib()
-    sh = dataclasses.replace(synth.C4, L=2, H_q=8, H_k=4, T=40, T_q=5, k=8, name="C4-small")
-    every, sys_len = 6, 11
+    sh = dataclasses.replace(synth.C4, name=name, **geom)
+    need = 2 * sh.L * sh.T * sh.H_k * sh.N_in * sh.d * 2 * 1.5
+    if torch.cuda.mem_get_info()[0] < need:
+        pytest.skip("not enough free device memory for this stream")
     K, V = synth.kv_stream(sh)                                       # [L][T][H_k][196][d]
     keep = synth.keep_mask(sh, 0, sh.T)                              # [T][50]
     ocfg, gcfg = P.oracle_cfg(orc, sh), P.gpu_cfg(oqm, sh)
