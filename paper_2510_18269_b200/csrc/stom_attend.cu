@@ -311,6 +311,10 @@ __global__ void __launch_bounds__(kAtMaxThreads, 1) attend_kernel(const AttendPa
         else named_sync(1 + team, 32 * TW);
     };
 
+    // The launch may overlap the tail of the kernel ahead of it in the stream (programmatic dependent launch): what
+    // follows up to the wait touches shared memory only; the kernel behind this one may be scheduled from here on
+    // and does its own waiting.
+    grid_launch_dependents();
     if (wj == 0 && lane == 0) {
         for (int s = 0; s < S; ++s) mbar_init(bar0 + 8 * s, 1);
         if (warp == 0) {
@@ -399,6 +403,8 @@ __global__ void __launch_bounds__(kAtMaxThreads, 1) attend_kernel(const AttendPa
         }
     };
 
+    // everything above is arithmetic on the arguments; from here on global memory is read
+    grid_dependency_wait();  // indices, the query rows or the bank may come from the kernel just ahead in the stream
     for (int h0 = 0; h0 < p.rep; h0 += kAtHeads) {
         const int nh = min(kAtHeads, p.rep - h0);
         // ---- start the first units on their way, then fetch this warp's share of the query rows behind them
@@ -949,13 +955,15 @@ static int32_t attend_launch(KernelT kernel, const AttendResidency &res, const A
     lc.dynamicSmemBytes = sh.smem;
     lc.stream = s;
     lc.gridDim = dim3((unsigned)plan.c, (unsigned)p.g.H, (unsigned)layers);
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = (unsigned)plan.c;
     at[0].val.clusterDim.y = 1;
     at[0].val.clusterDim.z = 1;
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // see the kernel's prologue
+    at[1].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = at;
-    lc.numAttrs = 1;
+    lc.numAttrs = 2;
     const cudaError_t e = cudaLaunchKernelEx(&lc, kernel, q);
     if (e != cudaSuccess) {
         set_last_cuda_error(e);
