@@ -424,6 +424,9 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
     const uint32_t full0 = smem_u32(bars), empty0 = full0 + 2 * kMaxSlots * 8;
     auto full_bar = [&](int slot, uint32_t round) -> uint32_t { return full0 + 8 * ((round & 1u) * kMaxSlots + slot); };
 
+    // The launch may overlap the tail of the kernel ahead of it in the stream (programmatic dependent launch): the
+    // barriers are set up meanwhile, and every thread waits for that kernel before it touches global memory.
+    grid_launch_dependents();
     if (threadIdx.x == 0) {
         for (int i = 0; i < N; ++i) {
             mbar_init(full0 + 8 * i, 1);
@@ -436,6 +439,7 @@ __global__ void __launch_bounds__(kQuantThreads, 1) quantize_kernel(const QuantP
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    grid_dependency_wait();  // the frames may come from, and the bank may still be read by, the kernel just ahead
 
     // tiles of this block: tau = blockIdx.x + n * gridDim.x, n = 0 .. my_count-1
     const uint32_t my_count = p.n_tiles > blockIdx.x ? (p.n_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u;
@@ -774,7 +778,11 @@ static int32_t launch_quantize(QuantParams p, cudaStream_t stream) {
         return STOM_ERR_CUDA;
     }
     const unsigned grid = p.n_tiles < (uint32_t)sms ? p.n_tiles : (unsigned)sms;
-    quantize_kernel<T, C, BITS, MD><<<grid, kQuantThreads, smem, stream>>>(p);
+    e = launch_after_producer(quantize_kernel<T, C, BITS, MD>, dim3(grid), dim3(kQuantThreads), smem, stream, p);
+    if (e != cudaSuccess) {
+        set_last_cuda_error(e);
+        return STOM_ERR_CUDA;
+    }
     return finish_launch();
 }
 
