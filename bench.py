@@ -41,7 +41,7 @@ FALLBACK_HBM_GBS = 6650.0
 # case of the same kernel and scaled by the units one launch processes; see profiles/*.md.  None = not captured.
 NCU_TRAFFIC_PER_UNIT = {
     # all figures are per kv head of the unit named (the captures ran the 4-head 7B geometry)
-    "quantize_kernel": 137535.0 / 4,    # bytes per (layer, frame): 3.943 GB over 28 x 1024 units
+    "quantize_kernel": 137448.0 / 4,    # bytes per (layer, frame): 3.941 GB over 28 x 1024 units
     # bytes per (layer, selected group): 186.0 MB over 28 x 64 units; of the 183.5 MB the kernel writes only
     # 125.4 MB had left L2 when it ended (the rest is written back later), so this undercounts by design
     "dequant_gather_kernel": 103805.0 / 4,
