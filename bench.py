@@ -854,6 +854,7 @@ def run_ctr(args):
 
     ret = torch.empty(T, G, D, dtype=F.dtype, device=dev)
     rpos = torch.empty(T, G, dtype=torch.int32, device=dev)
+    mflags = torch.zeros(1, dtype=torch.int32, device=dev)
 
     def step(timers=None):
         flush.fill_(1)       # evict everything ...
@@ -864,7 +865,7 @@ def run_ctr(args):
         e[1].record()
         oqm.stom_ctr_select(sim, alpha, T, N, G, c["tau_c"], ks, kd, si, di)
         e[2].record()
-        oqm.stom_ctr_merge(F, T, N, D, (N * D, D), ks, kd, si, di, G, 5, ret, rpos)
+        oqm.stom_ctr_merge(F, T, N, D, (N * D, D), ks, kd, si, di, G, 5, ret, rpos, dev_flags=mflags)
         e[3].record()
         if timers is not None:
             timers.append(e)
@@ -881,6 +882,8 @@ def run_ctr(args):
         step(timers)
     torch.cuda.synchronize()
     sdist.barrier()
+    if int(mflags.item()) != 0:
+        raise RuntimeError(f"stom_ctr_merge raised device flags {int(mflags.item()):#x}: its timing is void")
     clocks = sampler.result()
     sim_ms = sdist.max_over_ranks(statistics.mean(t[0].elapsed_time(t[1]) for t in timers))
     sel_ms = sdist.max_over_ranks(statistics.mean(t[1].elapsed_time(t[2]) for t in timers))
