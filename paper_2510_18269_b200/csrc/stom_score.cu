@@ -63,7 +63,9 @@ extern "C" int32_t stom_oqm_score_groups(const stom_oqm_config *cfg, const stom_
     }
     if ((rc = finish_launch())) return rc;
 
-    // about eight blocks per SM over the whole grid, each with a contiguous run of groups (at least 32)
+    // about two blocks per SM over the whole grid, each with a long contiguous run of groups (at least 32): a block's
+    // first loads and its last reduction are paid once per run.  The kernel is launched so that its blocks may be
+    // scheduled under the tail of the embedding kernel; it waits for that kernel before it reads the embeddings.
     int dev = 0, sms = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
@@ -71,7 +73,7 @@ extern "C" int32_t stom_oqm_score_groups(const stom_oqm_config *cfg, const stom_
         set_last_cuda_error(e);
         return STOM_ERR_CUDA;
     }
-    int chunks = (8 * sms + layer_count - 1) / layer_count;
+    int chunks = (2 * sms) / layer_count;
     if (chunks > (n_groups + 31) / 32) chunks = (n_groups + 31) / 32;
     if (chunks < 1) chunks = 1;
     p.groups_per_block = (n_groups + chunks - 1) / chunks;
@@ -79,17 +81,18 @@ extern "C" int32_t stom_oqm_score_groups(const stom_oqm_config *cfg, const stom_
     const size_t smem = (size_t)cfg->n_kv_heads * (cfg->head_dim + 1) * sizeof(float);
     const int HD = cfg->n_kv_heads * cfg->head_dim;
     const bool fast = !p.per_head && cfg->n_kv_heads <= 32;
+    cudaError_t le = cudaSuccess;
 #define STOM_SCORE_LAUNCH(KT_)                                                                       \
     switch (score_fast_v4(HD, fast, cfg->meta_dtype)) {                                             \
-    case 4: score_kernel<4, KT_><<<g2, kScoreWarps * 32, smem, s>>>(p); break; /* 4 kv heads x 128 */ \
-    case 8: score_kernel<8, KT_><<<g2, kScoreWarps * 32, smem, s>>>(p); break; /* 8 kv heads x 128 */ \
-    case 2: score_kernel<2, KT_><<<g2, kScoreWarps * 32, smem, s>>>(p); break;                      \
+    case 4: le = launch_after_producer(score_kernel<4, KT_>, g2, dim3(kScoreWarps * 32), smem, s, p); break; /* 4 kv heads x 128 */ \
+    case 8: le = launch_after_producer(score_kernel<8, KT_>, g2, dim3(kScoreWarps * 32), smem, s, p); break; /* 8 kv heads x 128 */ \
+    case 2: le = launch_after_producer(score_kernel<2, KT_>, g2, dim3(kScoreWarps * 32), smem, s, p); break;                      \
     case 1:                                                                                         \
         if constexpr (sizeof(KT_) == 4) {                                                           \
-            score_kernel<1, KT_><<<g2, kScoreWarps * 32, smem, s>>>(p);                             \
+            le = launch_after_producer(score_kernel<1, KT_>, g2, dim3(kScoreWarps * 32), smem, s, p);                             \
             break;                                                                                  \
         }                                                                                           \
-    default: score_kernel<0, KT_><<<g2, kScoreWarps * 32, smem, s>>>(p); break;                     \
+    default: le = launch_after_producer(score_kernel<0, KT_>, g2, dim3(kScoreWarps * 32), smem, s, p); break;                     \
     }
     switch (cfg->meta_dtype) {
     case STOM_BF16: STOM_SCORE_LAUNCH(__nv_bfloat16) break;
@@ -97,6 +100,10 @@ extern "C" int32_t stom_oqm_score_groups(const stom_oqm_config *cfg, const stom_
     default: STOM_SCORE_LAUNCH(float) break;
     }
 #undef STOM_SCORE_LAUNCH
+    if (le != cudaSuccess) {
+        set_last_cuda_error(le);
+        return STOM_ERR_CUDA;
+    }
     return finish_launch();
 }
 

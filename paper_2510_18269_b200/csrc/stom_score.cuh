@@ -30,6 +30,7 @@ template <typename T>
 __global__ void __launch_bounds__(kEmbedThreads) query_embed_kernel(const ScoreParams p) {
     __shared__ __align__(16) float part[kEmbedThreads / 8][256 + 4];  // [row group <= 32][channel <= 256]
     __shared__ float red[kEmbedThreads / 32];
+    grid_launch_dependents();  // the scoring kernel behind this one may be scheduled; it waits before it reads
     const int h = blockIdx.x, li = blockIdx.y, d = p.g.d;
     const int lanes_per_row = d >> 3;                 // threads across one row (8 channels each): 8, 16 or 32
     const int RG = kEmbedThreads / lanes_per_row;     // row groups: 32, 16 or 8
@@ -272,6 +273,7 @@ template <int V4, typename KT>
 __global__ void __launch_bounds__(kScoreWarps * 32) score_kernel(const ScoreParams p) {
     extern __shared__ __align__(16) float sq[];  // q of this layer: H*d floats, then H norms
     const int li = blockIdx.y, H = p.g.H, HD = H * p.g.d;
+    grid_dependency_wait();  // the embeddings come from the kernel just ahead in the stream
     for (int i = threadIdx.x; i < HD; i += blockDim.x) sq[i] = p.qemb[(int64_t)li * HD + i];
     float *qn = sq + HD;
     if (threadIdx.x < H) qn[threadIdx.x] = p.qnorm2[(int64_t)li * H + threadIdx.x];
