@@ -45,7 +45,7 @@ NCU_TRAFFIC_PER_UNIT = {
     # bytes per (layer, selected group): 186.0 MB over 28 x 64 units; of the 183.5 MB the kernel writes only
     # 125.4 MB had left L2 when it ended (the rest is written back later), so this undercounts by design
     "dequant_gather_kernel": 103805.0 / 4,
-    "score_kernel": 2071.0 / 4,         # bytes per (layer, stored group): 59.39 MB over 28 x 1024 units
+    "score_kernel": 2067.0 / 4,         # bytes per (layer, stored group): 59.26 MB over 28 x 1024 units
     "retrieve_kernel": 2188.0 / 4,      # bytes per (layer, stored group): 62.75 MB over 28 x 1024 units (Q read per cluster)
     # bytes per frame of 196 tokens x 1152 bf16 channels (not per kv head): 561.8 MB over 1200 frames
     "ctr_similarity_kernel": 468181.0,
