@@ -88,8 +88,8 @@ int32_t stom_ctr_reduce(const void *F, const void *prev, int32_t dtype, int32_t 
  *             the densest token of all takes its largest distance
  *   the k_s tokens of largest rho_i * delta_i are the centres (equal products: the earlier token)
  *   every other static token joins its nearest centre (equal distances: the earlier centre)
- *   a cluster becomes ONE token: the mean of its members' features (binary32 sums in ascending token order, true
- *   division), rounded to the feature type, standing at its centre's position
+ *   a cluster becomes ONE token: the mean of its members' features (binary32 sums in ascending token order, the
+ *   correctly rounded binary32 quotient), rounded to the feature type, standing at its centre's position
  * Retained group: the k_d selected dynamic rows, copied unchanged, and the k_s merged rows, in ascending position.
  *   F            as for stom_ctr_similarity; dtype STOM_BF16 or STOM_FP16 (the Gram matrix runs on the tensor cores)
  *   k_s, k_d, static_idx, dyn_idx   the outputs of stom_ctr_select for the same T frames

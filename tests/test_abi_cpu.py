@@ -1,10 +1,11 @@
 """CPU-only checks of the C-ABI library: it builds, loads, exports every symbol the
 header declares, and its host-side logic (layout, K formula, argument validation)
-behaves as documented.  No kernel is launched here."""
+behaves as documented; and an arithmetic identity one kernel relies on.  No kernel is launched here."""
 import ctypes as C
 import re
 from pathlib import Path
 
+import numpy as np
 import pytest
 
 ROOT = Path(__file__).resolve().parent.parent
@@ -160,3 +161,18 @@ def test_binding_fails_loudly_without_library(monkeypatch, tmp_path):
     monkeypatch.setattr(m, "LIB_PATH", tmp_path / "absent.so")
     with pytest.raises(ImportError):
         m.lib()
+
+
+def test_quotient_by_reciprocal_and_one_correction_is_the_correctly_rounded_one():
+    """The merge kernel divides a cluster's binary32 sums by its size n with y = rn(1/n), q = rn(s y), r = s - q n
+    (exact), q' = rn(q + r y).  That this equals the correctly rounded s / n -- which is what the oracle's binary64
+    mean, rounded once, is compared with -- is checked here in numpy for every n a frame can have."""
+    rng = np.random.default_rng(97)
+    for n in range(1, 225):
+        y = np.float32(1) / np.float32(n)
+        s = (rng.standard_normal(20000) * rng.choice([0.01, 1.0, 300.0], 20000)).astype(np.float32)
+        q = (s * y).astype(np.float32)
+        r = (s.astype(np.float64) - q.astype(np.float64) * n).astype(np.float32)      # exact: one FMA on the GPU
+        got = (q.astype(np.float64) + r.astype(np.float64) * float(y)).astype(np.float32)
+        want = (s.astype(np.float64) / n).astype(np.float32)
+        assert np.array_equal(got, want), n
