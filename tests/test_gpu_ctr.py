@@ -226,6 +226,8 @@ def _blob_stream(T, N, D, n_blobs, seed, dtype):
     (6, 224, 256, 224, 5, "bf16", 40),      # the largest frame; G = N
     (8, 33, 64, 9, 0, "bf16", 6),           # no neighbours in the density: rho = 1, delta alone decides
     (8, 64, 192, 16, 8, "fp16", 10),        # the most neighbours
+    (6, 128, 128, 32, 5, "bf16", 16),       # exactly one 128-row tile of the Gram product
+    (6, 144, 320, 40, 5, "fp16", 20),       # two tiles that overlap in all but 16 rows; five slabs through a ring of three
 ])
 def test_merge_matches_oracle_on_clustered_features(orc, T, N, D, G, knn, dtype, n_blobs):
     oqm = _lib()
