@@ -31,6 +31,7 @@
 // The layer counters live in the caller's workspace and are zeroed by a
 // memset enqueued ahead of the kernel; the selecting block also puts its
 // counter back to zero.
+#include "stom_async.cuh"
 #include "stom_score.cuh"
 #include "stom_topk.cuh"
 
@@ -182,41 +183,6 @@ __device__ __forceinline__ void embed_layer(const ScoreParams &p, int li, float 
         // part is rewritten by the next group only after that group's loads; the barrier below orders it for all
         __syncthreads();
     }
-}
-
-// Thread-block cluster primitives (sm_90+).  A kernel launched without a cluster dimension is a cluster of one.
-__device__ __forceinline__ uint32_t cluster_rank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ uint32_t cluster_size() {
-    uint32_t n;
-    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(n));
-    return n;
-}
-// Hardware barrier over all threads of the cluster; every thread of every block must call it (no spinning involved)
-__device__ __forceinline__ void cluster_sync() {
-    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// The word(s) at the same shared-memory offset as `mine` in block `rank` of the cluster
-__device__ __forceinline__ uint32_t cluster_addr(const void *mine, uint32_t rank) {
-    uint32_t a = (uint32_t)__cvta_generic_to_shared(mine), ra;
-    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(a), "r"(rank));
-    return ra;
-}
-__device__ __forceinline__ float4 ld_cluster_f4(const float4 *mine, uint32_t rank) {
-    float4 v;
-    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];"
-                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                 : "r"(cluster_addr(mine, rank))
-                 : "memory");
-    return v;
-}
-__device__ __forceinline__ float ld_cluster_f(const float *mine, uint32_t rank) {
-    float v;
-    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(cluster_addr(mine, rank)) : "memory");
-    return v;
 }
 
 // grid (chunks, layer_count), kFusedThreads threads, optionally in clusters of consecutive chunks of a layer.
