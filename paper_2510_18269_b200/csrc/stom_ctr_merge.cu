@@ -321,6 +321,8 @@ __global__ void __launch_bounds__(kMgThreads, 2) ctr_merge_kernel(const MergePar
                 }
             }
         }
+        if (dead)  // gave up (flagged): the clustering below still runs, on distances that are all zero, so that
+            for (int i = tid; i < L.rows * (L.rows + 1) / 2; i += kMgThreads) d2[i] = 0.0f;  // every index it forms is valid
         tc_fence_before_sync();
         __syncthreads();
         if (warp == 0) tmem_dealloc(tmem, kMgTmemCols);  // the tensor memory goes back before the clustering starts
