@@ -177,6 +177,8 @@ def oracle_sample(sh, K_cpu, V_cpu, Q_cpu, frames, threads=0):
     from paper_2510_18269_b200 import synth
     import numpy as np
     k = min(sh.k, frames)
+    # all the cores this process may run on, also under a launcher that exports OMP_NUM_THREADS=1 for its children
+    threads = threads or orc.host_cores()
     cfg = orc.make_config(sh.L, sh.H_q, sh.H_k, sh.d, sh.G, frames, 4, {"bf16": 0, "fp16": 1, "fp32": 2}[sh.dtype],
                           meta_dtype=META_CODE[meta_of(sh)])
     st = orc.Store(cfg)
@@ -194,7 +196,7 @@ def oracle_sample(sh, K_cpu, V_cpu, Q_cpu, frames, threads=0):
     assert orc.dequant_gather(cfg, st, 0, sh.L, idx, k, frames, ka, va, orc.BF16,
                               (sh.H_k * S * sh.d, S * sh.d, sh.d), 0, n_threads=threads) == 0
     t2 = time.perf_counter()
-    return {"quantize_s": t1 - t0, "retrieve_s": t2 - t1, "k": k, "threads": orc.max_threads() if threads == 0 else threads,
+    return {"quantize_s": t1 - t0, "retrieve_s": t2 - t1, "k": k, "threads": threads,
             "cores": orc.host_cores()}
 
 
