@@ -113,7 +113,7 @@ __device__ __forceinline__ int tri(int a, int b) { return a >= b ? a * (a + 1) /
 // Shared-memory layout (bytes): the slab ring (later the triangle), then the per-token arrays
 struct MergeLayout {
     int rows, slab_bytes, off_tri, off_nrm, off_rho, off_gam, off_slist, off_cid, off_clist, off_member, off_coff, off_slot,
-        off_flag, off_bar, total;
+        off_flag, off_wcnt, off_bar, total;
 };
 __host__ __device__ inline MergeLayout merge_layout(int N) {
     MergeLayout l;
@@ -135,6 +135,7 @@ __host__ __device__ inline MergeLayout merge_layout(int N) {
     l.off_slot = off; off += l.rows * 4;     // retained slot of every cluster
     l.off_flag = off; off += l.rows;         // per token: 1 static, 3 centre
     off = (off + 15) / 16 * 16;
+    l.off_wcnt = off; off += (kMgMaxTokens / 32) * l.rows * 4;  // [warp of 32 static tokens][cluster]: members it holds
     l.off_bar = off; off += kMgSlabs * 8 + 16;  // one mbarrier per slab, the tensor-memory base address, the abort word
     l.total = (off + 15) / 16 * 16;
     return l;
@@ -336,10 +337,12 @@ __global__ void __launch_bounds__(kMgThreads, 2) ctr_merge_kernel(const MergePar
         const bool mine = a < n_s;
         const int ia = mine ? slist[a] : 0, row = ia * (ia + 1) / 2;
         float far2 = 0.0f;  // the token's largest squared distance to another static token
-        {
-            float best[kMgMaxKnn];  // the smallest squared distances among this thread's candidates, ascending
+        // KD: slots of the insertion list, at least knn (5, the usual choice, or the maximum of 8)
+        auto density = [&](auto kd_tag) {
+            constexpr int KD = decltype(kd_tag)::value;
+            float best[KD];  // the smallest squared distances among this thread's candidates, ascending
 #pragma unroll
-            for (int q = 0; q < kMgMaxKnn; ++q) best[q] = INFINITY;
+            for (int q = 0; q < KD; ++q) best[q] = INFINITY;
             if (mine) {
 #pragma unroll 4
                 for (int b = hf; b < n_s; b += 2) {
@@ -348,7 +351,7 @@ __global__ void __launch_bounds__(kMgThreads, 2) ctr_merge_kernel(const MergePar
                     far2 = fmaxf(far2, v);          // (the token itself adds 0)
                     v = b == a ? INFINITY : v;      // ... and is no neighbour of itself
 #pragma unroll
-                    for (int q = 0; q < kMgMaxKnn; ++q) {  // insertion: v sinks to its place, the largest falls out
+                    for (int q = 0; q < KD; ++q) {  // insertion: v sinks to its place, the largest falls out
                         const float lo = fminf(best[q], v);
                         v = fmaxf(best[q], v);
                         best[q] = lo;
@@ -356,15 +359,15 @@ __global__ void __launch_bounds__(kMgThreads, 2) ctr_merge_kernel(const MergePar
                 }
             }
             // the partner's list sinks into this one: both threads end with the smallest of all candidates
-            float theirs[kMgMaxKnn];
+            float theirs[KD];
 #pragma unroll
-            for (int q = 0; q < kMgMaxKnn; ++q) theirs[q] = __shfl_xor_sync(0xffffffffu, best[q], 1);
+            for (int q = 0; q < KD; ++q) theirs[q] = __shfl_xor_sync(0xffffffffu, best[q], 1);
             far2 = fmaxf(far2, __shfl_xor_sync(0xffffffffu, far2, 1));
 #pragma unroll
-            for (int e = 0; e < kMgMaxKnn; ++e) {
+            for (int e = 0; e < KD; ++e) {
                 float v = theirs[e];
 #pragma unroll
-                for (int q = 0; q < kMgMaxKnn; ++q) {
+                for (int q = 0; q < KD; ++q) {
                     const float lo = fminf(best[q], v);
                     v = fmaxf(best[q], v);
                     best[q] = lo;
@@ -372,10 +375,12 @@ __global__ void __launch_bounds__(kMgThreads, 2) ctr_merge_kernel(const MergePar
             }
             float sum = 0.0f;
 #pragma unroll
-            for (int q = 0; q < kMgMaxKnn; ++q)
+            for (int q = 0; q < KD; ++q)
                 if (q < kk) sum += best[q];
             if (mine && hf == 0) rho[a] = kk > 0 ? expf(-sum / (float)kk) : 1.0f;
-        }
+        };
+        if (p.knn <= 5) density(std::integral_constant<int, 5>{});
+        else density(std::integral_constant<int, kMgMaxKnn>{});
         __syncthreads();
         {
             const float ra = mine ? rho[a] : 0.0f;
@@ -402,44 +407,76 @@ __global__ void __launch_bounds__(kMgThreads, 2) ctr_merge_kernel(const MergePar
             if (mine && hf == 0 && rank < k_s) flag[ia] = 3;
         }
         __syncthreads();
-        for (int a = tid; a < n_s; a += kMgThreads) {
-            if (flag[slist[a]] == 3) {
-                int before = 0;
-                for (int b = 0; b < a; ++b) before += flag[slist[b]] == 3;
-                clist[before] = slist[a];
-                cid[slist[a]] = before;
+        // the centres in ascending token order: one thread per static token from here on, a warp's share counted by
+        // ballot, the warps before it added up (coff is free until the members are sorted)
+        const int a1 = tid;
+        const int tok1 = a1 < n_s ? slist[a1] : 0;
+        {
+            const bool is_c = a1 < n_s && flag[tok1] == 3;
+            const unsigned bal = __ballot_sync(0xffffffffu, is_c);
+            if (lane == 0) coff[warp] = __popc(bal);
+            __syncthreads();
+            int before = __popc(bal & ((1u << lane) - 1u));
+            for (int w = 0; w < warp; ++w) before += coff[w];
+            if (is_c) {
+                clist[before] = tok1;
+                cid[tok1] = before;
             }
         }
+        int32_t *wcnt = reinterpret_cast<int32_t *>(smem + L.off_wcnt);
+        for (int i = tid; i < (kMgMaxTokens / 32) * L.rows; i += kMgThreads) wcnt[i] = 0;
         __syncthreads();
-        // every other static token joins its nearest centre (the earlier centre among equals)
-        for (int a = tid; a < n_s; a += kMgThreads) {
-            const int ia = slist[a];
-            if (flag[ia] != 3) {
-                int best = 0;
-                float bd = d2[tri(ia, clist[0])];
-                for (int j = 1; j < k_s; ++j) {
+        // every other static token joins its nearest centre (the earlier centre among equals): the token's two threads
+        // take the even and the odd centres
+        {
+            float bd = INFINITY;
+            int best = 0x7fffffff;
+            const bool joins = mine && flag[ia] != 3;
+            if (joins) {
+#pragma unroll 4
+                for (int j = hf; j < k_s; j += 2) {
                     const float v = d2[tri(ia, clist[j])];
                     if (v < bd) {
                         bd = v;
                         best = j;
                     }
                 }
-                cid[ia] = best;
+            }
+            const float obd = __shfl_xor_sync(0xffffffffu, bd, 1);
+            const int ob = __shfl_xor_sync(0xffffffffu, best, 1);
+            if (obd < bd || (obd == bd && ob < best)) best = ob;
+            if (joins && hf == 0) cid[ia] = best;
+        }
+        __syncthreads();
+        // members ordered by cluster, ascending token inside a cluster.  A warp holds 32 consecutive static tokens:
+        // the lanes of one cluster find each other (match), the first of them records how many they are, and a
+        // token's place is its cluster's start + the members in the warps before + those in lower lanes.
+        const int c1 = a1 < n_s ? cid[tok1] : -1 - lane;  // (lanes without a token match nobody)
+        const unsigned same = __match_any_sync(0xffffffffu, c1);
+        if (a1 < n_s && (same & ((1u << lane) - 1u)) == 0) wcnt[warp * L.rows + c1] = __popc(same);
+        __syncthreads();
+        if (warp == 0) {  // where each cluster starts: a running sum over the clusters, 32 at a time
+            int carry = 0;
+            for (int j0 = 0; j0 <= k_s; j0 += 32) {
+                const int j = j0 + lane;
+                int n = 0;
+                if (j < k_s)
+                    for (int w = 0; w < kMgMaxTokens / 32; ++w) n += wcnt[w * L.rows + j];
+                int inc = n;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int v = __shfl_up_sync(0xffffffffu, inc, o);
+                    if (lane >= o) inc += v;
+                }
+                if (j <= k_s) coff[j] = carry + inc - n;
+                carry += __shfl_sync(0xffffffffu, inc, 31);
             }
         }
         __syncthreads();
-        // members ordered by cluster, ascending token inside a cluster (counting passes)
-        for (int j = tid; j <= k_s; j += kMgThreads) {
-            int n = 0;
-            for (int a = 0; a < n_s; ++a) n += cid[slist[a]] < j;
-            coff[j] = n;
-        }
-        __syncthreads();
-        for (int a = tid; a < n_s; a += kMgThreads) {
-            const int c = cid[slist[a]];
-            int within = 0;
-            for (int b = 0; b < a; ++b) within += cid[slist[b]] == c;
-            member[coff[c] + within] = slist[a];
+        if (a1 < n_s) {
+            int within = __popc(same & ((1u << lane) - 1u));
+            for (int w = 0; w < warp; ++w) within += wcnt[w * L.rows + c1];
+            member[coff[c1] + within] = tok1;
         }
     }
     __syncthreads();
