@@ -534,15 +534,20 @@ def run_ours(args, sh):
     # ---- the other workloads of the benchmark definition, single-GPU runs of the default line only
     if args.config == "C3" and world == 1 and not args.no_other_workloads and not (args.layers or args.frames):
         others = {}
-        r5 = measure_stream(args, synth.CONFIGS["C5"], dev, rank, world, sdist, peak, peak_src, steps=max(2, args.steps // 3),
-                            warmup=3, extras=False)
-        s5 = workload_summary(r5, world, peak)
-        s5["clocks"] = r5["clocks"]
-        s5["roofline_all"] = r5["roofs"]
-        s5["steps"] = max(2, args.steps // 3)
-        others["C5-72B"] = s5
-        del r5
-        torch.cuda.empty_cache()
+        c5 = synth.CONFIGS["C5"]
+        need = 2 * c5.L * c5.T * c5.H_k * c5.G * c5.d * 2 * 1.45 + (2 << 30)   # K, V, the bank, the flush buffers
+        if torch.cuda.mem_get_info(dev)[0] >= need:
+            r5 = measure_stream(args, c5, dev, rank, world, sdist, peak, peak_src, steps=max(2, args.steps // 3),
+                                warmup=3, extras=False)
+            s5 = workload_summary(r5, world, peak)
+            s5["clocks"] = r5["clocks"]
+            s5["roofline_all"] = r5["roofs"]
+            s5["steps"] = max(2, args.steps // 3)
+            others["C5-72B"] = s5
+            del r5
+            torch.cuda.empty_cache()
+        else:
+            others["C5-72B"] = {"skipped": f"needs {need / 2**30:.0f} GiB of free device memory"}
         import dataclasses
         c4 = dataclasses.replace(synth.CONFIGS["C4"], T=240)
         others["C4-7B-interleave-240-frames"] = run_stream(args, c4, dev)
