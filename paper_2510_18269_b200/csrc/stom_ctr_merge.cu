@@ -3,7 +3,9 @@
 // by a density-based clustering and fixes none of that method's parameters; the reading implemented here
 // is the k-nearest-neighbour form of density-peak clustering (see include/stom_ctr.h for the rule, step by step).
 //
-// One block per frame.
+// One block of 16 warps per frame, two blocks per multiprocessor: the tensor memory a block's Gram stage needs is
+// allocated when that stage starts and given back as soon as the accumulators are read, so the blocks of a
+// multiprocessor take turns at it and one frame's load-bound Gram stage runs beside another's clustering.
 //   Gram     all pairwise inner products of the frame's N feature rows: a [N x D] . [D x N] contraction, the one dense
 //            product of CTR, on the fifth-generation tensor cores (tcgen05.mma, kind::f16, binary32 accumulators in
 //            tensor memory).  The rows arrive in shared memory in slabs of 64 channels (cp.async, a ring of slabs) in
@@ -15,9 +17,11 @@
 //            16 warps read the accumulators from tensor memory (a warp reaches the 32 lanes of its quarter), and the
 //            squared distances d2(i,j) = (|x_i|^2 + |x_j|^2 - 2 x_i.x_j) / D, j <= i, go to a packed triangle that
 //            takes the slabs' place.
-//   cluster  a thread per token: density from the k nearest static neighbours, distance to the nearest denser token,
-//            rank count of gamma = rho * delta for the centres, nearest centre for the rest -- a few passes over rows
-//            of the triangle, N is a few hundred at most.
+//   cluster  two threads per static token (neighbours in a warp, combined by shuffle): density from the k nearest
+//            static neighbours, distance to the nearest denser token, rank count of gamma = rho * delta for the
+//            centres, nearest centre for the rest -- a few passes over rows of the triangle.  Orders and places
+//            (the centres in token order, a member's place in its cluster) come from warp ballots and matches over 32
+//            consecutive tokens and a small table of per-warp counts, never from a thread walking all tokens.
 //   merge    a cluster's mean, 8 channels per thread, members in ascending token order, written straight into the
 //            cluster's slot of the retained group; the selected dynamic rows are copied beside them.
 #include <type_traits>
