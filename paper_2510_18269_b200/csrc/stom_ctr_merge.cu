@@ -517,31 +517,48 @@ __global__ void __launch_bounds__(kMgThreads, 2) ctr_merge_kernel(const MergePar
         const int w = k_d + k_s + e / vec, c = e % vec;
         reinterpret_cast<uint4 *>(ret + (int64_t)w * D)[c] = make_uint4(0, 0, 0, 0);
     }
-    // a cluster's mean: 8 channels per thread, the members added up in ascending token order
-    for (int e = tid; e < k_s * vec; e += kMgThreads) {
-        const int j = e / vec, c = e - j * vec;
+    // a cluster's mean: 8 channels per thread, the members added up in ascending token order.  A thread works on two
+    // (cluster, column) items at a time and asks for the first four members of both before it adds any of them up:
+    // the rows come from DRAM (they have left L2 since the Gram pass), and what bounds this loop is how many of them
+    // are on their way.
+    const int n_items = k_s * vec;
+    auto first_members = [&](int e, int &j, int &c, int &m0, int &m1, uint4 (&v)[4]) {
+        j = e / vec;
+        c = e - j * vec;
+        m0 = m1 = 0;
+        if (e < n_items) {
+            m0 = coff[j];
+            m1 = coff[j + 1];
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u)
+            v[u] = m0 + u < m1 ? __ldg(reinterpret_cast<const uint4 *>(Ft + (int64_t)member[m0 + u] * p.st) + c) : make_uint4(0, 0, 0, 0);
+    };
+    auto add_up = [&](const uint4 (&v)[4], int m, int m1, float (&s8)[8]) {
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (m + u < m1) {
+                const uint32_t w4[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    float lo, hi;
+                    unpack2<T>(w4[q], lo, hi);
+                    s8[2 * q] += lo;
+                    s8[2 * q + 1] += hi;
+                }
+            }
+        }
+    };
+    auto finish = [&](int j, int c, int m0, int m1, uint4 (&v)[4]) {
         float s8[8];
 #pragma unroll
         for (int q = 0; q < 8; ++q) s8[q] = 0.0f;
-        const int m0 = coff[j], m1 = coff[j + 1];
-        for (int m = m0; m < m1; m += 4) {  // the loads of four members are in flight together; added in member order
-            uint4 v[4];
+        add_up(v, m0, m1, s8);
+        for (int m = m0 + 4; m < m1; m += 4) {  // a cluster of more than four: the rest, four at a time
 #pragma unroll
             for (int u = 0; u < 4; ++u)
                 v[u] = m + u < m1 ? __ldg(reinterpret_cast<const uint4 *>(Ft + (int64_t)member[m + u] * p.st) + c) : make_uint4(0, 0, 0, 0);
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                if (m + u < m1) {
-                    const uint32_t w4[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        float lo, hi;
-                        unpack2<T>(w4[q], lo, hi);
-                        s8[2 * q] += lo;
-                        s8[2 * q + 1] += hi;
-                    }
-                }
-            }
+            add_up(v, m, m1, s8);
         }
         // The binary32 sum of a few 16-bit values is exact, so a correctly rounded quotient is the correctly rounded
         // mean.  Eight divisions by the same small integer: y = rn(1 / cnt) once, then per value q = rn(s y), the exact
@@ -560,6 +577,14 @@ __global__ void __launch_bounds__(kMgThreads, 2) ctr_merge_kernel(const MergePar
         o.z = pack2<T>(mean[4], mean[5]);
         o.w = pack2<T>(mean[6], mean[7]);
         reinterpret_cast<uint4 *>(ret + (int64_t)slot[j] * D)[c] = o;
+    };
+    for (int e = tid; e < n_items; e += 2 * kMgThreads) {
+        int ja, ca, a0, a1, jb, cb, b0, b1;
+        uint4 va[4], vb[4];
+        first_members(e, ja, ca, a0, a1, va);
+        first_members(e + kMgThreads, jb, cb, b0, b1, vb);
+        finish(ja, ca, a0, a1, va);
+        if (e + kMgThreads < n_items) finish(jb, cb, b0, b1, vb);
     }
 }
 
